@@ -1,0 +1,238 @@
+/*
+ * dflash.h -- C ABI of the B200 (sm_100a) DFlash draft-block / verify-accept library.
+ *
+ * What the calls compute follows the paper "DFlash: Block Diffusion for Flash Speculative
+ * Decoding": Sec. 3.1 (speculative cycle, Eq. 1), Sec. 4.1 (context features, KV injection,
+ * single-pass block drafting) and App. A.3 (KV-injection equations).
+ *
+ * Conventions
+ *   - Plain C. Every pointer is tagged [host] or [device] below. The library allocates NO device
+ *     memory: weights, KV pool, page tables, lengths, outputs and the workspace are caller-owned
+ *     device buffers; the library keeps only borrowed pointers (dflash_set_weights) which must
+ *     stay valid while they are in use.
+ *   - Every compute call is asynchronous on the caller's stream (`stream` is a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream) and never synchronises. Errors the host can see
+ *     (bad arguments, unsupported shapes, small workspace, launch failures) come back as a negative
+ *     return code and nothing is launched. Errors only the device can see (token id >= vocab, page
+ *     index outside the pool, a bounded wait that ran out) OR bits into `*dev_status` (caller
+ *     zeroes it; may be NULL) and the affected work is skipped or clamped; no kernel traps.
+ *   - Lengths that chain from one call to the next (ctx_len, n_new, accept lengths) live in device
+ *     memory, so a decode cycle needs no host round trip.
+ *   - dtype: DFLASH_F32 or DFLASH_BF16 selects the storage type of weights, features, KV pool,
+ *     and activations handed across the ABI. Accumulation, norms and softmax are fp32 either way.
+ *   - All matrices are row-major [out_features, in_features].
+ *
+ * Paged KV pool layout (element type = config dtype):
+ *     pool[layer][page][K=0|V=1][kv_head][slot 0..page_size-1][head_dim]
+ *   Logical position p of sequence b lives in physical page page_table[b*max_pages + p/page_size],
+ *   slot p % page_size. Pages need not be contiguous or ordered. Context keys are stored already
+ *   position-encoded.
+ */
+#ifndef DFLASH_H_
+#define DFLASH_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes (host-visible) ---- */
+#define DFLASH_OK                    0
+#define DFLASH_ERR_INVALID_ARG      -1
+#define DFLASH_ERR_UNSUPPORTED      -2
+#define DFLASH_ERR_WORKSPACE        -3
+#define DFLASH_ERR_CUDA             -4
+#define DFLASH_ERR_NOT_READY        -5   /* weights not set */
+
+/* ---- bits OR-ed into *dev_status by kernels ---- */
+#define DFLASH_DEV_BAD_TOKEN         1   /* token id outside [0, vocab): row embedded as token 0 */
+#define DFLASH_DEV_BAD_PAGE          2   /* page index outside the pool: tile skipped            */
+#define DFLASH_DEV_CTX_OVERFLOW      4   /* position beyond page table capacity: row skipped     */
+#define DFLASH_DEV_TIMEOUT           8   /* a bounded on-chip wait expired: output invalid       */
+
+#define DFLASH_F32   0
+#define DFLASH_BF16  1
+
+#define DFLASH_ATTN_FULL    0   /* draft mode: block rows see each other in both directions */
+#define DFLASH_ATTN_CAUSAL  1   /* verify mode: block row r sees block rows <= r            */
+
+#define DFLASH_VERIFY_LOGITS 0
+#define DFLASH_VERIFY_IDS    1
+
+typedef struct dflash_handle dflash_handle;
+
+/* Shape of the drafter. Notation: N layers, D, Hq, Hkv, hd, F, V, k tapped target layers of width
+ * D_t (App. A.3: W_c is D x k*D_t), block size B. */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t n_feat_layers, d_target, block_size, page_size;
+    int32_t dtype;          /* DFLASH_F32 | DFLASH_BF16 */
+    int32_t mask_token_id;  /* id embedded at block rows 1..B-1 */
+    int32_t use_rope;       /* 1: rotary positions (rotate-half pairing) on q and k; 0: none */
+    float   rms_eps;
+    float   softmax_scale;  /* usually head_dim^-1/2 */
+} dflash_config;
+
+typedef struct {
+    const void* g1;        /* [device] [D]            pre-attention norm gain            */
+    const void* W_qkv;     /* [device] [(Hq+2Hkv)*hd, D]  rows: q heads, k heads, v heads */
+    const void* W_o;       /* [device] [D, Hq*hd]                                         */
+    const void* g2;        /* [device] [D]            pre-FFN norm gain                  */
+    const void* W_gateup;  /* [device] [2F, D]        row 2j = gate_j, row 2j+1 = up_j   */
+    const void* W_down;    /* [device] [D, F]                                             */
+} dflash_layer_weights;
+
+typedef struct {
+    const void* embed;                    /* [device] [V, D] token embedding (shared with target) */
+    const void* W_c;                      /* [device] [D, k*D_t] context fusion (App. A.3)        */
+    const void* g_c;                      /* [device] [D] gain of the fusion RMSNorm              */
+    const dflash_layer_weights* layers;   /* [host]   array of n_layers entries (copied)          */
+    const void* g_f;                      /* [device] [D] final norm gain                         */
+    const void* W_lm;                     /* [device] [V, D] LM head (shared with target)         */
+    const float* rope_cos;                /* [device] [rope_max_pos, hd/2] fp32                   */
+    const float* rope_sin;                /* [device] [rope_max_pos, hd/2] fp32                   */
+    int32_t rope_max_pos;
+} dflash_weights;
+
+/* ---- life cycle (host only, no CUDA work) ---- */
+
+/* Validates the configuration and builds a handle. Returns DFLASH_ERR_UNSUPPORTED for shapes the
+ * kernels do not cover (head_dim not in {64,128}, Hq % Hkv != 0, block_size > 32, ...). */
+int32_t dflash_create(const dflash_config* cfg /*[host]*/, dflash_handle** out /*[host]*/);
+void    dflash_destroy(dflash_handle* h);
+
+/* Borrow the weight pointers. The `layers` array is copied; the device buffers are not. */
+int32_t dflash_set_weights(dflash_handle* h, const dflash_weights* w /*[host]*/);
+
+/* Bytes of device workspace that any call below needs for up to `max_rows` rows in flight
+ * (rows = batch * block_size for a draft, batch * (gamma+1) for verify-side calls, batch * max_new
+ * for the context projection) and `max_batch` sequences. */
+int64_t dflash_workspace_bytes(const dflash_handle* h, int32_t max_batch, int32_t max_rows);
+
+/* ---- context-feature fusion and KV injection (App. A.3, first and second display) ----
+ * For each valid row (b, r), r < n_new[b]:
+ *   y = W_c * feats[b, r, :]                       (feats = k tapped hidden states, concatenated)
+ *   H_t = g_c * y / sqrt(mean(y^2) + eps)
+ *   for each draft layer i: K = RoPE(W_i^K H_t, pos), V = W_i^V H_t, pos = ctx_len[b] + r
+ *   written to pool[i][page_table[b][pos/page]][K|V][:][pos % page][:].
+ * ctx_len is read, never updated (the accept step produces the next value). */
+typedef struct {
+    const void*    feats;        /* [device] [batch, max_new, k*D_t], config dtype            */
+    int32_t        batch;
+    int32_t        max_new;      /* row slots per sequence                                    */
+    const int32_t* n_new;        /* [device] [batch] valid rows per sequence; NULL = max_new  */
+    const int32_t* ctx_len;      /* [device] [batch] position of row 0                        */
+    const int32_t* page_table;   /* [device] [batch, max_pages]                               */
+    int32_t        max_pages;
+    void*          kv_pool;      /* [device] pool, see layout above                           */
+    int32_t        n_pool_pages;
+    void*          workspace;    /* [device] >= dflash_workspace_bytes(h, batch, batch*max_new), 256-byte aligned */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;   /* [device] may be NULL                                      */
+} dflash_ctx_args;
+int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a /*[host]*/, void* stream);
+
+/* ---- single-pass block draft (Sec. 4.1 "Parallel diffusion drafting"; App. A.3) ----
+ * Per sequence b: rows r = 0..B-1 at positions ctx_len[b]+r; row 0 embeds anchor_ids[b], the others
+ * the mask token. N pre-norm layers: q,k,v projections (+RoPE), attention of every row over the
+ * ctx_len[b] cached context entries and ALL B block rows, output projection, SwiGLU FFN; final
+ * norm; LM head; draft_ids[b, r] = argmax_v logits (lowest index among equal maxima). Logits are
+ * never written unless logits_out is given. */
+typedef struct {
+    const int32_t* anchor_ids;   /* [device] [batch]                                          */
+    int32_t        batch;
+    const int32_t* ctx_len;      /* [device] [batch]                                          */
+    int32_t        max_ctx_len;  /* [host value] upper bound of ctx_len (sizes the KV split)  */
+    const int32_t* page_table;   /* [device] [batch, max_pages]                               */
+    int32_t        max_pages;
+    const void*    kv_pool;      /* [device]                                                  */
+    int32_t        n_pool_pages;
+    void*          workspace;    /* [device] >= dflash_workspace_bytes(h, batch, batch*B)     */
+    int64_t        workspace_bytes;
+    int32_t*       draft_ids;    /* [device] out [batch, B]                                   */
+    float*         top1;         /* [device] out [batch, B] winning logit; may be NULL        */
+    float*         margin;       /* [device] out [batch, B] top-1 minus top-2; may be NULL    */
+    float*         hidden_out;   /* [device] out [batch*B, D] fp32 residual stream after the last layer; may be NULL */
+    float*         logits_out;   /* [device] out [batch*B, V] fp32; may be NULL (tests only)  */
+    int32_t*       dev_status;   /* [device] may be NULL                                      */
+} dflash_draft_args;
+int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a /*[host]*/, void* stream);
+
+/* ---- greedy verify / accept (Sec. 3.1: tau in [1, gamma+1] incl. the bonus token) ----
+ * p_j = argmax_v logits[b, j, :] (mode LOGITS) or target_ids[b, j] (mode IDS), j = 0..gamma.
+ * a = length of the longest prefix with draft[b, i] == p_i, i < a;  tau = a + 1;
+ * out_tokens[b] = draft[b, 0..a-1], p_a, then -1; bonus[b] = p_a; new_ctx_len[b] = ctx_len[b]+tau. */
+typedef struct {
+    int32_t        mode;             /* DFLASH_VERIFY_LOGITS | DFLASH_VERIFY_IDS               */
+    const void*    logits;           /* [device] mode LOGITS: [batch, gamma+1, vocab]          */
+    int32_t        logits_dtype;     /* DFLASH_F32 | DFLASH_BF16                               */
+    int64_t        logits_row_stride;/* elements between rows j and j+1 (0 = vocab)            */
+    const int32_t* target_ids;       /* [device] mode IDS: [batch, gamma+1]                    */
+    const int32_t* draft_ids;        /* [device] first draft of sequence b at draft_ids + b*draft_stride */
+    int32_t        draft_stride;     /* elements                                               */
+    int32_t        batch, gamma, vocab;
+    const int32_t* ctx_len;          /* [device] [batch]                                       */
+    int32_t*       accept_len;       /* [device] out [batch] tau                               */
+    int32_t*       out_tokens;       /* [device] out [batch, gamma+1]                          */
+    int32_t*       bonus;            /* [device] out [batch]                                   */
+    int32_t*       new_ctx_len;      /* [device] out [batch]; may alias ctx_len                */
+    int32_t*       target_ids_out;   /* [device] out [batch, gamma+1] the p_j; may be NULL     */
+    void*          workspace;        /* [device] >= dflash_workspace_bytes(h, batch, batch*(gamma+1)) */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;
+} dflash_verify_args;
+int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a /*[host]*/, void* stream);
+
+/* ---- building block: attention of `rows` block rows per sequence over paged context + the block
+ * itself (App. A.3: K = [K_ctx ; K_block]_seq). FULL = draft mode, CAUSAL = the target's verify
+ * pass over (gamma+1) rows. Head geometry and dtype come from the handle. q and k_blk must already
+ * be position-encoded. */
+typedef struct {
+    int32_t        mode;         /* DFLASH_ATTN_FULL | DFLASH_ATTN_CAUSAL                     */
+    const void*    q;            /* [device] [batch, rows, Hq, hd]                            */
+    const void*    k_blk;        /* [device] [batch, rows, Hkv, hd]                           */
+    const void*    v_blk;        /* [device] [batch, rows, Hkv, hd]                           */
+    int32_t        batch, rows;  /* rows <= 32                                                */
+    const int32_t* ctx_len;      /* [device] [batch]                                          */
+    int32_t        max_ctx_len;  /* [host value] upper bound of ctx_len                       */
+    const int32_t* page_table;   /* [device] [batch, max_pages]                               */
+    int32_t        max_pages;
+    const void*    kv_pool;      /* [device] pool with the layout above                       */
+    int32_t        n_pool_pages;
+    int32_t        layer;        /* which pool layer to read                                  */
+    void*          out;          /* [device] [batch, rows, Hq, hd]                            */
+    void*          workspace;
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;
+} dflash_attn_args;
+int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a /*[host]*/, void* stream);
+
+/* ---- building block: LM head fused with row-wise argmax (Sec. 4.2: LM head shared with the
+ * target). ids[m] = argmax_v (W_lm z_m)_v with z = hidden (apply_norm = 0) or
+ * z = g_f * hidden / rms(hidden) (apply_norm = 1). */
+typedef struct {
+    const void* hidden;          /* [device] [n_rows, D]; config dtype, or fp32 if hidden_is_f32 */
+    int32_t     hidden_is_f32;
+    int32_t     n_rows;
+    int32_t     apply_norm;
+    int32_t*    ids;             /* [device] out [n_rows]                                     */
+    float*      top1;            /* [device] out [n_rows]; may be NULL                        */
+    float*      margin;          /* [device] out [n_rows]; may be NULL                        */
+    float*      logits_out;      /* [device] out [n_rows, V] fp32; may be NULL                */
+    void*       workspace;
+    int64_t     workspace_bytes;
+    int32_t*    dev_status;
+} dflash_lmhead_args;
+int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a /*[host]*/, void* stream);
+
+/* Static description of a return code. */
+const char* dflash_status_string(int32_t code);
+
+/* Number of kernel launches the library has issued since it was loaded (all handles). */
+int64_t dflash_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DFLASH_H_ */

@@ -1,0 +1,81 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "dflash.h"
+
+#define DFLASH_MAX_LAYERS 64
+
+struct dflash_handle {
+    dflash_config cfg;
+    dflash_layer_weights layers[DFLASH_MAX_LAYERS];
+    dflash_weights w;
+    bool has_weights;
+    int sm_count;
+};
+
+namespace dflash {
+
+// Counts kernel launches issued by the library (reported by dflash_launch_count).
+extern long long g_launches;
+
+inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline int elem_size(int dtype) { return dtype == DFLASH_F32 ? 4 : 2; }
+
+// Bump allocator over the caller's workspace; the same walk sizes it (base == nullptr).
+struct Arena {
+    char* base;
+    int64_t off;
+    explicit Arena(void* b) : base(static_cast<char*>(b)), off(0) {}
+    void* take(int64_t bytes) {
+        void* p = base ? base + off : nullptr;
+        off += align_up(bytes, 256);
+        return p;
+    }
+};
+
+// Activation buffers of one pass over `rows` rows (rows = batch * rows-per-sequence).
+struct Workspace {
+    float* x;        // [rows, D]   fp32 residual stream
+    void*  u;        // [rows, max(D, k*D_t?)] normalised operand, config dtype
+    float* tmp;      // [rows, max(QKV, 2F, D)] fp32 GEMM output before its epilogue
+    void*  q;        // [rows, Hq*hd]
+    void*  k_blk;    // [rows, Hkv*hd]
+    void*  v_blk;    // [rows, Hkv*hd]
+    void*  attn;     // [rows, Hq*hd]
+    void*  h;        // [rows, F]
+    float* logits;   // [min(rows, LOGIT_ROWS), V] fp32 (only the fp32 path stages logits)
+    int32_t* ids;    // [rows]
+    float* part;     // attention split-KV partials
+    int64_t bytes;
+};
+Workspace carve(const dflash_config& c, void* base, int batch, int rows);
+
+constexpr int LOGIT_ROWS = 64;
+
+struct Launch {
+    const dflash_handle* h;
+    cudaStream_t st;
+    int32_t* status;
+};
+
+// ---- generic (any dtype) kernels: the whole fp32 path, and the small steps of the bf16 path ----
+int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch);
+int launch_rmsnorm(const Launch& L, const void* in, bool in_is_f32, const void* g, bool apply,
+                   void* out, int rows, int dim);
+int launch_gemm_simt(const Launch& L, const void* X, const void* W, float* Y, int M, int N, int K,
+                     bool accumulate);
+int launch_rope_split(const Launch& L, const float* qkv, const int32_t* ctx_len, int rows_per_seq,
+                      int rows, void* q, void* k, void* v);
+int launch_swiglu(const Launch& L, const float* gu, void* h, int rows);
+int launch_attention_simt(const Launch& L, const dflash_attn_args& a);
+int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer);
+int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows,
+                      int vocab, int32_t* ids, float* top1, float* margin);
+int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids);
+int launch_copy_f32(const Launch& L, const float* src, float* dst, int64_t n);
+
+}  // namespace dflash

@@ -1,0 +1,545 @@
+// Generic CUDA-core kernels, templated on the storage type. They are the whole fp32 path (the
+// tiny configuration) and the small element-wise steps of the bf16 path; the bf16 contractions
+// and attention have tensor-core kernels of their own.
+#include "dflash_internal.h"
+
+#include <math_constants.h>
+
+namespace dflash {
+
+long long g_launches = 0;
+
+#define DFLASH_CHECK_LAUNCH()                                     \
+    do {                                                          \
+        ++g_launches;                                             \
+        if (cudaPeekAtLastError() != cudaSuccess) return DFLASH_ERR_CUDA; \
+    } while (0)
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Block-wide sum / max for blockDim.x <= 1024 (multiple of 32). `red` holds 32 floats.
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    float t = (lane < nw) ? red[lane] : 0.f;
+    return warp_sum(t);
+}
+__device__ __forceinline__ float block_max(float v, float* red) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    v = warp_max(v);
+    __syncthreads();
+    if (lane == 0) red[w] = v;
+    __syncthreads();
+    float t = (lane < nw) ? red[lane] : -CUDART_INF_F;
+    return warp_max(t);
+}
+
+// ------------------------------------------------------------------------------------------
+// embedding gather: row 0 of each block = anchor, rows 1.. = mask token (Sec. 4.2)
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ anchor,
+                             float* __restrict__ x, int B, int D, int V, int mask_id, int32_t* status) {
+    const int row = blockIdx.x, b = row / B, r = row % B;
+    int id = (r == 0) ? anchor[b] : mask_id;
+    if (id < 0 || id >= V) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_TOKEN);
+        id = 0;
+    }
+    const T* src = E + (size_t)id * D;
+    float* dst = x + (size_t)row * D;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = to_f(src[d]);
+}
+
+int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch) {
+    const dflash_config& c = L.h->cfg;
+    const int rows = batch * c.block_size;
+    if (c.dtype == DFLASH_F32)
+        embed_kernel<float><<<rows, 256, 0, L.st>>>((const float*)L.h->w.embed, anchor, x, c.block_size,
+                                                    c.d_model, c.vocab, c.mask_token_id, L.status);
+    else
+        embed_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>((const __nv_bfloat16*)L.h->w.embed, anchor, x,
+                                                            c.block_size, c.d_model, c.vocab,
+                                                            c.mask_token_id, L.status);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// RMSNorm (App. A.3): out = g * y * rsqrt(mean(y^2) + eps); statistics in fp32
+// ------------------------------------------------------------------------------------------
+template <typename Tin, typename Tg, typename Tout>
+__global__ void rmsnorm_kernel(const Tin* __restrict__ in, const Tg* __restrict__ g, Tout* __restrict__ out,
+                               int dim, float eps, int apply) {
+    __shared__ float red[32];
+    const Tin* src = in + (size_t)blockIdx.x * dim;
+    Tout* dst = out + (size_t)blockIdx.x * dim;
+    float scale = 1.f;
+    if (apply) {
+        float ss = 0.f;
+        for (int d = threadIdx.x; d < dim; d += blockDim.x) { float v = to_f(src[d]); ss += v * v; }
+        ss = block_sum(ss, red);
+        scale = rsqrtf(ss / (float)dim + eps);
+    }
+    for (int d = threadIdx.x; d < dim; d += blockDim.x) {
+        float v = to_f(src[d]);
+        dst[d] = from_f<Tout>(apply ? v * scale * to_f(g[d]) : v);
+    }
+}
+
+int launch_rmsnorm(const Launch& L, const void* in, bool in_is_f32, const void* g, bool apply, void* out,
+                   int rows, int dim) {
+    const dflash_config& c = L.h->cfg;
+    if (rows == 0) return DFLASH_OK;
+    const int ap = apply ? 1 : 0;
+    if (c.dtype == DFLASH_F32) {
+        rmsnorm_kernel<float, float, float><<<rows, 256, 0, L.st>>>((const float*)in, (const float*)g,
+                                                                    (float*)out, dim, c.rms_eps, ap);
+    } else if (in_is_f32) {
+        rmsnorm_kernel<float, __nv_bfloat16, __nv_bfloat16><<<rows, 256, 0, L.st>>>(
+            (const float*)in, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, dim, c.rms_eps, ap);
+    } else {
+        rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16><<<rows, 256, 0, L.st>>>(
+            (const __nv_bfloat16*)in, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, dim, c.rms_eps, ap);
+    }
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Y[M,N] (+)= X[M,K] * W[N,K]^T on CUDA cores, fp32 accumulate. 64x64 tile, 4x4 per thread.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ X, const T* __restrict__ W,
+                                                        float* __restrict__ Y, int M, int N, int K,
+                                                        int accumulate) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float sx[BK][BM + 1];
+    __shared__ float sw[BK][BN + 1];
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;   // tx -> n, ty -> m
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        // 64 rows x 16 k = 1024 elements per operand, 4 per thread
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = threadIdx.x + i * 256;
+            const int r = e / BK, kk = e % BK;
+            const int k = k0 + kk;
+            sx[kk][r] = (m0 + r < M && k < K) ? to_f(X[(size_t)(m0 + r) * K + k]) : 0.f;
+            sw[kk][r] = (n0 + r < N && k < K) ? to_f(W[(size_t)(n0 + r) * K + k]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = sx[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = sw[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= N) continue;
+            float* y = Y + (size_t)m * N + n;
+            *y = accumulate ? (*y + acc[i][j]) : acc[i][j];
+        }
+    }
+}
+
+int launch_gemm_simt(const Launch& L, const void* X, const void* W, float* Y, int M, int N, int K,
+                     bool accumulate) {
+    if (M == 0 || N == 0) return DFLASH_OK;
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    if (L.h->cfg.dtype == DFLASH_F32)
+        gemm_simt_kernel<float><<<grid, 256, 0, L.st>>>((const float*)X, (const float*)W, Y, M, N, K,
+                                                        accumulate ? 1 : 0);
+    else
+        gemm_simt_kernel<__nv_bfloat16><<<grid, 256, 0, L.st>>>((const __nv_bfloat16*)X,
+                                                                (const __nv_bfloat16*)W, Y, M, N, K,
+                                                                accumulate ? 1 : 0);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// split the fused projection into q, k, v and rotate q and k (rotate-half pairing)
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rope_split_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ ctx_len,
+                                  int rows_per_seq, T* __restrict__ q, T* __restrict__ k,
+                                  T* __restrict__ v, int Hq, int Hkv, int hd, int use_rope,
+                                  const float* __restrict__ cs, const float* __restrict__ sn, int max_pos,
+                                  int32_t* status) {
+    const int row = blockIdx.x, b = row / rows_per_seq, r = row % rows_per_seq;
+    const int half = hd / 2;
+    int pos = ctx_len[b] + r;
+    if (use_rope && (pos < 0 || pos >= max_pos)) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_CTX_OVERFLOW);
+        pos = pos < 0 ? 0 : max_pos - 1;
+    }
+    const int qdim = Hq * hd, kdim = Hkv * hd;
+    const float* src = qkv + (size_t)row * (qdim + 2 * kdim);
+    // rotated part: q heads then k heads
+    for (int e = threadIdx.x; e < (Hq + Hkv) * half; e += blockDim.x) {
+        const int head = e / half, i = e % half;
+        const float a = src[head * hd + i], bb = src[head * hd + i + half];
+        float c = 1.f, s = 0.f;
+        if (use_rope) { c = cs[(size_t)pos * half + i]; s = sn[(size_t)pos * half + i]; }
+        const float o1 = a * c - bb * s, o2 = bb * c + a * s;
+        if (head < Hq) {
+            q[(size_t)row * qdim + head * hd + i] = from_f<T>(o1);
+            q[(size_t)row * qdim + head * hd + i + half] = from_f<T>(o2);
+        } else {
+            const int kh = head - Hq;
+            k[(size_t)row * kdim + kh * hd + i] = from_f<T>(o1);
+            k[(size_t)row * kdim + kh * hd + i + half] = from_f<T>(o2);
+        }
+    }
+    for (int e = threadIdx.x; e < kdim; e += blockDim.x)
+        v[(size_t)row * kdim + e] = from_f<T>(src[qdim + kdim + e]);
+}
+
+int launch_rope_split(const Launch& L, const float* qkv, const int32_t* ctx_len, int rows_per_seq, int rows,
+                      void* q, void* k, void* v) {
+    const dflash_config& c = L.h->cfg;
+    if (rows == 0) return DFLASH_OK;
+    if (c.dtype == DFLASH_F32)
+        rope_split_kernel<float><<<rows, 256, 0, L.st>>>(qkv, ctx_len, rows_per_seq, (float*)q, (float*)k,
+                                                         (float*)v, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                                         c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin,
+                                                         L.h->w.rope_max_pos, L.status);
+    else
+        rope_split_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>(
+            qkv, ctx_len, rows_per_seq, (__nv_bfloat16*)q, (__nv_bfloat16*)k, (__nv_bfloat16*)v, c.n_q_heads,
+            c.n_kv_heads, c.head_dim, c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin, L.h->w.rope_max_pos,
+            L.status);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// SwiGLU on the interleaved gate/up projection: h_j = silu(gu[2j]) * gu[2j+1]
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ h, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float g = gu[2 * i], u = gu[2 * i + 1];
+    h[i] = from_f<T>(g / (1.f + __expf(-g)) * u);
+}
+
+int launch_swiglu(const Launch& L, const float* gu, void* h, int rows) {
+    const dflash_config& c = L.h->cfg;
+    const int64_t n = (int64_t)rows * c.d_ffn;
+    if (n == 0) return DFLASH_OK;
+    const int grid = (int)((n + 255) / 256);
+    if (c.dtype == DFLASH_F32) swiglu_kernel<float><<<grid, 256, 0, L.st>>>(gu, (float*)h, n);
+    else swiglu_kernel<__nv_bfloat16><<<grid, 256, 0, L.st>>>(gu, (__nv_bfloat16*)h, n);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// attention over [paged context ; block] on CUDA cores: one CTA per (row, q head, sequence),
+// keys in chunks of 128 with a running (max, sum) softmax.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) attention_simt_kernel(
+    const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
+    const T* __restrict__ pool, const int32_t* __restrict__ page_table, const int32_t* __restrict__ ctx_len,
+    T* __restrict__ out, int R, int Hq, int Hkv, int hd, int PG, int max_pages, int n_pages, int layer,
+    float scale, int causal, int32_t* status) {
+    __shared__ float sq[128];
+    __shared__ float sp[128];
+    __shared__ float red[32];
+    const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int kvh = h / (Hq / Hkv);
+    const int tid = threadIdx.x;
+    const int L = ctx_len[b];
+    const int n_keys = L + R;
+    const size_t row = (size_t)b * R + r;
+    if (tid < hd) sq[tid] = to_f(q[(row * Hq + h) * hd + tid]) * scale;
+    __syncthreads();
+
+    float m = -CUDART_INF_F, l = 0.f, acc = 0.f;
+    for (int j0 = 0; j0 < n_keys; j0 += 128) {
+        const int j = j0 + tid;
+        const T* kp = nullptr;
+        const T* vp = nullptr;
+        if (j < L) {
+            const int pidx = j / PG;
+            const int page = pidx < max_pages ? page_table[(size_t)b * max_pages + pidx] : -1;
+            if (page >= 0 && page < n_pages) {
+                const size_t base = ((((size_t)layer * n_pages + page) * 2) * Hkv + kvh) * PG * hd;
+                kp = pool + base + (size_t)(j % PG) * hd;
+                vp = kp + (size_t)Hkv * PG * hd;
+            } else if (status) {
+                atomicOr(status, DFLASH_DEV_BAD_PAGE);
+            }
+        } else if (j < n_keys) {
+            const int rr = j - L;
+            if (!causal || rr <= r) {
+                kp = k_blk + (((size_t)b * R + rr) * Hkv + kvh) * hd;
+                vp = v_blk + (((size_t)b * R + rr) * Hkv + kvh) * hd;
+            }
+        }
+        float s = -CUDART_INF_F;
+        if (kp) {
+            float d = 0.f;
+            for (int e = 0; e < hd; ++e) d = fmaf(sq[e], to_f(kp[e]), d);
+            s = d;
+        }
+        const float cmax = block_max(s, red);
+        const float m_new = fmaxf(m, cmax);          // finite: every chunk holds >= 1 visible key or m stays
+        float p = 0.f, corr = 1.f;
+        if (m_new > -CUDART_INF_F) {
+            p = kp ? __expf(s - m_new) : 0.f;
+            corr = (m > -CUDART_INF_F) ? __expf(m - m_new) : 0.f;
+        }
+        sp[tid] = p;
+        const float psum = block_sum(p, red);         // contains __syncthreads: sp is visible after it
+        l = l * corr + psum;
+        m = m_new;
+        // thread d accumulates output component d over the chunk's keys
+        if (tid < hd) {
+            float a = acc * corr;
+            const int lim = min(128, n_keys - j0);
+            for (int jj = 0; jj < lim; ++jj) {
+                const float pj = sp[jj];
+                if (pj == 0.f) continue;
+                const int jg = j0 + jj;
+                const T* vv;
+                if (jg < L) {
+                    const int page = page_table[(size_t)b * max_pages + jg / PG];
+                    vv = pool + (((((size_t)layer * n_pages + page) * 2 + 1) * Hkv + kvh) * PG + (jg % PG)) * hd;
+                } else {
+                    vv = v_blk + (((size_t)b * R + (jg - L)) * Hkv + kvh) * hd;
+                }
+                a = fmaf(pj, to_f(vv[tid]), a);
+            }
+            acc = a;
+        }
+        __syncthreads();
+    }
+    if (tid < hd) out[(row * Hq + h) * hd + tid] = from_f<T>(l > 0.f ? acc / l : 0.f);
+}
+
+int launch_attention_simt(const Launch& L, const dflash_attn_args& a) {
+    const dflash_config& c = L.h->cfg;
+    if (a.batch == 0 || a.rows == 0) return DFLASH_OK;
+    dim3 grid(a.rows, c.n_q_heads, a.batch);
+    const int causal = a.mode == DFLASH_ATTN_CAUSAL ? 1 : 0;
+    if (c.dtype == DFLASH_F32)
+        attention_simt_kernel<float><<<grid, 128, 0, L.st>>>(
+            (const float*)a.q, (const float*)a.k_blk, (const float*)a.v_blk, (const float*)a.kv_pool,
+            a.page_table, a.ctx_len, (float*)a.out, a.rows, c.n_q_heads, c.n_kv_heads, c.head_dim, c.page_size,
+            a.max_pages, a.n_pool_pages, a.layer, c.softmax_scale, causal, L.status);
+    else
+        attention_simt_kernel<__nv_bfloat16><<<grid, 128, 0, L.st>>>(
+            (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k_blk, (const __nv_bfloat16*)a.v_blk,
+            (const __nv_bfloat16*)a.kv_pool, a.page_table, a.ctx_len, (__nv_bfloat16*)a.out, a.rows,
+            c.n_q_heads, c.n_kv_heads, c.head_dim, c.page_size, a.max_pages, a.n_pool_pages, a.layer,
+            c.softmax_scale, causal, L.status);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// context K/V of one layer: rotate K, scatter K and V into the paged pool
+// kv: [rows, 2*Hkv*hd] fp32 (K heads then V heads)
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void ctx_scatter_kernel(const float* __restrict__ kv, const int32_t* __restrict__ n_new,
+                                   const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ page_table,
+                                   T* __restrict__ pool, int max_new, int Hkv, int hd, int PG, int max_pages,
+                                   int n_pages, int layer, int use_rope, const float* __restrict__ cs,
+                                   const float* __restrict__ sn, int max_pos, int32_t* status) {
+    const int row = blockIdx.x, b = row / max_new, r = row % max_new;
+    const int nn = n_new ? n_new[b] : max_new;
+    if (r >= nn) return;
+    const int pos = ctx_len[b] + r;
+    const int pidx = pos / PG;
+    if (pos < 0 || pidx >= max_pages || (use_rope && pos >= max_pos)) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_CTX_OVERFLOW);
+        return;
+    }
+    const int page = page_table[(size_t)b * max_pages + pidx];
+    if (page < 0 || page >= n_pages) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_PAGE);
+        return;
+    }
+    const int half = hd / 2, kdim = Hkv * hd;
+    const float* src = kv + (size_t)row * 2 * kdim;
+    T* kdst = pool + ((((size_t)layer * n_pages + page) * 2) * Hkv) * PG * hd + (size_t)(pos % PG) * hd;
+    T* vdst = kdst + (size_t)Hkv * PG * hd;
+    for (int e = threadIdx.x; e < Hkv * half; e += blockDim.x) {
+        const int head = e / half, i = e % half;
+        const float a = src[head * hd + i], bb = src[head * hd + i + half];
+        float c = 1.f, s = 0.f;
+        if (use_rope) { c = cs[(size_t)pos * half + i]; s = sn[(size_t)pos * half + i]; }
+        kdst[(size_t)head * PG * hd + i] = from_f<T>(a * c - bb * s);
+        kdst[(size_t)head * PG * hd + i + half] = from_f<T>(bb * c + a * s);
+    }
+    for (int e = threadIdx.x; e < kdim; e += blockDim.x) {
+        const int head = e / hd, i = e % hd;
+        vdst[(size_t)head * PG * hd + i] = from_f<T>(src[kdim + e]);
+    }
+}
+
+int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer) {
+    const dflash_config& c = L.h->cfg;
+    const int rows = a.batch * a.max_new;
+    if (rows == 0) return DFLASH_OK;
+    if (c.dtype == DFLASH_F32)
+        ctx_scatter_kernel<float><<<rows, 128, 0, L.st>>>(
+            kv, a.n_new, a.ctx_len, a.page_table, (float*)a.kv_pool, a.max_new, c.n_kv_heads, c.head_dim,
+            c.page_size, a.max_pages, a.n_pool_pages, layer, c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin,
+            L.h->w.rope_max_pos, L.status);
+    else
+        ctx_scatter_kernel<__nv_bfloat16><<<rows, 128, 0, L.st>>>(
+            kv, a.n_new, a.ctx_len, a.page_table, (__nv_bfloat16*)a.kv_pool, a.max_new, c.n_kv_heads,
+            c.head_dim, c.page_size, a.max_pages, a.n_pool_pages, layer, c.use_rope, L.h->w.rope_cos,
+            L.h->w.rope_sin, L.h->w.rope_max_pos, L.status);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// row-wise argmax with runner-up: lowest index among equal maxima, NaN never wins
+// ------------------------------------------------------------------------------------------
+struct Top2 {
+    float v1; int i1; float v2;
+};
+__device__ __forceinline__ void top2_push(Top2& t, float v, int i) {
+    if (v > t.v1 || (v == t.v1 && i < t.i1)) { t.v2 = t.v1; t.v1 = v; t.i1 = i; }
+    else if (v > t.v2) t.v2 = v;
+}
+__device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
+    Top2 r;
+    if (b.v1 > a.v1 || (b.v1 == a.v1 && b.i1 < a.i1)) { r.v1 = b.v1; r.i1 = b.i1; r.v2 = fmaxf(a.v1, b.v2); }
+    else { r.v1 = a.v1; r.i1 = a.i1; r.v2 = fmaxf(a.v2, b.v1); }
+    return r;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(512) row_argmax_kernel(const T* __restrict__ logits, int64_t row_stride,
+                                                         int vocab, int32_t* __restrict__ ids,
+                                                         float* __restrict__ top1, float* __restrict__ margin) {
+    __shared__ Top2 sh[16];
+    const T* src = logits + (size_t)blockIdx.x * row_stride;
+    Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
+    for (int i = threadIdx.x; i < vocab; i += blockDim.x) top2_push(t, to_f(src[i]), i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Top2 u;
+        u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t = top2_merge(t, u);
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) sh[w] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Top2 r = sh[0];
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i) r = top2_merge(r, sh[i]);
+        const int idx = (r.i1 == 0x7fffffff) ? 0 : r.i1;   // nothing compared greater than -inf
+        ids[blockIdx.x] = idx;
+        if (top1) top1[blockIdx.x] = r.v1;
+        if (margin) margin[blockIdx.x] = r.v1 - r.v2;
+    }
+}
+
+int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows, int vocab,
+                      int32_t* ids, float* top1, float* margin) {
+    if (rows == 0) return DFLASH_OK;
+    if (dtype == DFLASH_F32)
+        row_argmax_kernel<float><<<rows, 512, 0, L.st>>>((const float*)logits, row_stride, vocab, ids, top1, margin);
+    else
+        row_argmax_kernel<__nv_bfloat16><<<rows, 512, 0, L.st>>>((const __nv_bfloat16*)logits, row_stride, vocab,
+                                                                 ids, top1, margin);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// accept rule (Sec. 3.1): longest agreeing prefix + bonus token, one thread per sequence
+// ------------------------------------------------------------------------------------------
+__global__ void accept_kernel(const int32_t* __restrict__ target_ids, const int32_t* __restrict__ draft_ids,
+                              int draft_stride, int batch, int gamma, const int32_t* __restrict__ ctx_len,
+                              int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
+                              int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx_len,
+                              int32_t* __restrict__ target_ids_out) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int32_t* p = target_ids + (size_t)b * (gamma + 1);
+    const int32_t* d = draft_ids + (size_t)b * draft_stride;
+    int a = 0;
+    while (a < gamma && d[a] == p[a]) ++a;
+    int32_t* o = out_tokens + (size_t)b * (gamma + 1);
+    for (int i = 0; i <= gamma; ++i) o[i] = i < a ? d[i] : (i == a ? p[a] : -1);
+    const int32_t len = ctx_len[b];
+    accept_len[b] = a + 1;
+    bonus[b] = p[a];
+    new_ctx_len[b] = len + a + 1;
+    if (target_ids_out && target_ids_out != target_ids)
+        for (int i = 0; i <= gamma; ++i) target_ids_out[(size_t)b * (gamma + 1) + i] = p[i];
+}
+
+int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids) {
+    if (a.batch == 0) return DFLASH_OK;
+    accept_kernel<<<(a.batch + 127) / 128, 128, 0, L.st>>>(target_ids, a.draft_ids, a.draft_stride, a.batch,
+                                                           a.gamma, a.ctx_len, a.accept_len, a.out_tokens,
+                                                           a.bonus, a.new_ctx_len, a.target_ids_out);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+__global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = src[i];
+}
+int launch_copy_f32(const Launch& L, const float* src, float* dst, int64_t n) {
+    if (n == 0) return DFLASH_OK;
+    copy_f32_kernel<<<(int)((n + 255) / 256), 256, 0, L.st>>>(src, dst, n);
+    DFLASH_CHECK_LAUNCH();
+    return DFLASH_OK;
+}
+
+}  // namespace dflash

@@ -1,0 +1,117 @@
+"""Host-side checks that need no GPU: the library builds, loads, exports every symbol the header
+declares, its structs have the layout the binding assumes, and host-detectable errors come back as
+return codes."""
+import ctypes as C
+import os
+import re
+import subprocess
+import tempfile
+
+import pytest
+
+from paper_2602_06036_b200 import binding, build, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "dflash.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def _declared():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dflash_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert set(binding.EXPORTS) <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_struct_layouts_match_the_header():
+    structs = {"dflash_config": binding.Config, "dflash_layer_weights": binding.LayerWeights,
+               "dflash_weights": binding.Weights, "dflash_ctx_args": binding.CtxArgs,
+               "dflash_draft_args": binding.DraftArgs, "dflash_verify_args": binding.VerifyArgs,
+               "dflash_attn_args": binding.AttnArgs, "dflash_lmhead_args": binding.LmHeadArgs}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "dflash.h"', "int main(void){"]
+    for cname, st in structs.items():
+        lines.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
+        for f, _ in st._fields_:
+            lines.append(f'printf("{cname}.{f} %zu\\n", offsetof({cname}, {f}));')
+    lines.append("return 0;}")
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "t.c")
+        open(src, "w").write("\n".join(lines))
+        exe = os.path.join(d, "t")
+        subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), src, "-o", exe])
+        out = subprocess.check_output([exe], text=True)
+    got = dict(line.split() for line in out.strip().splitlines())
+    for cname, st in structs.items():
+        assert int(got[cname]) == C.sizeof(st), cname
+        for f, _ in st._fields_:
+            assert int(got[f"{cname}.{f}"]) == getattr(st, f).offset, (cname, f)
+
+
+def _cfg(**over):
+    c = synth.TINY
+    vals = dict(n_layers=c.n_layers, d_model=c.d_model, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
+                head_dim=c.head_dim, d_ffn=c.d_ffn, vocab=c.vocab, n_feat_layers=c.n_feat_layers,
+                d_target=c.d_target, block_size=c.block_size, page_size=64, dtype=0, mask_token_id=c.vocab - 1,
+                use_rope=1, rms_eps=1e-6, softmax_scale=0.125)
+    vals.update(over)
+    return binding.Config(**vals)
+
+
+def test_create_validates_on_the_host(lib):
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_cfg()), C.byref(h)) == 0 and h.value
+    # workspace grows with rows; invalid arguments are refused
+    a = lib.dflash_workspace_bytes(h, 1, 8)
+    b = lib.dflash_workspace_bytes(h, 4, 64)
+    assert 0 < a < b and a % 256 == 0
+    assert lib.dflash_workspace_bytes(h, -1, 8) < 0
+    # calls before set_weights are refused without touching CUDA
+    args = binding.DraftArgs()
+    args.batch = 1
+    assert lib.dflash_draft_block(h, C.byref(args), None) == -5
+    assert lib.dflash_draft_block(None, C.byref(args), None) == -1
+    lib.dflash_destroy(h)
+    for bad in (dict(head_dim=48), dict(n_q_heads=3), dict(block_size=33), dict(dtype=2), dict(page_size=48),
+                dict(n_layers=0), dict(mask_token_id=5000), dict(softmax_scale=0.0)):
+        h2 = C.c_void_p()
+        assert lib.dflash_create(C.byref(_cfg(**bad)), C.byref(h2)) < 0 and not h2.value, bad
+    assert lib.dflash_create(None, C.byref(h)) == -1
+
+
+def test_verify_args_validated_on_the_host(lib):
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_cfg()), C.byref(h)) == 0
+    a = binding.VerifyArgs()
+    a.batch, a.gamma, a.draft_stride = 1, 0, 8
+    assert lib.dflash_verify_accept(h, C.byref(a), None) == -1      # gamma < 1
+    a.gamma, a.draft_stride = 8, 4
+    assert lib.dflash_verify_accept(h, C.byref(a), None) == -1      # stride < gamma
+    a.draft_stride = 8
+    assert lib.dflash_verify_accept(h, C.byref(a), None) == -1      # null pointers
+    a.batch = 0
+    assert lib.dflash_verify_accept(h, C.byref(a), None) == 0       # empty batch: nothing to do
+    lib.dflash_destroy(h)
+
+
+def test_status_strings(lib):
+    seen = {lib.dflash_status_string(c).decode() for c in (0, -1, -2, -3, -4, -5)}
+    assert len(seen) == 6 and lib.dflash_status_string(-99).decode() == "unknown status"
+    assert lib.dflash_launch_count() >= 0
+
+
+def test_binding_has_no_cpu_fallback():
+    # the product path must not be able to reach the oracle
+    for mod in ("binding.py", "build.py", "synth.py", "__init__.py"):
+        text = open(os.path.join(ROOT, "paper_2602_06036_b200", mod)).read()
+        assert "import oracle" not in text and "from oracle" not in text

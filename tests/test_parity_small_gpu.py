@@ -1,0 +1,169 @@
+"""Element-by-element parity of the CUDA path against the CPU oracle on the tiny fp32 configuration
+and on a reduced bf16 shape (several weight tiles, ragged vocabulary tail, ragged batch, empty
+context), through the C ABI."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dflash_oracle as orc
+from paper_2602_06036_b200 import synth
+from tests.harness import Case, assert_close, TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_pool(case):
+    cfg = case.cfg
+    got = case.pool.float().cpu().numpy()
+    for b, L in enumerate(case.ctx_lens):
+        for i in range(cfg.n_layers):
+            gk, gv = orc.pool_read(got, case.page_table_cpu[b].numpy(), L, i, cfg.page_size)
+            rk, rv = orc.pool_read(case.pool_np, case.page_table_cpu[b].numpy(), L, i, cfg.page_size)
+            if L:
+                assert_close(gk, rk, cfg.dtype, f"ctx K seq {b} layer {i}")
+                assert_close(gv, rv, cfg.dtype, f"ctx V seq {b} layer {i}")
+    # pages nobody owns stay untouched (zero)
+    owned = set(int(p) for p in case.page_table_cpu.reshape(-1).tolist() if p >= 0)
+    free = [p for p in range(case.n_pages) if p not in owned]
+    assert free and float(np.abs(got[:, free]).max()) == 0.0
+
+
+@pytest.mark.parametrize("name", ["cfg0", "mid"])
+def test_full_cycle_matches_oracle(name):
+    wl = synth.workload(name)
+    case = Case(wl.cfg, wl.ctx_lens, seed=wl.seed)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    n_sure = case.check_draft(got)
+    assert n_sure >= case.S * wl.cfg.block_size // 2       # the id check is not vacuous
+
+
+def test_tiny_without_rope_and_paper_block_sizes():
+    for B, use_rope in ((8, 0), (1, 1), (10, 1)):
+        cfg = dataclasses.replace(synth.TINY, block_size=B, use_rope=use_rope)
+        case = Case(cfg, (65,), seed=3)
+        case.project_prefill()
+        got = case.run_draft()
+        case.check_draft(got)
+
+
+def test_decode_step_appends_at_ctx_len():
+    # second projection call with n_new < max_new appends rows at positions L..L+n-1 only
+    cfg = synth.MID
+    case = Case(cfg, (60, 130), seed=5)
+    case.project_prefill()
+    max_new = 17
+    n_new = [3, 17]
+    feats = synth.make_features(cfg, 2 * max_new, 5, "decode.feats").reshape(2, max_new, cfg.feat_dim)
+    before = case.pool.clone()
+    case.lib.dflash_ctx_project(feats.to(case.device), torch.tensor(n_new, dtype=torch.int32, device=case.device),
+                                case.ctx_len, case.page_table, case.pool)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) == 0
+    for b in range(2):
+        L, n = case.ctx_lens[b], n_new[b]
+        K, V = orc.ctx_project(synth.to_numpy_f32(feats[b, :n]), np.arange(L, L + n), case.w_np, cfg)
+        orc.pool_write(case.pool_np, case.page_table_cpu[b].numpy(), list(range(L, L + n)), K, V, cfg.page_size)
+    case.ctx_lens = [case.ctx_lens[b] + n_new[b] for b in range(2)]
+    _check_pool(case)
+    # rows beyond n_new were not written: slot L+3 of sequence 0 is still what it was
+    p = 60 + 3
+    page = int(case.page_table_cpu[0, p // cfg.page_size])
+    assert torch.equal(case.pool[:, page, :, :, p % cfg.page_size], before[:, page, :, :, p % cfg.page_size])
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("mode", ["full", "causal"])
+def test_block_attention_building_block(dtype, mode):
+    from paper_2602_06036_b200 import binding
+    cfg = synth.TINY if dtype == "fp32" else synth.MID
+    lens = (0, 1, 63, 64, 65, 300)
+    case = Case(cfg, lens, seed=7)
+    case.fill_pool_synthetic()
+    R = 9 if mode == "causal" else cfg.block_size
+    S = len(lens)
+    q = synth.normal((S, R, cfg.n_q_heads, cfg.head_dim), 1.0, 7, "attn.q", cfg.torch_dtype)
+    k = synth.normal((S, R, cfg.n_kv_heads, cfg.head_dim), 1.0, 7, "attn.k", cfg.torch_dtype)
+    v = synth.normal((S, R, cfg.n_kv_heads, cfg.head_dim), 1.0, 7, "attn.v", cfg.torch_dtype)
+    out = torch.zeros_like(q, device=case.device)
+    layer = cfg.n_layers - 1
+    case.lib.dflash_block_attention(binding.ATTN_CAUSAL if mode == "causal" else binding.ATTN_FULL,
+                                    q.to(case.device), k.to(case.device), v.to(case.device), case.ctx_len,
+                                    max(lens), case.page_table, case.pool, layer, out)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) == 0
+    for b, L in enumerate(lens):
+        kc, vc = orc.pool_read(case.pool_np, case.page_table_cpu[b].numpy(), L, layer, cfg.page_size)
+        ref = orc.block_attention(synth.to_numpy_f32(q[b]), kc, vc, synth.to_numpy_f32(k[b]),
+                                  synth.to_numpy_f32(v[b]), cfg.softmax_scale, causal=(mode == "causal"))
+        assert_close(out[b].float().cpu().numpy(), ref, dtype, f"attention seq {b} L={L}")
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_lmhead_argmax_building_block(dtype):
+    cfg = synth.TINY if dtype == "fp32" else synth.MID
+    case = Case(cfg, (0,), seed=9)
+    M = 70                                   # more rows than one logits staging chunk
+    hid = synth.normal((M, cfg.d_model), 1.0, 9, "lm.hidden", cfg.torch_dtype)
+    dev = case.device
+    ids = torch.zeros(M, dtype=torch.int32, device=dev)
+    top1 = torch.zeros(M, dtype=torch.float32, device=dev)
+    margin = torch.zeros(M, dtype=torch.float32, device=dev)
+    logits = torch.zeros((M, cfg.vocab), dtype=torch.float32, device=dev)
+    for apply_norm in (0, 1):
+        case.lib.dflash_lmhead_argmax(hid.to(dev), apply_norm, ids, top1, margin, logits)
+        torch.cuda.synchronize()
+        x = synth.to_numpy_f32(hid)
+        z = orc.rmsnorm(x, case.w_np["g_f"], cfg.rms_eps) if apply_norm else x
+        ref = orc.linear(z, case.w_np["W_lm"])
+        rid, rtop, rmargin = orc.argmax_top2(ref)
+        assert_close(logits.cpu().numpy(), ref, dtype, "lm-head logits")
+        sure = rmargin > TOL[dtype]["margin"]
+        assert sure.sum() > M // 3
+        assert np.array_equal(ids.cpu().numpy()[sure], rid[sure])
+        assert np.max(np.abs(top1.cpu().numpy() - ref[np.arange(M), ids.cpu().numpy()])) <= TOL[dtype]["max_abs"]
+        # the fused argmax agrees exactly with an argmax over the logits the same kernel wrote
+        # wherever those logits have a unique maximum
+        lg = logits.cpu().numpy()
+        srt = np.sort(lg, axis=-1)
+        uniq = srt[:, -1] > srt[:, -2]
+        assert np.array_equal(ids.cpu().numpy()[uniq], np.argmax(lg, axis=-1)[uniq])
+
+
+def test_bad_token_and_bad_page_are_flagged_not_fatal():
+    from paper_2602_06036_b200 import binding
+    cfg = synth.TINY
+    case = Case(cfg, (70,), seed=11)
+    case.fill_pool_synthetic()
+    dev = case.device
+    ids = torch.zeros((1, cfg.block_size), dtype=torch.int32, device=dev)
+    case.lib.status.zero_()
+    case.lib.dflash_draft_block(torch.tensor([cfg.vocab + 5], dtype=torch.int32, device=dev), case.ctx_len, 70,
+                                case.page_table, case.pool, ids)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) & binding.DEV_BAD_TOKEN
+    bad_table = case.page_table.clone()
+    bad_table[0, 1] = case.n_pages + 100
+    case.lib.status.zero_()
+    case.lib.dflash_draft_block(torch.tensor([3], dtype=torch.int32, device=dev), case.ctx_len, 70, bad_table,
+                                case.pool, ids)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) & binding.DEV_BAD_PAGE
+    # the context stays usable
+    case.lib.status.zero_()
+    got = case.run_draft()
+    case.check_draft(got)
+
+
+def test_empty_batch_is_a_no_op():
+    cfg = synth.TINY
+    case = Case(cfg, (5,), seed=1)
+    dev = case.device
+    e = torch.zeros(0, dtype=torch.int32, device=dev)
+    n0 = __import__("paper_2602_06036_b200.binding", fromlist=["x"]).launch_count()
+    case.lib.dflash_draft_block(e, e, 0, case.page_table[:0].contiguous().reshape(0, case.page_table.shape[1]),
+                                case.pool, e.reshape(0, cfg.block_size))
+    assert __import__("paper_2602_06036_b200.binding", fromlist=["x"]).launch_count() == n0
