@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the DFlash hot path on B200: one step = context projection of the rows committed by
+the previous cycle + one single-pass draft block + greedy verify/accept, for one batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl reference]
+
+Prints ONE JSON line (rank 0). `value` = draft tokens/s with all inputs resident in HBM; `e2e` = the
+same metric through the C ABI with host buffers (H2D of the step's inputs and D2H of its results
+inside the timed region). `roofline` describes the dominant kernel (LM head + argmax) against the
+measured HBM peak; `kernels` lists every kernel family. `cpu_baseline` is the CPU oracle timed on
+this machine's host cores (a reported baseline, not the target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_06036_b200 import synth  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic bytes (what the method must move): weights once per block, KV once per sequence/layer
+# ------------------------------------------------------------------------------------------------
+def algorithmic_bytes(cfg, ctx_lens, n_new_rows):
+    es = 4 if cfg.dtype == "fp32" else 2
+    D, F, V = cfg.d_model, cfg.d_ffn, cfg.vocab
+    qkv = (cfg.q_dim + 2 * cfg.kv_dim) * D * es
+    o = D * cfg.q_dim * es
+    gateup = 2 * F * D * es
+    down = D * F * es
+    lm = V * D * es
+    kv_layer = 2 * cfg.kv_dim * es * sum(ctx_lens)
+    ctx = (D * cfg.feat_dim + cfg.n_layers * 2 * cfg.kv_dim * D) * es + \
+        n_new_rows * (cfg.feat_dim * es + cfg.n_layers * 2 * cfg.kv_dim * es)
+    return {
+        "gemm_qkv": qkv, "gemm_o": o, "gemm_gateup": gateup, "gemm_down": down, "lmhead_argmax": lm,
+        "attention": kv_layer, "ctx_fuse": D * cfg.feat_dim * es + n_new_rows * cfg.feat_dim * es,
+        "ctx_kv": 2 * cfg.kv_dim * D * es,
+        "draft_block_total": cfg.n_layers * (qkv + o + gateup + down + kv_layer) + lm,
+        "ctx_project_total": ctx,
+    }
+
+
+class ClockSampler:
+    """nvidia-smi polling during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx = float(f[2])
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the step
+# ------------------------------------------------------------------------------------------------
+class Step:
+    def __init__(self, wl, device, seed=0):
+        from paper_2602_06036_b200 import binding
+        cfg = wl.cfg
+        self.wl, self.cfg, self.dev = wl, cfg, device
+        B, S = cfg.block_size, wl.batch
+        self.gamma = B
+        self.lib = binding.DFlash(cfg, str(device))
+        w = synth.make_weights(cfg, seed)
+        cos, sin = synth.rope_tables(cfg, max(wl.ctx_lens) + 4 * B + 8)
+        self.lib.set_weights(synth.pack_device_weights(cfg, w), cos, sin)
+        del w
+        caps = [L + 2 * B + 2 for L in wl.ctx_lens]
+        table, n_pages = synth.make_page_table(cfg, caps, seed)
+        self.page_table = table.to(device)
+        self.n_pages = n_pages
+        self.ctx_len = torch.tensor(wl.ctx_lens, dtype=torch.int32, device=device)
+        # context K/V: produced by the library's own context projection from N(0,1) features
+        self.pool = torch.zeros(synth.kv_pool_shape(cfg, n_pages), dtype=cfg.torch_dtype, device=device)
+        zero = torch.zeros(S, dtype=torch.int32, device=device)
+        chunk = 4096
+        for b, L in enumerate(wl.ctx_lens):
+            for p0 in range(0, L, chunk):
+                n = min(chunk, L - p0)
+                f = synth.make_features(cfg, n, seed, f"feats.seq{b}.{p0}").to(device).reshape(1, n, cfg.feat_dim)
+                self.lib.dflash_ctx_project(f, None, torch.tensor([p0], dtype=torch.int32, device=device),
+                                            self.page_table[b:b + 1].contiguous(), self.pool)
+        torch.cuda.synchronize()
+        # per-step inputs (host masters, pinned; device copies for the resident run)
+        g = self.gamma
+        self.h_feats = synth.make_features(cfg, S * (g + 1), seed, "step.feats").reshape(S, g + 1, cfg.feat_dim).pin_memory()
+        self.h_anchor = synth.make_anchors(cfg, S, seed).pin_memory()
+        logits, drafts, planted = synth.make_verify_case(S, g, cfg.vocab, wl.accept_p, seed, cfg.torch_dtype)
+        self.h_logits = logits.pin_memory()
+        self.planted = planted
+        self.d_feats = self.h_feats.to(device)
+        self.d_anchor = self.h_anchor.to(device)
+        self.d_logits = self.h_logits.to(device)
+        self.e_feats = torch.empty_like(self.d_feats)
+        self.e_anchor = torch.empty_like(self.d_anchor)
+        self.e_logits = torch.empty_like(self.d_logits)
+        self.n_new = (planted + 1).to(torch.int32).to(device)      # rows committed by the previous cycle
+        self.draft_ids = torch.zeros((S, B), dtype=torch.int32, device=device)
+        self.tau = torch.zeros(S, dtype=torch.int32, device=device)
+        self.out_tokens = torch.zeros((S, g + 1), dtype=torch.int32, device=device)
+        self.bonus = torch.zeros(S, dtype=torch.int32, device=device)
+        self.new_len = torch.zeros(S, dtype=torch.int32, device=device)
+        self.h_out = torch.zeros((S, B + g + 1 + 3), dtype=torch.int32).pin_memory()
+        self.d_out = torch.zeros((S, B + g + 1 + 3), dtype=torch.int32, device=device)
+        self.max_ctx = max(wl.ctx_lens)
+        self.rows_new = int(self.n_new.sum().item())
+
+    def run(self, feats, anchor, logits):
+        lib = self.lib
+        lib.dflash_ctx_project(feats, self.n_new, self.ctx_len, self.page_table, self.pool)
+        lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids)
+        # The target's verify pass is outside this library; its logits are an input. The drafts
+        # verified are synthetic ones with a planted agreeing prefix (the random-init drafter would
+        # never be accepted), so the accept kernel sees realistic accept lengths.
+        lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
+                                 self.out_tokens, self.bonus, self.new_len, logits=logits)
+
+    def step_resident(self):
+        self.run(self.d_feats, self.d_anchor, self.d_logits)
+
+    def step_e2e(self):
+        self.e_feats.copy_(self.h_feats, non_blocking=True)
+        self.e_anchor.copy_(self.h_anchor, non_blocking=True)
+        self.e_logits.copy_(self.h_logits, non_blocking=True)
+        self.run(self.e_feats, self.e_anchor, self.e_logits)
+        B, g = self.cfg.block_size, self.gamma
+        self.d_out[:, :B] = self.draft_ids
+        self.d_out[:, B:B + g + 1] = self.out_tokens
+        self.d_out[:, B + g + 1] = self.tau
+        self.d_out[:, B + g + 2] = self.bonus
+        self.d_out[:, B + g + 3] = self.new_len
+        self.h_out.copy_(self.d_out, non_blocking=True)
+
+    def e2e_bytes(self):
+        h2d = self.h_feats.numel() * self.h_feats.element_size() + self.h_anchor.numel() * 4 + \
+            self.h_logits.numel() * self.h_logits.element_size()
+        return h2d, self.h_out.numel() * 4
+
+
+def timed(fn, steps, warmup, dist_on):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl, seed=0, layers=1, vocab_frac=8):
+    """A bounded sample of one step for the CPU oracle: the context projection of the step's rows,
+    `layers` of the N draft layers over the full context, and the LM head over V/vocab_frac rows.
+    Returns (seconds, fraction of the step's algorithmic bytes covered, threads)."""
+    from oracle import dflash_oracle as orc
+    import dataclasses
+    cfg = wl.cfg
+    sub = dataclasses.replace(cfg, n_layers=layers)
+    B = cfg.block_size
+    Vs = max(cfg.vocab // vocab_frac, 2)
+    rng_w = synth.make_weights(dataclasses.replace(sub, vocab=Vs), seed)
+    w = synth.weights_to_numpy(rng_w)
+    b = 0
+    L = wl.ctx_lens[b]
+    ctxK = [synth.to_numpy_f32(synth.normal((L, cfg.n_kv_heads, cfg.head_dim), 1.0, seed, f"o.K{i}", cfg.torch_dtype))
+            for i in range(layers)]
+    ctxV = [synth.to_numpy_f32(synth.normal((L, cfg.n_kv_heads, cfg.head_dim), 1.0, seed, f"o.V{i}", cfg.torch_dtype))
+            for i in range(layers)]
+    feats = synth.to_numpy_f32(synth.make_features(cfg, B + 1, seed, "o.feats"))
+    logits, drafts, _ = synth.make_verify_case(1, B, cfg.vocab, wl.accept_p, seed, cfg.torch_dtype)
+    lg = synth.to_numpy_f32(logits[0])
+    sub_v = dataclasses.replace(sub, vocab=Vs)
+    t0 = time.perf_counter()
+    orc.ctx_project(feats, L + np.arange(B + 1), w, sub_v)
+    orc.draft_block(3, L, ctxK, ctxV, w, sub_v)
+    orc.verify_accept_logits(drafts[0].numpy(), lg, L)
+    dt = time.perf_counter() - t0
+    full = algorithmic_bytes(cfg, [L], B + 1)
+    es = 2 if cfg.dtype == "bf16" else 4
+    per_layer = (full["draft_block_total"] - full["lmhead_argmax"]) / cfg.n_layers
+    covered = layers * per_layer + full["lmhead_argmax"] / cfg.vocab * Vs + \
+        (cfg.d_model * cfg.feat_dim + layers * 2 * cfg.kv_dim * cfg.d_model) * es
+    total = full["draft_block_total"] + full["ctx_project_total"]
+    return dt, covered / total, (os.cpu_count() or 1)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = synth.workload(args.workload)
+    cores = len(os.sched_getaffinity(0))
+    B = wl.cfg.block_size
+    times = []
+    frac = 1.0
+    for i in range(args.warmup + args.steps):
+        dt, frac, _ = oracle_sample(wl)
+        if i >= args.warmup:
+            times.append(dt)
+    per_step = statistics.mean(times) / frac            # extrapolated to the whole step, one sequence
+    value = B / per_step
+    sample = (f"per step: ctx projection of {B + 1} rows + 1 of {wl.cfg.n_layers} draft layers over the full "
+              f"context + LM head over V/8 + accept, one sequence; {frac:.3f} of the step's algorithmic bytes, "
+              f"time scaled by 1/{frac:.3f}")
+    line = {
+        "impl": "reference", "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": 1, "block_size": B, "ctx_len": wl.ctx_lens[0]},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    if dist_on:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+
+    from paper_2602_06036_b200 import binding, build
+    build.build()
+    wl = synth.workload(args.workload)
+    cfg = wl.cfg
+    peaks = load_peaks()
+    # replicas: every rank runs the same batch on its own GPU; there is no data-path collective
+    step = Step(wl, device, seed=0)
+    S, B = wl.batch, cfg.block_size
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    n0 = binding.launch_count()
+    ms = timed(step.step_resident, args.steps, args.warmup, dist_on)
+    launches = (binding.launch_count() - n0) // (args.steps + args.warmup) * args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    ms_e2e = timed(step.step_e2e, args.steps, args.warmup, dist_on)
+
+    # per-kernel-family durations: a second pass of the same steps with event pairs around each launch
+    prof = step.lib.profile(step.step_resident, args.steps) if hasattr(step.lib, "profile") else {}
+
+    if rank != 0:
+        if dist_on:
+            torch.distributed.destroy_process_group()
+        return
+
+    per_step_ms = ms / args.steps
+    tokens = S * B * world
+    value = tokens / (per_step_ms * 1e-3)
+    e2e_value = tokens / (ms_e2e / args.steps * 1e-3)
+    h2d, d2h = step.e2e_bytes()
+    alg = algorithmic_bytes(cfg, wl.ctx_lens, step.rows_new)
+    hbm = peaks["hbm_gbs"]
+    kernels = {}
+    for fam, (us, n) in prof.items():
+        entry = {"us_per_launch": us, "launches_per_step": n}
+        if fam in alg and us > 0:
+            entry["alg_bytes"] = alg[fam]
+            entry["gbs"] = alg[fam] / (us * 1e-6) / 1e9
+            entry["frac_hbm"] = entry["gbs"] / hbm
+        kernels[fam] = entry
+    dom = kernels.get("lmhead_argmax")
+    roofline = None
+    if dom and "gbs" in dom:
+        roofline = {"kernel": "lmhead_argmax", "bound": "hbm", "achieved": dom["gbs"], "peak": hbm, "unit": "GB/s",
+                    "frac": dom["frac_hbm"], "traffic": None, "peak_source": peaks["_source"],
+                    "timing": "event pairs around each launch, separate pass of the same steps"}
+    step_bytes = alg["draft_block_total"] + alg["ctx_project_total"] + S * (B + 1) * cfg.vocab * 2
+    line = {
+        "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": per_step_ms, "us_per_draft_block": per_step_ms * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "batch": S, "block_size": B, "ctx_lens": list(wl.ctx_lens)[:8],
+                   "step": "ctx_project(n_new=tau) + draft_block + verify_accept(logits)",
+                   "l2": "per-step weight traffic (3.2 GB) exceeds the 126 MB L2; no flush",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "step_roofline": {"alg_bytes": step_bytes, "us_at_peak": step_bytes / (hbm * 1e9) * 1e6,
+                          "frac": step_bytes / (hbm * 1e9) / (per_step_ms * 1e-3)},
+        "roofline": roofline, "kernels": kernels, "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / args.steps},
+    }
+    if not args.no_cpu_baseline:
+        dt, frac, _ = oracle_sample(wl)
+        cores = len(os.sched_getaffinity(0))
+        line["cpu_baseline"] = {
+            "value": B / (dt / frac), "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"one sequence: ctx projection of {B + 1} rows + 1 of {cfg.n_layers} draft layers + LM head over "
+                      f"V/8 + accept = {frac:.3f} of the step's algorithmic bytes in {dt:.1f} s, scaled to the full step"}
+    print(json.dumps(line))
+    if dist_on:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -226,6 +226,16 @@ typedef struct {
 } dflash_lmhead_args;
 int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a /*[host]*/, void* stream);
 
+/* ---- per-kernel-family timing (host-side CUDA events; off by default) ----
+ * While enabled, every launch the library issues is bracketed by an event pair on the caller's
+ * stream. dflash_profile_read synchronises on the last event, adds the elapsed milliseconds and the
+ * launch counts per family into the two host arrays (DFLASH_N_FAMILIES entries each) and clears
+ * the record. Event pairs cost a little time per launch: never time a step with profiling on. */
+#define DFLASH_N_FAMILIES 14
+int32_t dflash_profile_enable(dflash_handle* h, int32_t on);
+int32_t dflash_profile_read(dflash_handle* h, float* ms /*[host]*/, int32_t* launches /*[host]*/);
+const char* dflash_family_name(int32_t family);
+
 /* Static description of a return code. */
 const char* dflash_status_string(int32_t code);
 

@@ -25,8 +25,10 @@ DEV_BAD_TOKEN, DEV_BAD_PAGE, DEV_CTX_OVERFLOW, DEV_TIMEOUT = 1, 2, 4, 8
 EXPORTS = (
     "dflash_create", "dflash_destroy", "dflash_set_weights", "dflash_workspace_bytes",
     "dflash_ctx_project", "dflash_draft_block", "dflash_verify_accept", "dflash_block_attention",
-    "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count",
+    "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
+    "dflash_profile_read", "dflash_family_name",
 )
+N_FAMILIES = 14
 
 
 class Config(C.Structure):
@@ -112,6 +114,12 @@ def load():
     lib.dflash_status_string.restype = C.c_char_p
     lib.dflash_launch_count.argtypes = []
     lib.dflash_launch_count.restype = C.c_int64
+    lib.dflash_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+    lib.dflash_profile_enable.restype = C.c_int32
+    lib.dflash_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.dflash_profile_read.restype = C.c_int32
+    lib.dflash_family_name.argtypes = [C.c_int32]
+    lib.dflash_family_name.restype = C.c_char_p
     _lib = lib
     return lib
 
@@ -200,6 +208,24 @@ class DFlash:
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._ws
+
+    def profile(self, fn, steps: int):
+        """Run `fn` `steps` times with an event pair around every launch of this handle.
+        Returns {family: (microseconds per launch, launches per step)}."""
+        _check(self.lib.dflash_profile_enable(self.h, 1))
+        ms = (C.c_float * N_FAMILIES)()
+        n = (C.c_int32 * N_FAMILIES)()
+        try:
+            for _ in range(steps):
+                fn()
+                _check(self.lib.dflash_profile_read(self.h, ms, n))
+        finally:
+            self.lib.dflash_profile_enable(self.h, 0)
+        out = {}
+        for f in range(N_FAMILIES):
+            if n[f]:
+                out[self.lib.dflash_family_name(f).decode()] = (1e3 * ms[f] / n[f], n[f] / steps)
+        return out
 
     # ---- the path -----------------------------------------------------------------------
     def dflash_ctx_project(self, feats, n_new, ctx_len, page_table, kv_pool, stream=None):

@@ -1,5 +1,6 @@
 // C ABI of the library: argument validation, workspace carving and the launch sequence of each call.
 #include "dflash_internal.h"
+#include "gemm_tc.cuh"
 
 #include <algorithm>
 #include <cstring>
@@ -9,14 +10,19 @@ using namespace dflash;
 
 namespace dflash {
 
-Workspace carve(const dflash_config& c, void* base, int batch, int rows) {
+Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
+    const dflash_config& c = h->cfg;
     Arena a(base);
     Workspace w{};
     const int es = elem_size(c.dtype);
     const int64_t R = std::max(rows, 1);
     const int qdim = c.n_q_heads * c.head_dim, kdim = c.n_kv_heads * c.head_dim;
-    const int64_t wide = std::max<int64_t>(std::max<int64_t>(qdim + 2 * kdim, 2 * (int64_t)c.d_ffn),
-                                           (int64_t)c.d_model);
+    const int feat = c.n_feat_layers * c.d_target;
+    const bool tc = c.dtype == DFLASH_BF16;
+    // fp32 staging of a projection before its element-wise epilogue (fp32 path), or the fused
+    // context projection's un-normalised output (both paths)
+    const int64_t wide = tc ? (int64_t)c.d_model
+                            : std::max<int64_t>(std::max<int64_t>(qdim + 2 * kdim, 2 * (int64_t)c.d_ffn), c.d_model);
     w.x = (float*)a.take(R * c.d_model * 4);
     w.u = a.take(R * std::max(c.d_model, qdim) * es);
     w.tmp = (float*)a.take(R * wide * 4);
@@ -25,9 +31,24 @@ Workspace carve(const dflash_config& c, void* base, int batch, int rows) {
     w.v_blk = a.take(R * kdim * es);
     w.attn = a.take(R * qdim * es);
     w.h = a.take(R * c.d_ffn * es);
-    w.logits = (float*)a.take(std::min<int64_t>(R, LOGIT_ROWS) * c.vocab * 4);
+    w.logits = (float*)a.take(tc ? 256 : std::min<int64_t>(R, LOGIT_ROWS) * c.vocab * 4);
     w.ids = (int32_t*)a.take(R * 4);
-    w.part = (float*)a.take(256);
+    int64_t part = 0, counters = 256;
+    if (tc) {
+        const int M = (int)R, sm = h->sm_count;
+        const int shapes[7][2] = {{qdim + 2 * kdim, c.d_model}, {c.d_model, qdim}, {2 * c.d_ffn, c.d_model},
+                                  {c.d_model, c.d_ffn},         {c.d_model, feat}, {2 * kdim, c.d_model},
+                                  {c.vocab, c.d_model}};
+        for (auto& s : shapes) {
+            part = std::max(part, gemm_tc_part_bytes(M, s[0], s[1], sm));
+            counters = std::max(counters, gemm_tc_counter_bytes(M, s[0]));
+        }
+    }
+    w.part = (float*)a.take(std::max<int64_t>(part, 256));
+    w.counter_bytes = align_up(counters, 256);
+    w.counters = (int32_t*)a.take(w.counter_bytes);
+    w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
+    w.attn_part = (float*)a.take(256);
     (void)batch;
     w.bytes = a.off;
     return w;
@@ -36,6 +57,88 @@ Workspace carve(const dflash_config& c, void* base, int batch, int rows) {
 }  // namespace dflash
 
 static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+static const char* kFamilyNames[DFLASH_N_FAMILIES] = {
+    "embed", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gateup", "gemm_down", "lmhead_argmax",
+    "argmax_finish", "row_argmax", "accept", "ctx_fuse", "ctx_kv", "misc"};
+
+// ---- per-launch event pairs -------------------------------------------------------------------
+static void prof_begin(const Launch& L, int fam) {
+    dflash_handle* h = L.h;
+    if (!h->prof_on) return;
+    if (h->prof_used == h->prof_cap) {
+        const int cap = h->prof_cap ? h->prof_cap * 2 : 256;
+        dflash_profile_rec* n = new (std::nothrow) dflash_profile_rec[cap];
+        if (!n) { h->prof_on = false; return; }
+        for (int i = 0; i < h->prof_cap; ++i) n[i] = h->prof[i];
+        for (int i = h->prof_cap; i < cap; ++i) {
+            cudaEventCreate(&n[i].e0);
+            cudaEventCreate(&n[i].e1);
+        }
+        delete[] h->prof;
+        h->prof = n;
+        h->prof_cap = cap;
+    }
+    h->prof[h->prof_used].family = fam;
+    cudaEventRecord(h->prof[h->prof_used].e0, L.st);
+}
+static void prof_end(const Launch& L) {
+    dflash_handle* h = L.h;
+    if (!h->prof_on) return;
+    cudaEventRecord(h->prof[h->prof_used].e1, L.st);
+    ++h->prof_used;
+}
+
+#define DFLASH_TRY(expr)                    \
+    do {                                    \
+        int rc__ = (expr);                  \
+        if (rc__ != DFLASH_OK) return rc__; \
+    } while (0)
+
+#define RUN(fam, expr)              \
+    do {                            \
+        prof_begin(L, fam);         \
+        int rc2__ = (expr);         \
+        prof_end(L);                \
+        if (rc2__ != DFLASH_OK) return rc2__; \
+    } while (0)
+
+static int check_ws(const dflash_handle* h, void* ws, int64_t bytes, int batch, int rows, Workspace* out) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return DFLASH_ERR_WORKSPACE;
+    *out = carve(h, ws, batch, rows);
+    if (out->bytes > bytes) return DFLASH_ERR_WORKSPACE;
+    return DFLASH_OK;
+}
+
+static int zero_counters(const Launch& L, const Workspace& ws) {
+    if (L.h->cfg.dtype != DFLASH_BF16) return DFLASH_OK;
+    return cudaMemsetAsync(ws.counters, 0, ws.counter_bytes, L.st) == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+// LM head + argmax over `rows` normalised rows z (config dtype)
+static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, int rows, int32_t* ids, float* top1,
+                       float* margin, float* logits_out) {
+    const dflash_config& c = L.h->cfg;
+    if (c.dtype == DFLASH_BF16) {
+        GemmArgs g{};
+        g.X = z; g.W = L.h->w.W_lm; g.M = rows; g.N = c.vocab; g.K = c.d_model;
+        g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters;
+        g.top2 = (Top2Entry*)ws.top2; g.logits_out = logits_out;
+        RUN(FAM_LMHEAD, launch_gemm_tc(L, g));
+        RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, ids, top1, margin));
+        return DFLASH_OK;
+    }
+    const int es = elem_size(c.dtype);
+    for (int r0 = 0; r0 < rows; r0 += LOGIT_ROWS) {
+        const int n = std::min(LOGIT_ROWS, rows - r0);
+        float* lg = logits_out ? logits_out + (size_t)r0 * c.vocab : ws.logits;
+        RUN(FAM_LMHEAD, launch_gemm_simt(L, (const char*)z + (size_t)r0 * c.d_model * es, L.h->w.W_lm, lg, n, c.vocab,
+                                         c.d_model, false));
+        RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, lg, DFLASH_F32, c.vocab, n, c.vocab, ids + r0, top1 ? top1 + r0 : nullptr,
+                                              margin ? margin + r0 : nullptr));
+    }
+    return DFLASH_OK;
+}
 
 extern "C" {
 
@@ -50,6 +153,8 @@ const char* dflash_status_string(int32_t code) {
         default: return "unknown status";
     }
 }
+
+const char* dflash_family_name(int32_t f) { return (f >= 0 && f < DFLASH_N_FAMILIES) ? kFamilyNames[f] : "?"; }
 
 int64_t dflash_launch_count(void) { return (int64_t)g_launches; }
 
@@ -69,16 +174,49 @@ int32_t dflash_create(const dflash_config* cfg, dflash_handle** out) {
     if (c.block_size > 32) return DFLASH_ERR_UNSUPPORTED;
     if (!is_pow2(c.page_size) || c.page_size > 256) return DFLASH_ERR_UNSUPPORTED;
     if (c.d_model % 8 || c.d_ffn % 8 || (c.n_feat_layers * c.d_target) % 8) return DFLASH_ERR_UNSUPPORTED;
+    // the bf16 epilogues pair rows of whole heads inside a 128-row weight tile
+    if (c.dtype == DFLASH_BF16 && ((c.n_q_heads * c.head_dim) % 128 || (c.n_kv_heads * c.head_dim) % 128))
+        return DFLASH_ERR_UNSUPPORTED;
     dflash_handle* h = new (std::nothrow) dflash_handle();
     if (!h) return DFLASH_ERR_INVALID_ARG;
     h->cfg = c;
     h->has_weights = false;
     h->sm_count = 148;
+    h->prof_on = false;
+    h->prof = nullptr;
+    h->prof_cap = h->prof_used = 0;
     *out = h;
     return DFLASH_OK;
 }
 
-void dflash_destroy(dflash_handle* h) { delete h; }
+void dflash_destroy(dflash_handle* h) {
+    if (!h) return;
+    for (int i = 0; i < h->prof_cap; ++i) {
+        cudaEventDestroy(h->prof[i].e0);
+        cudaEventDestroy(h->prof[i].e1);
+    }
+    delete[] h->prof;
+    delete h;
+}
+
+int32_t dflash_profile_enable(dflash_handle* h, int32_t on) {
+    if (!h) return DFLASH_ERR_INVALID_ARG;
+    h->prof_on = on != 0;
+    return DFLASH_OK;
+}
+
+int32_t dflash_profile_read(dflash_handle* h, float* ms, int32_t* launches) {
+    if (!h || !ms || !launches) return DFLASH_ERR_INVALID_ARG;
+    if (h->prof_used > 0 && cudaEventSynchronize(h->prof[h->prof_used - 1].e1) != cudaSuccess) return DFLASH_ERR_CUDA;
+    for (int i = 0; i < h->prof_used; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, h->prof[i].e0, h->prof[i].e1) != cudaSuccess) return DFLASH_ERR_CUDA;
+        ms[h->prof[i].family] += t;
+        launches[h->prof[i].family] += 1;
+    }
+    h->prof_used = 0;
+    return DFLASH_OK;
+}
 
 int32_t dflash_set_weights(dflash_handle* h, const dflash_weights* w) {
     if (!h || !w || !w->layers) return DFLASH_ERR_INVALID_ARG;
@@ -97,21 +235,8 @@ int32_t dflash_set_weights(dflash_handle* h, const dflash_weights* w) {
 
 int64_t dflash_workspace_bytes(const dflash_handle* h, int32_t max_batch, int32_t max_rows) {
     if (!h || max_batch < 0 || max_rows < 0) return DFLASH_ERR_INVALID_ARG;
-    return carve(h->cfg, nullptr, max_batch, max_rows).bytes;
+    return carve(h, nullptr, max_batch, max_rows).bytes;
 }
-
-static int check_ws(const dflash_handle* h, void* ws, int64_t bytes, int batch, int rows, Workspace* out) {
-    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return DFLASH_ERR_WORKSPACE;
-    *out = carve(h->cfg, ws, batch, rows);
-    if (out->bytes > bytes) return DFLASH_ERR_WORKSPACE;
-    return DFLASH_OK;
-}
-
-#define DFLASH_TRY(expr)            \
-    do {                            \
-        int rc__ = (expr);          \
-        if (rc__ != DFLASH_OK) return rc__; \
-    } while (0)
 
 int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* stream) {
     if (!h || !a) return DFLASH_ERR_INVALID_ARG;
@@ -126,30 +251,31 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
     const dflash_config& c = h->cfg;
     Launch L{h, (cudaStream_t)stream, a->dev_status};
-    const int kdim = c.n_kv_heads * c.head_dim;
+    const int kdim = c.n_kv_heads * c.head_dim, feat = c.n_feat_layers * c.d_target;
+    const bool tc = c.dtype == DFLASH_BF16;
+    DFLASH_TRY(zero_counters(L, ws));
     // y = W_c [h^(l1); ...; h^(lk)]  ->  H_t = RMSNorm(y)
-    DFLASH_TRY(launch_gemm_simt(L, a->feats, h->w.W_c, ws.tmp, rows, c.d_model, c.n_feat_layers * c.d_target, false));
-    DFLASH_TRY(launch_rmsnorm(L, ws.tmp, true, h->w.g_c, true, ws.u, rows, c.d_model));
+    if (tc) {
+        GemmArgs g{};
+        g.X = a->feats; g.W = h->w.W_c; g.M = rows; g.N = c.d_model; g.K = feat;
+        g.epilogue = EPI_STORE_F32; g.out_f32 = ws.tmp; g.ld_out = c.d_model; g.part = ws.part; g.counters = ws.counters;
+        RUN(FAM_CTX_FUSE, launch_gemm_tc(L, g));
+    } else {
+        RUN(FAM_CTX_FUSE, launch_gemm_simt(L, a->feats, h->w.W_c, ws.tmp, rows, c.d_model, feat, false));
+    }
+    RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.tmp, true, h->w.g_c, true, ws.u, rows, c.d_model));
     for (int i = 0; i < c.n_layers; ++i) {
         // rows Hq*hd .. of W_qkv are W_i^K then W_i^V
         const char* Wkv = (const char*)h->layers[i].W_qkv + (size_t)c.n_q_heads * c.head_dim * c.d_model * elem_size(c.dtype);
-        DFLASH_TRY(launch_gemm_simt(L, ws.u, Wkv, ws.tmp, rows, 2 * kdim, c.d_model, false));
-        DFLASH_TRY(launch_ctx_scatter(L, ws.tmp, *a, i));
-    }
-    return DFLASH_OK;
-}
-
-static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, int rows, int32_t* ids, float* top1,
-                       float* margin, float* logits_out) {
-    const dflash_config& c = L.h->cfg;
-    const int es = elem_size(c.dtype);
-    for (int r0 = 0; r0 < rows; r0 += LOGIT_ROWS) {
-        const int n = std::min(LOGIT_ROWS, rows - r0);
-        float* lg = logits_out ? logits_out + (size_t)r0 * c.vocab : ws.logits;
-        DFLASH_TRY(launch_gemm_simt(L, (const char*)z + (size_t)r0 * c.d_model * es, L.h->w.W_lm, lg, n, c.vocab,
-                                    c.d_model, false));
-        DFLASH_TRY(launch_row_argmax(L, lg, DFLASH_F32, c.vocab, n, c.vocab, ids + r0, top1 ? top1 + r0 : nullptr,
-                                     margin ? margin + r0 : nullptr));
+        if (tc) {
+            GemmArgs g{};
+            g.X = ws.u; g.W = Wkv; g.M = rows; g.N = 2 * kdim; g.K = c.d_model;
+            g.epilogue = EPI_CTX_KV; g.ctx = a; g.layer = i; g.part = ws.part; g.counters = ws.counters;
+            RUN(FAM_CTX_KV, launch_gemm_tc(L, g));
+        } else {
+            RUN(FAM_CTX_KV, launch_gemm_simt(L, ws.u, Wkv, ws.tmp, rows, 2 * kdim, c.d_model, false));
+            RUN(FAM_CTX_KV, launch_ctx_scatter(L, ws.tmp, *a, i));
+        }
     }
     return DFLASH_OK;
 }
@@ -166,14 +292,26 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
     Launch L{h, (cudaStream_t)stream, a->dev_status};
-    const int qdim = c.n_q_heads * c.head_dim;
+    const int qdim = c.n_q_heads * c.head_dim, kdim = c.n_kv_heads * c.head_dim;
+    const bool tc = c.dtype == DFLASH_BF16;
+    DFLASH_TRY(zero_counters(L, ws));
 
-    DFLASH_TRY(launch_embed(L, a->anchor_ids, ws.x, a->batch));
+    RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, ws.x, a->batch));
     for (int i = 0; i < c.n_layers; ++i) {
         const dflash_layer_weights& lw = h->layers[i];
-        DFLASH_TRY(launch_rmsnorm(L, ws.x, true, lw.g1, true, ws.u, rows, c.d_model));
-        DFLASH_TRY(launch_gemm_simt(L, ws.u, lw.W_qkv, ws.tmp, rows, qdim + 2 * c.n_kv_heads * c.head_dim, c.d_model, false));
-        DFLASH_TRY(launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk));
+        // attention half: u = RMSNorm(x); q,k,v = W u (+RoPE); x += W_o attention(q, [K_ctx; k], [V_ctx; v])
+        RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g1, true, ws.u, rows, c.d_model));
+        if (tc) {
+            GemmArgs g{};
+            g.X = ws.u; g.W = lw.W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model;
+            g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
+            g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
+            g.part = ws.part; g.counters = ws.counters;
+            RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g));
+        } else {
+            RUN(FAM_GEMM_QKV, launch_gemm_simt(L, ws.u, lw.W_qkv, ws.tmp, rows, qdim + 2 * kdim, c.d_model, false));
+            RUN(FAM_GEMM_QKV, launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk));
+        }
         dflash_attn_args at{};
         at.mode = DFLASH_ATTN_FULL;
         at.q = ws.q; at.k_blk = ws.k_blk; at.v_blk = ws.v_blk;
@@ -182,17 +320,35 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
         at.page_table = a->page_table; at.max_pages = a->max_pages;
         at.kv_pool = a->kv_pool; at.n_pool_pages = a->n_pool_pages; at.layer = i;
         at.out = ws.attn;
-        DFLASH_TRY(launch_attention_simt(L, at));
-        DFLASH_TRY(launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));
-        DFLASH_TRY(launch_rmsnorm(L, ws.x, true, lw.g2, true, ws.u, rows, c.d_model));
-        DFLASH_TRY(launch_gemm_simt(L, ws.u, lw.W_gateup, ws.tmp, rows, 2 * c.d_ffn, c.d_model, false));
-        DFLASH_TRY(launch_swiglu(L, ws.tmp, ws.h, rows));
-        DFLASH_TRY(launch_gemm_simt(L, ws.h, lw.W_down, ws.x, rows, c.d_model, c.d_ffn, true));
+        RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+        if (tc) {
+            GemmArgs g{};
+            g.X = ws.attn; g.W = lw.W_o; g.M = rows; g.N = c.d_model; g.K = qdim;
+            g.epilogue = EPI_RESIDUAL; g.out_f32 = ws.x; g.ld_out = c.d_model; g.part = ws.part; g.counters = ws.counters;
+            RUN(FAM_GEMM_O, launch_gemm_tc(L, g));
+        } else {
+            RUN(FAM_GEMM_O, launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));
+        }
+        // FFN half: u = RMSNorm(x); x += W_down (silu(W_gate u) * W_up u)
+        RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g2, true, ws.u, rows, c.d_model));
+        if (tc) {
+            GemmArgs g{};
+            g.X = ws.u; g.W = lw.W_gateup; g.M = rows; g.N = 2 * c.d_ffn; g.K = c.d_model;
+            g.epilogue = EPI_SWIGLU; g.h = (__nv_bfloat16*)ws.h; g.part = ws.part; g.counters = ws.counters;
+            RUN(FAM_GEMM_GATEUP, launch_gemm_tc(L, g));
+            GemmArgs d{};
+            d.X = ws.h; d.W = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
+            d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part; d.counters = ws.counters;
+            RUN(FAM_GEMM_DOWN, launch_gemm_tc(L, d));
+        } else {
+            RUN(FAM_GEMM_GATEUP, launch_gemm_simt(L, ws.u, lw.W_gateup, ws.tmp, rows, 2 * c.d_ffn, c.d_model, false));
+            RUN(FAM_GEMM_GATEUP, launch_swiglu(L, ws.tmp, ws.h, rows));
+            RUN(FAM_GEMM_DOWN, launch_gemm_simt(L, ws.h, lw.W_down, ws.x, rows, c.d_model, c.d_ffn, true));
+        }
     }
-    if (a->hidden_out) DFLASH_TRY(launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
-    DFLASH_TRY(launch_rmsnorm(L, ws.x, true, h->w.g_f, true, ws.u, rows, c.d_model));
-    DFLASH_TRY(lmhead_rows(L, ws, ws.u, rows, a->draft_ids, a->top1, a->margin, a->logits_out));
-    return DFLASH_OK;
+    if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
+    RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, h->w.g_f, true, ws.u, rows, c.d_model));
+    return lmhead_rows(L, ws, ws.u, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
 }
 
 int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void* stream) {
@@ -205,7 +361,8 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
     const int rows = a->batch * (a->gamma + 1);
     if (a->mode == DFLASH_VERIFY_IDS) {
         if (!a->target_ids) return DFLASH_ERR_INVALID_ARG;
-        return launch_accept(L, *a, a->target_ids);
+        RUN(FAM_ACCEPT, launch_accept(L, *a, a->target_ids));
+        return DFLASH_OK;
     }
     if (a->mode != DFLASH_VERIFY_LOGITS) return DFLASH_ERR_INVALID_ARG;
     if (!a->logits || a->vocab < 2) return DFLASH_ERR_INVALID_ARG;
@@ -218,8 +375,9 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
         DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
         ids = ws.ids;
     }
-    DFLASH_TRY(launch_row_argmax(L, a->logits, a->logits_dtype, stride, rows, a->vocab, ids, nullptr, nullptr));
-    return launch_accept(L, *a, ids);
+    RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, a->logits, a->logits_dtype, stride, rows, a->vocab, ids, nullptr, nullptr));
+    RUN(FAM_ACCEPT, launch_accept(L, *a, ids));
+    return DFLASH_OK;
 }
 
 int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void* stream) {
@@ -232,7 +390,8 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     if (!a->q || !a->k_blk || !a->v_blk || !a->ctx_len || !a->page_table || !a->kv_pool || !a->out)
         return DFLASH_ERR_INVALID_ARG;
     Launch L{h, (cudaStream_t)stream, a->dev_status};
-    return launch_attention_simt(L, *a);
+    RUN(FAM_ATTENTION, launch_attention_simt(L, *a));
+    return DFLASH_OK;
 }
 
 int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a, void* stream) {
@@ -247,7 +406,8 @@ int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a, void
     Launch L{h, (cudaStream_t)stream, a->dev_status};
     const dflash_config& c = h->cfg;
     const bool f32in = a->hidden_is_f32 || c.dtype == DFLASH_F32;
-    DFLASH_TRY(launch_rmsnorm(L, a->hidden, f32in, h->w.g_f, a->apply_norm != 0, ws.u, a->n_rows, c.d_model));
+    DFLASH_TRY(zero_counters(L, ws));
+    RUN(FAM_RMSNORM, launch_rmsnorm(L, a->hidden, f32in, h->w.g_f, a->apply_norm != 0, ws.u, a->n_rows, c.d_model));
     return lmhead_rows(L, ws, ws.u, a->n_rows, a->ids, a->top1, a->margin, a->logits_out);
 }
 

@@ -9,12 +9,27 @@
 
 #define DFLASH_MAX_LAYERS 64
 
+enum DflashFamily : int {
+    FAM_EMBED = 0, FAM_RMSNORM, FAM_GEMM_QKV, FAM_ATTENTION, FAM_GEMM_O, FAM_GEMM_GATEUP, FAM_GEMM_DOWN,
+    FAM_LMHEAD, FAM_ARGMAX_FINISH, FAM_ROW_ARGMAX, FAM_ACCEPT, FAM_CTX_FUSE, FAM_CTX_KV, FAM_MISC,
+};
+static_assert(FAM_MISC + 1 == DFLASH_N_FAMILIES, "family table out of step with the header");
+
+struct dflash_profile_rec {
+    cudaEvent_t e0, e1;
+    int family;
+};
+
 struct dflash_handle {
     dflash_config cfg;
     dflash_layer_weights layers[DFLASH_MAX_LAYERS];
     dflash_weights w;
     bool has_weights;
     int sm_count;
+    // optional per-launch event pairs
+    bool prof_on;
+    dflash_profile_rec* prof;
+    int prof_cap, prof_used;
 };
 
 namespace dflash {
@@ -49,15 +64,19 @@ struct Workspace {
     void*  h;        // [rows, F]
     float* logits;   // [min(rows, LOGIT_ROWS), V] fp32 (only the fp32 path stages logits)
     int32_t* ids;    // [rows]
-    float* part;     // attention split-KV partials
+    float* part;     // split-K partial sums of the tensor-core contractions
+    int32_t* counters;   // split-K tickets (zeroed at the start of each call)
+    int64_t counter_bytes;
+    void* top2;      // [vocab tiles, rows] per-tile winners of the fused LM-head argmax
+    float* attn_part;    // attention split-KV partials
     int64_t bytes;
 };
-Workspace carve(const dflash_config& c, void* base, int batch, int rows);
+Workspace carve(const dflash_handle* h, void* base, int batch, int rows);
 
 constexpr int LOGIT_ROWS = 64;
 
 struct Launch {
-    const dflash_handle* h;
+    dflash_handle* h;
     cudaStream_t st;
     int32_t* status;
 };
