@@ -1,6 +1,7 @@
 // C ABI of the library: argument validation, workspace carving and the launch sequence of each call.
 #include "dflash_internal.h"
 #include "gemm_tc.cuh"
+#include "attn_tc.cuh"
 
 #include <algorithm>
 #include <cstring>
@@ -45,11 +46,14 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
         }
     }
     w.part = (float*)a.take(std::max<int64_t>(part, 256));
-    w.counter_bytes = align_up(counters, 256);
+    // tickets of the contractions, then tickets of the attention splits: one memset clears both
+    const int64_t gemm_counters = align_up(counters, 256);
+    const int64_t attn_counters = tc ? align_up(attn_tc_counter_bytes(c, std::max(batch, 1)), 256) : 0;
+    w.counter_bytes = gemm_counters + attn_counters;
     w.counters = (int32_t*)a.take(w.counter_bytes);
+    w.attn_counters = w.counters ? (int32_t*)((char*)w.counters + gemm_counters) : nullptr;
     w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
-    w.attn_part = (float*)a.take(256);
-    (void)batch;
+    w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), h->sm_count) : 256);
     w.bytes = a.off;
     return w;
 }
@@ -320,7 +324,8 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
         at.page_table = a->page_table; at.max_pages = a->max_pages;
         at.kv_pool = a->kv_pool; at.n_pool_pages = a->n_pool_pages; at.layer = i;
         at.out = ws.attn;
-        RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+        if (tc && attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
+        else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
         if (tc) {
             GemmArgs g{};
             g.X = ws.attn; g.W = lw.W_o; g.M = rows; g.N = c.d_model; g.K = qdim;
@@ -390,7 +395,14 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     if (!a->q || !a->k_blk || !a->v_blk || !a->ctx_len || !a->page_table || !a->kv_pool || !a->out)
         return DFLASH_ERR_INVALID_ARG;
     Launch L{h, (cudaStream_t)stream, a->dev_status};
-    RUN(FAM_ATTENTION, launch_attention_simt(L, *a));
+    if (attn_tc_supported(h->cfg, a->rows)) {
+        Workspace ws;
+        DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, a->batch * a->rows, &ws));
+        DFLASH_TRY(zero_counters(L, ws));
+        RUN(FAM_ATTENTION, launch_attention_tc(L, *a, ws.attn_part, ws.attn_counters));
+    } else {
+        RUN(FAM_ATTENTION, launch_attention_simt(L, *a));
+    }
     return DFLASH_OK;
 }
 

@@ -1,0 +1,460 @@
+// Block attention on tcgen05 tensor cores (bf16, head_dim 128, 64-token pages):
+//   every block row of a sequence attends over [paged context K/V ; the block's own K/V].
+// One CTA works on one (sequence, kv head, range of KV tiles). The queries of all block rows and of
+// the q heads that share the kv head (rows x group <= 128) are the 128-row "M" operand; a KV tile
+// is one 64-token page (or the block's own rows). Per tile:
+//   S = Q K^T           tcgen05.mma, S in TMEM (two buffers, so the next tile's S is computed while
+//                       this one is in the softmax)
+//   softmax             one thread per query row reads its S row from TMEM (no cross-thread
+//                       reduction), running max / sum in the log2 domain, P -> shared memory (bf16)
+//   O_tile = P V        tcgen05.mma with V as an MN-major operand straight from the page layout
+//   acc = acc*alpha + O_tile   in registers, one row per thread
+// K/V tiles stream through a TMA ring that runs ahead of the math. Long contexts are split across
+// CTAs; partial (max, sum, acc) are merged in split order by the last CTA to arrive at a ticket
+// counter (no waiting, bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block
+// row r sees block rows <= r. Every mbarrier wait is bounded.
+#include "attn_tc.cuh"
+
+#include "ptx_sm100.cuh"
+
+#include <math_constants.h>
+
+#include <algorithm>
+
+namespace dflash {
+namespace {
+
+using namespace ptx;
+
+constexpr int HD = 128;          // head_dim
+constexpr int PG = 64;           // tokens per page = keys per tile
+constexpr int NS = 5;            // K/V ring depth
+constexpr int Q_BYTES = 128 * HD * 2;          // 32 KiB: two 64-wide halves of 128 rows
+constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
+constexpr int P_BYTES = 128 * PG * 2;          // 16 KiB
+constexpr int PART_LD = HD + 2;                // acc[128], running max, running sum
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + P_BYTES + 512;
+constexpr uint32_t TMEM_COLS = 256;            // S0 | S1 (64 each) | O (128)
+constexpr int N_THREADS = 192;
+
+struct AParams {
+    int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks;
+    float scale_log2;
+    const int32_t* ctx_len;
+    const int32_t* page_table;
+    __nv_bfloat16* out;
+    float* part;
+    int32_t* counters;
+    int32_t* status;
+};
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// MN-major operand (V: [key][head_dim], head_dim contiguous) in two 64-column halves of 64 rows x
+// 128 bytes, 128-byte swizzle: leading byte offset = distance between the halves (8 KiB), stride
+// byte offset = distance between 8-key groups (1 KiB).
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// D fp32, A bf16 K-major, B bf16 MN-major
+__host__ __device__ constexpr uint32_t instr_desc_bf16_bmn(int m, int n) {
+    return instr_desc_bf16(m, n) | (1u << 16);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+__global__ void __launch_bounds__(N_THREADS, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPool,
+               const __grid_constant__ CUtensorMap tmKb, const __grid_constant__ CUtensorMap tmVb, const AParams p) {
+    // ---- which work unit ----
+    const int chunk = blockIdx.x % p.n_chunks;
+    const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
+    const int b = blockIdx.x / (p.n_chunks * p.Hkv);
+    const int L = max(p.ctx_len[b], 0);
+    const int n_ctx_tiles = (L + PG - 1) / PG;
+    const int T = n_ctx_tiles + 1;                       // + the block's own rows
+    const int t_lo = chunk * p.tiles_per_unit;
+    if (t_lo >= T) return;                               // whole CTA leaves before touching any barrier
+    const int t_hi = min(t_lo + p.tiles_per_unit, T);
+    const int n_tiles = t_hi - t_lo;
+    const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;
+    uint8_t* sKV = sQ + Q_BYTES;
+    uint8_t* sP = sKV + NS * KV_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
+    uint64_t* q_full = bars;
+    uint64_t* kv_full = bars + 1;
+    uint64_t* kv_empty = kv_full + NS;
+    uint64_t* s_full = kv_empty + NS;
+    uint64_t* s_empty = s_full + 2;
+    uint64_t* p_full = s_empty + 2;
+    uint64_t* p_empty = p_full + 1;
+    uint64_t* o_full = p_empty + 1;
+    uint64_t* o_empty = o_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
+    volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] last arriver
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 4); }
+        mbar_init(p_full, 4); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 4);
+        flags[0] = 0; flags[1] = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            const uint64_t pol_kv = policy_evict_first(), pol_q = policy_evict_last();
+            mbar_expect_tx(q_full, Q_BYTES);
+            // q viewed as [S*R][Hkv][group][hd]: box = 64 x group x 1 x (128/group) -> rows ordered (r, j)
+            tma_load_4d(sQ, &tmQ, 0, 0, g, b * p.R, q_full, pol_q);
+            tma_load_4d(sQ + Q_BYTES / 2, &tmQ, 64, 0, g, b * p.R, q_full, pol_q);
+            bool ok = true;
+            for (int i = 0; i < n_tiles; ++i) {
+                const int st = i % NS;
+                const uint32_t ph = (i / NS) & 1;
+                if (!mbar_wait(&kv_empty[st], ph ^ 1, &flags[0])) { ok = false; break; }
+                uint8_t* dK = sKV + (size_t)st * KV_STAGE_BYTES;
+                uint8_t* dV = dK + KV_STAGE_BYTES / 2;
+                mbar_expect_tx(&kv_full[st], KV_STAGE_BYTES);
+                const int t = t_lo + i;
+                if (t < n_ctx_tiles) {
+                    int page = t < p.max_pages ? p.page_table[(size_t)b * p.max_pages + t] : -1;
+                    if (page < 0 || page >= p.n_pages) {
+                        if (p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
+                        page = 0;      // loaded but fully masked by the softmax warps
+                    }
+                    // pool rows: ((((layer*n_pages + page)*2 + kv)*Hkv + head)*PG + slot), hd contiguous
+                    const int rowK = ((((p.layer * p.n_pages + page) * 2 + 0) * p.Hkv + g) * PG);
+                    const int rowV = rowK + p.Hkv * PG;
+                    tma_load_2d(dK, &tmPool, 0, rowK, &kv_full[st], pol_kv);
+                    tma_load_2d(dK + 8192, &tmPool, 64, rowK, &kv_full[st], pol_kv);
+                    tma_load_2d(dV, &tmPool, 0, rowV, &kv_full[st], pol_kv);
+                    tma_load_2d(dV + 8192, &tmPool, 64, rowV, &kv_full[st], pol_kv);
+                } else {
+                    // the block's own k/v: [S*R][Hkv*hd]; rows past this sequence are masked
+                    tma_load_2d(dK, &tmKb, g * HD, b * p.R, &kv_full[st], pol_q);
+                    tma_load_2d(dK + 8192, &tmKb, g * HD + 64, b * p.R, &kv_full[st], pol_q);
+                    tma_load_2d(dV, &tmVb, g * HD, b * p.R, &kv_full[st], pol_q);
+                    tma_load_2d(dV + 8192, &tmVb, g * HD + 64, b * p.R, &kv_full[st], pol_q);
+                }
+            }
+            if (!ok) {
+                flags[0] = 1;
+                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc_bf16(128, PG);
+            constexpr uint32_t idesc_o = instr_desc_bf16_bmn(128, HD);
+            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+            bool ok = mbar_wait(q_full, 0, &flags[0]);
+            auto issue_s = [&](int i) -> bool {
+                const int st = i % NS;
+                const uint32_t sb = i & 1;
+                if (!mbar_wait(&kv_full[st], (i / NS) & 1, &flags[0])) return false;
+                if (!mbar_wait(&s_empty[sb], ((i >> 1) & 1) ^ 1, &flags[0])) return false;
+                tc_fence_after();
+                const uint32_t k_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_bf16(tmem_S + sb * PG, smem_desc_sw128(q_addr + (kk >> 2) * (Q_BYTES / 2) + (kk & 3) * 32),
+                             smem_desc_sw128(k_addr + (kk >> 2) * 8192 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
+                mma_commit(&s_full[sb]);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                if (i + 1 < n_tiles) { ok = issue_s(i + 1); if (!ok) break; }
+                const int st = i % NS;
+                if (!mbar_wait(p_full, i & 1, &flags[0])) { ok = false; break; }
+                if (!mbar_wait(o_empty, (i & 1) ^ 1, &flags[0])) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t v_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES + KV_STAGE_BYTES / 2);
+#pragma unroll
+                for (int kk = 0; kk < PG / 16; ++kk)
+                    mma_bf16(tmem_O, smem_desc_sw128(p_addr + kk * 32), smem_desc_sw128_mn(v_addr + kk * 2048), idesc_o,
+                             kk > 0 ? 1u : 0u);
+                mma_commit(o_full);
+                mma_commit(p_empty);
+                mma_commit(&kv_empty[st]);
+            }
+            if (!ok) {
+                flags[0] = 1;
+                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+            }
+        }
+    } else {
+        // ---------------- softmax + accumulation: thread = query row ----------------
+        const int ew = warp & 3;
+        const int row = ew * 32 + lane;                    // TMEM lane
+        const int r = row / p.group, j = row % p.group;    // block row, q head inside the group
+        const uint32_t lane_sel = (uint32_t)(ew * 32) << 16;
+        float acc[HD];
+#pragma unroll
+        for (int d = 0; d < HD; ++d) acc[d] = 0.f;
+        float m_run = -CUDART_INF_F, l_run = 0.f;
+        bool ok = true;
+        for (int i = 0; i < n_tiles; ++i) {
+            const int t = t_lo + i;
+            const uint32_t sb = i & 1;
+            const int st = i % NS;
+            // how many keys of this tile exist, and from which one on they are hidden from this row
+            int n_valid, n_vis;
+            if (t < n_ctx_tiles) {
+                n_valid = min(PG, L - t * PG);
+                const int page = t < p.max_pages ? p.page_table[(size_t)b * p.max_pages + t] : -1;
+                if (page < 0 || page >= p.n_pages) n_valid = 0;
+                n_vis = n_valid;
+            } else {
+                n_valid = p.R;
+                n_vis = p.causal ? min(r + 1, p.R) : p.R;
+            }
+            if (!mbar_wait(&s_full[sb], (i >> 1) & 1, &flags[0])) { ok = false; break; }
+            tc_fence_after();
+            float s[PG];
+            tmem_ld32(tmem_S + sb * PG + lane_sel, s);
+            tmem_ld32(tmem_S + sb * PG + 32 + lane_sel, s + 32);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[sb]);
+            float mx = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < PG; ++c) {
+                s[c] = (c < n_vis) ? s[c] * p.scale_log2 : -CUDART_INF_F;
+                mx = fmaxf(mx, s[c]);
+            }
+            const float m_new = fmaxf(m_run, mx);
+            float alpha = 1.f, psum = 0.f;
+            if (m_new > -CUDART_INF_F) {
+                alpha = exp2f(m_run - m_new);
+#pragma unroll
+                for (int c = 0; c < PG; ++c) { s[c] = exp2f(s[c] - m_new); psum += s[c]; }
+            } else {
+#pragma unroll
+                for (int c = 0; c < PG; ++c) s[c] = 0.f;
+            }
+            l_run = l_run * alpha + psum;
+            m_run = m_new;
+            // P (bf16) into its swizzled K-major tile once the previous P.V has finished reading it
+            if (!mbar_wait(p_empty, (i & 1) ^ 1, &flags[0])) { ok = false; break; }
+            uint8_t* prow = sP + row * 128;
+#pragma unroll
+            for (int ck = 0; ck < 8; ++ck) {
+                uint4 w;
+                w.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
+                w.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
+                w.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
+                w.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
+                *reinterpret_cast<uint4*>(prow + ((ck ^ (row & 7)) << 4)) = w;
+            }
+            // keys that do not exist must not poison P.V with whatever the page holds there
+            if (n_valid < PG) {
+                uint8_t* dV = sKV + (size_t)st * KV_STAGE_BYTES + KV_STAGE_BYTES / 2;
+                const int n_bad = PG - n_valid;                  // rows n_valid..63, two halves, 8 chunks each
+                for (int e = row; e < n_bad * 16; e += 128) {
+                    const int kr = n_valid + e / 16, part = e % 16;
+                    *reinterpret_cast<uint4*>(dV + (part >> 3) * 8192 + kr * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+            // O_tile -> running accumulator
+            if (!mbar_wait(o_full, i & 1, &flags[0])) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int c4 = 0; c4 < HD / 32; ++c4) {
+                float o[32];
+                tmem_ld32(tmem_O + c4 * 32 + lane_sel, o);
+#pragma unroll
+                for (int d = 0; d < 32; ++d) acc[c4 * 32 + d] = acc[c4 * 32 + d] * alpha + o[d];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_empty);
+        }
+        if (!ok) {
+            flags[0] = 1;
+            if (lane == 0 && p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+        }
+        epi_bar();
+        if (!flags[0]) {
+            const bool row_valid = r < p.R;
+            __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD;
+            if (n_splits == 1) {
+                if (row_valid) {
+                    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+#pragma unroll
+                    for (int d = 0; d < HD; d += 8) {
+                        uint4 w;
+                        w.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
+                        w.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
+                        w.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
+                        w.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + d) = w;
+                    }
+                }
+            } else {
+                const int bg = b * p.Hkv + g;
+                float* mine = p.part + (((size_t)bg * p.n_chunks + chunk) * 128 + row) * PART_LD;
+                if (row_valid) {
+#pragma unroll
+                    for (int d = 0; d < HD; d += 2) *reinterpret_cast<float2*>(mine + d) = make_float2(acc[d], acc[d + 1]);
+                    *reinterpret_cast<float2*>(mine + HD) = make_float2(m_run, l_run);
+                }
+                __threadfence();
+                epi_bar();
+                if (row == 0) {
+                    const int old = atomicAdd(p.counters + bg, 1);
+                    flags[1] = (old == n_splits - 1) ? 1 : 0;
+                    if (old == n_splits - 1) p.counters[bg] = 0;
+                }
+                epi_bar();
+                if (flags[1] && row_valid) {
+                    __threadfence();
+                    float M = -CUDART_INF_F;
+                    for (int s2 = 0; s2 < n_splits; ++s2)
+                        M = fmaxf(M, __ldcg(p.part + (((size_t)bg * p.n_chunks + s2) * 128 + row) * PART_LD + HD));
+                    float Lsum = 0.f;
+#pragma unroll
+                    for (int d = 0; d < HD; ++d) acc[d] = 0.f;
+                    for (int s2 = 0; s2 < n_splits; ++s2) {
+                        const float* src = p.part + (((size_t)bg * p.n_chunks + s2) * 128 + row) * PART_LD;
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + HD));
+                        const float w = (ml.x > -CUDART_INF_F) ? exp2f(ml.x - M) : 0.f;
+                        Lsum += ml.y * w;
+#pragma unroll
+                        for (int d = 0; d < HD; d += 2) {
+                            const float2 a = __ldcg(reinterpret_cast<const float2*>(src + d));
+                            acc[d] += a.x * w;
+                            acc[d + 1] += a.y * w;
+                        }
+                    }
+                    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+#pragma unroll
+                    for (int d = 0; d < HD; d += 8) {
+                        uint4 w;
+                        w.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
+                        w.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
+                        w.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
+                        w.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + d) = w;
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+bool attn_tc_supported(const dflash_config& c, int rows) {
+    if (c.dtype != DFLASH_BF16 || c.head_dim != HD || c.page_size != PG) return false;
+    const int group = c.n_q_heads / c.n_kv_heads;
+    return group >= 1 && 128 % group == 0 && rows * group <= 128 && rows <= PG;
+}
+
+static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
+    const int64_t Tmax = (max_ctx_len + PG - 1) / PG + 1;
+    const int64_t c = ((int64_t)batch * Hkv * Tmax + 2 * sm_count - 1) / (2 * sm_count);
+    return (int)std::max<int64_t>(2, c);
+}
+
+int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int sm_count) {
+    // units never exceed 2*SMs + 2*batch*Hkv (see tiles_per_unit)
+    const int64_t units = 2 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
+    return units * 128 * PART_LD * 4;
+}
+int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
+
+int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters) {
+    const dflash_config& c = L.h->cfg;
+    if (a.batch == 0 || a.rows == 0) return DFLASH_OK;
+    AParams p{};
+    p.S = a.batch; p.R = a.rows; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.group = c.n_q_heads / c.n_kv_heads;
+    p.max_pages = a.max_pages; p.n_pages = a.n_pool_pages; p.layer = a.layer;
+    p.causal = a.mode == DFLASH_ATTN_CAUSAL ? 1 : 0;
+    p.tiles_per_unit = tiles_per_unit(a.batch, c.n_kv_heads, a.max_ctx_len, L.h->sm_count);
+    const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
+    p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
+    p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
+    p.ctx_len = a.ctx_len; p.page_table = a.page_table;
+    p.out = (__nv_bfloat16*)a.out; p.part = part; p.counters = counters; p.status = L.status;
+
+    CUtensorMap tq, tpool, tkb, tvb;
+    {   // q as [S*R][Hkv][group][hd]
+        const uint64_t dims[4] = {(uint64_t)HD, (uint64_t)p.group, (uint64_t)p.Hkv, (uint64_t)a.batch * a.rows};
+        const uint64_t str[3] = {(uint64_t)HD * 2, (uint64_t)p.group * HD * 2, (uint64_t)p.Hq * HD * 2};
+        const uint32_t box[4] = {64, (uint32_t)p.group, 1, (uint32_t)(128 / p.group)};
+        if (!tmap_encode_bf16(&tq, a.q, 4, dims, str, box)) return DFLASH_ERR_CUDA;
+    }
+    {   // the whole pool as rows of head_dim
+        const uint64_t rows = (uint64_t)c.n_layers * a.n_pool_pages * 2 * p.Hkv * PG;
+        const uint64_t dims[2] = {(uint64_t)HD, rows};
+        const uint64_t str[1] = {(uint64_t)HD * 2};
+        const uint32_t box[2] = {64, (uint32_t)PG};
+        if (!tmap_encode_bf16(&tpool, a.kv_pool, 2, dims, str, box)) return DFLASH_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)p.Hkv * HD, (uint64_t)a.batch * a.rows};
+        const uint64_t str[1] = {(uint64_t)p.Hkv * HD * 2};
+        const uint32_t box[2] = {64, (uint32_t)PG};
+        if (!tmap_encode_bf16(&tkb, a.k_blk, 2, dims, str, box)) return DFLASH_ERR_CUDA;
+        if (!tmap_encode_bf16(&tvb, a.v_blk, 2, dims, str, box)) return DFLASH_ERR_CUDA;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return DFLASH_ERR_CUDA;
+        attr_set = true;
+    }
+    const int grid = a.batch * p.Hkv * p.n_chunks;
+    attn_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, L.st>>>(tq, tpool, tkb, tvb, p);
+    ++g_launches;
+    return cudaPeekAtLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+}  // namespace dflash

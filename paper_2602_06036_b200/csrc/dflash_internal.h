@@ -67,6 +67,7 @@ struct Workspace {
     float* part;     // split-K partial sums of the tensor-core contractions
     int32_t* counters;   // split-K tickets (zeroed at the start of each call)
     int64_t counter_bytes;
+    int32_t* attn_counters;   // split-KV tickets of the attention kernel (inside the same region)
     void* top2;      // [vocab tiles, rows] per-tile winners of the fused LM-head argmax
     float* attn_part;    // attention split-KV partials
     int64_t bytes;
