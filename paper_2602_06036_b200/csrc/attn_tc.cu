@@ -10,9 +10,9 @@
 //   O_tile = P V        tcgen05.mma with V as an MN-major operand straight from the page layout
 //   acc = acc*alpha + O_tile   in registers, one row per thread
 // K/V tiles stream through a TMA ring that runs ahead of the math. Long contexts are split across
-// CTAs; partial (max, sum, acc) are merged in split order by the last CTA to arrive at a ticket
-// counter (no waiting, bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block
-// row r sees block rows <= r. Every mbarrier wait is bounded.
+// CTAs; each writes its partial (acc, max, sum) and a small second kernel merges them in split
+// order (bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block row r sees
+// block rows <= r. Every mbarrier wait is bounded.
 #include "attn_tc.cuh"
 
 #include "ptx_sm100.cuh"
@@ -32,7 +32,7 @@ constexpr int NS = 5;            // K/V ring depth
 constexpr int Q_BYTES = 128 * HD * 2;          // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
 constexpr int P_BYTES = 128 * PG * 2;          // 16 KiB
-constexpr int PART_LD = HD + 2;                // acc[128], running max, running sum
+constexpr int PART_LD = HD + 4;                // acc[128], running max, running sum, 2 pad (16-byte rows)
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + P_BYTES + 512;
 constexpr uint32_t TMEM_COLS = 256;            // S0 | S1 (64 each) | O (128)
 constexpr int N_THREADS = 192;
@@ -77,6 +77,12 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16_bmn(int m, int n) {
     return instr_desc_bf16(m, n) | (1u << 16);
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&t);
@@ -96,7 +102,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (t_lo >= T) return;                               // whole CTA leaves before touching any barrier
     const int t_hi = min(t_lo + p.tiles_per_unit, T);
     const int n_tiles = t_hi - t_lo;
-    const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
+    const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;   // CTAs sharing this (sequence, kv head)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -114,7 +120,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t* o_full = p_empty + 1;
     uint64_t* o_empty = o_full + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
-    volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] last arriver
+    volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -261,9 +267,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const float m_new = fmaxf(m_run, mx);
             float alpha = 1.f, psum = 0.f;
             if (m_new > -CUDART_INF_F) {
-                alpha = exp2f(m_run - m_new);
+                alpha = fast_exp2(m_run - m_new);
 #pragma unroll
-                for (int c = 0; c < PG; ++c) { s[c] = exp2f(s[c] - m_new); psum += s[c]; }
+                for (int c = 0; c < PG; ++c) { s[c] = fast_exp2(s[c] - m_new); psum += s[c]; }
             } else {
 #pragma unroll
                 for (int c = 0; c < PG; ++c) s[c] = 0.f;
@@ -330,52 +336,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                 }
             } else {
-                const int bg = b * p.Hkv + g;
-                float* mine = p.part + (((size_t)bg * p.n_chunks + chunk) * 128 + row) * PART_LD;
+                // partial result of this KV range: rows staged through the (now idle) K/V ring so the
+                // global write is one contiguous, coalesced copy
+                float* stage = reinterpret_cast<float*>(sKV);
                 if (row_valid) {
+                    float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);
 #pragma unroll
-                    for (int d = 0; d < HD; d += 2) *reinterpret_cast<float2*>(mine + d) = make_float2(acc[d], acc[d + 1]);
-                    *reinterpret_cast<float2*>(mine + HD) = make_float2(m_run, l_run);
-                }
-                __threadfence();
-                epi_bar();
-                if (row == 0) {
-                    const int old = atomicAdd(p.counters + bg, 1);
-                    flags[1] = (old == n_splits - 1) ? 1 : 0;
-                    if (old == n_splits - 1) p.counters[bg] = 0;
+                    for (int d = 0; d < HD; d += 4) srow[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
+                    srow[HD >> 2] = make_float4(m_run, l_run, 0.f, 0.f);
                 }
                 epi_bar();
-                if (flags[1] && row_valid) {
-                    __threadfence();
-                    float M = -CUDART_INF_F;
-                    for (int s2 = 0; s2 < n_splits; ++s2)
-                        M = fmaxf(M, __ldcg(p.part + (((size_t)bg * p.n_chunks + s2) * 128 + row) * PART_LD + HD));
-                    float Lsum = 0.f;
-#pragma unroll
-                    for (int d = 0; d < HD; ++d) acc[d] = 0.f;
-                    for (int s2 = 0; s2 < n_splits; ++s2) {
-                        const float* src = p.part + (((size_t)bg * p.n_chunks + s2) * 128 + row) * PART_LD;
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + HD));
-                        const float w = (ml.x > -CUDART_INF_F) ? exp2f(ml.x - M) : 0.f;
-                        Lsum += ml.y * w;
-#pragma unroll
-                        for (int d = 0; d < HD; d += 2) {
-                            const float2 a = __ldcg(reinterpret_cast<const float2*>(src + d));
-                            acc[d] += a.x * w;
-                            acc[d + 1] += a.y * w;
-                        }
-                    }
-                    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-#pragma unroll
-                    for (int d = 0; d < HD; d += 8) {
-                        uint4 w;
-                        w.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
-                        w.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
-                        w.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
-                        w.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
-                        *reinterpret_cast<uint4*>(dst + d) = w;
-                    }
-                }
+                const int n_valid_rows = min(128, p.R * p.group);
+                const int bg = b * p.Hkv + g;
+                float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * 128 * PART_LD);
+                const float4* src4 = reinterpret_cast<const float4*>(stage);
+                for (int e = row; e < n_valid_rows * (PART_LD / 4); e += 128) dst4[e] = src4[e];
             }
         }
     }
@@ -389,6 +364,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
 }
 
+// Merge of the per-range partials of one (sequence, kv head): one warp per query row, lanes over
+// head_dim, ranges visited in order. Sequences whose context fitted one range were already written.
+__global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
+    const int rows_valid = min(128, p.R * p.group);
+    const int row_blocks = (rows_valid + 3) / 4;
+    const int bg = blockIdx.x / row_blocks;
+    const int row = (blockIdx.x % row_blocks) * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int b = bg / p.Hkv, g = bg % p.Hkv;
+    const int L = max(p.ctx_len[b], 0);
+    const int T = (L + PG - 1) / PG + 1;
+    const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
+    if (n_splits <= 1 || row >= rows_valid) return;
+    const float* base = p.part + ((size_t)bg * p.n_chunks * 128 + row) * PART_LD;
+    const size_t unit_stride = (size_t)128 * PART_LD;
+    float M = -CUDART_INF_F;
+    for (int s = lane; s < n_splits; s += 32) M = fmaxf(M, __ldcg(base + s * unit_stride + HD));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float Lsum = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float* src = base + s * unit_stride;
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + HD));
+        const float w = (ml.x > -CUDART_INF_F) ? exp2f(ml.x - M) : 0.f;
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(src) + lane);
+        Lsum += ml.y * w;
+        acc.x += a.x * w; acc.y += a.y * w; acc.z += a.z * w; acc.w += a.w * w;
+    }
+    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+    const int r = row / p.group, j = row % p.group;
+    __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD + lane * 4;
+    uint2 w2;
+    w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+    w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(dst) = w2;
+}
+
 }  // namespace
 
 bool attn_tc_supported(const dflash_config& c, int rows) {
@@ -397,14 +410,18 @@ bool attn_tc_supported(const dflash_config& c, int rows) {
     return group >= 1 && 128 % group == 0 && rows * group <= 128 && rows <= PG;
 }
 
+// Keys are split into ranges of `tiles_per_unit` 64-key tiles so that the grid is about one wave of
+// CTAs (the longest sequence decides; shorter ones leave empty units that exit at once).
 static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
-    const int64_t Tmax = (max_ctx_len + PG - 1) / PG + 1;
-    const int64_t c = ((int64_t)batch * Hkv * Tmax + 2 * sm_count - 1) / (2 * sm_count);
-    return (int)std::max<int64_t>(2, c);
+    const int Tmax = (max_ctx_len + PG - 1) / PG + 1;
+    const int64_t bh = (int64_t)batch * Hkv;
+    for (int c = 2; c < Tmax; ++c)
+        if (bh * ((Tmax + c - 1) / c) <= sm_count) return c;
+    return std::max(2, Tmax);
 }
 
 int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int sm_count) {
-    // units never exceed 2*SMs + 2*batch*Hkv (see tiles_per_unit)
+    // units never exceed max(SMs, batch*Hkv*ceil(Tmax/2)) <= 2*SMs + 2*batch*Hkv (see tiles_per_unit)
     const int64_t units = 2 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
     return units * 128 * PART_LD * 4;
 }
@@ -454,7 +471,14 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     const int grid = a.batch * p.Hkv * p.n_chunks;
     attn_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, L.st>>>(tq, tpool, tkb, tvb, p);
     ++g_launches;
-    return cudaPeekAtLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    if (cudaPeekAtLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
+    if (p.n_chunks > 1) {
+        const int rows_valid = std::min(128, a.rows * p.group);
+        attn_combine_kernel<<<a.batch * p.Hkv * ((rows_valid + 3) / 4), 128, 0, L.st>>>(p);
+        ++g_launches;
+        if (cudaPeekAtLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
+    }
+    return DFLASH_OK;
 }
 
 }  // namespace dflash
