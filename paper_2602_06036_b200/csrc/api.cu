@@ -54,6 +54,7 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     w.attn_counters = w.counters ? (int32_t*)((char*)w.counters + gemm_counters) : nullptr;
     w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
     w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), h->sm_count) : 256);
+    w.seg = (float4*)a.take(R * 64 * 16);
     w.bytes = a.off;
     return w;
 }
@@ -138,7 +139,7 @@ static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, int 
         float* lg = logits_out ? logits_out + (size_t)r0 * c.vocab : ws.logits;
         RUN(FAM_LMHEAD, launch_gemm_simt(L, (const char*)z + (size_t)r0 * c.d_model * es, L.h->w.W_lm, lg, n, c.vocab,
                                          c.d_model, false));
-        RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, lg, DFLASH_F32, c.vocab, n, c.vocab, ids + r0, top1 ? top1 + r0 : nullptr,
+        RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, lg, DFLASH_F32, c.vocab, n, c.vocab, ws.seg, ids + r0, top1 ? top1 + r0 : nullptr,
                                               margin ? margin + r0 : nullptr));
     }
     return DFLASH_OK;
@@ -374,13 +375,10 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
     if (a->logits_dtype != DFLASH_F32 && a->logits_dtype != DFLASH_BF16) return DFLASH_ERR_UNSUPPORTED;
     const int64_t stride = a->logits_row_stride ? a->logits_row_stride : a->vocab;
     if (stride < a->vocab) return DFLASH_ERR_INVALID_ARG;
-    int32_t* ids = a->target_ids_out;
-    if (!ids) {
-        Workspace ws;
-        DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
-        ids = ws.ids;
-    }
-    RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, a->logits, a->logits_dtype, stride, rows, a->vocab, ids, nullptr, nullptr));
+    Workspace ws;
+    DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
+    int32_t* ids = a->target_ids_out ? a->target_ids_out : ws.ids;
+    RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, a->logits, a->logits_dtype, stride, rows, a->vocab, ws.seg, ids, nullptr, nullptr));
     RUN(FAM_ACCEPT, launch_accept(L, *a, ids));
     return DFLASH_OK;
 }

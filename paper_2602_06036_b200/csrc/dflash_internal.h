@@ -70,6 +70,7 @@ struct Workspace {
     int32_t* attn_counters;   // split-KV tickets of the attention kernel (inside the same region)
     void* top2;      // [vocab tiles, rows] per-tile winners of the fused LM-head argmax
     float* attn_part;    // attention split-KV partials
+    float4* seg;         // [rows, 64] per-segment winners of the row argmax over given logits
     int64_t bytes;
 };
 Workspace carve(const dflash_handle* h, void* base, int batch, int rows);
@@ -93,8 +94,9 @@ int launch_rope_split(const Launch& L, const float* qkv, const int32_t* ctx_len,
 int launch_swiglu(const Launch& L, const float* gu, void* h, int rows);
 int launch_attention_simt(const Launch& L, const dflash_attn_args& a);
 int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer);
+// two-stage row argmax; seg_scratch holds rows * 64 float4 entries
 int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows,
-                      int vocab, int32_t* ids, float* top1, float* margin);
+                      int vocab, float4* seg_scratch, int32_t* ids, float* top1, float* margin);
 int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids);
 int launch_copy_f32(const Launch& L, const float* src, float* dst, int64_t n);
 

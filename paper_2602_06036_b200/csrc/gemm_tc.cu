@@ -79,11 +79,15 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
         case EPI_STORE_F32:
         case EPI_RESIDUAL: {
             if (f < p.N) {
-                for (int c = 0; c < n_tok; ++c) {
-                    float* o = p.out_f32 + (size_t)(tok0 + c) * p.ld_out + f;
-                    const float a = sAcc[row * ACC_LD + c];
-                    *o = (p.epi == EPI_RESIDUAL) ? (*o + a) : a;
-                }
+                float* o = p.out_f32 + (size_t)tok0 * p.ld_out + f;
+                float prev[CH];
+                // all loads first: they are independent and must not queue behind the stores
+#pragma unroll
+                for (int c = 0; c < CH; ++c)
+                    prev[c] = (p.epi == EPI_RESIDUAL && c < n_tok) ? __ldcg(o + (size_t)c * p.ld_out) : 0.f;
+#pragma unroll
+                for (int c = 0; c < CH; ++c)
+                    if (c < n_tok) o[(size_t)c * p.ld_out] = prev[c] + sAcc[row * ACC_LD + c];
             }
         } break;
         case EPI_QKV_ROPE: {
@@ -93,23 +97,32 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
                 const int partner = row ^ half;
                 const int qdim = p.Hq * hd, kdim = p.Hkv * hd;
                 const bool rot = p.use_rope && head < p.Hq + p.Hkv;
-                for (int c = 0; c < n_tok; ++c) {
-                    const int tok = tok0 + c;
-                    float val = sAcc[row * ACC_LD + c];
-                    if (rot) {
-                        int pos = p.ctx_len[tok / p.rows_per_seq] + tok % p.rows_per_seq;
+                float cs[CH], sn[CH];
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    cs[c] = 1.f; sn[c] = 0.f;
+                    if (rot && c < n_tok) {
+                        const int tok = tok0 + c;
+                        int pos = __ldg(p.ctx_len + tok / p.rows_per_seq) + tok % p.rows_per_seq;
                         if (pos < 0 || pos >= p.max_pos) {
                             if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
                             pos = pos < 0 ? 0 : p.max_pos - 1;
                         }
-                        const float b = sAcc[partner * ACC_LD + c];
-                        const float cs = p.cs[(size_t)pos * half + i], sn = p.sn[(size_t)pos * half + i];
-                        val = hrow < half ? (val * cs - b * sn) : (val * cs + b * sn);
+                        cs[c] = __ldg(p.cs + (size_t)pos * half + i);
+                        sn[c] = __ldg(p.sn + (size_t)pos * half + i);
                     }
-                    const __nv_bfloat16 o = __float2bfloat16_rn(val);
-                    if (head < p.Hq) p.q[(size_t)tok * qdim + f] = o;
-                    else if (head < p.Hq + p.Hkv) p.k[(size_t)tok * kdim + (f - qdim)] = o;
-                    else p.v[(size_t)tok * kdim + (f - qdim - kdim)] = o;
+                }
+                __nv_bfloat16* dst;
+                int ld;
+                if (head < p.Hq) { dst = p.q + f; ld = qdim; }
+                else if (head < p.Hq + p.Hkv) { dst = p.k + (f - qdim); ld = kdim; }
+                else { dst = p.v + (f - qdim - kdim); ld = kdim; }
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    if (c >= n_tok) break;
+                    const float a = sAcc[row * ACC_LD + c], b = sAcc[partner * ACC_LD + c];
+                    const float val = hrow < half ? (a * cs[c] - b * sn[c]) : (a * cs[c] + b * sn[c]);
+                    dst[(size_t)(tok0 + c) * ld] = __float2bfloat16_rn(val);
                 }
             }
         } break;
@@ -427,7 +440,7 @@ int gemm_tc_splits(int M, int N, int K, int sm_count) {
     const int nt = pick_nt(M);
     const int base = ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt);
     const int chunks = (K + BK - 1) / BK;
-    if (base * 10 >= sm_count * 9) return 1;
+    if (base >= 4 * sm_count) return 1;   // enough units: the tail imbalance is already small
     int best = 1;
     double best_eff = 0.0;
     for (int s = 1; s <= 16; ++s) {

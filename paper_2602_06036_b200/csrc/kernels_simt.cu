@@ -5,6 +5,8 @@
 
 #include <math_constants.h>
 
+#include <algorithm>
+
 namespace dflash {
 
 long long g_launches = 0;
@@ -457,14 +459,34 @@ __device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
     return r;
 }
 
+// Stage 1: grid (segments, rows). Each CTA scans one contiguous segment of one row with 16-byte
+// loads (scalar at a misaligned head/tail) and writes that segment's (max, index, runner-up).
 template <typename T>
-__global__ void __launch_bounds__(512) row_argmax_kernel(const T* __restrict__ logits, int64_t row_stride,
-                                                         int vocab, int32_t* __restrict__ ids,
-                                                         float* __restrict__ top1, float* __restrict__ margin) {
-    __shared__ Top2 sh[16];
-    const T* src = logits + (size_t)blockIdx.x * row_stride;
+__global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict__ logits, int64_t row_stride,
+                                                             int vocab, int seg_len, float4* __restrict__ out) {
+    __shared__ Top2 sh[8];
+    constexpr int VEC = 16 / (int)sizeof(T);
+    const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
+    const T* src = logits + (size_t)row * row_stride;
+    const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
     Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-    for (int i = threadIdx.x; i < vocab; i += blockDim.x) top2_push(t, to_f(src[i]), i);
+    if (lo < hi) {
+        // first index at or after lo whose address is 16-byte aligned
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(src + lo);
+        int head = (int)(((16 - (addr & 15)) & 15) / sizeof(T));
+        head = min(head, hi - lo);
+        const int body = (hi - lo - head) / VEC;
+        for (int i = threadIdx.x; i < head; i += blockDim.x) top2_push(t, to_f(src[lo + i]), lo + i);
+        const uint4* v = reinterpret_cast<const uint4*>(src + lo + head);
+        for (int i = threadIdx.x; i < body; i += blockDim.x) {
+            const uint4 w = __ldg(v + i);
+            const T* e = reinterpret_cast<const T*>(&w);
+            const int base = lo + head + i * VEC;
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) top2_push(t, to_f(e[k]), base + k);
+        }
+        for (int i = lo + head + body * VEC + threadIdx.x; i < hi; i += blockDim.x) top2_push(t, to_f(src[i]), i);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         Top2 u;
@@ -479,21 +501,57 @@ __global__ void __launch_bounds__(512) row_argmax_kernel(const T* __restrict__ l
     if (threadIdx.x == 0) {
         Top2 r = sh[0];
         for (int i = 1; i < (int)(blockDim.x >> 5); ++i) r = top2_merge(r, sh[i]);
-        const int idx = (r.i1 == 0x7fffffff) ? 0 : r.i1;   // nothing compared greater than -inf
-        ids[blockIdx.x] = idx;
-        if (top1) top1[blockIdx.x] = r.v1;
-        if (margin) margin[blockIdx.x] = r.v1 - r.v2;
+        out[(size_t)row * nseg + seg] = make_float4(r.v1, __int_as_float(r.i1), r.v2, 0.f);
     }
 }
 
+// Stage 2: one warp per row merges the segments.
+__global__ void __launch_bounds__(256) row_argmax_merge_kernel(const float4* __restrict__ seg, int nseg, int rows,
+                                                               int32_t* __restrict__ ids, float* __restrict__ top1,
+                                                               float* __restrict__ margin) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int lane = threadIdx.x & 31;
+    Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
+    for (int i = lane; i < nseg; i += 32) {
+        const float4 e = seg[(size_t)row * nseg + i];
+        t = top2_merge(t, Top2{e.x, __float_as_int(e.y), e.z});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Top2 u;
+        u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t = top2_merge(t, u);
+    }
+    if (lane == 0) {
+        ids[row] = (t.i1 == 0x7fffffff) ? 0 : t.i1;      // nothing compared greater than -inf
+        if (top1) top1[row] = t.v1;
+        if (margin) margin[row] = t.v1 - t.v2;
+    }
+}
+
+int row_argmax_segments(int rows, int vocab, int sm_count) {
+    int nseg = (4 * sm_count + rows - 1) / std::max(rows, 1);
+    nseg = std::max(1, std::min(nseg, 64));
+    nseg = std::min(nseg, std::max(1, vocab / 2048));
+    return std::max(nseg, 1);
+}
+
 int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows, int vocab,
-                      int32_t* ids, float* top1, float* margin) {
+                      float4* seg_scratch, int32_t* ids, float* top1, float* margin) {
     if (rows == 0) return DFLASH_OK;
+    const int nseg = row_argmax_segments(rows, vocab, L.h->sm_count);
+    const int seg_len = ((vocab + nseg - 1) / nseg + 7) / 8 * 8;
+    dim3 grid(nseg, rows);
     if (dtype == DFLASH_F32)
-        row_argmax_kernel<float><<<rows, 512, 0, L.st>>>((const float*)logits, row_stride, vocab, ids, top1, margin);
+        row_argmax_seg_kernel<float><<<grid, 256, 0, L.st>>>((const float*)logits, row_stride, vocab, seg_len, seg_scratch);
     else
-        row_argmax_kernel<__nv_bfloat16><<<rows, 512, 0, L.st>>>((const __nv_bfloat16*)logits, row_stride, vocab,
-                                                                 ids, top1, margin);
+        row_argmax_seg_kernel<__nv_bfloat16><<<grid, 256, 0, L.st>>>((const __nv_bfloat16*)logits, row_stride, vocab,
+                                                                     seg_len, seg_scratch);
+    DFLASH_CHECK_LAUNCH();
+    row_argmax_merge_kernel<<<(rows + 7) / 8, 256, 0, L.st>>>(seg_scratch, nseg, rows, ids, top1, margin);
     DFLASH_CHECK_LAUNCH();
     return DFLASH_OK;
 }

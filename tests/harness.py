@@ -41,7 +41,7 @@ def assert_ids_match(got_ids, ref_ids, ref_margin, dtype, what=""):
 class Case:
     """One model + batch of sequences with paged context, on both sides."""
 
-    def __init__(self, cfg, ctx_lens, seed=0, weights=None, headroom=None, device="cuda:0"):
+    def __init__(self, cfg, ctx_lens, seed=0, weights=None, headroom=None, device="cuda:0", w_np=None, lib=None):
         from paper_2602_06036_b200 import binding
         self.cfg = cfg
         self.dtype = cfg.dtype
@@ -54,11 +54,14 @@ class Case:
         if weights is None:
             weights = synth.make_weights(cfg, seed)
         self.w_cpu = weights
-        self.w_np = synth.weights_to_numpy(weights)
+        self.w_np = w_np if w_np is not None else synth.weights_to_numpy(weights)
         self.max_pos = max(self.ctx_lens + [0]) + self.headroom + 1
         cos, sin = synth.rope_tables(cfg, self.max_pos)
-        self.lib = binding.DFlash(cfg, device)
-        self.lib.set_weights(synth.pack_device_weights(cfg, weights), cos, sin)
+        if lib is None:
+            self.lib = binding.DFlash(cfg, device)
+            self.lib.set_weights(synth.pack_device_weights(cfg, weights), cos, sin)
+        else:                      # a handle that already holds these weights (rope tables long enough)
+            self.lib = lib
         caps = [L + self.headroom for L in self.ctx_lens]
         self.page_table_cpu, self.n_pages = synth.make_page_table(cfg, caps, seed)
         self.page_table = self.page_table_cpu.to(self.device)
