@@ -198,6 +198,14 @@ class Step:
         return h2d, self.h_out.numel() * 4
 
 
+def capture(fn):
+    """Capture one step into a CUDA graph (after the eager warm-up has sized every buffer)."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g.replay
+
+
 def timed(fn, steps, warmup, dist_on):
     for _ in range(warmup):
         fn()
@@ -296,6 +304,7 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
 
@@ -323,13 +332,23 @@ def main():
     S, B = wl.batch, cfg.block_size
 
     sampler = ClockSampler(local)
+    run_resident, run_e2e = step.step_resident, step.step_e2e
+    for _ in range(2):           # eager warm-up: sizes the workspace, sets kernel attributes
+        run_resident()
+        run_e2e()
+    torch.cuda.synchronize()
+    n0 = binding.launch_count()
+    run_resident()
+    launches_per_step = binding.launch_count() - n0
+    if not args.no_graph:
+        run_resident = capture(step.step_resident)
+        run_e2e = capture(step.step_e2e)
     if rank == 0:
         sampler.start()
-    n0 = binding.launch_count()
-    ms = timed(step.step_resident, args.steps, args.warmup, dist_on)
-    launches = (binding.launch_count() - n0) // (args.steps + args.warmup) * args.steps
+    ms = timed(run_resident, args.steps, args.warmup, dist_on)
+    launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
-    ms_e2e = timed(step.step_e2e, args.steps, args.warmup, dist_on)
+    ms_e2e = timed(run_e2e, args.steps, args.warmup, dist_on)
 
     # per-kernel-family durations: a second pass of the same steps with event pairs around each launch
     prof = step.lib.profile(step.step_resident, args.steps) if hasattr(step.lib, "profile") else {}
@@ -368,6 +387,7 @@ def main():
         "config": {"workload": wl.name, "batch": S, "block_size": B, "ctx_lens": list(wl.ctx_lens)[:8],
                    "step": "ctx_project(n_new=tau) + draft_block + verify_accept(logits)",
                    "l2": "per-step weight traffic (3.2 GB) exceeds the 126 MB L2; no flush",
+                   "launch": "eager" if args.no_graph else "cuda graph replay of one step",
                    "parallelism": "replicas" if world > 1 else "single"},
         "step_roofline": {"alg_bytes": step_bytes, "us_at_peak": step_bytes / (hbm * 1e9) * 1e6,
                           "frac": step_bytes / (hbm * 1e9) / (per_step_ms * 1e-3)},

@@ -37,12 +37,13 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     int64_t part = 0, counters = 256;
     if (tc) {
         const int M = (int)R, sm = h->sm_count;
-        const int shapes[7][2] = {{qdim + 2 * kdim, c.d_model}, {c.d_model, qdim}, {2 * c.d_ffn, c.d_model},
-                                  {c.d_model, c.d_ffn},         {c.d_model, feat}, {2 * kdim, c.d_model},
-                                  {c.vocab, c.d_model}};
+        const int kv_groups = std::min(c.n_layers, GEMM_MAX_GROUPS);
+        const int shapes[7][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
+                                  {c.d_model, c.d_ffn, 1},         {c.d_model, feat, 1}, {2 * kdim, c.d_model, kv_groups},
+                                  {c.vocab, c.d_model, 1}};
         for (auto& s : shapes) {
-            part = std::max(part, gemm_tc_part_bytes(M, s[0], s[1], sm));
-            counters = std::max(counters, gemm_tc_counter_bytes(M, s[0]));
+            part = std::max(part, gemm_tc_part_bytes(M, s[0], s[1], s[2], sm));
+            counters = std::max(counters, gemm_tc_counter_bytes(M, s[0], s[2]));
         }
     }
     w.part = (float*)a.take(std::max<int64_t>(part, 256));
@@ -55,6 +56,7 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
     w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), h->sm_count) : 256);
     w.seg = (float4*)a.take(R * 64 * 16);
+    w.ssq = (float*)a.take((int64_t)((c.d_model + 127) / 128) * R * 4);
     w.bytes = a.off;
     return w;
 }
@@ -121,13 +123,14 @@ static int zero_counters(const Launch& L, const Workspace& ws) {
 }
 
 // LM head + argmax over `rows` normalised rows z (config dtype)
-static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, int rows, int32_t* ids, float* top1,
-                       float* margin, float* logits_out) {
+// (bf16 path: if ssq_in is given, z holds gain-scaled rows and the per-token rsqrt is applied inside)
+static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, const float* ssq_in, int rows, int32_t* ids,
+                       float* top1, float* margin, float* logits_out) {
     const dflash_config& c = L.h->cfg;
     if (c.dtype == DFLASH_BF16) {
         GemmArgs g{};
-        g.X = z; g.W = L.h->w.W_lm; g.M = rows; g.N = c.vocab; g.K = c.d_model;
-        g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters;
+        g.X = z; g.W[0] = L.h->w.W_lm; g.M = rows; g.N = c.vocab; g.K = c.d_model;
+        g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters; g.ssq_in = ssq_in;
         g.top2 = (Top2Entry*)ws.top2; g.logits_out = logits_out;
         RUN(FAM_LMHEAD, launch_gemm_tc(L, g));
         RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, ids, top1, margin));
@@ -259,28 +262,32 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
     const int kdim = c.n_kv_heads * c.head_dim, feat = c.n_feat_layers * c.d_target;
     const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
-    // y = W_c [h^(l1); ...; h^(lk)]  ->  H_t = RMSNorm(y)
+    // y = W_c [h^(l1); ...; h^(lk)]  ->  H_t = RMSNorm(y)  ->  per layer K = RoPE(W^K H_t), V = W^V H_t
+    const size_t kv_off = (size_t)c.n_q_heads * c.head_dim * c.d_model * elem_size(c.dtype);   // rows Hq*hd.. of W_qkv
     if (tc) {
+        // the norm is folded: the first contraction emits g_c*y (bf16) and sums of squares, the second
+        // scales its accumulator by the per-token rsqrt
         GemmArgs g{};
-        g.X = a->feats; g.W = h->w.W_c; g.M = rows; g.N = c.d_model; g.K = feat;
-        g.epilogue = EPI_STORE_F32; g.out_f32 = ws.tmp; g.ld_out = c.d_model; g.part = ws.part; g.counters = ws.counters;
+        g.X = a->feats; g.W[0] = h->w.W_c; g.M = rows; g.N = c.d_model; g.K = feat;
+        g.epilogue = EPI_STORE_F32; g.g_next = h->w.g_c; g.xn_out = (__nv_bfloat16*)ws.u; g.ssq_out = ws.ssq;
+        g.part = ws.part; g.counters = ws.counters;
         RUN(FAM_CTX_FUSE, launch_gemm_tc(L, g));
-    } else {
-        RUN(FAM_CTX_FUSE, launch_gemm_simt(L, a->feats, h->w.W_c, ws.tmp, rows, c.d_model, feat, false));
+        for (int i0 = 0; i0 < c.n_layers; i0 += GEMM_MAX_GROUPS) {
+            GemmArgs k{};
+            k.n_groups = std::min(GEMM_MAX_GROUPS, c.n_layers - i0);
+            for (int j = 0; j < k.n_groups; ++j) k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
+            k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
+            k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part; k.counters = ws.counters;
+            RUN(FAM_CTX_KV, launch_gemm_tc(L, k));
+        }
+        return DFLASH_OK;
     }
+    RUN(FAM_CTX_FUSE, launch_gemm_simt(L, a->feats, h->w.W_c, ws.tmp, rows, c.d_model, feat, false));
     RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.tmp, true, h->w.g_c, true, ws.u, rows, c.d_model));
     for (int i = 0; i < c.n_layers; ++i) {
-        // rows Hq*hd .. of W_qkv are W_i^K then W_i^V
-        const char* Wkv = (const char*)h->layers[i].W_qkv + (size_t)c.n_q_heads * c.head_dim * c.d_model * elem_size(c.dtype);
-        if (tc) {
-            GemmArgs g{};
-            g.X = ws.u; g.W = Wkv; g.M = rows; g.N = 2 * kdim; g.K = c.d_model;
-            g.epilogue = EPI_CTX_KV; g.ctx = a; g.layer = i; g.part = ws.part; g.counters = ws.counters;
-            RUN(FAM_CTX_KV, launch_gemm_tc(L, g));
-        } else {
-            RUN(FAM_CTX_KV, launch_gemm_simt(L, ws.u, Wkv, ws.tmp, rows, 2 * kdim, c.d_model, false));
-            RUN(FAM_CTX_KV, launch_ctx_scatter(L, ws.tmp, *a, i));
-        }
+        const char* Wkv = (const char*)h->layers[i].W_qkv + kv_off;
+        RUN(FAM_CTX_KV, launch_gemm_simt(L, ws.u, Wkv, ws.tmp, rows, 2 * kdim, c.d_model, false));
+        RUN(FAM_CTX_KV, launch_ctx_scatter(L, ws.tmp, *a, i));
     }
     return DFLASH_OK;
 }
@@ -301,60 +308,70 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
 
+    dflash_attn_args at{};
+    at.mode = DFLASH_ATTN_FULL;
+    at.q = ws.q; at.k_blk = ws.k_blk; at.v_blk = ws.v_blk;
+    at.batch = a->batch; at.rows = B;
+    at.ctx_len = a->ctx_len; at.max_ctx_len = a->max_ctx_len;
+    at.page_table = a->page_table; at.max_pages = a->max_pages;
+    at.kv_pool = a->kv_pool; at.n_pool_pages = a->n_pool_pages;
+    at.out = ws.attn;
+
+    if (tc) {
+        // bf16: tensor-core contractions with the norms folded into their epilogues.
+        // ws.u always holds bf16(gain * x) of the rows about to be projected, ws.ssq their sums of squares.
+        __nv_bfloat16* xn = (__nv_bfloat16*)ws.u;
+        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, ws.x, h->layers[0].g1, xn, ws.ssq));
+        for (int i = 0; i < c.n_layers; ++i) {
+            const dflash_layer_weights& lw = h->layers[i];
+            GemmArgs g{};      // q,k,v = W_qkv RMSNorm(x), rotated
+            g.X = xn; g.W[0] = lw.W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model; g.ssq_in = ws.ssq;
+            g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
+            g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
+            g.part = ws.part; g.counters = ws.counters;
+            RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g));
+            at.layer = i;
+            if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
+            else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+            GemmArgs o{};      // x += W_o attn; emits the FFN norm inputs
+            o.X = ws.attn; o.W[0] = lw.W_o; o.M = rows; o.N = c.d_model; o.K = qdim;
+            o.epilogue = EPI_RESIDUAL; o.out_f32 = ws.x; o.ld_out = c.d_model; o.part = ws.part; o.counters = ws.counters;
+            o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq;
+            RUN(FAM_GEMM_O, launch_gemm_tc(L, o));
+            GemmArgs u{};      // h = silu(W_gate u) * (W_up u)
+            u.X = xn; u.W[0] = lw.W_gateup; u.M = rows; u.N = 2 * c.d_ffn; u.K = c.d_model; u.ssq_in = ws.ssq;
+            u.epilogue = EPI_SWIGLU; u.h = (__nv_bfloat16*)ws.h; u.part = ws.part; u.counters = ws.counters;
+            RUN(FAM_GEMM_GATEUP, launch_gemm_tc(L, u));
+            GemmArgs d{};      // x += W_down h; emits the next layer's (or the final) norm inputs
+            d.X = ws.h; d.W[0] = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
+            d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part; d.counters = ws.counters;
+            d.g_next = (i + 1 < c.n_layers) ? h->layers[i + 1].g1 : h->w.g_f; d.xn_out = xn; d.ssq_out = ws.ssq;
+            RUN(FAM_GEMM_DOWN, launch_gemm_tc(L, d));
+        }
+        if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
+        return lmhead_rows(L, ws, xn, ws.ssq, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
+    }
+
+    // fp32: CUDA-core kernels, one step per launch
     RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, ws.x, a->batch));
     for (int i = 0; i < c.n_layers; ++i) {
         const dflash_layer_weights& lw = h->layers[i];
         // attention half: u = RMSNorm(x); q,k,v = W u (+RoPE); x += W_o attention(q, [K_ctx; k], [V_ctx; v])
         RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g1, true, ws.u, rows, c.d_model));
-        if (tc) {
-            GemmArgs g{};
-            g.X = ws.u; g.W = lw.W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model;
-            g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
-            g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
-            g.part = ws.part; g.counters = ws.counters;
-            RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g));
-        } else {
-            RUN(FAM_GEMM_QKV, launch_gemm_simt(L, ws.u, lw.W_qkv, ws.tmp, rows, qdim + 2 * kdim, c.d_model, false));
-            RUN(FAM_GEMM_QKV, launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk));
-        }
-        dflash_attn_args at{};
-        at.mode = DFLASH_ATTN_FULL;
-        at.q = ws.q; at.k_blk = ws.k_blk; at.v_blk = ws.v_blk;
-        at.batch = a->batch; at.rows = B;
-        at.ctx_len = a->ctx_len; at.max_ctx_len = a->max_ctx_len;
-        at.page_table = a->page_table; at.max_pages = a->max_pages;
-        at.kv_pool = a->kv_pool; at.n_pool_pages = a->n_pool_pages; at.layer = i;
-        at.out = ws.attn;
-        if (tc && attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
-        else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
-        if (tc) {
-            GemmArgs g{};
-            g.X = ws.attn; g.W = lw.W_o; g.M = rows; g.N = c.d_model; g.K = qdim;
-            g.epilogue = EPI_RESIDUAL; g.out_f32 = ws.x; g.ld_out = c.d_model; g.part = ws.part; g.counters = ws.counters;
-            RUN(FAM_GEMM_O, launch_gemm_tc(L, g));
-        } else {
-            RUN(FAM_GEMM_O, launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));
-        }
+        RUN(FAM_GEMM_QKV, launch_gemm_simt(L, ws.u, lw.W_qkv, ws.tmp, rows, qdim + 2 * kdim, c.d_model, false));
+        RUN(FAM_GEMM_QKV, launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk));
+        at.layer = i;
+        RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+        RUN(FAM_GEMM_O, launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));
         // FFN half: u = RMSNorm(x); x += W_down (silu(W_gate u) * W_up u)
         RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g2, true, ws.u, rows, c.d_model));
-        if (tc) {
-            GemmArgs g{};
-            g.X = ws.u; g.W = lw.W_gateup; g.M = rows; g.N = 2 * c.d_ffn; g.K = c.d_model;
-            g.epilogue = EPI_SWIGLU; g.h = (__nv_bfloat16*)ws.h; g.part = ws.part; g.counters = ws.counters;
-            RUN(FAM_GEMM_GATEUP, launch_gemm_tc(L, g));
-            GemmArgs d{};
-            d.X = ws.h; d.W = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
-            d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part; d.counters = ws.counters;
-            RUN(FAM_GEMM_DOWN, launch_gemm_tc(L, d));
-        } else {
-            RUN(FAM_GEMM_GATEUP, launch_gemm_simt(L, ws.u, lw.W_gateup, ws.tmp, rows, 2 * c.d_ffn, c.d_model, false));
-            RUN(FAM_GEMM_GATEUP, launch_swiglu(L, ws.tmp, ws.h, rows));
-            RUN(FAM_GEMM_DOWN, launch_gemm_simt(L, ws.h, lw.W_down, ws.x, rows, c.d_model, c.d_ffn, true));
-        }
+        RUN(FAM_GEMM_GATEUP, launch_gemm_simt(L, ws.u, lw.W_gateup, ws.tmp, rows, 2 * c.d_ffn, c.d_model, false));
+        RUN(FAM_GEMM_GATEUP, launch_swiglu(L, ws.tmp, ws.h, rows));
+        RUN(FAM_GEMM_DOWN, launch_gemm_simt(L, ws.h, lw.W_down, ws.x, rows, c.d_model, c.d_ffn, true));
     }
     if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
     RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, h->w.g_f, true, ws.u, rows, c.d_model));
-    return lmhead_rows(L, ws, ws.u, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
+    return lmhead_rows(L, ws, ws.u, nullptr, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
 }
 
 int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void* stream) {
@@ -418,7 +435,7 @@ int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a, void
     const bool f32in = a->hidden_is_f32 || c.dtype == DFLASH_F32;
     DFLASH_TRY(zero_counters(L, ws));
     RUN(FAM_RMSNORM, launch_rmsnorm(L, a->hidden, f32in, h->w.g_f, a->apply_norm != 0, ws.u, a->n_rows, c.d_model));
-    return lmhead_rows(L, ws, ws.u, a->n_rows, a->ids, a->top1, a->margin, a->logits_out);
+    return lmhead_rows(L, ws, ws.u, nullptr, a->n_rows, a->ids, a->top1, a->margin, a->logits_out);
 }
 
 }  // extern "C"

@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPool,
                const __grid_constant__ CUtensorMap tmKb, const __grid_constant__ CUtensorMap tmVb, const AParams p) {
     // ---- which work unit ----
+    pdl_trigger();
+    pdl_wait();      // lengths, page table, q and the block's k/v come from earlier kernels
     const int chunk = blockIdx.x % p.n_chunks;
     const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
     const int b = blockIdx.x / (p.n_chunks * p.Hkv);
@@ -182,6 +184,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
             }
         }
+        __syncwarp();     // the whole warp must reach the closing barrier together
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
@@ -224,6 +227,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
             }
         }
+        __syncwarp();
     } else {
         // ---------------- softmax + accumulation: thread = query row ----------------
         const int ew = warp & 3;
@@ -367,6 +371,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 // Merge of the per-range partials of one (sequence, kv head): one warp per query row, lanes over
 // head_dim, ranges visited in order. Sequences whose context fitted one range were already written.
 __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
+    pdl_trigger();
+    pdl_wait();
     const int rows_valid = min(128, p.R * p.group);
     const int row_blocks = (rows_valid + 3) / 4;
     const int bg = blockIdx.x / row_blocks;
@@ -469,14 +475,14 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
         attr_set = true;
     }
     const int grid = a.batch * p.Hkv * p.n_chunks;
-    attn_tc_kernel<<<grid, N_THREADS, SMEM_BYTES, L.st>>>(tq, tpool, tkb, tvb, p);
+    if (launch_pdl(attn_tc_kernel, dim3(grid), dim3(N_THREADS), (size_t)SMEM_BYTES, L.st, tq, tpool, tkb, tvb, p) != cudaSuccess)
+        return DFLASH_ERR_CUDA;
     ++g_launches;
-    if (cudaPeekAtLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
     if (p.n_chunks > 1) {
         const int rows_valid = std::min(128, a.rows * p.group);
-        attn_combine_kernel<<<a.batch * p.Hkv * ((rows_valid + 3) / 4), 128, 0, L.st>>>(p);
+        if (launch_pdl(attn_combine_kernel, dim3(a.batch * p.Hkv * ((rows_valid + 3) / 4)), dim3(128), 0, L.st, p) != cudaSuccess)
+            return DFLASH_ERR_CUDA;
         ++g_launches;
-        if (cudaPeekAtLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
     }
     return DFLASH_OK;
 }

@@ -71,6 +71,7 @@ struct Workspace {
     void* top2;      // [vocab tiles, rows] per-tile winners of the fused LM-head argmax
     float* attn_part;    // attention split-KV partials
     float4* seg;         // [rows, 64] per-segment winners of the row argmax over given logits
+    float* ssq;          // [D/128, rows] per-tile sums of squares feeding the folded RMSNorm
     int64_t bytes;
 };
 Workspace carve(const dflash_handle* h, void* base, int batch, int rows);

@@ -4,9 +4,16 @@
 // (16..256 columns), so the tensor core runs full-height instructions however few tokens there
 // are. A CTA is one TMA producer warp, one MMA-issuing warp and four epilogue warps; operands
 // stream through a ring of 128-byte-swizzled shared-memory stages, accumulators live in two TMEM
-// buffers so the epilogue of one work unit overlaps the main loop of the next. Work units are
-// (feature tile, token tile, K split), walked persistently; K splits meet in a fixed-order sum done
-// by whichever CTA arrives last at a ticket counter (no waiting, bit-reproducible).
+// buffers so the epilogue of one piece of work overlaps the main loop of the next. The work is the
+// sequence of all (output tile, K chunk) pairs, cut into one contiguous, equally long range per CTA
+// ("stream-K"): every SM streams the same number of weight bytes whatever the tile count. A range
+// that covers a whole output tile goes straight to the epilogue; tiles shared by several CTAs meet
+// in a fixed-order sum done by whichever CTA arrives last at a ticket counter (no waiting,
+// bit-reproducible). RMSNorm never runs as a kernel of its own: epilogues that produce residual
+// rows also emit the gain-scaled bf16 operand and per-tile sums of squares, and the consuming
+// contraction scales its accumulator columns by the per-token rsqrt.
+// Launched with programmatic dependent launch: barrier set-up, TMEM allocation and the first ring
+// of WEIGHT tiles (which no earlier kernel writes) are issued before griddepcontrol.wait.
 // Every wait on an mbarrier is bounded; on expiry the kernel raises DFLASH_DEV_TIMEOUT, drains its
 // outstanding copies, frees its TMEM and returns.
 #include "gemm_tc.cuh"
@@ -28,14 +35,24 @@ constexpr int CH = 16;                           // token columns handled per ep
 constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB
 constexpr int MAX_STAGES = 12;
 constexpr int ACC_LD = CH + 1;
-constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + (2 * MAX_STAGES + 4) * 8 + 64;
+constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64;
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int N_THREADS = 192;
 
+struct WMaps {
+    CUtensorMap m[GEMM_MAX_GROUPS];
+};
+
 struct KParams {
-    int M, N, K, epi, splits, chunks_total, chunks_per_split, n_ftiles, n_ttiles, stages;
+    int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, stages;
     float* part;
     int32_t* counters;
+    const float* ssq_in;
+    int n_parts_in;
+    float inv_dim_in, eps;
+    const __nv_bfloat16* g_next;
+    __nv_bfloat16* xn_out;
+    float* ssq_out;
     float* out_f32;
     int ld_out;
     __nv_bfloat16 *q, *k, *v;
@@ -50,9 +67,49 @@ struct KParams {
     __nv_bfloat16* pool;
     const int32_t* n_new;
     const int32_t* page_table;
-    int max_new, max_pages, n_pages, PG, layer;
+    int max_new, max_pages, n_pages, PG, first_layer;
     int32_t* status;
 };
+
+// One piece of a CTA's chunk range: chunks [c0, c1) of output tile `tile`.
+struct Unit {
+    int tile, g, ft, tt, c0, c1;
+    int slot;      // 0 = first piece of this CTA's range, 1 = a later one (partial pieces only: first or last)
+    int full;      // covers every chunk of the tile
+};
+
+// Walks the pieces of CTA `cta` out of `n_ctas`: range [cta*T/G, (cta+1)*T/G) of the T = n_tiles *
+// chunks_total (tile, chunk) pairs, tiles ordered token-tile fastest so neighbours share weights.
+struct PieceWalk {
+    long long cur, hi;
+    int first;
+    __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas) {
+        const long long T = (long long)p.n_tiles * p.chunks_total;
+        cur = (long long)cta * T / n_ctas;
+        hi = (long long)(cta + 1) * T / n_ctas;
+        first = 1;
+    }
+    __device__ __forceinline__ bool done() const { return cur >= hi; }
+    __device__ __forceinline__ Unit next(const KParams& p) {
+        Unit u;
+        u.tile = (int)(cur / p.chunks_total);
+        u.c0 = (int)(cur % p.chunks_total);
+        const long long left = hi - cur;
+        u.c1 = (int)min((long long)p.chunks_total, u.c0 + left);
+        u.full = (u.c0 == 0 && u.c1 == p.chunks_total) ? 1 : 0;
+        u.slot = first ? 0 : 1;
+        int t = u.tile;
+        u.tt = t % p.n_ttiles;
+        t /= p.n_ttiles;
+        u.ft = t % p.n_ftiles;
+        u.g = t / p.n_ftiles;
+        cur += u.c1 - u.c0;
+        first = 0;
+        return u;
+    }
+};
+// CTA that owns (tile, chunk) pair number x:  largest j with floor(j*T/G) <= x
+__device__ __forceinline__ int cta_of_pair(long long x, long long T, int G) { return (int)(((x + 1) * G + T - 1) / T - 1); }
 
 // ---------------------------------------------------------------------------------------------
 // epilogues: 128 threads, thread `row` owns feature f0 + row; sAcc[row][c] holds 16 token columns
@@ -71,23 +128,57 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
     else a.v2 = fmaxf(a.v2, v1);
 }
 
-__device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sAcc, Top2Entry* sRed, int ft, int tok0,
+// Every one of the 128 epilogue threads calls this (it contains named barriers).
+__device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
                                                int row) {
-    const int f = ft * TILE_F + row;
+    const int f = un.ft * TILE_F + row;
     const int n_tok = min(CH, p.M - tok0);
     switch (p.epi) {
         case EPI_STORE_F32:
         case EPI_RESIDUAL: {
+            float xv[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) xv[c] = 0.f;
             if (f < p.N) {
-                float* o = p.out_f32 + (size_t)tok0 * p.ld_out + f;
-                float prev[CH];
+                float* o = p.out_f32 ? p.out_f32 + (size_t)tok0 * p.ld_out + f : nullptr;
                 // all loads first: they are independent and must not queue behind the stores
+                if (p.epi == EPI_RESIDUAL) {
 #pragma unroll
-                for (int c = 0; c < CH; ++c)
-                    prev[c] = (p.epi == EPI_RESIDUAL && c < n_tok) ? __ldcg(o + (size_t)c * p.ld_out) : 0.f;
+                    for (int c = 0; c < CH; ++c)
+                        if (c < n_tok) xv[c] = __ldcg(o + (size_t)c * p.ld_out);
+                }
 #pragma unroll
-                for (int c = 0; c < CH; ++c)
-                    if (c < n_tok) o[(size_t)c * p.ld_out] = prev[c] + sAcc[row * ACC_LD + c];
+                for (int c = 0; c < CH; ++c) {
+                    if (c < n_tok) {
+                        xv[c] += sAcc[row * ACC_LD + c];
+                        if (o) o[(size_t)c * p.ld_out] = xv[c];
+                    }
+                }
+                if (p.g_next) {
+                    const float gv = __bfloat162float(p.g_next[f]);
+#pragma unroll
+                    for (int c = 0; c < CH; ++c)
+                        if (c < n_tok) p.xn_out[(size_t)(tok0 + c) * p.N + f] = __float2bfloat16_rn(gv * xv[c]);
+                }
+            }
+            if (p.ssq_out) {
+                // per-token sum of squares over this tile's 128 features
+#pragma unroll
+                for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = xv[c] * xv[c];
+                epi_bar();
+                const int c = row & 15, g8 = row >> 4;
+                float s = 0.f;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) s += sAcc[(g8 * 16 + r) * ACC_LD + c];
+                float* red = reinterpret_cast<float*>(sRed);
+                red[g8 * 16 + c] = s;
+                epi_bar();
+                if (row < n_tok) {
+                    float t = 0.f;
+#pragma unroll
+                    for (int gg = 0; gg < 8; ++gg) t += red[gg * 16 + row];
+                    p.ssq_out[(size_t)un.ft * p.M + tok0 + row] = t;
+                }
             }
         } break;
         case EPI_QKV_ROPE: {
@@ -103,7 +194,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
                     cs[c] = 1.f; sn[c] = 0.f;
                     if (rot && c < n_tok) {
                         const int tok = tok0 + c;
-                        int pos = __ldg(p.ctx_len + tok / p.rows_per_seq) + tok % p.rows_per_seq;
+                        int pos = __ldcg(p.ctx_len + tok / p.rows_per_seq) + tok % p.rows_per_seq;
                         if (pos < 0 || pos >= p.max_pos) {
                             if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
                             pos = pos < 0 ? 0 : p.max_pos - 1;
@@ -142,7 +233,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
             T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
-                const int rr = g * 16 + r, ff = ft * TILE_F + rr;
+                const int rr = g * 16 + r, ff = un.ft * TILE_F + rr;
                 if (ff < p.N) t2_push(t, sAcc[rr * ACC_LD + c], ff);
             }
             sRed[g * 16 + c] = Top2Entry{t.v1, t.i1, t.v2, 0};
@@ -151,7 +242,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
                 T2 m{sRed[row].v1, sRed[row].i1, sRed[row].v2};
 #pragma unroll
                 for (int gg = 1; gg < 8; ++gg) t2_merge(m, sRed[gg * 16 + row].v1, sRed[gg * 16 + row].i1, sRed[gg * 16 + row].v2);
-                p.top2[(size_t)ft * p.M + tok0 + row] = Top2Entry{m.v1, m.i1, m.v2, 0};
+                p.top2[(size_t)un.ft * p.M + tok0 + row] = Top2Entry{m.v1, m.i1, m.v2, 0};
             }
         } break;
         case EPI_CTX_KV: {
@@ -162,31 +253,45 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
                 const int fh = f - is_v * kdim;
                 const int head = fh / hd, hrow = fh % hd, i = hrow % half;
                 const int partner = row ^ half;
-                for (int c = 0; c < n_tok; ++c) {
+                const int layer = p.first_layer + un.g;
+                // gather every token's destination and rotation first, then write
+                long long dst[CH];
+                float cs[CH], sn[CH];
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    dst[c] = -1; cs[c] = 1.f; sn[c] = 0.f;
+                    if (c >= n_tok) continue;
                     const int tok = tok0 + c;
                     const int b = tok / p.max_new, r = tok % p.max_new;
-                    const int nn = p.n_new ? p.n_new[b] : p.max_new;
+                    const int nn = p.n_new ? __ldcg(p.n_new + b) : p.max_new;
                     if (r >= nn) continue;
-                    const int pos = p.ctx_len[b] + r;
+                    const int pos = __ldcg(p.ctx_len + b) + r;
                     const int pidx = pos / p.PG;
                     if (pos < 0 || pidx >= p.max_pages || (p.use_rope && pos >= p.max_pos)) {
                         if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
                         continue;
                     }
-                    const int page = p.page_table[(size_t)b * p.max_pages + pidx];
+                    const int page = __ldcg(p.page_table + (size_t)b * p.max_pages + pidx);
                     if (page < 0 || page >= p.n_pages) {
                         if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
                         continue;
                     }
+                    if (!is_v && p.use_rope) {
+                        cs[c] = __ldg(p.cs + (size_t)pos * half + i);
+                        sn[c] = __ldg(p.sn + (size_t)pos * half + i);
+                    }
+                    dst[c] = (long long)((((((size_t)layer * p.n_pages + page) * 2 + is_v) * p.Hkv + head) * p.PG +
+                                          (pos % p.PG)) * hd + hrow);
+                }
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    if (dst[c] < 0) continue;
                     float val = sAcc[row * ACC_LD + c];
                     if (!is_v && p.use_rope) {
                         const float bb = sAcc[partner * ACC_LD + c];
-                        const float cs = p.cs[(size_t)pos * half + i], sn = p.sn[(size_t)pos * half + i];
-                        val = hrow < half ? (val * cs - bb * sn) : (val * cs + bb * sn);
+                        val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
                     }
-                    const size_t dst = (((((size_t)p.layer * p.n_pages + page) * 2 + is_v) * p.Hkv + head) * p.PG +
-                                        (pos % p.PG)) * hd + hrow;
-                    p.pool[dst] = __float2bfloat16_rn(val);
+                    p.pool[dst[c]] = __float2bfloat16_rn(val);
                 }
             }
         } break;
@@ -199,7 +304,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, const float* sA
 // ---------------------------------------------------------------------------------------------
 template <int NT>
 __global__ void __launch_bounds__(N_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const KParams p) {
+gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtensorMap tmX, const KParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int X_STAGE_BYTES = NT * BK * 2;
@@ -209,7 +314,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     uint8_t* sX = sW + (size_t)stages * W_STAGE_BYTES;
     float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE_BYTES);
     Top2Entry* sRed = reinterpret_cast<Top2Entry*>(sAcc + TILE_F * ACC_LD);
-    uint64_t* full = reinterpret_cast<uint64_t*>(sRed + 128);
+    float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [256] per-token rsqrt of this token tile
+    uint64_t* full = reinterpret_cast<uint64_t*>(sRstd + 256);
     uint64_t* empty = full + MAX_STAGES;
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -230,25 +336,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_trigger();
 
-    const int total_units = p.n_ftiles * p.n_ttiles * p.splits;
+    const int G = gridDim.x;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+            // Before the grid dependency is resolved: fill the ring with WEIGHT tiles only (weights
+            // are never written by a kernel). The matching activation tiles follow after the wait.
+            int n_pre = 0;
+            for (PieceWalk w(p, blockIdx.x, G); !w.done() && n_pre < stages;) {
+                const Unit un = w.next(p);
+                for (int c = un.c0; c < un.c1 && n_pre < stages; ++c, ++n_pre) {
+                    mbar_expect_tx(&full[n_pre], W_STAGE_BYTES + X_STAGE_BYTES);
+                    tma_load_2d(sW + (size_t)n_pre * W_STAGE_BYTES, &tmW.m[un.g], c * BK, un.ft * TILE_F, &full[n_pre], pol_w);
+                }
+            }
+            pdl_wait();
             uint32_t it = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-                const int s = u % p.splits, tt = (u / p.splits) % p.n_ttiles, ft = u / (p.splits * p.n_ttiles);
-                const int c0 = s * p.chunks_per_split, c1 = min(c0 + p.chunks_per_split, p.chunks_total);
-                for (int c = c0; c < c1; ++c, ++it) {
+            for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok;) {
+                const Unit un = w.next(p);
+                for (int c = un.c0; c < un.c1; ++c, ++it) {
                     const int st = it % stages;
                     const uint32_t ph = (it / stages) & 1;
-                    if (!mbar_wait(&empty[st], ph ^ 1, &flags[0])) { ok = false; break; }
-                    mbar_expect_tx(&full[st], W_STAGE_BYTES + X_STAGE_BYTES);
-                    tma_load_2d(sW + (size_t)st * W_STAGE_BYTES, &tmW, c * BK, ft * TILE_F, &full[st], pol_w);
-                    tma_load_2d(sX + (size_t)st * X_STAGE_BYTES, &tmX, c * BK, tt * NT, &full[st], pol_x);
+                    if ((int)it >= n_pre) {
+                        if (!mbar_wait(&empty[st], ph ^ 1, &flags[0])) { ok = false; break; }
+                        mbar_expect_tx(&full[st], W_STAGE_BYTES + X_STAGE_BYTES);
+                        tma_load_2d(sW + (size_t)st * W_STAGE_BYTES, &tmW.m[un.g], c * BK, un.ft * TILE_F, &full[st], pol_w);
+                    }
+                    tma_load_2d(sX + (size_t)st * X_STAGE_BYTES, &tmX, c * BK, un.tt * NT, &full[st], pol_x);
                 }
             }
             if (!ok) {
@@ -263,20 +382,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 }
             }
         }
+        __syncwarp();     // the whole warp must reach the closing barrier together
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_bf16(TILE_F, NT);
             uint32_t it = 0, ui = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++ui) {
-                const int s = u % p.splits;
-                const int c0 = s * p.chunks_per_split, c1 = min(c0 + p.chunks_per_split, p.chunks_total);
+            for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok; ++ui) {
+                const Unit un = w.next(p);
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
                 if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * NT;
-                for (int c = c0; c < c1; ++c, ++it) {
+                for (int c = un.c0; c < un.c1; ++c, ++it) {
                     const int st = it % stages;
                     const uint32_t ph = (it / stages) & 1;
                     if (!mbar_wait(&full[st], ph, &flags[0])) { ok = false; break; }
@@ -286,7 +405,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk)
                         mma_bf16(d_tmem, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32), idesc,
-                                 (c > c0 || kk > 0) ? 1u : 0u);
+                                 (c > un.c0 || kk > 0) ? 1u : 0u);
                     mma_commit(&empty[st]);
                 }
                 if (ok) mma_commit(&acc_full[buf]);
@@ -296,48 +415,67 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
             }
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
         const int ew = warp & 3;
         const int row = ew * 32 + lane;
+        const long long T = (long long)p.n_tiles * p.chunks_total;
+        pdl_wait();
         uint32_t ui = 0;
-        for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++ui) {
-            const int s = u % p.splits, tt = (u / p.splits) % p.n_ttiles, ft = u / (p.splits * p.n_ttiles);
+        int rstd_tt = -1;
+        for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
+            const Unit un = w.next(p);
+            const int tok_base = un.tt * NT;
+            // per-token rsqrt(mean square) of the operand rows, once per token tile
+            if (p.ssq_in && rstd_tt != un.tt) {
+                for (int t = row; t < NT; t += 128) {
+                    float rs = 1.f;
+                    if (tok_base + t < p.M) {
+                        float s = 0.f;
+                        for (int q = 0; q < p.n_parts_in; ++q) s += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
+                        rs = rsqrtf(s * p.inv_dim_in + p.eps);
+                    }
+                    sRstd[t] = rs;
+                }
+                rstd_tt = un.tt;
+                // made visible by the barrier below
+            }
             const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
             const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
             if (!got) flags[2] = 1;
             epi_bar();
             if (flags[2]) break;   // uniform over the four warps
             tc_fence_after();
-            const int tok_base = tt * NT;
             const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
-            const int unit_tile = ft * p.n_ttiles + tt;
             for (int ch = 0; ch < n_ch; ++ch) {
                 float v[CH];
                 tmem_ld16(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
-                if (p.splits > 1) {
-                    float* dst = p.part + (((size_t)unit_tile * p.splits + s) * NT + ch * CH) * TILE_F + row;
+                if (!un.full) {
+                    float* dst = p.part + (((size_t)blockIdx.x * 2 + un.slot) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
                     for (int c = 0; c < CH; ++c) dst[(size_t)c * TILE_F] = v[c];
                 } else {
 #pragma unroll
-                    for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = v[c];
+                    for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[ch * CH + c] : v[c];
                     epi_bar();
-                    apply_epilogue(p, sAcc, sRed, ft, tok_base + ch * CH, row);
+                    apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
                     epi_bar();
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (p.splits > 1) {
-                // ticket: the CTA that completes the set sums the slices in split order
+            if (!un.full) {
+                // the tile is shared: ticket; the CTA that completes the set sums the pieces in CTA order
+                const long long x0 = (long long)un.tile * p.chunks_total;
+                const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
                 __threadfence();
                 epi_bar();
                 if (row == 0) {
-                    const int old = atomicAdd(p.counters + unit_tile, 1);
-                    flags[1] = (old == p.splits - 1) ? 1 : 0;
-                    if (old == p.splits - 1) p.counters[unit_tile] = 0;   // ready for the next launch
+                    const int old = atomicAdd(p.counters + un.tile, 1);
+                    flags[1] = (old == j1 - j0) ? 1 : 0;
+                    if (old == j1 - j0) p.counters[un.tile] = 0;   // ready for the next launch
                 }
                 epi_bar();
                 if (flags[1]) {
@@ -346,19 +484,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                         float acc[CH];
 #pragma unroll
                         for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                        for (int ss = 0; ss < p.splits; ++ss) {
-                            const float* src = p.part + (((size_t)unit_tile * p.splits + ss) * NT + ch * CH) * TILE_F + row;
+                        for (int j = j0; j <= j1; ++j) {
+                            // CTA j's piece of this tile is the first of its range iff its range starts inside the tile
+                            const int sl = ((long long)j * T / G >= x0) ? 0 : 1;
+                            const float* src = p.part + (((size_t)j * 2 + sl) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
                             for (int c = 0; c < CH; ++c) acc[c] += __ldcg(src + (size_t)c * TILE_F);
                         }
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = acc[c];
+                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[ch * CH + c] : acc[c];
                         epi_bar();
-                        apply_epilogue(p, sAcc, sRed, ft, tok_base + ch * CH, row);
+                        apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
                         epi_bar();
                     }
                 }
-                epi_bar();   // flags[1] is rewritten by the next unit
+                epi_bar();   // flags[1] is rewritten by the next piece
             }
         }
         if (flags[2] && row == 0) {
@@ -375,11 +515,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
 }
 
-// one CTA per token: merge the per-tile winners in tile order (index-aware, so order-independent)
+// one CTA per token: merge the per-tile winners (index-aware, so order-independent)
 __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __restrict__ top2, int n_tiles, int M,
                                                             int32_t* __restrict__ ids, float* __restrict__ top1,
                                                             float* __restrict__ margin) {
     __shared__ Top2Entry sh[4];
+    pdl_trigger();
+    pdl_wait();
     const int tok = blockIdx.x;
     T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
@@ -404,9 +546,37 @@ __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __r
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// host side
-// ---------------------------------------------------------------------------------------------
+// block row 0 of each sequence = anchor, rows 1.. = mask token; also the first layer's norm inputs
+__global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __restrict__ E,
+                                                         const int32_t* __restrict__ anchor, float* __restrict__ x,
+                                                         const __nv_bfloat16* __restrict__ g,
+                                                         __nv_bfloat16* __restrict__ xn, float* __restrict__ ssq, int B,
+                                                         int D, int V, int mask_id, int M, int32_t* status) {
+    pdl_trigger();
+    pdl_wait();
+    const int row = blockIdx.x, b = row / B, r = row % B;
+    int id = (r == 0) ? anchor[b] : mask_id;
+    if (id < 0 || id >= V) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_TOKEN);
+        id = 0;
+    }
+    const __nv_bfloat16* src = E + (size_t)id * D;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (D + 127) / 128;
+    for (int t = warp; t < n_tiles; t += (blockDim.x >> 5)) {
+        float s = 0.f;
+        for (int d = t * 128 + lane; d < min(D, (t + 1) * 128); d += 32) {
+            const float v = __bfloat162float(src[d]);
+            x[(size_t)row * D + d] = v;
+            xn[(size_t)row * D + d] = __float2bfloat16_rn(v * __bfloat162float(g[d]));
+            s += v * v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) ssq[(size_t)t * M + row] = s;
+    }
+}
+
 // [rows, K] bf16 row-major; box = 64 K-elements x box_rows rows
 bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)rows};
@@ -421,7 +591,7 @@ int pick_nt(int M) {
 }
 
 template <int NT>
-int launch_nt(const Launch& L, const CUtensorMap& tw, const CUtensorMap& tx, const KParams& p, int grid) {
+int launch_nt(const Launch& L, const WMaps& tw, const CUtensorMap& tx, const KParams& p, int grid) {
     static bool attr_set = false;
     const int smem = 1024 + p.stages * (W_STAGE_BYTES + NT * BK * 2) + SMEM_FIXED;
     if (!attr_set) {
@@ -429,43 +599,27 @@ int launch_nt(const Launch& L, const CUtensorMap& tw, const CUtensorMap& tx, con
             return DFLASH_ERR_CUDA;
         attr_set = true;
     }
-    gemm_tc_kernel<NT><<<grid, N_THREADS, smem, L.st>>>(tw, tx, p);
+    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, p);
     ++g_launches;
-    return cudaPeekAtLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 }  // namespace
 
-int gemm_tc_splits(int M, int N, int K, int sm_count) {
-    const int nt = pick_nt(M);
-    const int base = ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt);
-    const int chunks = (K + BK - 1) / BK;
-    if (base >= 4 * sm_count) return 1;   // enough units: the tail imbalance is already small
-    int best = 1;
-    double best_eff = 0.0;
-    for (int s = 1; s <= 16; ++s) {
-        const int cps = (chunks + s - 1) / s;
-        if (cps < 4 && s > 1) break;
-        if ((chunks + cps - 1) / cps != s) continue;   // would leave an empty split
-        const int units = base * s;
-        const int waves = (units + sm_count - 1) / sm_count;
-        const double eff = (double)units / ((double)waves * sm_count);
-        if (eff > best_eff + 0.03) { best_eff = eff; best = s; }
-    }
-    return best;
+// Grid: one CTA per SM unless the whole problem is so small that ranges would drop under 4 chunks.
+static int gemm_grid(int n_tiles, int chunks, int sm_count) {
+    const long long T = (long long)n_tiles * chunks;
+    return (int)std::max<long long>(1, std::min<long long>(sm_count, T / 4));
 }
 
-int64_t gemm_tc_part_bytes(int M, int N, int K, int sm_count) {
-    const int s = gemm_tc_splits(M, N, K, sm_count);
-    if (s == 1) return 0;
-    const int nt = pick_nt(M);
-    const int64_t tiles = (int64_t)((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt);
-    return tiles * s * nt * TILE_F * 4;
+int64_t gemm_tc_part_bytes(int M, int N, int K, int n_groups, int sm_count) {
+    (void)N; (void)K; (void)n_groups;
+    return (int64_t)sm_count * 2 * pick_nt(M) * TILE_F * 4;    // two partial pieces per CTA at most
 }
 
-int64_t gemm_tc_counter_bytes(int M, int N) {
+int64_t gemm_tc_counter_bytes(int M, int N, int n_groups) {
     const int nt = pick_nt(M);
-    return (int64_t)((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt) * 4;
+    return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt) * 4;
 }
 
 int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
@@ -473,16 +627,20 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
     if (a.K % 8 != 0) return DFLASH_ERR_UNSUPPORTED;
     const dflash_config& c = L.h->cfg;
     const int nt = pick_nt(a.M);
+    const int groups = std::max(a.n_groups, 1);
+    if (groups > GEMM_MAX_GROUPS) return DFLASH_ERR_UNSUPPORTED;
     KParams p{};
     p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epilogue;
+    p.n_groups = groups;
     p.n_ftiles = (a.N + TILE_F - 1) / TILE_F;
     p.n_ttiles = (a.M + nt - 1) / nt;
     p.chunks_total = (a.K + BK - 1) / BK;
-    p.splits = gemm_tc_splits(a.M, a.N, a.K, L.h->sm_count);
-    if (p.splits > 1 && (!a.part || !a.counters)) p.splits = 1;
-    p.chunks_per_split = (p.chunks_total + p.splits - 1) / p.splits;
+    p.n_tiles = groups * p.n_ftiles * p.n_ttiles;
+    if (!a.part || !a.counters) return DFLASH_ERR_INVALID_ARG;
     p.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - SMEM_FIXED) / (W_STAGE_BYTES + nt * BK * 2));
     p.part = a.part; p.counters = a.counters;
+    p.ssq_in = a.ssq_in; p.n_parts_in = (a.K + 127) / 128; p.inv_dim_in = 1.f / (float)a.K; p.eps = c.rms_eps;
+    p.g_next = (const __nv_bfloat16*)a.g_next; p.xn_out = a.xn_out; p.ssq_out = a.ssq_out;
     p.out_f32 = a.out_f32; p.ld_out = a.ld_out;
     p.q = a.q; p.k = a.k; p.v = a.v; p.ctx_len = a.ctx_len; p.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : 1;
     p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.hd = c.head_dim; p.use_rope = c.use_rope;
@@ -494,13 +652,16 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
         p.ctx_len = a.ctx->ctx_len;
         p.max_new = a.ctx->max_new; p.max_pages = a.ctx->max_pages; p.n_pages = a.ctx->n_pool_pages;
     }
-    p.PG = c.page_size; p.layer = a.layer;
+    p.PG = c.page_size; p.first_layer = a.first_layer;
     p.status = L.status;
 
-    CUtensorMap tw, tx;
-    if (!make_map(&tw, a.W, a.N, a.K, TILE_F) || !make_map(&tx, a.X, a.M, a.K, nt)) return DFLASH_ERR_CUDA;
-    const int units = p.n_ftiles * p.n_ttiles * p.splits;
-    const int grid = std::min(units, L.h->sm_count);
+    WMaps tw;
+    CUtensorMap tx;
+    for (int g = 0; g < groups; ++g)
+        if (!make_map(&tw.m[g], a.W[g], a.N, a.K, TILE_F)) return DFLASH_ERR_CUDA;
+    for (int g = groups; g < GEMM_MAX_GROUPS; ++g) tw.m[g] = tw.m[0];
+    if (!make_map(&tx, a.X, a.M, a.K, nt)) return DFLASH_ERR_CUDA;
+    const int grid = gemm_grid(p.n_tiles, p.chunks_total, L.h->sm_count);
     switch (nt) {
         case 16: return launch_nt<16>(L, tw, tx, p, grid);
         case 32: return launch_nt<32>(L, tw, tx, p, grid);
@@ -513,9 +674,21 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,
                          float* margin) {
     if (M <= 0) return DFLASH_OK;
-    argmax_finish_kernel<<<M, 128, 0, L.st>>>(top2, n_tiles, M, ids, top1, margin);
+    const cudaError_t e = launch_pdl(argmax_finish_kernel, dim3(M), dim3(128), 0, L.st, top2, n_tiles, M, ids, top1, margin);
     ++g_launches;
-    return cudaPeekAtLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, float* x, const void* g, __nv_bfloat16* xn,
+                      float* ssq) {
+    const dflash_config& c = L.h->cfg;
+    const int rows = batch * c.block_size;
+    if (rows <= 0) return DFLASH_OK;
+    const cudaError_t e = launch_pdl(embed_norm_kernel, dim3(rows), dim3(256), 0, L.st,
+                                     (const __nv_bfloat16*)L.h->w.embed, anchor, x, (const __nv_bfloat16*)g, xn, ssq,
+                                     c.block_size, c.d_model, c.vocab, c.mask_token_id, rows, L.status);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 }  // namespace dflash

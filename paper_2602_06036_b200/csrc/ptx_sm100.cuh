@@ -6,12 +6,33 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace dflash {
 
 // bf16 tensor map with 128-byte swizzle and zero fill outside the tensor. dims/box are listed
 // innermost first; strides_bytes has rank-1 entries (dimension 0 is contiguous).
 bool tmap_encode_bf16(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                       const uint32_t* box);
+
+// Launch with the programmatic-stream-serialization attribute: the grid may begin before its
+// predecessor in the stream has drained, and must call ptx::pdl_wait() before it touches anything
+// a predecessor writes.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 namespace ptx {
 
@@ -55,6 +76,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (clock64() - t0 > limit) return false;
     }
 }
+
+// Programmatic dependent launch: `pdl_wait` blocks until the grids this one depends on have
+// completed and their writes are visible (a no-op for a normally launched grid); `pdl_trigger`
+// lets the next grid in the stream start its own prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
