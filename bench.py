@@ -304,6 +304,7 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
@@ -352,6 +353,14 @@ def main():
 
     # per-kernel-family durations: a second pass of the same steps with event pairs around each launch
     prof = step.lib.profile(step.step_resident, args.steps) if hasattr(step.lib, "profile") else {}
+
+    if args.trace and rank == 0:
+        rows = step.lib.trace(step.step_resident)
+        with open(args.trace, "w") as f:
+            f.write("# kernel family, first CTA start, dependency resolved, main loop end, last CTA exit (us since first start)\n")
+            for fam, a, b, c, d in rows:
+                us = lambda v: "      -" if v is None else f"{v / 1e3:8.2f}"
+                f.write(f"{fam:16s} {us(a)} {us(b)} {us(c)} {us(d)}\n")
 
     if rank != 0:
         if dist_on:

@@ -236,6 +236,17 @@ int32_t dflash_profile_enable(dflash_handle* h, int32_t on);
 int32_t dflash_profile_read(dflash_handle* h, float* ms /*[host]*/, int32_t* launches /*[host]*/);
 const char* dflash_family_name(int32_t family);
 
+/* ---- device-side timeline (off by default) ----
+ * While a trace buffer is set, every tensor-core kernel the library launches records four device
+ * timestamps (nanoseconds of the GPU's global timer) into the next 4-word record of `dev_buf`:
+ *   [0] ~(earliest CTA start)   [1] ~(earliest moment a CTA saw its grid dependency resolved)
+ *   [2] latest end of a CTA's main loop   [3] latest CTA exit
+ * (the first two are stored complemented so that every word is a running maximum and the caller
+ * only has to zero the buffer). dflash_trace_read returns, per record written since the last read,
+ * the kernel family that wrote it, and rewinds. Passing NULL switches tracing off. */
+int32_t dflash_trace_enable(dflash_handle* h, uint64_t* dev_buf /*[device]*/, int32_t capacity_records);
+int32_t dflash_trace_read(dflash_handle* h, int32_t* families /*[host] capacity entries*/, int32_t* n_records /*[host]*/);
+
 /* Static description of a return code. */
 const char* dflash_status_string(int32_t code);
 

@@ -26,7 +26,7 @@ EXPORTS = (
     "dflash_create", "dflash_destroy", "dflash_set_weights", "dflash_workspace_bytes",
     "dflash_ctx_project", "dflash_draft_block", "dflash_verify_accept", "dflash_block_attention",
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
-    "dflash_profile_read", "dflash_family_name",
+    "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
 )
 N_FAMILIES = 14
 
@@ -118,6 +118,10 @@ def load():
     lib.dflash_profile_enable.restype = C.c_int32
     lib.dflash_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.dflash_profile_read.restype = C.c_int32
+    lib.dflash_trace_enable.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+    lib.dflash_trace_enable.restype = C.c_int32
+    lib.dflash_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.dflash_trace_read.restype = C.c_int32
     lib.dflash_family_name.argtypes = [C.c_int32]
     lib.dflash_family_name.restype = C.c_char_p
     _lib = lib
@@ -226,6 +230,34 @@ class DFlash:
             if n[f]:
                 out[self.lib.dflash_family_name(f).decode()] = (1e3 * ms[f] / n[f], n[f] / steps)
         return out
+
+    def trace(self, fn, capacity: int = 256):
+        """Run `fn` once with the device-side timeline on. Returns a list of
+        (family, start_ns, dependency_resolved_ns, main_loop_end_ns, end_ns) relative to the first start."""
+        buf = torch.zeros(capacity * 4, dtype=torch.int64, device=self.device)
+        _check(self.lib.dflash_trace_enable(self.h, C.c_void_p(buf.data_ptr()), capacity))
+        try:
+            fn()
+            torch.cuda.synchronize()
+            fam = (C.c_int32 * capacity)()
+            n = C.c_int32()
+            _check(self.lib.dflash_trace_read(self.h, fam, C.byref(n)))
+        finally:
+            self.lib.dflash_trace_enable(self.h, None, 0)
+        rec = buf.cpu().view(capacity, 4).tolist()
+        inv = lambda v: (~v) & 0xFFFFFFFFFFFFFFFF if v else 0
+        fix = lambda v: v & 0xFFFFFFFFFFFFFFFF
+        rows = []
+        for i in range(n.value):
+            r = rec[i]
+            if r[3] == 0 and r[0] == 0:
+                continue
+            rows.append((self.lib.dflash_family_name(fam[i]).decode(), inv(fix(r[0])), inv(fix(r[1])), fix(r[2]), fix(r[3])))
+        if not rows:
+            return rows
+        t0 = min(r[1] for r in rows if r[1])
+        return [(f, a - t0 if a else None, b - t0 if b else None, c - t0 if c else None, d - t0 if d else None)
+                for f, a, b, c, d in rows]
 
     # ---- the path -----------------------------------------------------------------------
     def dflash_ctx_project(self, feats, n_new, ctx_len, page_table, kv_pool, stream=None):

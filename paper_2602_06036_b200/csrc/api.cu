@@ -96,6 +96,17 @@ static void prof_end(const Launch& L) {
     ++h->prof_used;
 }
 
+// next timeline record (attention takes two: main kernel + combine)
+static unsigned long long* trace_slot(dflash_handle* h, int fam) {
+    if (!h->trace_buf) return nullptr;
+    const int n = fam == FAM_ATTENTION ? 2 : 1;
+    if (h->trace_used + n > h->trace_cap) return nullptr;
+    unsigned long long* r = h->trace_buf + (size_t)h->trace_used * 4;
+    for (int i = 0; i < n; ++i) h->trace_fam[h->trace_used + i] = fam;
+    h->trace_used += n;
+    return r;
+}
+
 #define DFLASH_TRY(expr)                    \
     do {                                    \
         int rc__ = (expr);                  \
@@ -104,6 +115,7 @@ static void prof_end(const Launch& L) {
 
 #define RUN(fam, expr)              \
     do {                            \
+        L.trace = trace_slot(L.h, fam); \
         prof_begin(L, fam);         \
         int rc2__ = (expr);         \
         prof_end(L);                \
@@ -124,7 +136,7 @@ static int zero_counters(const Launch& L, const Workspace& ws) {
 
 // LM head + argmax over `rows` normalised rows z (config dtype)
 // (bf16 path: if ssq_in is given, z holds gain-scaled rows and the per-token rsqrt is applied inside)
-static int lmhead_rows(const Launch& L, const Workspace& ws, const void* z, const float* ssq_in, int rows, int32_t* ids,
+static int lmhead_rows(Launch& L, const Workspace& ws, const void* z, const float* ssq_in, int rows, int32_t* ids,
                        float* top1, float* margin, float* logits_out) {
     const dflash_config& c = L.h->cfg;
     if (c.dtype == DFLASH_BF16) {
@@ -193,6 +205,9 @@ int32_t dflash_create(const dflash_config* cfg, dflash_handle** out) {
     h->prof_on = false;
     h->prof = nullptr;
     h->prof_cap = h->prof_used = 0;
+    h->trace_buf = nullptr;
+    h->trace_cap = h->trace_used = 0;
+    h->trace_fam = nullptr;
     *out = h;
     return DFLASH_OK;
 }
@@ -204,6 +219,7 @@ void dflash_destroy(dflash_handle* h) {
         cudaEventDestroy(h->prof[i].e1);
     }
     delete[] h->prof;
+    delete[] h->trace_fam;
     delete h;
 }
 
@@ -223,6 +239,29 @@ int32_t dflash_profile_read(dflash_handle* h, float* ms, int32_t* launches) {
         launches[h->prof[i].family] += 1;
     }
     h->prof_used = 0;
+    return DFLASH_OK;
+}
+
+int32_t dflash_trace_enable(dflash_handle* h, uint64_t* dev_buf, int32_t capacity_records) {
+    if (!h || capacity_records < 0) return DFLASH_ERR_INVALID_ARG;
+    delete[] h->trace_fam;
+    h->trace_fam = nullptr;
+    h->trace_buf = nullptr;
+    h->trace_cap = h->trace_used = 0;
+    if (dev_buf && capacity_records > 0) {
+        h->trace_fam = new (std::nothrow) int[capacity_records];
+        if (!h->trace_fam) return DFLASH_ERR_INVALID_ARG;
+        h->trace_buf = reinterpret_cast<unsigned long long*>(dev_buf);
+        h->trace_cap = capacity_records;
+    }
+    return DFLASH_OK;
+}
+
+int32_t dflash_trace_read(dflash_handle* h, int32_t* families, int32_t* n_records) {
+    if (!h || !families || !n_records) return DFLASH_ERR_INVALID_ARG;
+    for (int i = 0; i < h->trace_used; ++i) families[i] = h->trace_fam[i];
+    *n_records = h->trace_used;
+    h->trace_used = 0;
     return DFLASH_OK;
 }
 
@@ -258,7 +297,7 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
     const dflash_config& c = h->cfg;
-    Launch L{h, (cudaStream_t)stream, a->dev_status};
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const int kdim = c.n_kv_heads * c.head_dim, feat = c.n_feat_layers * c.d_target;
     const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
@@ -303,7 +342,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     const int B = c.block_size, rows = a->batch * B;
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
-    Launch L{h, (cudaStream_t)stream, a->dev_status};
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const int qdim = c.n_q_heads * c.head_dim, kdim = c.n_kv_heads * c.head_dim;
     const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
@@ -380,7 +419,7 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
     if (a->batch == 0) return DFLASH_OK;
     if (!a->draft_ids || !a->ctx_len || !a->accept_len || !a->out_tokens || !a->bonus || !a->new_ctx_len)
         return DFLASH_ERR_INVALID_ARG;
-    Launch L{h, (cudaStream_t)stream, a->dev_status};
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const int rows = a->batch * (a->gamma + 1);
     if (a->mode == DFLASH_VERIFY_IDS) {
         if (!a->target_ids) return DFLASH_ERR_INVALID_ARG;
@@ -409,7 +448,7 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     if (a->batch == 0 || a->rows == 0) return DFLASH_OK;
     if (!a->q || !a->k_blk || !a->v_blk || !a->ctx_len || !a->page_table || !a->kv_pool || !a->out)
         return DFLASH_ERR_INVALID_ARG;
-    Launch L{h, (cudaStream_t)stream, a->dev_status};
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     if (attn_tc_supported(h->cfg, a->rows)) {
         Workspace ws;
         DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, a->batch * a->rows, &ws));
@@ -430,7 +469,7 @@ int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a, void
     if (a->n_rows > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, 1, a->n_rows, &ws));
-    Launch L{h, (cudaStream_t)stream, a->dev_status};
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const dflash_config& c = h->cfg;
     const bool f32in = a->hidden_is_f32 || c.dtype == DFLASH_F32;
     DFLASH_TRY(zero_counters(L, ws));

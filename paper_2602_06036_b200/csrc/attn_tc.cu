@@ -46,6 +46,7 @@ struct AParams {
     float* part;
     int32_t* counters;
     int32_t* status;
+    unsigned long long* trace;
 };
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
@@ -92,8 +93,10 @@ __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPool,
                const __grid_constant__ CUtensorMap tmKb, const __grid_constant__ CUtensorMap tmVb, const AParams p) {
     // ---- which work unit ----
+    if (threadIdx.x == 0) trace_min(p.trace, 0);
     pdl_trigger();
     pdl_wait();      // lengths, page table, q and the block's k/v come from earlier kernels
+    if (threadIdx.x == 0) trace_min(p.trace, 1);
     const int chunk = blockIdx.x % p.n_chunks;
     const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
     const int b = blockIdx.x / (p.n_chunks * p.Hkv);
@@ -366,13 +369,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    if (threadIdx.x == 0) trace_max(p.trace, 3);
 }
 
 // Merge of the per-range partials of one (sequence, kv head): one warp per query row, lanes over
 // head_dim, ranges visited in order. Sequences whose context fitted one range were already written.
 __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
+    unsigned long long* trace = p.trace ? p.trace + 4 : nullptr;   // the record after the main kernel's
+    if (threadIdx.x == 0) trace_min(trace, 0);
     pdl_trigger();
     pdl_wait();
+    if (threadIdx.x == 0) trace_min(trace, 1);
     const int rows_valid = min(128, p.R * p.group);
     const int row_blocks = (rows_valid + 3) / 4;
     const int bg = blockIdx.x / row_blocks;
@@ -406,6 +413,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     w2.x = pack_bf16(acc.x * inv, acc.y * inv);
     w2.y = pack_bf16(acc.z * inv, acc.w * inv);
     *reinterpret_cast<uint2*>(dst) = w2;
+    if (lane == 0) trace_max(trace, 3);
 }
 
 }  // namespace
@@ -445,7 +453,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
     p.ctx_len = a.ctx_len; p.page_table = a.page_table;
-    p.out = (__nv_bfloat16*)a.out; p.part = part; p.counters = counters; p.status = L.status;
+    p.out = (__nv_bfloat16*)a.out; p.part = part; p.counters = counters; p.status = L.status; p.trace = L.trace;
 
     CUtensorMap tq, tpool, tkb, tvb;
     {   // q as [S*R][Hkv][group][hd]

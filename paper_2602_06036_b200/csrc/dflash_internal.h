@@ -30,6 +30,10 @@ struct dflash_handle {
     bool prof_on;
     dflash_profile_rec* prof;
     int prof_cap, prof_used;
+    // optional device-side timeline
+    unsigned long long* trace_buf;
+    int trace_cap, trace_used;
+    int* trace_fam;
 };
 
 namespace dflash {
@@ -82,6 +86,7 @@ struct Launch {
     dflash_handle* h;
     cudaStream_t st;
     int32_t* status;
+    unsigned long long* trace;   // 4-word timeline record of the launch being issued, or nullptr
 };
 
 // ---- generic (any dtype) kernels: the whole fp32 path, and the small steps of the bf16 path ----

@@ -69,6 +69,7 @@ struct KParams {
     const int32_t* page_table;
     int max_new, max_pages, n_pages, PG, first_layer;
     int32_t* status;
+    unsigned long long* trace;
 };
 
 // One piece of a CTA's chunk range: chunks [c0, c1) of output tile `tile`.
@@ -305,6 +306,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 template <int NT>
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtensorMap tmX, const KParams p) {
+    if (threadIdx.x == 0) trace_min(p.trace, 0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int X_STAGE_BYTES = NT * BK * 2;
@@ -355,6 +357,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
                 }
             }
             pdl_wait();
+            trace_min(p.trace, 1);
             uint32_t it = 0;
             bool ok = true;
             for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok;) {
@@ -410,6 +413,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
                 }
                 if (ok) mma_commit(&acc_full[buf]);
             }
+            trace_max(p.trace, 2);
             if (!ok) {
                 flags[0] = 1;
                 if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
@@ -513,15 +517,18 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    if (threadIdx.x == 0) trace_max(p.trace, 3);
 }
 
 // one CTA per token: merge the per-tile winners (index-aware, so order-independent)
 __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __restrict__ top2, int n_tiles, int M,
                                                             int32_t* __restrict__ ids, float* __restrict__ top1,
-                                                            float* __restrict__ margin) {
+                                                            float* __restrict__ margin, unsigned long long* trace) {
     __shared__ Top2Entry sh[4];
+    if (threadIdx.x == 0) trace_min(trace, 0);
     pdl_trigger();
     pdl_wait();
+    if (threadIdx.x == 0) trace_min(trace, 1);
     const int tok = blockIdx.x;
     T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
@@ -543,6 +550,7 @@ __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __r
         ids[tok] = r.i1 == 0x7fffffff ? 0 : r.i1;
         if (top1) top1[tok] = r.v1;
         if (margin) margin[tok] = r.v1 - r.v2;
+        trace_max(trace, 3);
     }
 }
 
@@ -551,9 +559,12 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __
                                                          const int32_t* __restrict__ anchor, float* __restrict__ x,
                                                          const __nv_bfloat16* __restrict__ g,
                                                          __nv_bfloat16* __restrict__ xn, float* __restrict__ ssq, int B,
-                                                         int D, int V, int mask_id, int M, int32_t* status) {
+                                                         int D, int V, int mask_id, int M, int32_t* status,
+                                                         unsigned long long* trace) {
+    if (threadIdx.x == 0) trace_min(trace, 0);
     pdl_trigger();
     pdl_wait();
+    if (threadIdx.x == 0) trace_min(trace, 1);
     const int row = blockIdx.x, b = row / B, r = row % B;
     int id = (r == 0) ? anchor[b] : mask_id;
     if (id < 0 || id >= V) {
@@ -575,6 +586,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (lane == 0) ssq[(size_t)t * M + row] = s;
     }
+    if (threadIdx.x == 0) trace_max(trace, 3);
 }
 
 // [rows, K] bf16 row-major; box = 64 K-elements x box_rows rows
@@ -654,6 +666,7 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
     }
     p.PG = c.page_size; p.first_layer = a.first_layer;
     p.status = L.status;
+    p.trace = L.trace;
 
     WMaps tw;
     CUtensorMap tx;
@@ -674,7 +687,7 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,
                          float* margin) {
     if (M <= 0) return DFLASH_OK;
-    const cudaError_t e = launch_pdl(argmax_finish_kernel, dim3(M), dim3(128), 0, L.st, top2, n_tiles, M, ids, top1, margin);
+    const cudaError_t e = launch_pdl(argmax_finish_kernel, dim3(M), dim3(128), 0, L.st, top2, n_tiles, M, ids, top1, margin, L.trace);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
@@ -686,7 +699,7 @@ int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, float* 
     if (rows <= 0) return DFLASH_OK;
     const cudaError_t e = launch_pdl(embed_norm_kernel, dim3(rows), dim3(256), 0, L.st,
                                      (const __nv_bfloat16*)L.h->w.embed, anchor, x, (const __nv_bfloat16*)g, xn, ssq,
-                                     c.block_size, c.d_model, c.vocab, c.mask_token_id, rows, L.status);
+                                     c.block_size, c.d_model, c.vocab, c.mask_token_id, rows, L.status, L.trace);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
