@@ -231,7 +231,7 @@ int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a /*[ho
  * stream. dflash_profile_read synchronises on the last event, adds the elapsed milliseconds and the
  * launch counts per family into the two host arrays (DFLASH_N_FAMILIES entries each) and clears
  * the record. Event pairs cost a little time per launch: never time a step with profiling on. */
-#define DFLASH_N_FAMILIES 14
+#define DFLASH_N_FAMILIES 15
 int32_t dflash_profile_enable(dflash_handle* h, int32_t on);
 int32_t dflash_profile_read(dflash_handle* h, float* ms /*[host]*/, int32_t* launches /*[host]*/);
 const char* dflash_family_name(int32_t family);

@@ -28,7 +28,7 @@ EXPORTS = (
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
 )
-N_FAMILIES = 14
+N_FAMILIES = 15
 
 
 class Config(C.Structure):

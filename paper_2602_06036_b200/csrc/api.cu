@@ -34,25 +34,30 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     w.h = a.take(R * c.d_ffn * es);
     w.logits = (float*)a.take(tc ? 256 : std::min<int64_t>(R, LOGIT_ROWS) * c.vocab * 4);
     w.ids = (int32_t*)a.take(R * 4);
-    int64_t part = 0, counters = 256;
+    int64_t part = 0, counters = 0;
     if (tc) {
         const int M = (int)R, sm = h->sm_count;
         const int kv_groups = std::min(c.n_layers, GEMM_MAX_GROUPS);
-        const int shapes[7][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
-                                  {c.d_model, c.d_ffn, 1},         {c.d_model, feat, 1}, {2 * kdim, c.d_model, kv_groups},
-                                  {c.vocab, c.d_model, 1}};
-        for (auto& s : shapes) {
-            part = std::max(part, gemm_tc_part_bytes(M, s[0], s[1], s[2], sm));
-            counters = std::max(counters, gemm_tc_counter_bytes(M, s[0], s[2]));
+        // order = Workspace::CNT_* : every contraction shape has its own ticket range
+        const int shapes[Workspace::CNT_N][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
+                                                 {c.d_model, c.d_ffn, 1},         {c.vocab, c.d_model, 1}, {c.d_model, feat, 1},
+                                                 {2 * kdim, c.d_model, kv_groups}};
+        for (int i = 0; i < Workspace::CNT_N; ++i) {
+            part = std::max(part, gemm_tc_part_bytes(M, shapes[i][0], shapes[i][1], shapes[i][2], sm));
+            w.cnt_off[i] = (int)(counters / 4);
+            counters += align_up(gemm_tc_counter_bytes(M, shapes[i][0], shapes[i][2]), 256);
         }
     }
     w.part = (float*)a.take(std::max<int64_t>(part, 256));
-    // tickets of the contractions, then tickets of the attention splits: one memset clears both
-    const int64_t gemm_counters = align_up(counters, 256);
+    // one zeroing per call clears: tickets of the contractions, chain phase flags, attention tickets
+    const int64_t gemm_counters = std::max<int64_t>(counters, 256);
+    w.n_flag_sets = 2 * c.n_layers + 8;
+    const int64_t flag_bytes = tc ? align_up((int64_t)w.n_flag_sets * GEMM_MAX_PHASES * 4, 256) : 0;
     const int64_t attn_counters = tc ? align_up(attn_tc_counter_bytes(c, std::max(batch, 1)), 256) : 0;
-    w.counter_bytes = gemm_counters + attn_counters;
+    w.counter_bytes = gemm_counters + flag_bytes + attn_counters;
     w.counters = (int32_t*)a.take(w.counter_bytes);
-    w.attn_counters = w.counters ? (int32_t*)((char*)w.counters + gemm_counters) : nullptr;
+    w.flags = w.counters ? (int32_t*)((char*)w.counters + gemm_counters) : nullptr;
+    w.attn_counters = w.counters ? (int32_t*)((char*)w.counters + gemm_counters + flag_bytes) : nullptr;
     w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
     w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), h->sm_count) : 256);
     w.seg = (float4*)a.take(R * 64 * 16);
@@ -67,7 +72,7 @@ static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
 static const char* kFamilyNames[DFLASH_N_FAMILIES] = {
     "embed", "rmsnorm", "gemm_qkv", "attention", "gemm_o", "gemm_gateup", "gemm_down", "lmhead_argmax",
-    "argmax_finish", "row_argmax", "accept", "ctx_fuse", "ctx_kv", "misc"};
+    "argmax_finish", "row_argmax", "accept", "ctx_fuse", "ctx_kv", "misc", "gemm_chain"};
 
 // ---- per-launch event pairs -------------------------------------------------------------------
 static void prof_begin(const Launch& L, int fam) {
@@ -142,9 +147,9 @@ static int lmhead_rows(Launch& L, const Workspace& ws, const void* z, const floa
     if (c.dtype == DFLASH_BF16) {
         GemmArgs g{};
         g.X = z; g.W[0] = L.h->w.W_lm; g.M = rows; g.N = c.vocab; g.K = c.d_model;
-        g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters; g.ssq_in = ssq_in;
+        g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_LM]; g.ssq_in = ssq_in;
         g.top2 = (Top2Entry*)ws.top2; g.logits_out = logits_out;
-        RUN(FAM_LMHEAD, launch_gemm_tc(L, g));
+        RUN(FAM_LMHEAD, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * (ws.n_flag_sets - 1)));
         RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, ids, top1, margin));
         return DFLASH_OK;
     }
@@ -309,15 +314,18 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
         GemmArgs g{};
         g.X = a->feats; g.W[0] = h->w.W_c; g.M = rows; g.N = c.d_model; g.K = feat;
         g.epilogue = EPI_STORE_F32; g.g_next = h->w.g_c; g.xn_out = (__nv_bfloat16*)ws.u; g.ssq_out = ws.ssq;
-        g.part = ws.part; g.counters = ws.counters;
-        RUN(FAM_CTX_FUSE, launch_gemm_tc(L, g));
+        g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_FUSE];
+        int flag_set = 0;
+        RUN(FAM_CTX_FUSE, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
         for (int i0 = 0; i0 < c.n_layers; i0 += GEMM_MAX_GROUPS) {
             GemmArgs k{};
             k.n_groups = std::min(GEMM_MAX_GROUPS, c.n_layers - i0);
             for (int j = 0; j < k.n_groups; ++j) k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
             k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
-            k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part; k.counters = ws.counters;
-            RUN(FAM_CTX_KV, launch_gemm_tc(L, k));
+            k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part;
+            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV];
+            if (flag_set >= ws.n_flag_sets - 1) return DFLASH_ERR_UNSUPPORTED;
+            RUN(FAM_CTX_KV, launch_gemm_tc(L, k, ws.flags + GEMM_MAX_PHASES * flag_set++));
         }
         return DFLASH_OK;
     }
@@ -359,36 +367,75 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     if (tc) {
         // bf16: tensor-core contractions with the norms folded into their epilogues.
         // ws.u always holds bf16(gain * x) of the rows about to be projected, ws.ssq their sums of squares.
+        // Launches: embed | QKV_0 | attention_0 | [O_0, gate/up_0, down_0, QKV_1] | attention_1 | ... |
+        //           [O_last, gate/up_last, down_last, LM head] | argmax finish. Each [...] is one chained launch
+        //           that keeps the weight stream running across its phases.
         __nv_bfloat16* xn = (__nv_bfloat16*)ws.u;
-        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, ws.x, h->layers[0].g1, xn, ws.ssq));
-        for (int i = 0; i < c.n_layers; ++i) {
-            const dflash_layer_weights& lw = h->layers[i];
+        int flag_set = 0;
+        auto qkv_args = [&](int i) {
             GemmArgs g{};      // q,k,v = W_qkv RMSNorm(x), rotated
-            g.X = xn; g.W[0] = lw.W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model; g.ssq_in = ws.ssq;
+            g.X = xn; g.W[0] = h->layers[i].W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model; g.ssq_in = ws.ssq;
             g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
             g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
-            g.part = ws.part; g.counters = ws.counters;
-            RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g));
+            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV];
+            return g;
+        };
+        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, ws.x, h->layers[0].g1, xn, ws.ssq));
+        {
+            const GemmArgs g = qkv_args(0);
+            RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
+        }
+        for (int i = 0; i < c.n_layers; ++i) {
+            const dflash_layer_weights& lw = h->layers[i];
+            const bool last = i + 1 == c.n_layers;
             at.layer = i;
             if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
             else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
-            GemmArgs o{};      // x += W_o attn; emits the FFN norm inputs
+            GemmArgs ph[4];
+            int fam[4];
+            GemmArgs& o = ph[0];      // x += W_o attn; emits the FFN norm inputs
+            o = GemmArgs{};
             o.X = ws.attn; o.W[0] = lw.W_o; o.M = rows; o.N = c.d_model; o.K = qdim;
-            o.epilogue = EPI_RESIDUAL; o.out_f32 = ws.x; o.ld_out = c.d_model; o.part = ws.part; o.counters = ws.counters;
+            o.epilogue = EPI_RESIDUAL; o.out_f32 = ws.x; o.ld_out = c.d_model; o.part = ws.part;
+            o.counters = ws.counters + ws.cnt_off[Workspace::CNT_O];
             o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq;
-            RUN(FAM_GEMM_O, launch_gemm_tc(L, o));
-            GemmArgs u{};      // h = silu(W_gate u) * (W_up u)
+            fam[0] = FAM_GEMM_O;
+            GemmArgs& u = ph[1];      // h = silu(W_gate u) * (W_up u)
+            u = GemmArgs{};
             u.X = xn; u.W[0] = lw.W_gateup; u.M = rows; u.N = 2 * c.d_ffn; u.K = c.d_model; u.ssq_in = ws.ssq;
-            u.epilogue = EPI_SWIGLU; u.h = (__nv_bfloat16*)ws.h; u.part = ws.part; u.counters = ws.counters;
-            RUN(FAM_GEMM_GATEUP, launch_gemm_tc(L, u));
-            GemmArgs d{};      // x += W_down h; emits the next layer's (or the final) norm inputs
+            u.epilogue = EPI_SWIGLU; u.h = (__nv_bfloat16*)ws.h; u.part = ws.part;
+            u.counters = ws.counters + ws.cnt_off[Workspace::CNT_GATEUP];
+            fam[1] = FAM_GEMM_GATEUP;
+            GemmArgs& d = ph[2];      // x += W_down h; emits the next layer's (or the final) norm inputs
+            d = GemmArgs{};
             d.X = ws.h; d.W[0] = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
-            d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part; d.counters = ws.counters;
-            d.g_next = (i + 1 < c.n_layers) ? h->layers[i + 1].g1 : h->w.g_f; d.xn_out = xn; d.ssq_out = ws.ssq;
-            RUN(FAM_GEMM_DOWN, launch_gemm_tc(L, d));
+            d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part;
+            d.counters = ws.counters + ws.cnt_off[Workspace::CNT_DOWN];
+            d.g_next = last ? h->w.g_f : h->layers[i + 1].g1; d.xn_out = xn; d.ssq_out = ws.ssq;
+            fam[2] = FAM_GEMM_DOWN;
+            if (!last) {
+                ph[3] = qkv_args(i + 1);
+                fam[3] = FAM_GEMM_QKV;
+            } else {              // LM head on the final-normed rows, fused with the per-tile argmax
+                GemmArgs& g = ph[3];
+                g = GemmArgs{};
+                g.X = xn; g.W[0] = h->w.W_lm; g.M = rows; g.N = c.vocab; g.K = c.d_model; g.ssq_in = ws.ssq;
+                g.epilogue = EPI_ARGMAX; g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_LM];
+                g.top2 = (Top2Entry*)ws.top2; g.logits_out = a->logits_out;
+                fam[3] = FAM_LMHEAD;
+            }
+            unsigned long long* tr[4];
+            for (int k = 0; k < 4; ++k) tr[k] = trace_slot(h, fam[k]);
+            if (flag_set >= ws.n_flag_sets - 1) return DFLASH_ERR_UNSUPPORTED;
+            prof_begin(L, FAM_GEMM_CHAIN);
+            const int rc = launch_gemm_chain(L, ph, 4, ws.flags + GEMM_MAX_PHASES * flag_set++, tr);
+            prof_end(L);
+            if (rc != DFLASH_OK) return rc;
         }
+        RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, a->draft_ids,
+                                                    a->top1, a->margin));
         if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
-        return lmhead_rows(L, ws, xn, ws.ssq, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
+        return DFLASH_OK;
     }
 
     // fp32: CUDA-core kernels, one step per launch

@@ -11,9 +11,9 @@
 
 enum DflashFamily : int {
     FAM_EMBED = 0, FAM_RMSNORM, FAM_GEMM_QKV, FAM_ATTENTION, FAM_GEMM_O, FAM_GEMM_GATEUP, FAM_GEMM_DOWN,
-    FAM_LMHEAD, FAM_ARGMAX_FINISH, FAM_ROW_ARGMAX, FAM_ACCEPT, FAM_CTX_FUSE, FAM_CTX_KV, FAM_MISC,
+    FAM_LMHEAD, FAM_ARGMAX_FINISH, FAM_ROW_ARGMAX, FAM_ACCEPT, FAM_CTX_FUSE, FAM_CTX_KV, FAM_MISC, FAM_GEMM_CHAIN,
 };
-static_assert(FAM_MISC + 1 == DFLASH_N_FAMILIES, "family table out of step with the header");
+static_assert(FAM_GEMM_CHAIN + 1 == DFLASH_N_FAMILIES, "family table out of step with the header");
 
 struct dflash_profile_rec {
     cudaEvent_t e0, e1;
@@ -69,7 +69,11 @@ struct Workspace {
     float* logits;   // [min(rows, LOGIT_ROWS), V] fp32 (only the fp32 path stages logits)
     int32_t* ids;    // [rows]
     float* part;     // split-K partial sums of the tensor-core contractions
-    int32_t* counters;   // split-K tickets (zeroed at the start of each call)
+    enum { CNT_QKV = 0, CNT_O, CNT_GATEUP, CNT_DOWN, CNT_LM, CNT_FUSE, CNT_KV, CNT_N };
+    int32_t* counters;   // tickets of shared output tiles (zeroed at the start of each call)
+    int cnt_off[CNT_N];  // first ticket of each contraction shape (int32 units)
+    int32_t* flags;      // [n_flag_sets][4] phase-completion counters of chained launches
+    int n_flag_sets;
     int64_t counter_bytes;
     int32_t* attn_counters;   // split-KV tickets of the attention kernel (inside the same region)
     void* top2;      // [vocab tiles, rows] per-tile winners of the fused LM-head argmax

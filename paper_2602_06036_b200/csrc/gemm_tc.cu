@@ -12,6 +12,12 @@
 // bit-reproducible). RMSNorm never runs as a kernel of its own: epilogues that produce residual
 // rows also emit the gain-scaled bf16 operand and per-tile sums of squares, and the consuming
 // contraction scales its accumulator columns by the per-token rsqrt.
+// One launch runs a CHAIN of up to four such contractions ("phases": e.g. output projection ->
+// gate/up -> down -> next layer's QKV), each consuming what the previous one's epilogues wrote.
+// The producer warp never stops streaming WEIGHT tiles: only the activation tile of a ring slot
+// waits until every CTA has signalled the end of the previous phase (a counter in global memory,
+// polled with a bound), so the tail of one phase - partial sums, tickets, epilogues - overlaps the
+// weight stream of the next and HBM stays busy across the chain.
 // Launched with programmatic dependent launch: barrier set-up, TMEM allocation and the first ring
 // of WEIGHT tiles (which no earlier kernel writes) are issued before griddepcontrol.wait.
 // Every wait on an mbarrier is bounded; on expiry the kernel raises DFLASH_DEV_TIMEOUT, drains its
@@ -35,7 +41,7 @@ constexpr int CH = 16;                           // token columns handled per ep
 constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB
 constexpr int MAX_STAGES = 12;
 constexpr int ACC_LD = CH + 1;
-constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64;
+constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int N_THREADS = 192;
 
@@ -44,7 +50,7 @@ struct WMaps {
 };
 
 struct KParams {
-    int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, stages;
+    int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, w_map0, x_map;
     float* part;
     int32_t* counters;
     const float* ssq_in;
@@ -69,7 +75,19 @@ struct KParams {
     const int32_t* page_table;
     int max_new, max_pages, n_pages, PG, first_layer;
     int32_t* status;
-    unsigned long long* trace;
+    unsigned long long* trace;   // this phase's timeline record
+};
+
+constexpr int MAX_PHASES = 4;
+struct XMaps {
+    CUtensorMap m[MAX_PHASES];
+};
+// A launch = a chain of phases that share the token tile size and the ring.
+struct MParams {
+    int n_phases, stages;
+    int32_t* phase_done;         // [MAX_PHASES] CTAs that finished each phase (zero on entry)
+    int32_t* status;
+    KParams ph[MAX_PHASES];
 };
 
 // One piece of a CTA's chunk range: chunks [c0, c1) of output tile `tile`.
@@ -303,15 +321,22 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
+// Bounded poll of a global counter written by other CTAs (release/acquire through L2).
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 template <int NT>
 __global__ void __launch_bounds__(N_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtensorMap tmX, const KParams p) {
-    if (threadIdx.x == 0) trace_min(p.trace, 0);
+gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps tmX, const __grid_constant__ MParams mp) {
+    if (threadIdx.x == 0) trace_min(mp.ph[0].trace, 0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int X_STAGE_BYTES = NT * BK * 2;
     constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
-    const int stages = p.stages;
+    const int stages = mp.stages;
     uint8_t* sW = smem;
     uint8_t* sX = sW + (size_t)stages * W_STAGE_BYTES;
     float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE_BYTES);
@@ -323,6 +348,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] last-arriver, [2] epilogue abort
+    int* sPend = const_cast<int*>(flags) + 4;                               // [3 * MAX_STAGES] producer's queue
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -344,45 +370,87 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        // WEIGHT tiles are issued as soon as a ring slot is free. The ACTIVATION tile of a slot needs
+        // the phase's inputs (phase 0: the grid dependency; later phases: every CTA has finished the
+        // previous phase). While they are missing, the slot is queued and the weight stream goes on;
+        // queued slots are completed, in order, as soon as the inputs exist. In the steady state the
+        // queue is empty and both tiles are issued back to back.
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-            // Before the grid dependency is resolved: fill the ring with WEIGHT tiles only (weights
-            // are never written by a kernel). The matching activation tiles follow after the wait.
-            int n_pre = 0;
-            for (PieceWalk w(p, blockIdx.x, G); !w.done() && n_pre < stages;) {
-                const Unit un = w.next(p);
-                for (int c = un.c0; c < un.c1 && n_pre < stages; ++c, ++n_pre) {
-                    mbar_expect_tx(&full[n_pre], W_STAGE_BYTES + X_STAGE_BYTES);
-                    tma_load_2d(sW + (size_t)n_pre * W_STAGE_BYTES, &tmW.m[un.g], c * BK, un.ft * TILE_F, &full[n_pre], pol_w);
+            int* q_ph = sPend;                      // queued slots: phase, chunk, token tile (ring order)
+            int* q_c = sPend + MAX_STAGES;
+            int* q_tt = sPend + 2 * MAX_STAGES;
+            int q_head = 0, q_count = 0;            // q_head = ring slot of the oldest queued entry
+            int ready_ph = -1;                      // phases 0..ready_ph have their inputs
+            int st = 0;
+            uint32_t par = 0;
+            bool ok = true;
+            // completes queued slots while their phase is ready; returns false if the head still waits
+            auto flush = [&]() {
+                while (q_count > 0) {
+                    const int ph = q_ph[q_head];
+                    if (ph > ready_ph) {
+                        if (ph == 0) {
+                            pdl_wait();
+                            trace_min(mp.ph[0].trace, 1);
+                        } else {
+                            if (ld_acquire(mp.phase_done + ph - 1) < G) return;
+                            fence_proxy_async_all();      // other CTAs' stores -> this CTA's TMA reads
+                            trace_min(mp.ph[ph].trace, 0);
+                            trace_min(mp.ph[ph].trace, 1);
+                        }
+                        ready_ph = ph;
+                    }
+                    tma_load_2d(sX + (size_t)q_head * X_STAGE_BYTES, &tmX.m[mp.ph[ph].x_map], q_c[q_head] * BK, q_tt[q_head] * NT,
+                                &full[q_head], pol_x);
+                    q_head = (q_head + 1 == stages) ? 0 : q_head + 1;
+                    --q_count;
+                }
+            };
+            for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
+                const KParams& p = mp.ph[ph];
+                const CUtensorMap* xm = &tmX.m[p.x_map];
+                for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok;) {
+                    const Unit un = w.next(p);
+                    const CUtensorMap* wm = &tmW.m[p.w_map0 + un.g];
+                    const int y_w = un.ft * TILE_F, y_x = un.tt * NT;
+                    for (int c = un.c0; c < un.c1; ++c) {
+                        if (!mbar_try_wait(&empty[st], par ^ 1)) {
+                            const long long t0 = clock64();
+                            while (!mbar_try_wait(&empty[st], par ^ 1)) {
+                                flush();                  // a full ring of queued slots frees nothing by itself
+                                if (flags[0] || clock64() - t0 > SPIN_LIMIT) { ok = false; break; }
+                            }
+                            if (!ok) break;
+                        }
+                        mbar_expect_tx(&full[st], W_STAGE_BYTES + X_STAGE_BYTES);
+                        tma_load_2d(sW + (size_t)st * W_STAGE_BYTES, wm, c * BK, y_w, &full[st], pol_w);
+                        if (q_count == 0 && ph <= ready_ph) {
+                            tma_load_2d(sX + (size_t)st * X_STAGE_BYTES, xm, c * BK, y_x, &full[st], pol_x);
+                        } else {
+                            if (q_count == 0) q_head = st;
+                            q_ph[st] = ph; q_c[st] = c; q_tt[st] = un.tt;
+                            ++q_count;
+                            flush();
+                        }
+                        if (++st == stages) { st = 0; par ^= 1; }
+                    }
                 }
             }
-            pdl_wait();
-            trace_min(p.trace, 1);
-            uint32_t it = 0;
-            bool ok = true;
-            for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok;) {
-                const Unit un = w.next(p);
-                for (int c = un.c0; c < un.c1; ++c, ++it) {
-                    const int st = it % stages;
-                    const uint32_t ph = (it / stages) & 1;
-                    if ((int)it >= n_pre) {
-                        if (!mbar_wait(&empty[st], ph ^ 1, &flags[0])) { ok = false; break; }
-                        mbar_expect_tx(&full[st], W_STAGE_BYTES + X_STAGE_BYTES);
-                        tma_load_2d(sW + (size_t)st * W_STAGE_BYTES, &tmW.m[un.g], c * BK, un.ft * TILE_F, &full[st], pol_w);
-                    }
-                    tma_load_2d(sX + (size_t)st * X_STAGE_BYTES, &tmX, c * BK, un.tt * NT, &full[st], pol_x);
+            if (ok && q_count > 0) {
+                const long long t0 = clock64();
+                while (q_count > 0) {
+                    flush();
+                    if (flags[0] || clock64() - t0 > SPIN_LIMIT) { ok = false; break; }
                 }
             }
             if (!ok) {
                 flags[0] = 1;
-                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
-                // give copies already issued a chance to land before the CTA goes away
-                const int n_out = min((int)it, stages);
-                for (int j = 0; j < n_out; ++j) {
-                    const uint32_t jt = it - 1 - j;
-                    volatile int never = 0;
-                    mbar_wait(&full[jt % stages], (jt / stages) & 1, &never, DRAIN_LIMIT);
-                }
+                if (mp.status) atomicOr(mp.status, DFLASH_DEV_TIMEOUT);
+                // weight tiles already in flight must land before the CTA goes away; their barriers
+                // never complete without the activation tile, so wait on time instead
+                const long long t0 = clock64();
+                while (clock64() - t0 < DRAIN_LIMIT) {}
             }
         }
         __syncwarp();     // the whole warp must reach the closing barrier together
@@ -392,31 +460,34 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
             constexpr uint32_t idesc = instr_desc_bf16(TILE_F, NT);
             uint32_t it = 0, ui = 0;
             bool ok = true;
-            for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok; ++ui) {
-                const Unit un = w.next(p);
-                const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
-                if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * NT;
-                for (int c = un.c0; c < un.c1; ++c, ++it) {
-                    const int st = it % stages;
-                    const uint32_t ph = (it / stages) & 1;
-                    if (!mbar_wait(&full[st], ph, &flags[0])) { ok = false; break; }
+            for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
+                const KParams& p = mp.ph[ph];
+                for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok; ++ui) {
+                    const Unit un = w.next(p);
+                    const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
+                    if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(sW + (size_t)st * W_STAGE_BYTES);
-                    const uint32_t b_addr = smem_u32(sX + (size_t)st * X_STAGE_BYTES);
+                    const uint32_t d_tmem = tmem_base + buf * NT;
+                    for (int c = un.c0; c < un.c1; ++c, ++it) {
+                        const int st = it % stages;
+                        const uint32_t phs = (it / stages) & 1;
+                        if (!mbar_wait(&full[st], phs, &flags[0])) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = smem_u32(sW + (size_t)st * W_STAGE_BYTES);
+                        const uint32_t b_addr = smem_u32(sX + (size_t)st * X_STAGE_BYTES);
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        mma_bf16(d_tmem, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32), idesc,
-                                 (c > un.c0 || kk > 0) ? 1u : 0u);
-                    mma_commit(&empty[st]);
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            mma_bf16(d_tmem, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32), idesc,
+                                     (c > un.c0 || kk > 0) ? 1u : 0u);
+                        mma_commit(&empty[st]);
+                    }
+                    if (ok) mma_commit(&acc_full[buf]);
                 }
-                if (ok) mma_commit(&acc_full[buf]);
+                trace_max(p.trace, 2);
             }
-            trace_max(p.trace, 2);
             if (!ok) {
                 flags[0] = 1;
-                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+                if (mp.status) atomicOr(mp.status, DFLASH_DEV_TIMEOUT);
             }
         }
         __syncwarp();
@@ -424,90 +495,117 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
         // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
         const int ew = warp & 3;
         const int row = ew * 32 + lane;
-        const long long T = (long long)p.n_tiles * p.chunks_total;
-        pdl_wait();
         uint32_t ui = 0;
-        int rstd_tt = -1;
-        for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
-            const Unit un = w.next(p);
-            const int tok_base = un.tt * NT;
-            // per-token rsqrt(mean square) of the operand rows, once per token tile
-            if (p.ssq_in && rstd_tt != un.tt) {
-                for (int t = row; t < NT; t += 128) {
-                    float rs = 1.f;
-                    if (tok_base + t < p.M) {
-                        float s = 0.f;
-                        for (int q = 0; q < p.n_parts_in; ++q) s += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
-                        rs = rsqrtf(s * p.inv_dim_in + p.eps);
-                    }
-                    sRstd[t] = rs;
-                }
-                rstd_tt = un.tt;
-                // made visible by the barrier below
-            }
-            const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
-            const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
-            if (!got) flags[2] = 1;
-            epi_bar();
-            if (flags[2]) break;   // uniform over the four warps
-            tc_fence_after();
-            const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
-            for (int ch = 0; ch < n_ch; ++ch) {
-                float v[CH];
-                tmem_ld16(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
-                if (!un.full) {
-                    float* dst = p.part + (((size_t)blockIdx.x * 2 + un.slot) * NT + ch * CH) * TILE_F + row;
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) dst[(size_t)c * TILE_F] = v[c];
-                } else {
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[ch * CH + c] : v[c];
-                    epi_bar();
-                    apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
-                    epi_bar();
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (!un.full) {
-                // the tile is shared: ticket; the CTA that completes the set sums the pieces in CTA order
-                const long long x0 = (long long)un.tile * p.chunks_total;
-                const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
-                __threadfence();
+        bool alive = true;
+        for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
+            const KParams& p = mp.ph[ph];
+            const long long T = (long long)p.n_tiles * p.chunks_total;
+            int rstd_tt = -1;
+            for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
+                const Unit un = w.next(p);
+                const int tok_base = un.tt * NT;
+                const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
+                const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
+                if (!got) flags[2] = 1;
                 epi_bar();
-                if (row == 0) {
-                    const int old = atomicAdd(p.counters + un.tile, 1);
-                    flags[1] = (old == j1 - j0) ? 1 : 0;
-                    if (old == j1 - j0) p.counters[un.tile] = 0;   // ready for the next launch
-                }
-                epi_bar();
-                if (flags[1]) {
-                    __threadfence();
-                    for (int ch = 0; ch < n_ch; ++ch) {
-                        float acc[CH];
-#pragma unroll
-                        for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                        for (int j = j0; j <= j1; ++j) {
-                            // CTA j's piece of this tile is the first of its range iff its range starts inside the tile
-                            const int sl = ((long long)j * T / G >= x0) ? 0 : 1;
-                            const float* src = p.part + (((size_t)j * 2 + sl) * NT + ch * CH) * TILE_F + row;
-#pragma unroll
-                            for (int c = 0; c < CH; ++c) acc[c] += __ldcg(src + (size_t)c * TILE_F);
+                if (flags[2]) { alive = false; break; }   // uniform over the four warps
+                tc_fence_after();
+                // The accumulator exists, so this phase's inputs do too (phase 0: wait for the grid
+                // dependency explicitly, the producer may be the only thread that did).
+                if (ph == 0 && ui == 0) pdl_wait();
+                // per-token rsqrt(mean square) of the operand rows, once per token tile
+                if (p.ssq_in && rstd_tt != un.tt) {
+                    for (int t = row; t < NT; t += 128) {
+                        float rs = 1.f;
+                        if (tok_base + t < p.M) {
+                            float s = 0.f;
+                            for (int q = 0; q < p.n_parts_in; ++q) s += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
+                            rs = rsqrtf(s * p.inv_dim_in + p.eps);
                         }
+                        sRstd[t] = rs;
+                    }
+                    rstd_tt = un.tt;
+                    epi_bar();
+                }
+                const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
+                for (int ch = 0; ch < n_ch; ++ch) {
+                    float v[CH];
+                    tmem_ld16(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
+                    if (!un.full) {
+                        float* dst = p.part + (((size_t)blockIdx.x * 2 + un.slot) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[ch * CH + c] : acc[c];
+                        for (int c = 0; c < CH; ++c) dst[(size_t)c * TILE_F] = v[c];
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[ch * CH + c] : v[c];
                         epi_bar();
                         apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
                         epi_bar();
                     }
                 }
-                epi_bar();   // flags[1] is rewritten by the next piece
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (!un.full) {
+                    // the tile is shared: ticket; the CTA that completes the set sums the pieces in CTA order
+                    const long long x0 = (long long)un.tile * p.chunks_total;
+                    const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
+                    __threadfence();
+                    epi_bar();
+                    if (row == 0) {
+                        const int old = atomicAdd(p.counters + un.tile, 1);
+                        flags[1] = (old == j1 - j0) ? 1 : 0;
+                        if (old == j1 - j0) p.counters[un.tile] = 0;   // ready for the next launch
+                    }
+                    epi_bar();
+                    if (flags[1]) {
+                        __threadfence();
+                        for (int ch = 0; ch < n_ch; ++ch) {
+                            float acc[CH];
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) acc[c] = 0.f;
+                            // pieces are summed in CTA order; two are fetched at a time so their
+                            // loads overlap
+                            int j = j0;
+                            for (; j + 1 <= j1; j += 2) {
+                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
+                                const int sb = ((long long)(j + 1) * T / G >= x0) ? 0 : 1;
+                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+                                const float* pb = p.part + (((size_t)(j + 1) * 2 + sb) * NT + ch * CH) * TILE_F + row;
+                                float va[CH], vb[CH];
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) { va[c] = __ldcg(pa + (size_t)c * TILE_F); vb[c] = __ldcg(pb + (size_t)c * TILE_F); }
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) acc[c] = (acc[c] + va[c]) + vb[c];
+                            }
+                            if (j <= j1) {
+                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
+                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) acc[c] += __ldcg(pa + (size_t)c * TILE_F);
+                            }
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[ch * CH + c] : acc[c];
+                            epi_bar();
+                            apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
+                            epi_bar();
+                        }
+                    }
+                    epi_bar();   // flags[1] is rewritten by the next piece
+                }
+            }
+            if (!alive) break;
+            // this CTA's share of the phase is done and visible: tell the others
+            __threadfence();
+            epi_bar();
+            if (row == 0) {
+                trace_max(p.trace, 3);
+                atomicAdd(mp.phase_done + ph, 1);
             }
         }
         if (flags[2] && row == 0) {
             flags[0] = 1;
-            if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+            if (mp.status) atomicOr(mp.status, DFLASH_DEV_TIMEOUT);
         }
     }
 
@@ -517,7 +615,6 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ CUtens
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
-    if (threadIdx.x == 0) trace_max(p.trace, 3);
 }
 
 // one CTA per token: merge the per-tile winners (index-aware, so order-independent)
@@ -603,26 +700,20 @@ int pick_nt(int M) {
 }
 
 template <int NT>
-int launch_nt(const Launch& L, const WMaps& tw, const CUtensorMap& tx, const KParams& p, int grid) {
+int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
     static bool attr_set = false;
-    const int smem = 1024 + p.stages * (W_STAGE_BYTES + NT * BK * 2) + SMEM_FIXED;
+    const int smem = 1024 + mp.stages * (W_STAGE_BYTES + NT * BK * 2) + SMEM_FIXED;
     if (!attr_set) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         attr_set = true;
     }
-    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, p);
+    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 }  // namespace
-
-// Grid: one CTA per SM unless the whole problem is so small that ranges would drop under 4 chunks.
-static int gemm_grid(int n_tiles, int chunks, int sm_count) {
-    const long long T = (long long)n_tiles * chunks;
-    return (int)std::max<long long>(1, std::min<long long>(sm_count, T / 4));
-}
 
 int64_t gemm_tc_part_bytes(int M, int N, int K, int n_groups, int sm_count) {
     (void)N; (void)K; (void)n_groups;
@@ -634,14 +725,11 @@ int64_t gemm_tc_counter_bytes(int M, int N, int n_groups) {
     return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt) * 4;
 }
 
-int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
-    if (a.M <= 0 || a.N <= 0) return DFLASH_OK;
+static int fill_phase(const Launch& L, const GemmArgs& a, int nt, KParams& p) {
     if (a.K % 8 != 0) return DFLASH_ERR_UNSUPPORTED;
     const dflash_config& c = L.h->cfg;
-    const int nt = pick_nt(a.M);
     const int groups = std::max(a.n_groups, 1);
-    if (groups > GEMM_MAX_GROUPS) return DFLASH_ERR_UNSUPPORTED;
-    KParams p{};
+    p = KParams{};
     p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epilogue;
     p.n_groups = groups;
     p.n_ftiles = (a.N + TILE_F - 1) / TILE_F;
@@ -649,7 +737,6 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
     p.chunks_total = (a.K + BK - 1) / BK;
     p.n_tiles = groups * p.n_ftiles * p.n_ttiles;
     if (!a.part || !a.counters) return DFLASH_ERR_INVALID_ARG;
-    p.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - SMEM_FIXED) / (W_STAGE_BYTES + nt * BK * 2));
     p.part = a.part; p.counters = a.counters;
     p.ssq_in = a.ssq_in; p.n_parts_in = (a.K + 127) / 128; p.inv_dim_in = 1.f / (float)a.K; p.eps = c.rms_eps;
     p.g_next = (const __nv_bfloat16*)a.g_next; p.xn_out = a.xn_out; p.ssq_out = a.ssq_out;
@@ -666,22 +753,58 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a) {
     }
     p.PG = c.page_size; p.first_layer = a.first_layer;
     p.status = L.status;
-    p.trace = L.trace;
+    return DFLASH_OK;
+}
 
+int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int32_t* phase_done,
+                      unsigned long long* const* traces) {
+    if (n_phases < 1 || n_phases > MAX_PHASES) return DFLASH_ERR_INVALID_ARG;
+    const int M = phases[0].M;
+    if (M <= 0) return DFLASH_OK;
+    const int nt = pick_nt(M);
+    MParams mp{};
     WMaps tw;
-    CUtensorMap tx;
-    for (int g = 0; g < groups; ++g)
-        if (!make_map(&tw.m[g], a.W[g], a.N, a.K, TILE_F)) return DFLASH_ERR_CUDA;
-    for (int g = groups; g < GEMM_MAX_GROUPS; ++g) tw.m[g] = tw.m[0];
-    if (!make_map(&tx, a.X, a.M, a.K, nt)) return DFLASH_ERR_CUDA;
-    const int grid = gemm_grid(p.n_tiles, p.chunks_total, L.h->sm_count);
-    switch (nt) {
-        case 16: return launch_nt<16>(L, tw, tx, p, grid);
-        case 32: return launch_nt<32>(L, tw, tx, p, grid);
-        case 64: return launch_nt<64>(L, tw, tx, p, grid);
-        case 128: return launch_nt<128>(L, tw, tx, p, grid);
-        default: return launch_nt<256>(L, tw, tx, p, grid);
+    XMaps tx;
+    mp.n_phases = n_phases;
+    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - SMEM_FIXED) / (W_STAGE_BYTES + nt * BK * 2));
+    mp.phase_done = phase_done;
+    mp.status = L.status;
+
+    int n_maps = 0;
+    long long min_pairs = -1;
+    for (int i = 0; i < n_phases; ++i) {
+        const GemmArgs& a = phases[i];
+        if (a.M != M || a.N <= 0) return DFLASH_ERR_INVALID_ARG;
+        const int rc = fill_phase(L, a, nt, mp.ph[i]);
+        if (rc != DFLASH_OK) return rc;
+        KParams& p = mp.ph[i];
+        p.trace = traces ? traces[i] : nullptr;
+        if (n_maps + p.n_groups > GEMM_MAX_GROUPS) return DFLASH_ERR_UNSUPPORTED;
+        p.w_map0 = n_maps;
+        for (int g = 0; g < p.n_groups; ++g)
+            if (!make_map(&tw.m[n_maps++], a.W[g], a.N, a.K, TILE_F)) return DFLASH_ERR_CUDA;
+        p.x_map = i;
+        if (!make_map(&tx.m[i], a.X, a.M, a.K, nt)) return DFLASH_ERR_CUDA;
+        const long long pairs = (long long)p.n_tiles * p.chunks_total;
+        min_pairs = min_pairs < 0 ? pairs : std::min(min_pairs, pairs);
     }
+    for (int g = n_maps; g < GEMM_MAX_GROUPS; ++g) tw.m[g] = tw.m[0];
+    for (int i = n_phases; i < MAX_PHASES; ++i) tx.m[i] = tx.m[0];
+    // one CTA per SM unless the smallest phase would leave ranges under 4 chunks
+    const int grid = (int)std::max<long long>(1, std::min<long long>(L.h->sm_count, min_pairs / 4));
+    switch (nt) {
+        case 16: return launch_nt<16>(L, tw, tx, mp, grid);
+        case 32: return launch_nt<32>(L, tw, tx, mp, grid);
+        case 64: return launch_nt<64>(L, tw, tx, mp, grid);
+        case 128: return launch_nt<128>(L, tw, tx, mp, grid);
+        default: return launch_nt<256>(L, tw, tx, mp, grid);
+    }
+}
+
+int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done) {
+    if (a.M <= 0 || a.N <= 0) return DFLASH_OK;
+    unsigned long long* tr[1] = {L.trace};
+    return launch_gemm_chain(L, &a, 1, phase_done, tr);
 }
 
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,
