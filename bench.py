@@ -206,6 +206,13 @@ def capture(fn):
     return g.replay
 
 
+def max_over_ranks(ms, device):
+    """The slowest rank's time (replicas run independently; the job is as slow as its slowest rank)."""
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
 def timed(fn, steps, warmup, dist_on):
     for _ in range(warmup):
         fn()
@@ -221,9 +228,7 @@ def timed(fn, steps, warmup, dist_on):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     if dist_on:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+        ms = max_over_ranks(ms, "cuda")
     return ms
 
 
@@ -231,19 +236,19 @@ def timed(fn, steps, warmup, dist_on):
 # CPU oracle arm
 # ------------------------------------------------------------------------------------------------
 def oracle_sample(wl, seed=0, layers=1, vocab_frac=8):
-    """A bounded sample of one step for the CPU oracle: the context projection of the step's rows,
-    `layers` of the N draft layers over the full context, and the LM head over V/vocab_frac rows.
-    Returns (seconds, fraction of the step's algorithmic bytes covered, threads)."""
+    """A bounded sample of one step for the CPU oracle, one sequence: the context projection of the
+    step's rows, `layers` of the N draft layers over the full context, the LM head over
+    V/vocab_frac rows, and the accept rule on full-vocabulary logits.
+    Returns (seconds, fraction of the step's algorithmic bytes covered)."""
     from oracle import dflash_oracle as orc
     import dataclasses
     cfg = wl.cfg
-    sub = dataclasses.replace(cfg, n_layers=layers)
+    layers = min(layers, cfg.n_layers)
     B = cfg.block_size
     Vs = max(cfg.vocab // vocab_frac, 2)
-    rng_w = synth.make_weights(dataclasses.replace(sub, vocab=Vs), seed)
-    w = synth.weights_to_numpy(rng_w)
-    b = 0
-    L = wl.ctx_lens[b]
+    sub_v = dataclasses.replace(cfg, n_layers=layers, vocab=Vs)
+    w = synth.weights_to_numpy(synth.make_weights(sub_v, seed))
+    L = wl.ctx_lens[0]
     ctxK = [synth.to_numpy_f32(synth.normal((L, cfg.n_kv_heads, cfg.head_dim), 1.0, seed, f"o.K{i}", cfg.torch_dtype))
             for i in range(layers)]
     ctxV = [synth.to_numpy_f32(synth.normal((L, cfg.n_kv_heads, cfg.head_dim), 1.0, seed, f"o.V{i}", cfg.torch_dtype))
@@ -251,7 +256,6 @@ def oracle_sample(wl, seed=0, layers=1, vocab_frac=8):
     feats = synth.to_numpy_f32(synth.make_features(cfg, B + 1, seed, "o.feats"))
     logits, drafts, _ = synth.make_verify_case(1, B, cfg.vocab, wl.accept_p, seed, cfg.torch_dtype)
     lg = synth.to_numpy_f32(logits[0])
-    sub_v = dataclasses.replace(sub, vocab=Vs)
     t0 = time.perf_counter()
     orc.ctx_project(feats, L + np.arange(B + 1), w, sub_v)
     orc.draft_block(3, L, ctxK, ctxV, w, sub_v)
@@ -263,7 +267,7 @@ def oracle_sample(wl, seed=0, layers=1, vocab_frac=8):
     covered = layers * per_layer + full["lmhead_argmax"] / cfg.vocab * Vs + \
         (cfg.d_model * cfg.feat_dim + layers * 2 * cfg.kv_dim * cfg.d_model) * es
     total = full["draft_block_total"] + full["ctx_project_total"]
-    return dt, covered / total, (os.cpu_count() or 1)
+    return dt, min(covered / total, 1.0)
 
 
 def run_reference(args):
@@ -276,7 +280,7 @@ def run_reference(args):
     times = []
     frac = 1.0
     for i in range(args.warmup + args.steps):
-        dt, frac, _ = oracle_sample(wl)
+        dt, frac = oracle_sample(wl)
         if i >= args.warmup:
             times.append(dt)
     per_step = statistics.mean(times) / frac            # extrapolated to the whole step, one sequence
@@ -295,6 +299,30 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_kernel_only(args, step, device):
+    """One building block alone, launched eagerly `steps` times after `warmup` (profiler captures)."""
+    from paper_2602_06036_b200 import binding
+    cfg, wl = step.cfg, step.wl
+    S, B = wl.batch, cfg.block_size
+    if args.kernel == "lmhead":
+        hid = torch.randn(S * B, cfg.d_model, device=device).to(cfg.torch_dtype)
+        ids = torch.zeros(S * B, dtype=torch.int32, device=device)
+        fn = lambda: step.lib.dflash_lmhead_argmax(hid, 1, ids)
+        nbytes = algorithmic_bytes(cfg, wl.ctx_lens, 0)["lmhead_argmax"]
+    else:
+        q = torch.randn(S, B, cfg.n_q_heads, cfg.head_dim, device=device).to(cfg.torch_dtype)
+        k = torch.randn(S, B, cfg.n_kv_heads, cfg.head_dim, device=device).to(cfg.torch_dtype)
+        v = torch.randn(S, B, cfg.n_kv_heads, cfg.head_dim, device=device).to(cfg.torch_dtype)
+        out = torch.zeros_like(q)
+        fn = lambda: step.lib.dflash_block_attention(binding.ATTN_FULL, q, k, v, step.ctx_len, step.max_ctx,
+                                                     step.page_table, step.pool, 0, out)
+        nbytes = algorithmic_bytes(cfg, wl.ctx_lens, 0)["attention"]
+    ms = timed(fn, args.steps, args.warmup, False)
+    us = ms / args.steps * 1e3
+    print(json.dumps({"kernel": args.kernel, "workload": wl.name, "us_per_call": us, "alg_bytes": nbytes,
+                      "gbs": nbytes / (us * 1e-6) / 1e9}))
+
+
 # ------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -304,6 +332,8 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention"],
+                    help="run one building block alone (for profiler captures) instead of the step")
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
@@ -332,6 +362,10 @@ def main():
     step = Step(wl, device, seed=0)
     S, B = wl.batch, cfg.block_size
 
+    if args.kernel:
+        run_kernel_only(args, step, device)
+        return
+
     sampler = ClockSampler(local)
     run_resident, run_e2e = step.step_resident, step.step_e2e
     for _ in range(2):           # eager warm-up: sizes the workspace, sets kernel attributes
@@ -351,11 +385,23 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     ms_e2e = timed(run_e2e, args.steps, args.warmup, dist_on)
 
-    # per-kernel-family durations: a second pass of the same steps with event pairs around each launch
-    prof = step.lib.profile(step.step_resident, args.steps) if hasattr(step.lib, "profile") else {}
-
+    # Per-kernel figures. Chained launches hide their phases from CUDA events, so the library's
+    # device-side timeline (global-timer stamps written by the kernels themselves) is read for one
+    # extra, eager step: a phase's interval runs from max(its inputs ready, previous record's end) to
+    # the moment its last CTA signalled completion.
+    trace_rows = step.lib.trace(step.step_resident) if rank == 0 else []
+    # The dominant kernel alone, timed with CUDA event pairs around each of its launches.
+    lm_us = None
+    if rank == 0:
+        hid = torch.randn(S * B, cfg.d_model, device=device).to(cfg.torch_dtype)
+        ids = torch.zeros(S * B, dtype=torch.int32, device=device)
+        lm_call = lambda: step.lib.dflash_lmhead_argmax(hid, 1, ids)
+        for _ in range(3):
+            lm_call()
+        prof_lm = step.lib.profile(lm_call, max(args.steps, 10))
+        lm_us = prof_lm.get("lmhead_argmax", (None, 0))[0]
     if args.trace and rank == 0:
-        rows = step.lib.trace(step.step_resident)
+        rows = trace_rows
         with open(args.trace, "w") as f:
             f.write("# kernel family, first CTA start, dependency resolved, main loop end, last CTA exit (us since first start)\n")
             for fam, a, b, c, d in rows:
@@ -375,19 +421,42 @@ def main():
     alg = algorithmic_bytes(cfg, wl.ctx_lens, step.rows_new)
     hbm = peaks["hbm_gbs"]
     kernels = {}
-    for fam, (us, n) in prof.items():
-        entry = {"us_per_launch": us, "launches_per_step": n}
-        if fam in alg and us > 0:
-            entry["alg_bytes"] = alg[fam]
-            entry["gbs"] = alg[fam] / (us * 1e-6) / 1e9
-            entry["frac_hbm"] = entry["gbs"] / hbm
-        kernels[fam] = entry
-    dom = kernels.get("lmhead_argmax")
+    prev_end = None
+    for fam, t_start, t_dep, t_loop, t_end in trace_rows:
+        if t_end is None:
+            continue
+        cands = [v for v in (t_dep, prev_end) if v is not None]
+        begin = max(cands) if cands else t_start
+        dur = max(t_end - begin, 0) / 1e3
+        prev_end = t_end if prev_end is None else max(prev_end, t_end)
+        e = kernels.setdefault(fam, {"us_total": 0.0, "launches_per_step": 0})
+        e["us_total"] += dur
+        e["launches_per_step"] += 1
+    for fam, e in kernels.items():
+        n = e["launches_per_step"]
+        e["us_per_launch"] = e.pop("us_total") / n
+        if fam == "attention":
+            e["us_per_launch"] *= 2          # two records (main kernel + merge) make one attention
+            e["launches_per_step"] = n // 2
+        if fam in alg and e["us_per_launch"] > 0:
+            e["alg_bytes"] = alg[fam]
+            e["gbs"] = alg[fam] / (e["us_per_launch"] * 1e-6) / 1e9
+            e["frac_hbm"] = e["gbs"] / hbm
     roofline = None
-    if dom and "gbs" in dom:
-        roofline = {"kernel": "lmhead_argmax", "bound": "hbm", "achieved": dom["gbs"], "peak": hbm, "unit": "GB/s",
-                    "frac": dom["frac_hbm"], "traffic": None, "peak_source": peaks["_source"],
-                    "timing": "event pairs around each launch, separate pass of the same steps"}
+    if lm_us:
+        traffic = None
+        prof_file = os.path.join(ROOT, "profiles", "lmhead_argmax_cfg1.md")
+        if os.path.exists(prof_file):
+            for line in open(prof_file):
+                if line.startswith("dram_bytes_per_launch:"):
+                    traffic = int(line.split(":")[1].strip().split()[0])
+        gbs = alg["lmhead_argmax"] / (lm_us * 1e-6) / 1e9
+        roofline = {"kernel": "gemm_tc_kernel<16> as LM head + argmax (V x D weights, 16 rows)", "bound": "hbm",
+                    "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm, "traffic": traffic,
+                    "peak_source": peaks["_source"] + " (copy bandwidth)", "us_per_launch": lm_us,
+                    "timing": "CUDA event pair around each launch of the kernel run alone (dflash_lmhead_argmax), "
+                              "same weights and row count as in the step",
+                    "in_step_us": kernels.get("lmhead_argmax", {}).get("us_per_launch")}
     step_bytes = alg["draft_block_total"] + alg["ctx_project_total"] + S * (B + 1) * cfg.vocab * 2
     line = {
         "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -400,17 +469,25 @@ def main():
                    "parallelism": "replicas" if world > 1 else "single"},
         "step_roofline": {"alg_bytes": step_bytes, "us_at_peak": step_bytes / (hbm * 1e9) * 1e6,
                           "frac": step_bytes / (hbm * 1e9) / (per_step_ms * 1e-3)},
-        "roofline": roofline, "kernels": kernels, "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": roofline, "kernels": kernels,
+        "kernels_note": "device-side timeline of one eager step: per phase, from inputs ready to last CTA done",
+        "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
     }
     if not args.no_cpu_baseline:
-        dt, frac, _ = oracle_sample(wl)
+        # the whole step (all layers, full vocabulary) for one sequence: about 10-30 s of host work
+        reps, spent = [], 0.0
+        while spent < 10.0 and len(reps) < 8:
+            dt, frac = oracle_sample(wl, layers=cfg.n_layers, vocab_frac=1)
+            reps.append(dt)
+            spent += dt
+        dt = statistics.mean(reps)
         cores = len(os.sched_getaffinity(0))
         line["cpu_baseline"] = {
             "value": B / (dt / frac), "unit": "tokens/s", "cores": cores, "kind": "oracle",
-            "sample": f"one sequence: ctx projection of {B + 1} rows + 1 of {cfg.n_layers} draft layers + LM head over "
-                      f"V/8 + accept = {frac:.3f} of the step's algorithmic bytes in {dt:.1f} s, scaled to the full step"}
+            "sample": f"one sequence of the batch, whole step (ctx projection of {B + 1} rows, all {cfg.n_layers} draft layers "
+                      f"over its full context, full-vocabulary LM head, accept): mean of {len(reps)} runs, {dt:.1f} s each, float64 numpy"}
     print(json.dumps(line))
     if dist_on:
         torch.distributed.destroy_process_group()
