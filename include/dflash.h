@@ -184,6 +184,23 @@ typedef struct {
 } dflash_verify_args;
 int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a /*[host]*/, void* stream);
 
+/* ---- verify/accept from logits without any caller-provided scratch ----
+ * (No counterpart in the paper: this entry point exists for integration reasons only.)
+ * Same result as dflash_verify_accept in mode DFLASH_VERIFY_LOGITS, for callers that cannot allocate
+ * device memory for a workspace (all GPU memory already committed to a cache pool, no tolerance for
+ * cudaMalloc's device-wide synchronisation, or a stream being captured into a graph). The scratch
+ * is a fixed array inside the library image: about 1.1 MB that every GPU loading the library holds
+ * until the process exits. `workspace` / `workspace_bytes` are ignored.
+ *   - at most DFLASH_STATIC_MAX_ROWS = batch * (gamma+1) rows; more returns DFLASH_ERR_UNSUPPORTED
+ *   - the array is shared by all calls on a device and keeps the previous call's contents (no entry
+ *     needs to start at zero); calls that overlap on the GPU race on it, so order them on one stream
+ *     or with events
+ *   - the first call on each device resolves the array's device address on the host: issue it
+ *     before any stream capture begins
+ *   - allocates and frees nothing */
+#define DFLASH_STATIC_MAX_ROWS 1088
+int32_t dflash_verify_accept_static(dflash_handle* h, const dflash_verify_args* a /*[host]*/, void* stream);
+
 /* ---- building block: attention of `rows` block rows per sequence over paged context + the block
  * itself (App. A.3: K = [K_ctx ; K_block]_seq). FULL = draft mode, CAUSAL = the target's verify
  * pass over (gamma+1) rows. Head geometry and dtype come from the handle. q and k_blk must already

@@ -27,6 +27,7 @@ EXPORTS = (
     "dflash_ctx_project", "dflash_draft_block", "dflash_verify_accept", "dflash_block_attention",
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
+    "dflash_verify_accept_static",
 )
 N_FAMILIES = 15
 
@@ -105,7 +106,7 @@ def load():
     lib.dflash_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib.dflash_workspace_bytes.restype = C.c_int64
     for name, st in (("dflash_ctx_project", CtxArgs), ("dflash_draft_block", DraftArgs),
-                     ("dflash_verify_accept", VerifyArgs), ("dflash_block_attention", AttnArgs),
+                     ("dflash_verify_accept", VerifyArgs), ("dflash_verify_accept_static", VerifyArgs), ("dflash_block_attention", AttnArgs),
                      ("dflash_lmhead_argmax", LmHeadArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(st), C.c_void_p]
@@ -293,6 +294,18 @@ class DFlash:
                        _ptr(ctx_len), _ptr(accept_len), _ptr(out_tokens), _ptr(bonus), _ptr(new_ctx_len),
                        _ptr(target_ids_out), _ptr(ws), ws.numel(), _ptr(self.status))
         _check(self.lib.dflash_verify_accept(self.h, C.byref(a), _stream(stream)))
+
+    def dflash_verify_accept_static(self, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus,
+                                    new_ctx_len, logits, target_ids_out=None, stream=None):
+        """Logits-mode verify/accept on the library's built-in scratch: no workspace is passed, nothing is
+        allocated. For callers that cannot allocate device memory; at most DFLASH_STATIC_MAX_ROWS rows, and
+        calls must not overlap on the GPU (they share the scratch)."""
+        S = ctx_len.shape[0]
+        ldt = F32 if logits.dtype == torch.float32 else BF16
+        a = VerifyArgs(VERIFY_LOGITS, _ptr(logits), ldt, 0, None, _ptr(draft_ids), draft_stride, S, gamma,
+                       logits.shape[-1], _ptr(ctx_len), _ptr(accept_len), _ptr(out_tokens), _ptr(bonus),
+                       _ptr(new_ctx_len), _ptr(target_ids_out), None, 0, _ptr(self.status))
+        _check(self.lib.dflash_verify_accept_static(self.h, C.byref(a), _stream(stream)))
 
     def dflash_block_attention(self, mode, q, k_blk, v_blk, ctx_len, max_ctx_len, page_table, kv_pool, layer,
                                out, stream=None):
