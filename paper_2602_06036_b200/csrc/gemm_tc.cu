@@ -41,7 +41,7 @@ constexpr int CH = 16;                           // token columns handled per ep
 constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB
 constexpr int MAX_STAGES = 12;
 constexpr int ACC_LD = CH + 1;
-constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
+constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 3 * 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int N_THREADS = 192;
 
@@ -149,7 +149,8 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
 
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
-                                               int row) {
+                                               int row, const int* tPos, const int* tPage) {
+    // tPos / tPage: position and physical page of the 16 tokens of this pass (-1 = skip the token)
     const int f = un.ft * TILE_F + row;
     const int n_tok = min(CH, p.M - tok0);
     switch (p.epi) {
@@ -210,17 +211,10 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 float cs[CH], sn[CH];
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    cs[c] = 1.f; sn[c] = 0.f;
-                    if (rot && c < n_tok) {
-                        const int tok = tok0 + c;
-                        int pos = __ldcg(p.ctx_len + tok / p.rows_per_seq) + tok % p.rows_per_seq;
-                        if (pos < 0 || pos >= p.max_pos) {
-                            if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
-                            pos = pos < 0 ? 0 : p.max_pos - 1;
-                        }
-                        cs[c] = __ldg(p.cs + (size_t)pos * half + i);
-                        sn[c] = __ldg(p.sn + (size_t)pos * half + i);
-                    }
+                    const int pos = tPos[c];
+                    const bool on = rot && c < n_tok && pos >= 0;
+                    cs[c] = on ? __ldg(p.cs + (size_t)pos * half + i) : 1.f;
+                    sn[c] = on ? __ldg(p.sn + (size_t)pos * half + i) : 0.f;
                 }
                 __nv_bfloat16* dst;
                 int ld;
@@ -273,44 +267,27 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 const int head = fh / hd, hrow = fh % hd, i = hrow % half;
                 const int partner = row ^ half;
                 const int layer = p.first_layer + un.g;
-                // gather every token's destination and rotation first, then write
-                long long dst[CH];
                 float cs[CH], sn[CH];
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    dst[c] = -1; cs[c] = 1.f; sn[c] = 0.f;
-                    if (c >= n_tok) continue;
-                    const int tok = tok0 + c;
-                    const int b = tok / p.max_new, r = tok % p.max_new;
-                    const int nn = p.n_new ? __ldcg(p.n_new + b) : p.max_new;
-                    if (r >= nn) continue;
-                    const int pos = __ldcg(p.ctx_len + b) + r;
-                    const int pidx = pos / p.PG;
-                    if (pos < 0 || pidx >= p.max_pages || (p.use_rope && pos >= p.max_pos)) {
-                        if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
-                        continue;
-                    }
-                    const int page = __ldcg(p.page_table + (size_t)b * p.max_pages + pidx);
-                    if (page < 0 || page >= p.n_pages) {
-                        if (row == 0 && p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
-                        continue;
-                    }
-                    if (!is_v && p.use_rope) {
-                        cs[c] = __ldg(p.cs + (size_t)pos * half + i);
-                        sn[c] = __ldg(p.sn + (size_t)pos * half + i);
-                    }
-                    dst[c] = (long long)((((((size_t)layer * p.n_pages + page) * 2 + is_v) * p.Hkv + head) * p.PG +
-                                          (pos % p.PG)) * hd + hrow);
+                    const int pos = tPos[c];
+                    const bool on = !is_v && p.use_rope && c < n_tok && pos >= 0;
+                    cs[c] = on ? __ldg(p.cs + (size_t)pos * half + i) : 1.f;
+                    sn[c] = on ? __ldg(p.sn + (size_t)pos * half + i) : 0.f;
                 }
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    if (dst[c] < 0) continue;
-                    float val = sAcc[row * ACC_LD + c];
-                    if (!is_v && p.use_rope) {
-                        const float bb = sAcc[partner * ACC_LD + c];
-                        val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
+                    const int pos = tPos[c], page = tPage[c];
+                    if (c < n_tok && pos >= 0 && page >= 0) {
+                        float val = sAcc[row * ACC_LD + c];
+                        if (!is_v && p.use_rope) {
+                            const float bb = sAcc[partner * ACC_LD + c];
+                            val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
+                        }
+                        const size_t dst = (((((size_t)layer * p.n_pages + page) * 2 + is_v) * p.Hkv + head) * p.PG +
+                                            (pos % p.PG)) * hd + hrow;
+                        p.pool[dst] = __float2bfloat16_rn(val);
                     }
-                    p.pool[dst[c]] = __float2bfloat16_rn(val);
                 }
             }
         } break;
@@ -321,6 +298,44 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
+// Position (and, for the context projection, physical page) of every token of a token tile, worked
+// out once per phase by the epilogue threads so that the per-pass epilogues carry no dependent loads.
+__device__ __forceinline__ void token_info(const KParams& p, int tok_base, int nt, int row, int* sPos, int* sPage) {
+    for (int t = row; t < nt; t += 128) {
+        const int tok = tok_base + t;
+        int pos = -1, page = -1;
+        if (tok < p.M) {
+            if (p.epi == EPI_QKV_ROPE) {
+                pos = __ldcg(p.ctx_len + tok / p.rows_per_seq) + tok % p.rows_per_seq;
+                if (p.use_rope && (pos < 0 || pos >= p.max_pos)) {
+                    if (p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
+                    pos = pos < 0 ? 0 : p.max_pos - 1;
+                }
+            } else if (p.epi == EPI_CTX_KV) {
+                const int b = tok / p.max_new, r = tok % p.max_new;
+                const int nn = p.n_new ? __ldcg(p.n_new + b) : p.max_new;
+                if (r < nn) {
+                    pos = __ldcg(p.ctx_len + b) + r;
+                    const int pidx = pos / p.PG;
+                    if (pos < 0 || pidx >= p.max_pages || (p.use_rope && pos >= p.max_pos)) {
+                        if (p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
+                        pos = -1;
+                    } else {
+                        page = __ldcg(p.page_table + (size_t)b * p.max_pages + pidx);
+                        if (page < 0 || page >= p.n_pages) {
+                            if (p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
+                            pos = -1;
+                            page = -1;
+                        }
+                    }
+                }
+            }
+        }
+        sPos[t] = pos;
+        sPage[t] = page;
+    }
+}
+
 // Bounded poll of a global counter written by other CTAs (release/acquire through L2).
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     int v;
@@ -342,7 +357,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE_BYTES);
     Top2Entry* sRed = reinterpret_cast<Top2Entry*>(sAcc + TILE_F * ACC_LD);
     float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [256] per-token rsqrt of this token tile
-    uint64_t* full = reinterpret_cast<uint64_t*>(sRstd + 256);
+    int* sPos = reinterpret_cast<int*>(sRstd + 256);              // [256] per-token position (-1: skip)
+    int* sPage = sPos + 256;                                      // [256] per-token physical page
+    uint64_t* full = reinterpret_cast<uint64_t*>(sPage + 256);
     uint64_t* empty = full + MAX_STAGES;
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -497,32 +514,35 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         const int row = ew * 32 + lane;
         uint32_t ui = 0;
         bool alive = true;
+        pdl_wait();      // lengths, page tables, residual rows ... come from earlier kernels
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
             const long long T = (long long)p.n_tiles * p.chunks_total;
-            int rstd_tt = -1;
+            int rstd_tt = -1, info_tt = -1;
             for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
+                // token positions / pages do not depend on this chain: work them out while the main loop runs
+                if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && info_tt != un.tt) {
+                    token_info(p, tok_base, NT, row, sPos, sPage);
+                    info_tt = un.tt;     // visible after the barrier below
+                }
                 const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
                 if (!got) flags[2] = 1;
                 epi_bar();
                 if (flags[2]) { alive = false; break; }   // uniform over the four warps
                 tc_fence_after();
-                // The accumulator exists, so this phase's inputs do too (phase 0: wait for the grid
-                // dependency explicitly, the producer may be the only thread that did).
-                if (ph == 0 && ui == 0) pdl_wait();
-                // per-token rsqrt(mean square) of the operand rows, once per token tile
+                // The accumulator exists, so the previous phase is complete and its sums of squares are final:
+                // per-token rsqrt(mean square), one warp per token, lanes over the 128-feature tiles.
                 if (p.ssq_in && rstd_tt != un.tt) {
-                    for (int t = row; t < NT; t += 128) {
-                        float rs = 1.f;
-                        if (tok_base + t < p.M) {
-                            float s = 0.f;
-                            for (int q = 0; q < p.n_parts_in; ++q) s += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
-                            rs = rsqrtf(s * p.inv_dim_in + p.eps);
-                        }
-                        sRstd[t] = rs;
+                    for (int t = ew; t < NT; t += 4) {
+                        float sum = 0.f;
+                        if (tok_base + t < p.M)
+                            for (int q = lane; q < p.n_parts_in; q += 32) sum += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                        if (lane == 0) sRstd[t] = (tok_base + t < p.M) ? rsqrtf(sum * p.inv_dim_in + p.eps) : 1.f;
                     }
                     rstd_tt = un.tt;
                     epi_bar();
@@ -539,7 +559,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 #pragma unroll
                         for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[ch * CH + c] : v[c];
                         epi_bar();
-                        apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
+                        apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + ch * CH, sPage + ch * CH);
                         epi_bar();
                     }
                 }
@@ -587,7 +607,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 #pragma unroll
                             for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[ch * CH + c] : acc[c];
                             epi_bar();
-                            apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row);
+                            apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + ch * CH, sPage + ch * CH);
                             epi_bar();
                         }
                     }
