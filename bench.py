@@ -59,7 +59,7 @@ def algorithmic_bytes(cfg, ctx_lens, n_new_rows):
     return {
         "gemm_qkv": qkv, "gemm_o": o, "gemm_gateup": gateup, "gemm_down": down, "lmhead_argmax": lm,
         "attention": kv_layer, "ctx_fuse": D * cfg.feat_dim * es + n_new_rows * cfg.feat_dim * es,
-        "ctx_kv": 2 * cfg.kv_dim * D * es,
+        "ctx_kv": cfg.n_layers * 2 * cfg.kv_dim * D * es + n_new_rows * cfg.n_layers * 2 * cfg.kv_dim * es,
         "draft_block_total": cfg.n_layers * (qkv + o + gateup + down + kv_layer) + lm,
         "ctx_project_total": ctx,
     }

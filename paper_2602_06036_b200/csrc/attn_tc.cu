@@ -392,19 +392,46 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     if (n_splits <= 1 || row >= rows_valid) return;
     const float* base = p.part + ((size_t)bg * p.n_chunks * 128 + row) * PART_LD;
     const size_t unit_stride = (size_t)128 * PART_LD;
-    float M = -CUDART_INF_F;
-    for (int s = lane; s < n_splits; s += 32) M = fmaxf(M, __ldcg(base + s * unit_stride + HD));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float Lsum = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float* src = base + s * unit_stride;
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + HD));
-        const float w = (ml.x > -CUDART_INF_F) ? exp2f(ml.x - M) : 0.f;
-        const float4 a = __ldcg(reinterpret_cast<const float4*>(src) + lane);
-        Lsum += ml.y * w;
-        acc.x += a.x * w; acc.y += a.y * w; acc.z += a.z * w; acc.w += a.w * w;
+    // Few dependent round trips: lane s fetches (max, sum) of range s (all ranges in flight at once),
+    // the weights travel by shuffle, and the accumulator rows are fetched sixteen at a time.
+    // More than 32 ranges: a first pass over (max, sum) finds the global maximum.
+    float M = -CUDART_INF_F;
+    float2 ml0 = make_float2(-CUDART_INF_F, 0.f);
+    for (int s0 = 0; s0 < n_splits; s0 += 32) {
+        const int s = s0 + lane;
+        if (s < n_splits) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(base + s * unit_stride + HD));
+            if (s0 == 0) ml0 = ml;
+            M = fmaxf(M, ml.x);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    for (int s0 = 0; s0 < n_splits; s0 += 32) {
+        const int s = s0 + lane;
+        float2 ml = ml0;
+        if (s0 > 0) ml = (s < n_splits) ? __ldcg(reinterpret_cast<const float2*>(base + s * unit_stride + HD))
+                                        : make_float2(-CUDART_INF_F, 0.f);
+        const float w_mine = (s < n_splits && ml.x > -CUDART_INF_F) ? exp2f(ml.x - M) : 0.f;
+        float l_mine = ml.y * w_mine;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) l_mine += __shfl_xor_sync(0xffffffffu, l_mine, o);
+        Lsum += l_mine;
+        const int n_here = min(32, n_splits - s0);
+        for (int k0 = 0; k0 < n_here; k0 += 16) {
+            float4 a[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                a[k] = (k0 + k < n_here) ? __ldcg(reinterpret_cast<const float4*>(base + (s0 + k0 + k) * unit_stride) + lane)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float w = __shfl_sync(0xffffffffu, w_mine, (k0 + k) & 31);
+                acc.x += a[k].x * w; acc.y += a[k].y * w; acc.z += a[k].z * w; acc.w += a[k].w * w;
+            }
+        }
     }
     const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
     const int r = row / p.group, j = row % p.group;

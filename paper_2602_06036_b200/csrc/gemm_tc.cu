@@ -37,11 +37,14 @@ using namespace ptx;
 
 constexpr int TILE_F = 128;                      // weight rows per tile = MMA M
 constexpr int BK = 64;                           // K elements per stage = one 128-byte swizzle row
-constexpr int CH = 16;                           // token columns handled per epilogue pass
 constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB
 constexpr int MAX_STAGES = 12;
-constexpr int ACC_LD = CH + 1;
-constexpr int SMEM_FIXED = TILE_F * ACC_LD * 4 + 128 * 16 + 3 * 256 * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
+constexpr int TOK_CACHE = 1024;                  // per-token scale / position / page kept for this many rows
+// token columns handled per epilogue pass (each of the 128 epilogue threads holds CH accumulators)
+constexpr int pass_cols(int nt) { return nt < 64 ? nt : (nt == 256 ? 32 : 64); }   // 256: keep shared memory for ring stages
+constexpr int smem_fixed(int nt) {
+    return TILE_F * (pass_cols(nt) + 1) * 4 + 128 * 16 + 3 * TOK_CACHE * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
+}
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int N_THREADS = 192;
 
@@ -148,9 +151,12 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
 }
 
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
+template <int CH>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
                                                int row, const int* tPos, const int* tPage) {
     // tPos / tPage: position and physical page of the 16 tokens of this pass (-1 = skip the token)
+    constexpr int ACC_LD = CH + 1;
+    constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
     const int f = un.ft * TILE_F + row;
     const int n_tok = min(CH, p.M - tok0);
     switch (p.epi) {
@@ -186,17 +192,17 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 #pragma unroll
                 for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = xv[c] * xv[c];
                 epi_bar();
-                const int c = row & 15, g8 = row >> 4;
+                const int c = row % CH, g8 = row / CH;
                 float s = 0.f;
 #pragma unroll
-                for (int r = 0; r < 16; ++r) s += sAcc[(g8 * 16 + r) * ACC_LD + c];
+                for (int r = 0; r < CH; ++r) s += sAcc[(g8 * CH + r) * ACC_LD + c];
                 float* red = reinterpret_cast<float*>(sRed);
-                red[g8 * 16 + c] = s;
+                red[g8 * CH + c] = s;
                 epi_bar();
                 if (row < n_tok) {
                     float t = 0.f;
 #pragma unroll
-                    for (int gg = 0; gg < 8; ++gg) t += red[gg * 16 + row];
+                    for (int gg = 0; gg < GROUPS; ++gg) t += red[gg * CH + row];
                     p.ssq_out[(size_t)un.ft * p.M + tok0 + row] = t;
                 }
             }
@@ -242,19 +248,19 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
         case EPI_ARGMAX: {
             if (p.logits_out && f < p.N)
                 for (int c = 0; c < n_tok; ++c) p.logits_out[(size_t)(tok0 + c) * p.N + f] = sAcc[row * ACC_LD + c];
-            const int c = row & 15, g = row >> 4;
+            const int c = row % CH, g = row / CH;
             T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                const int rr = g * 16 + r, ff = un.ft * TILE_F + rr;
+#pragma unroll 16
+            for (int r = 0; r < CH; ++r) {
+                const int rr = g * CH + r, ff = un.ft * TILE_F + rr;
                 if (ff < p.N) t2_push(t, sAcc[rr * ACC_LD + c], ff);
             }
-            sRed[g * 16 + c] = Top2Entry{t.v1, t.i1, t.v2, 0};
+            sRed[g * CH + c] = Top2Entry{t.v1, t.i1, t.v2, 0};
             epi_bar();
             if (row < n_tok) {
                 T2 m{sRed[row].v1, sRed[row].i1, sRed[row].v2};
 #pragma unroll
-                for (int gg = 1; gg < 8; ++gg) t2_merge(m, sRed[gg * 16 + row].v1, sRed[gg * 16 + row].i1, sRed[gg * 16 + row].v2);
+                for (int gg = 1; gg < GROUPS; ++gg) t2_merge(m, sRed[gg * CH + row].v1, sRed[gg * CH + row].i1, sRed[gg * CH + row].v2);
                 p.top2[(size_t)un.ft * p.M + tok0 + row] = Top2Entry{m.v1, m.i1, m.v2, 0};
             }
         } break;
@@ -301,7 +307,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 // Position (and, for the context projection, physical page) of every token of a token tile, worked
 // out once per phase by the epilogue threads so that the per-pass epilogues carry no dependent loads.
 __device__ __forceinline__ void token_info(const KParams& p, int tok_base, int nt, int row, int* sPos, int* sPage) {
-    for (int t = row; t < nt; t += 128) {
+    for (int t = row; t < nt; t += 128) {      // sPos[t] describes token tok_base + t
         const int tok = tok_base + t;
         int pos = -1, page = -1;
         if (tok < p.M) {
@@ -336,6 +342,29 @@ __device__ __forceinline__ void token_info(const KParams& p, int tok_base, int n
     }
 }
 
+// rsqrt(mean square) of operand rows tok_base .. tok_base+nt-1 from the per-tile sums of squares:
+// one thread per token, eight partial sums in flight.
+__device__ __forceinline__ void token_rstd(const KParams& p, int tok_base, int nt, int row, float* sRstd) {
+    for (int t = row; t < nt; t += 128) {
+        const int tok = tok_base + t;
+        float rs = 1.f;
+        if (tok < p.M) {
+            float s[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) s[k] = 0.f;
+            const float* src = p.ssq_in + tok;
+            for (int q = 0; q < p.n_parts_in; q += 8) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (q + k < p.n_parts_in) s[k] += __ldcg(src + (size_t)(q + k) * p.M);
+            }
+            const float sum = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
+            rs = rsqrtf(sum * p.inv_dim_in + p.eps);
+        }
+        sRstd[t] = rs;
+    }
+}
+
 // Bounded poll of a global counter written by other CTAs (release/acquire through L2).
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     int v;
@@ -350,16 +379,18 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int X_STAGE_BYTES = NT * BK * 2;
+    constexpr int CH = pass_cols(NT);
+    constexpr int ACC_LD = CH + 1;
     constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
     const int stages = mp.stages;
     uint8_t* sW = smem;
     uint8_t* sX = sW + (size_t)stages * W_STAGE_BYTES;
     float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE_BYTES);
     Top2Entry* sRed = reinterpret_cast<Top2Entry*>(sAcc + TILE_F * ACC_LD);
-    float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [256] per-token rsqrt of this token tile
-    int* sPos = reinterpret_cast<int*>(sRstd + 256);              // [256] per-token position (-1: skip)
-    int* sPage = sPos + 256;                                      // [256] per-token physical page
-    uint64_t* full = reinterpret_cast<uint64_t*>(sPage + 256);
+    float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [TOK_CACHE] per-token rsqrt(mean square)
+    int* sPos = reinterpret_cast<int*>(sRstd + TOK_CACHE);        // [TOK_CACHE] per-token position (-1: skip)
+    int* sPage = sPos + TOK_CACHE;                                // [TOK_CACHE] per-token physical page
+    uint64_t* full = reinterpret_cast<uint64_t*>(sPage + TOK_CACHE);
     uint64_t* empty = full + MAX_STAGES;
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -523,9 +554,13 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
+                // Per-token data is cached for the whole phase when the rows fit (else per token tile).
+                const bool all_tok = p.M <= TOK_CACHE;
+                const int tok_off = all_tok ? tok_base : 0;          // index of this tile's first token in the caches
                 // token positions / pages do not depend on this chain: work them out while the main loop runs
-                if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && info_tt != un.tt) {
-                    token_info(p, tok_base, NT, row, sPos, sPage);
+                if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && (all_tok ? info_tt < 0 : info_tt != un.tt)) {
+                    if (all_tok) token_info(p, 0, p.M, row, sPos, sPage);
+                    else token_info(p, tok_base, NT, row, sPos, sPage);
                     info_tt = un.tt;     // visible after the barrier below
                 }
                 const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
@@ -533,33 +568,26 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 epi_bar();
                 if (flags[2]) { alive = false; break; }   // uniform over the four warps
                 tc_fence_after();
-                // The accumulator exists, so the previous phase is complete and its sums of squares are final:
-                // per-token rsqrt(mean square), one warp per token, lanes over the 128-feature tiles.
-                if (p.ssq_in && rstd_tt != un.tt) {
-                    for (int t = ew; t < NT; t += 4) {
-                        float sum = 0.f;
-                        if (tok_base + t < p.M)
-                            for (int q = lane; q < p.n_parts_in; q += 32) sum += __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t);
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                        if (lane == 0) sRstd[t] = (tok_base + t < p.M) ? rsqrtf(sum * p.inv_dim_in + p.eps) : 1.f;
-                    }
+                // The accumulator exists, so the previous phase is complete and its sums of squares are final.
+                if (p.ssq_in && (all_tok ? rstd_tt < 0 : rstd_tt != un.tt)) {
+                    if (all_tok) token_rstd(p, 0, p.M, row, sRstd);
+                    else token_rstd(p, tok_base, NT, row, sRstd);
                     rstd_tt = un.tt;
                     epi_bar();
                 }
                 const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
                 for (int ch = 0; ch < n_ch; ++ch) {
                     float v[CH];
-                    tmem_ld16(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
+                    tmem_ld_cols<CH>(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
                     if (!un.full) {
                         float* dst = p.part + (((size_t)blockIdx.x * 2 + un.slot) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
                         for (int c = 0; c < CH; ++c) dst[(size_t)c * TILE_F] = v[c];
                     } else {
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[ch * CH + c] : v[c];
+                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[tok_off + ch * CH + c] : v[c];
                         epi_bar();
-                        apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + ch * CH, sPage + ch * CH);
+                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
                         epi_bar();
                     }
                 }
@@ -584,30 +612,20 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                             float acc[CH];
 #pragma unroll
                             for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                            // pieces are summed in CTA order; two are fetched at a time so their
-                            // loads overlap
-                            int j = j0;
-                            for (; j + 1 <= j1; j += 2) {
-                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
-                                const int sb = ((long long)(j + 1) * T / G >= x0) ? 0 : 1;
-                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
-                                const float* pb = p.part + (((size_t)(j + 1) * 2 + sb) * NT + ch * CH) * TILE_F + row;
-                                float va[CH], vb[CH];
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) { va[c] = __ldcg(pa + (size_t)c * TILE_F); vb[c] = __ldcg(pb + (size_t)c * TILE_F); }
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) acc[c] = (acc[c] + va[c]) + vb[c];
-                            }
-                            if (j <= j1) {
+                            // pieces are summed in CTA order; the CH loads of a piece are all in flight together
+                            for (int j = j0; j <= j1; ++j) {
                                 const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
                                 const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+                                float va[CH];
 #pragma unroll
-                                for (int c = 0; c < CH; ++c) acc[c] += __ldcg(pa + (size_t)c * TILE_F);
+                                for (int c = 0; c < CH; ++c) va[c] = __ldcg(pa + (size_t)c * TILE_F);
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) acc[c] += va[c];
                             }
 #pragma unroll
-                            for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[ch * CH + c] : acc[c];
+                            for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
                             epi_bar();
-                            apply_epilogue(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + ch * CH, sPage + ch * CH);
+                            apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
                             epi_bar();
                         }
                     }
@@ -722,7 +740,7 @@ int pick_nt(int M) {
 template <int NT>
 int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
     static bool attr_set = false;
-    const int smem = 1024 + mp.stages * (W_STAGE_BYTES + NT * BK * 2) + SMEM_FIXED;
+    const int smem = 1024 + mp.stages * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
     if (!attr_set) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
@@ -786,7 +804,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     WMaps tw;
     XMaps tx;
     mp.n_phases = n_phases;
-    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - SMEM_FIXED) / (W_STAGE_BYTES + nt * BK * 2));
+    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (W_STAGE_BYTES + nt * BK * 2));
     mp.phase_done = phase_done;
     mp.status = L.status;
 

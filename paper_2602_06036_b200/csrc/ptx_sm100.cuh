@@ -177,5 +177,24 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 }
 
 
+// CH consecutive fp32 columns of this warp's 32 TMEM lanes (CH = 16, 32 or 64), one row per thread
+template <int CH>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
+    static_assert(CH == 16 || CH == 32 || CH == 64, "unsupported pass width");
+#pragma unroll
+    for (int c0 = 0; c0 < CH; c0 += 16) {
+        uint32_t r[16];
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+              "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+            : "r"(taddr + c0)
+            : "memory");
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[c0 + i] = __uint_as_float(r[i]);
+    }
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 }  // namespace ptx
 }  // namespace dflash
