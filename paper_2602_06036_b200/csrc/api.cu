@@ -59,7 +59,7 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     w.flags = w.counters ? (int32_t*)((char*)w.counters + gemm_counters) : nullptr;
     w.attn_counters = w.counters ? (int32_t*)((char*)w.counters + gemm_counters + flag_bytes) : nullptr;
     w.top2 = a.take(tc ? (int64_t)((c.vocab + 127) / 128) * R * (int64_t)sizeof(Top2Entry) : 256);
-    w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), h->sm_count) : 256);
+    w.attn_part = (float*)a.take(tc ? attn_tc_part_bytes(c, std::max(batch, 1), (int)std::min<int64_t>(32, (R + std::max(batch, 1) - 1) / std::max(batch, 1)), h->sm_count) : 256);
     w.seg = (float4*)a.take(R * 64 * 16);
     w.ssq = (float*)a.take((int64_t)((c.d_model + 127) / 128) * R * 4);
     w.bytes = a.off;

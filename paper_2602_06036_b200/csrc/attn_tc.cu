@@ -2,17 +2,21 @@
 //   every block row of a sequence attends over [paged context K/V ; the block's own K/V].
 // One CTA works on one (sequence, kv head, range of KV tiles). The queries of all block rows and of
 // the q heads that share the kv head (rows x group <= 128) are the 128-row "M" operand; a KV tile
-// is one 64-token page (or the block's own rows). Per tile:
-//   S = Q K^T           tcgen05.mma, S in TMEM (two buffers, so the next tile's S is computed while
-//                       this one is in the softmax)
-//   softmax             one thread per query row reads its S row from TMEM (no cross-thread
-//                       reduction), running max / sum in the log2 domain, P -> shared memory (bf16)
-//   O_tile = P V        tcgen05.mma with V as an MN-major operand straight from the page layout
-//   acc = acc*alpha + O_tile   in registers, one row per thread
-// K/V tiles stream through a TMA ring that runs ahead of the math. Long contexts are split across
-// CTAs; each writes its partial (acc, max, sum) and a small second kernel merges them in split
-// order (bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block row r sees
-// block rows <= r. Every mbarrier wait is bounded.
+// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (4-deep K/V ring that
+// runs ahead of the math), an MMA-issuing warp, and TWO softmax warpgroups that take alternate
+// tiles, each with its own S buffer, P buffer and output accumulator:
+//   S_w = Q K^T          tcgen05.mma into TMEM
+//   softmax              one thread per query row reads its S row from TMEM (no cross-thread
+//                        reduction), exponentials in the log2 domain against a running maximum that
+//                        is only raised when a tile exceeds it by more than 2^8 (then the row of O_w
+//                        in TMEM is rescaled in place), P -> shared memory (bf16)
+//   O_w += P V           tcgen05.mma accumulating in TMEM, V as an MN-major operand straight from
+//                        the page layout
+// so the softmax of one tile overlaps the contractions of the next, and the output never leaves
+// TMEM until the end, where the two accumulators are merged. Long contexts are split across CTAs;
+// each writes its partial (acc, max, sum) and a small second kernel merges them in range order
+// (bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block row r sees block
+// rows <= r. Every mbarrier wait is bounded.
 #include "attn_tc.cuh"
 
 #include "ptx_sm100.cuh"
@@ -28,23 +32,23 @@ using namespace ptx;
 
 constexpr int HD = 128;          // head_dim
 constexpr int PG = 64;           // tokens per page = keys per tile
-constexpr int NS = 5;            // K/V ring depth
-constexpr int Q_BYTES = 128 * HD * 2;          // 32 KiB: two 64-wide halves of 128 rows
+constexpr int NS = 4;            // K/V ring depth
+constexpr int Q_BYTES = 128 * HD * 2;            // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
-constexpr int P_BYTES = 128 * PG * 2;          // 16 KiB
-constexpr int PART_LD = HD + 4;                // acc[128], running max, running sum, 2 pad (16-byte rows)
-constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + P_BYTES + 512;
-constexpr uint32_t TMEM_COLS = 256;            // S0 | S1 (64 each) | O (128)
-constexpr int N_THREADS = 192;
+constexpr int P_BYTES = 128 * PG * 2;            // 16 KiB per warpgroup
+constexpr int PART_LD = HD + 4;                  // acc[128], running max, running sum, 2 pad (16-byte rows)
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512;
+constexpr uint32_t TMEM_COLS = 512;              // S0 | S1 (64 each) | O0 | O1 (128 each)
+constexpr int N_THREADS = 320;                   // producer, MMA issuer, 2 x 4 softmax warps
+constexpr float RESCALE_GAP = 8.f;               // log2 units
 
 struct AParams {
-    int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks;
+    int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks, rows_valid;
     float scale_log2;
     const int32_t* ctx_len;
     const int32_t* page_table;
     __nv_bfloat16* out;
     float* part;
-    int32_t* counters;
     int32_t* status;
     unsigned long long* trace;
 };
@@ -65,6 +69,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+        "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+        "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // MN-major operand (V: [key][head_dim], head_dim contiguous) in two 64-column halves of 64 rows x
 // 128 bytes, 128-byte swizzle: leading byte offset = distance between the halves (8 KiB), stride
@@ -88,6 +108,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&t);
 }
+// named barrier over the 128 threads of one softmax warpgroup (ids 1 and 2), and over both (id 3)
+__device__ __forceinline__ void wg_bar(int wg) { asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory"); }
+__device__ __forceinline__ void both_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
 
 __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPool,
@@ -113,27 +136,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;
     uint8_t* sKV = sQ + Q_BYTES;
-    uint8_t* sP = sKV + NS * KV_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
+    uint8_t* sP = sKV + NS * KV_STAGE_BYTES;             // two P tiles
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * P_BYTES);
     uint64_t* q_full = bars;
     uint64_t* kv_full = bars + 1;
     uint64_t* kv_empty = kv_full + NS;
-    uint64_t* s_full = kv_empty + NS;
-    uint64_t* s_empty = s_full + 2;
-    uint64_t* p_full = s_empty + 2;
-    uint64_t* p_empty = p_full + 1;
-    uint64_t* o_full = p_empty + 1;
-    uint64_t* o_empty = o_full + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
+    uint64_t* s_full = kv_empty + NS;      // [2] S_w written by the tensor core
+    uint64_t* s_free = s_full + 2;         // [2] S_w read by its warpgroup
+    uint64_t* p_full = s_free + 2;         // [2] P_w written (and O_w rescaled if needed)
+    uint64_t* pv_done = p_full + 2;        // [2] O_w += P_w V finished (P_w reusable, O_w consistent)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
         for (int s = 0; s < NS; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 4); }
-        mbar_init(p_full, 4); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 4);
-        flags[0] = 0; flags[1] = 0;
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&p_full[s], 4); mbar_init(&pv_done[s], 1);
+        }
+        flags[0] = 0;
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -142,7 +164,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -193,37 +214,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc_bf16(128, PG);
             constexpr uint32_t idesc_o = instr_desc_bf16_bmn(128, HD);
-            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+            const uint32_t q_addr = smem_u32(sQ);
             bool ok = mbar_wait(q_full, 0, &flags[0]);
+            // tile i belongs to warpgroup w = i & 1 and is that warpgroup's (i >> 1)-th tile
             auto issue_s = [&](int i) -> bool {
                 const int st = i % NS;
-                const uint32_t sb = i & 1;
+                const uint32_t w = i & 1, k = (uint32_t)i >> 1;
                 if (!mbar_wait(&kv_full[st], (i / NS) & 1, &flags[0])) return false;
-                if (!mbar_wait(&s_empty[sb], ((i >> 1) & 1) ^ 1, &flags[0])) return false;
+                if (!mbar_wait(&s_free[w], (k & 1) ^ 1, &flags[0])) return false;
                 tc_fence_after();
                 const uint32_t k_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_bf16(tmem_S + sb * PG, smem_desc_sw128(q_addr + (kk >> 2) * (Q_BYTES / 2) + (kk & 3) * 32),
+                    mma_bf16(tmem_base + w * PG, smem_desc_sw128(q_addr + (kk >> 2) * (Q_BYTES / 2) + (kk & 3) * 32),
                              smem_desc_sw128(k_addr + (kk >> 2) * 8192 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-                mma_commit(&s_full[sb]);
+                mma_commit(&s_full[w]);
                 return true;
             };
             if (ok) ok = issue_s(0);
+            if (ok && n_tiles > 1) ok = issue_s(1);
             for (int i = 0; i < n_tiles && ok; ++i) {
-                if (i + 1 < n_tiles) { ok = issue_s(i + 1); if (!ok) break; }
                 const int st = i % NS;
-                if (!mbar_wait(p_full, i & 1, &flags[0])) { ok = false; break; }
-                if (!mbar_wait(o_empty, (i & 1) ^ 1, &flags[0])) { ok = false; break; }
+                const uint32_t w = i & 1, k = (uint32_t)i >> 1;
+                if (!mbar_wait(&p_full[w], k & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t v_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES + KV_STAGE_BYTES / 2);
+                const uint32_t p_addr = smem_u32(sP + w * P_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < PG / 16; ++kk)
-                    mma_bf16(tmem_O, smem_desc_sw128(p_addr + kk * 32), smem_desc_sw128_mn(v_addr + kk * 2048), idesc_o,
-                             kk > 0 ? 1u : 0u);
-                mma_commit(o_full);
-                mma_commit(p_empty);
+                    mma_bf16(tmem_base + 128 + w * HD, smem_desc_sw128(p_addr + kk * 32), smem_desc_sw128_mn(v_addr + kk * 2048),
+                             idesc_o, (k > 0 || kk > 0) ? 1u : 0u);      // a warpgroup's first tile starts its accumulator
+                mma_commit(&pv_done[w]);
                 mma_commit(&kv_empty[st]);
+                if (i + 2 < n_tiles) ok = issue_s(i + 2);
             }
             if (!ok) {
                 flags[0] = 1;
@@ -232,19 +255,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         __syncwarp();
     } else {
-        // ---------------- softmax + accumulation: thread = query row ----------------
-        const int ew = warp & 3;
-        const int row = ew * 32 + lane;                    // TMEM lane
-        const int r = row / p.group, j = row % p.group;    // block row, q head inside the group
+        // ---------------- softmax warpgroups: thread = query row ----------------
+        const int wg = (warp - 2) >> 2;                     // 0: even tiles, 1: odd tiles
+        const int ew = warp & 3;                            // TMEM lane quadrant of this warp
+        const int row = ew * 32 + lane;                     // query row = TMEM lane
+        const int r = row / p.group, j = row % p.group;     // block row, q head inside the group
         const uint32_t lane_sel = (uint32_t)(ew * 32) << 16;
-        float acc[HD];
-#pragma unroll
-        for (int d = 0; d < HD; ++d) acc[d] = 0.f;
-        float m_run = -CUDART_INF_F, l_run = 0.f;
+        const uint32_t tmem_S = tmem_base + wg * PG + lane_sel;
+        const uint32_t tmem_O = tmem_base + 128 + wg * HD + lane_sel;
+        uint8_t* myP = sP + wg * P_BYTES;
+        float m_run = -CUDART_INF_F, l_run = 0.f;           // log2-domain reference maximum, running sum
         bool ok = true;
-        for (int i = 0; i < n_tiles; ++i) {
+        int k = 0;                                          // index of this warpgroup's tile
+        for (int i = wg; i < n_tiles; i += 2, ++k) {
             const int t = t_lo + i;
-            const uint32_t sb = i & 1;
             const int st = i % NS;
             // how many keys of this tile exist, and from which one on they are hidden from this row
             int n_valid, n_vis;
@@ -257,43 +281,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 n_valid = p.R;
                 n_vis = p.causal ? min(r + 1, p.R) : p.R;
             }
-            if (!mbar_wait(&s_full[sb], (i >> 1) & 1, &flags[0])) { ok = false; break; }
+            if (!mbar_wait(&s_full[wg], k & 1, &flags[0])) { ok = false; break; }
             tc_fence_after();
             float s[PG];
-            tmem_ld32(tmem_S + sb * PG + lane_sel, s);
-            tmem_ld32(tmem_S + sb * PG + 32 + lane_sel, s + 32);
+            tmem_ld32(tmem_S, s);
+            tmem_ld32(tmem_S + 32, s + 32);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&s_empty[sb]);
+            if (lane == 0) mbar_arrive(&s_free[wg]);
             float mx = -CUDART_INF_F;
 #pragma unroll
             for (int c = 0; c < PG; ++c) {
                 s[c] = (c < n_vis) ? s[c] * p.scale_log2 : -CUDART_INF_F;
                 mx = fmaxf(mx, s[c]);
             }
-            const float m_new = fmaxf(m_run, mx);
-            float alpha = 1.f, psum = 0.f;
-            if (m_new > -CUDART_INF_F) {
-                alpha = fast_exp2(m_run - m_new);
+            // raise the reference maximum only when this tile tops it by more than the gap
+            const bool raise = mx > m_run + RESCALE_GAP || (m_run == -CUDART_INF_F && mx > -CUDART_INF_F);
+            const float m_new = raise ? mx : m_run;
+            const float alpha = (raise && m_run > -CUDART_INF_F) ? fast_exp2(m_run - m_new) : 1.f;
+            const float m_use = (m_new > -CUDART_INF_F) ? m_new : 0.f;
+            float psum = 0.f;
 #pragma unroll
-                for (int c = 0; c < PG; ++c) { s[c] = fast_exp2(s[c] - m_new); psum += s[c]; }
-            } else {
-#pragma unroll
-                for (int c = 0; c < PG; ++c) s[c] = 0.f;
-            }
+            for (int c = 0; c < PG; ++c) { s[c] = fast_exp2(s[c] - m_use); psum += s[c]; }
             l_run = l_run * alpha + psum;
             m_run = m_new;
-            // P (bf16) into its swizzled K-major tile once the previous P.V has finished reading it
-            if (!mbar_wait(p_empty, (i & 1) ^ 1, &flags[0])) { ok = false; break; }
-            uint8_t* prow = sP + row * 128;
+            // the previous P_w V of this warpgroup must be finished before P_w is rewritten or O_w rescaled
+            if (!mbar_wait(&pv_done[wg], (k & 1) ^ 1, &flags[0])) { ok = false; break; }
+            if (k > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                tc_fence_after();
+#pragma unroll
+                for (int c4 = 0; c4 < HD / 32; ++c4) {
+                    float o[32];
+                    tmem_ld32(tmem_O + c4 * 32, o);
+#pragma unroll
+                    for (int d = 0; d < 32; ++d) o[d] *= alpha;
+                    tmem_st32(tmem_O + c4 * 32, o);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+            }
+            uint8_t* prow = myP + row * 128;
 #pragma unroll
             for (int ck = 0; ck < 8; ++ck) {
-                uint4 w;
-                w.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
-                w.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
-                w.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
-                w.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
-                *reinterpret_cast<uint4*>(prow + ((ck ^ (row & 7)) << 4)) = w;
+                uint4 w4;
+                w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
+                w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
+                w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
+                w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
+                *reinterpret_cast<uint4*>(prow + ((ck ^ (row & 7)) << 4)) = w4;
             }
             // keys that do not exist must not poison P.V with whatever the page holds there
             if (n_valid < PG) {
@@ -306,58 +341,83 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             fence_proxy_async();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full);
-            // O_tile -> running accumulator
-            if (!mbar_wait(o_full, i & 1, &flags[0])) { ok = false; break; }
-            tc_fence_after();
-#pragma unroll
-            for (int c4 = 0; c4 < HD / 32; ++c4) {
-                float o[32];
-                tmem_ld32(tmem_O + c4 * 32 + lane_sel, o);
-#pragma unroll
-                for (int d = 0; d < 32; ++d) acc[c4 * 32 + d] = acc[c4 * 32 + d] * alpha + o[d];
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_empty);
+            if (lane == 0) mbar_arrive(&p_full[wg]);
         }
+        // this warpgroup's last P.V
+        if (ok && k > 0 && !mbar_wait(&pv_done[wg], (k & 1) ^ 1, &flags[0])) ok = false;
         if (!ok) {
             flags[0] = 1;
             if (lane == 0 && p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
         }
-        epi_bar();
-        if (!flags[0]) {
-            const bool row_valid = r < p.R;
+        tc_fence_after();
+        // ---- merge the two accumulators: warpgroup 1 hands (max, sum, O_1 row) over through the idle ring
+        float* stage = reinterpret_cast<float*>(sKV);
+        const bool row_valid = r < p.R;
+        both_bar();              // every contraction of both warpgroups is complete: the ring is idle
+        if (wg == 1 && !flags[0]) {
+            float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);
+            if (k > 0) {
+#pragma unroll
+                for (int c4 = 0; c4 < HD / 32; ++c4) {
+                    float o[32];
+                    tmem_ld32(tmem_O + c4 * 32, o);
+#pragma unroll
+                    for (int d = 0; d < 32; d += 4) srow[(c4 * 32 + d) >> 2] = make_float4(o[d], o[d + 1], o[d + 2], o[d + 3]);
+                }
+            }
+            srow[HD >> 2] = make_float4(k > 0 ? m_run : -CUDART_INF_F, k > 0 ? l_run : 0.f, 0.f, 0.f);
+        }
+        both_bar();
+        if (wg == 0 && !flags[0]) {
+            const float4* orow = reinterpret_cast<const float4*>(stage + row * PART_LD);
+            const float4 ml1 = orow[HD >> 2];
+            const float M = fmaxf(m_run, ml1.x);
+            const float w0 = (m_run > -CUDART_INF_F) ? fast_exp2(m_run - M) : 0.f;
+            const float w1 = (ml1.x > -CUDART_INF_F) ? fast_exp2(ml1.x - M) : 0.f;
+            const float l_tot = l_run * w0 + ml1.y * w1;
+            float acc[HD];
+#pragma unroll
+            for (int c4 = 0; c4 < HD / 32; ++c4) {
+                float o[32];
+                tmem_ld32(tmem_O + c4 * 32, o);
+#pragma unroll
+                for (int d = 0; d < 32; d += 4) {
+                    float4 o1 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (w1 > 0.f) o1 = orow[(c4 * 32 + d) >> 2];
+                    acc[c4 * 32 + d + 0] = o[d + 0] * w0 + o1.x * w1;
+                    acc[c4 * 32 + d + 1] = o[d + 1] * w0 + o1.y * w1;
+                    acc[c4 * 32 + d + 2] = o[d + 2] * w0 + o1.z * w1;
+                    acc[c4 * 32 + d + 3] = o[d + 3] * w0 + o1.w * w1;
+                }
+            }
             __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD;
             if (n_splits == 1) {
                 if (row_valid) {
-                    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
 #pragma unroll
                     for (int d = 0; d < HD; d += 8) {
-                        uint4 w;
-                        w.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
-                        w.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
-                        w.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
-                        w.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
-                        *reinterpret_cast<uint4*>(dst + d) = w;
+                        uint4 w4;
+                        w4.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
+                        w4.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
+                        w4.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
+                        w4.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + d) = w4;
                     }
                 }
             } else {
-                // partial result of this KV range: rows staged through the (now idle) K/V ring so the
-                // global write is one contiguous, coalesced copy
-                float* stage = reinterpret_cast<float*>(sKV);
+                // partial result of this KV range: rows staged so that the global write is one contiguous copy
+                wg_bar(0);               // every row of the hand-over area has been read
                 if (row_valid) {
                     float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);
 #pragma unroll
                     for (int d = 0; d < HD; d += 4) srow[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-                    srow[HD >> 2] = make_float4(m_run, l_run, 0.f, 0.f);
+                    srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
                 }
-                epi_bar();
-                const int n_valid_rows = min(128, p.R * p.group);
+                wg_bar(0);
                 const int bg = b * p.Hkv + g;
-                float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * 128 * PART_LD);
+                float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * p.rows_valid * PART_LD);
                 const float4* src4 = reinterpret_cast<const float4*>(stage);
-                for (int e = row; e < n_valid_rows * (PART_LD / 4); e += 128) dst4[e] = src4[e];
+                for (int e = row; e < p.rows_valid * (PART_LD / 4); e += 128) dst4[e] = src4[e];
             }
         }
     }
@@ -365,7 +425,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -380,7 +439,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     pdl_trigger();
     pdl_wait();
     if (threadIdx.x == 0) trace_min(trace, 1);
-    const int rows_valid = min(128, p.R * p.group);
+    const int rows_valid = p.rows_valid;
     const int row_blocks = (rows_valid + 3) / 4;
     const int bg = blockIdx.x / row_blocks;
     const int row = (blockIdx.x % row_blocks) * 4 + (threadIdx.x >> 5);
@@ -390,8 +449,8 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     const int T = (L + PG - 1) / PG + 1;
     const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
     if (n_splits <= 1 || row >= rows_valid) return;
-    const float* base = p.part + ((size_t)bg * p.n_chunks * 128 + row) * PART_LD;
-    const size_t unit_stride = (size_t)128 * PART_LD;
+    const float* base = p.part + ((size_t)bg * p.n_chunks * rows_valid + row) * PART_LD;
+    const size_t unit_stride = (size_t)rows_valid * PART_LD;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float Lsum = 0.f;
     // Few dependent round trips: lane s fetches (max, sum) of range s (all ranges in flight at once),
@@ -440,7 +499,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     w2.x = pack_bf16(acc.x * inv, acc.y * inv);
     w2.y = pack_bf16(acc.z * inv, acc.w * inv);
     *reinterpret_cast<uint2*>(dst) = w2;
-    if (lane == 0) trace_max(trace, 3);
+    if (threadIdx.x == 0) trace_max(trace, 3);
 }
 
 }  // namespace
@@ -451,20 +510,26 @@ bool attn_tc_supported(const dflash_config& c, int rows) {
     return group >= 1 && 128 % group == 0 && rows * group <= 128 && rows <= PG;
 }
 
-// Keys are split into ranges of `tiles_per_unit` 64-key tiles so that the grid is about one wave of
-// CTAs (the longest sequence decides; shorter ones leave empty units that exit at once).
+// Keys are split into ranges of `tiles_per_unit` 64-key tiles. One sequence: about one wave of equal
+// CTAs. A batch: lengths differ (shorter sequences leave empty units that exit at once), so ranges
+// of at least 8 tiles and enough of them for several waves.
 static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
     const int Tmax = (max_ctx_len + PG - 1) / PG + 1;
     const int64_t bh = (int64_t)batch * Hkv;
+    if (batch > 1) {
+        const int64_t c = (bh * Tmax + 8 * (int64_t)sm_count - 1) / (8 * (int64_t)sm_count);
+        return (int)std::min<int64_t>(std::max<int64_t>(8, c), std::max(2, Tmax));
+    }
     for (int c = 2; c < Tmax; ++c)
         if (bh * ((Tmax + c - 1) / c) <= sm_count) return c;
     return std::max(2, Tmax);
 }
 
-int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int sm_count) {
-    // units never exceed max(SMs, batch*Hkv*ceil(Tmax/2)) <= 2*SMs + 2*batch*Hkv (see tiles_per_unit)
-    const int64_t units = 2 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
-    return units * 128 * PART_LD * 4;
+int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count) {
+    // units: one sequence <= SMs (+ rounding); a batch <= 8*SMs + batch*Hkv (ranges of >= total/(8*SMs) tiles)
+    const int64_t units = 8 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
+    const int rows_valid = std::min(128, rows * (c.n_q_heads / c.n_kv_heads));
+    return units * rows_valid * PART_LD * 4;
 }
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
 
@@ -476,11 +541,13 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.max_pages = a.max_pages; p.n_pages = a.n_pool_pages; p.layer = a.layer;
     p.causal = a.mode == DFLASH_ATTN_CAUSAL ? 1 : 0;
     p.tiles_per_unit = tiles_per_unit(a.batch, c.n_kv_heads, a.max_ctx_len, L.h->sm_count);
+    p.rows_valid = std::min(128, a.rows * p.group);
     const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
     p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
     p.ctx_len = a.ctx_len; p.page_table = a.page_table;
-    p.out = (__nv_bfloat16*)a.out; p.part = part; p.counters = counters; p.status = L.status; p.trace = L.trace;
+    p.out = (__nv_bfloat16*)a.out; p.part = part; p.status = L.status; p.trace = L.trace;
+    (void)counters;
 
     CUtensorMap tq, tpool, tkb, tvb;
     {   // q as [S*R][Hkv][group][hd]
@@ -514,7 +581,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
         return DFLASH_ERR_CUDA;
     ++g_launches;
     if (p.n_chunks > 1) {
-        const int rows_valid = std::min(128, a.rows * p.group);
+        const int rows_valid = p.rows_valid;
         if (launch_pdl(attn_combine_kernel, dim3(a.batch * p.Hkv * ((rows_valid + 3) / 4)), dim3(128), 0, L.st, p) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         ++g_launches;

@@ -7,7 +7,7 @@ namespace dflash {
 
 // head_dim 128, 64-token pages, rows * (Hq/Hkv) <= 128
 bool attn_tc_supported(const dflash_config& c, int rows);
-int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int sm_count);
+int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count);
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
 // `part` / `counters`: split-KV scratch of the sizes above; counters must be zero on entry.
 int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters);
