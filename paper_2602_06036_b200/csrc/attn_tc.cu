@@ -2,9 +2,10 @@
 //   every block row of a sequence attends over [paged context K/V ; the block's own K/V].
 // One CTA works on one (sequence, kv head, range of KV tiles). The queries of all block rows and of
 // the q heads that share the kv head (rows x group <= 128) are the 128-row "M" operand; a KV tile
-// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (4-deep K/V ring that
-// runs ahead of the math), an MMA-issuing warp, and TWO softmax warpgroups that take alternate
-// tiles, each with its own S buffer, P buffer and output accumulator:
+// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (5-deep K/V ring that
+// runs ahead of the math) and TWO independent pipelines that take alternate tiles, each made of one
+// MMA-issuing warp and one softmax warpgroup with their own S buffers (two, so the next S is ready
+// before the current softmax ends), P buffer and output accumulator:
 //   S_w = Q K^T          tcgen05.mma into TMEM
 //   softmax              one thread per query row reads its S row from TMEM (no cross-thread
 //                        reduction), exponentials in the log2 domain against a running maximum that
@@ -32,14 +33,15 @@ using namespace ptx;
 
 constexpr int HD = 128;          // head_dim
 constexpr int PG = 64;           // tokens per page = keys per tile
-constexpr int NS = 4;            // K/V ring depth
+constexpr int NS = 5;            // K/V ring depth
 constexpr int Q_BYTES = 128 * HD * 2;            // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
 constexpr int P_BYTES = 128 * PG * 2;            // 16 KiB per warpgroup
 constexpr int PART_LD = HD + 4;                  // acc[128], running max, running sum, 2 pad (16-byte rows)
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512;
-constexpr uint32_t TMEM_COLS = 512;              // S0 | S1 (64 each) | O0 | O1 (128 each)
-constexpr int N_THREADS = 320;                   // producer, MMA issuer, 2 x 4 softmax warps
+constexpr uint32_t TMEM_COLS = 512;              // S[w][2] (4 x 64) | O0 | O1 (128 each)
+constexpr int N_THREADS = 352;                   // producer, MMA issuer 0, 2 x 4 softmax warps, MMA issuer 1
+constexpr uint32_t TMEM_O = 256;                 // first column of the output accumulators
 constexpr float RESCALE_GAP = 8.f;               // log2 units
 
 struct AParams {
@@ -141,25 +143,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t* q_full = bars;
     uint64_t* kv_full = bars + 1;
     uint64_t* kv_empty = kv_full + NS;
-    uint64_t* s_full = kv_empty + NS;      // [2] S_w written by the tensor core
-    uint64_t* s_free = s_full + 2;         // [2] S_w read by its warpgroup
-    uint64_t* p_full = s_free + 2;         // [2] P_w written (and O_w rescaled if needed)
+    uint64_t* s_full = kv_empty + NS;      // [2][2] S buffer (pipeline w, buffer) written by the tensor core
+    uint64_t* s_free = s_full + 4;         // [2][2] S buffer read by its warpgroup
+    uint64_t* p_full = s_free + 4;         // [2] P_w written (and O_w rescaled if needed)
     uint64_t* pv_done = p_full + 2;        // [2] O_w += P_w V finished (P_w reusable, O_w consistent)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort
+    volatile int* tile_ok = flags + 2;      // [NS] 0 if the ring stage holds a page that must be ignored
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
         for (int s = 0; s < NS; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&p_full[s], 4); mbar_init(&pv_done[s], 1);
-        }
+        for (int s = 0; s < 4; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&p_full[s], 4); mbar_init(&pv_done[s], 1); }
         flags[0] = 0;
         fence_barrier_init();
         fence_proxy_async();
     }
-    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);      // warp 1 owns the allocation
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -184,9 +186,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const int t = t_lo + i;
                 if (t < n_ctx_tiles) {
                     int page = t < p.max_pages ? p.page_table[(size_t)b * p.max_pages + t] : -1;
+                    tile_ok[st] = 1;
                     if (page < 0 || page >= p.n_pages) {
                         if (p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
                         page = 0;      // loaded but fully masked by the softmax warps
+                        tile_ok[st] = 0;
                     }
                     // pool rows: ((((layer*n_pages + page)*2 + kv)*Hkv + head)*PG + slot), hd contiguous
                     const int rowK = ((((p.layer * p.n_pages + page) * 2 + 0) * p.Hkv + g) * PG);
@@ -209,44 +213,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
         __syncwarp();     // the whole warp must reach the closing barrier together
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp == 1 || warp == 10) {
+        // ---------------- MMA issuers: warp 1 drives pipeline 0 (even tiles), warp 10 pipeline 1 ----------------
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc_bf16(128, PG);
             constexpr uint32_t idesc_o = instr_desc_bf16_bmn(128, HD);
-            const uint32_t q_addr = smem_u32(sQ);
+            const uint32_t w = (warp == 1) ? 0u : 1u;
+            const int n_mine = (n_tiles - (int)w + 1) / 2;          // tiles w, w+2, ...
+            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP + w * P_BYTES);
             bool ok = mbar_wait(q_full, 0, &flags[0]);
-            // tile i belongs to warpgroup w = i & 1 and is that warpgroup's (i >> 1)-th tile
-            auto issue_s = [&](int i) -> bool {
-                const int st = i % NS;
-                const uint32_t w = i & 1, k = (uint32_t)i >> 1;
+            // S of this pipeline's k-th tile into its buffer k & 1
+            auto issue_s = [&](int k) -> bool {
+                const int i = 2 * k + (int)w, st = i % NS;
+                const uint32_t bsel = k & 1;
                 if (!mbar_wait(&kv_full[st], (i / NS) & 1, &flags[0])) return false;
-                if (!mbar_wait(&s_free[w], (k & 1) ^ 1, &flags[0])) return false;
+                if (!mbar_wait(&s_free[w * 2 + bsel], ((k >> 1) & 1) ^ 1, &flags[0])) return false;
                 tc_fence_after();
                 const uint32_t k_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_bf16(tmem_base + w * PG, smem_desc_sw128(q_addr + (kk >> 2) * (Q_BYTES / 2) + (kk & 3) * 32),
+                    mma_bf16(tmem_base + (w * 2 + bsel) * PG, smem_desc_sw128(q_addr + (kk >> 2) * (Q_BYTES / 2) + (kk & 3) * 32),
                              smem_desc_sw128(k_addr + (kk >> 2) * 8192 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-                mma_commit(&s_full[w]);
+                mma_commit(&s_full[w * 2 + bsel]);
                 return true;
             };
-            if (ok) ok = issue_s(0);
-            if (ok && n_tiles > 1) ok = issue_s(1);
-            for (int i = 0; i < n_tiles && ok; ++i) {
-                const int st = i % NS;
-                const uint32_t w = i & 1, k = (uint32_t)i >> 1;
+            if (ok && n_mine > 0) ok = issue_s(0);
+            if (ok && n_mine > 1) ok = issue_s(1);
+            for (int k = 0; k < n_mine && ok; ++k) {
+                const int i = 2 * k + (int)w, st = i % NS;
                 if (!mbar_wait(&p_full[w], k & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t v_addr = smem_u32(sKV + (size_t)st * KV_STAGE_BYTES + KV_STAGE_BYTES / 2);
-                const uint32_t p_addr = smem_u32(sP + w * P_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < PG / 16; ++kk)
-                    mma_bf16(tmem_base + 128 + w * HD, smem_desc_sw128(p_addr + kk * 32), smem_desc_sw128_mn(v_addr + kk * 2048),
-                             idesc_o, (k > 0 || kk > 0) ? 1u : 0u);      // a warpgroup's first tile starts its accumulator
+                    mma_bf16(tmem_base + TMEM_O + w * HD, smem_desc_sw128(p_addr + kk * 32), smem_desc_sw128_mn(v_addr + kk * 2048),
+                             idesc_o, (k > 0 || kk > 0) ? 1u : 0u);      // a pipeline's first tile starts its accumulator
                 mma_commit(&pv_done[w]);
                 mma_commit(&kv_empty[st]);
-                if (i + 2 < n_tiles) ok = issue_s(i + 2);
+                if (k + 2 < n_mine) ok = issue_s(k + 2);
             }
             if (!ok) {
                 flags[0] = 1;
@@ -261,8 +265,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int row = ew * 32 + lane;                     // query row = TMEM lane
         const int r = row / p.group, j = row % p.group;     // block row, q head inside the group
         const uint32_t lane_sel = (uint32_t)(ew * 32) << 16;
-        const uint32_t tmem_S = tmem_base + wg * PG + lane_sel;
-        const uint32_t tmem_O = tmem_base + 128 + wg * HD + lane_sel;
+        const uint32_t tmem_O = tmem_base + TMEM_O + wg * HD + lane_sel;
         uint8_t* myP = sP + wg * P_BYTES;
         float m_run = -CUDART_INF_F, l_run = 0.f;           // log2-domain reference maximum, running sum
         bool ok = true;
@@ -274,36 +277,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             int n_valid, n_vis;
             if (t < n_ctx_tiles) {
                 n_valid = min(PG, L - t * PG);
-                const int page = t < p.max_pages ? p.page_table[(size_t)b * p.max_pages + t] : -1;
-                if (page < 0 || page >= p.n_pages) n_valid = 0;
                 n_vis = n_valid;
             } else {
                 n_valid = p.R;
                 n_vis = p.causal ? min(r + 1, p.R) : p.R;
             }
-            if (!mbar_wait(&s_full[wg], k & 1, &flags[0])) { ok = false; break; }
+            const uint32_t bsel = k & 1;
+            const uint32_t tmem_S = tmem_base + (wg * 2 + bsel) * PG + lane_sel;
+            if (!mbar_wait(&s_full[wg * 2 + bsel], (k >> 1) & 1, &flags[0])) { ok = false; break; }
             tc_fence_after();
-            float s[PG];
-            tmem_ld32(tmem_S, s);
-            tmem_ld32(tmem_S + 32, s + 32);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_free[wg]);
-            float mx = -CUDART_INF_F;
+            if (t < n_ctx_tiles && !tile_ok[st]) { n_valid = 0; n_vis = 0; }   // written by the producer before the tile's copy
+            // pass 1 over the S row (32 columns at a time, straight from TMEM): the row maximum
+            float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-            for (int c = 0; c < PG; ++c) {
-                s[c] = (c < n_vis) ? s[c] * p.scale_log2 : -CUDART_INF_F;
-                mx = fmaxf(mx, s[c]);
+            for (int h = 0; h < 2; ++h) {
+                float s[32];
+                tmem_ld32(tmem_S + h * 32, s);
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    if (h * 32 + c < n_vis) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
             }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;   // scale > 0
             // raise the reference maximum only when this tile tops it by more than the gap
             const bool raise = mx > m_run + RESCALE_GAP || (m_run == -CUDART_INF_F && mx > -CUDART_INF_F);
             const float m_new = raise ? mx : m_run;
             const float alpha = (raise && m_run > -CUDART_INF_F) ? fast_exp2(m_run - m_new) : 1.f;
             const float m_use = (m_new > -CUDART_INF_F) ? m_new : 0.f;
-            float psum = 0.f;
-#pragma unroll
-            for (int c = 0; c < PG; ++c) { s[c] = fast_exp2(s[c] - m_use); psum += s[c]; }
-            l_run = l_run * alpha + psum;
             m_run = m_new;
             // the previous P_w V of this warpgroup must be finished before P_w is rewritten or O_w rescaled
             if (!mbar_wait(&pv_done[wg], (k & 1) ^ 1, &flags[0])) { ok = false; break; }
@@ -320,16 +319,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 tmem_st_wait();
                 tc_fence_before();
             }
+            // pass 2: exponentials, row sum, P (bf16) into the swizzled K-major tile
+            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
             uint8_t* prow = myP + row * 128;
 #pragma unroll
-            for (int ck = 0; ck < 8; ++ck) {
-                uint4 w4;
-                w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
-                w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
-                w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
-                w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
-                *reinterpret_cast<uint4*>(prow + ((ck ^ (row & 7)) << 4)) = w4;
+            for (int h = 0; h < 2; ++h) {
+                float s[32];
+                tmem_ld32(tmem_S + h * 32, s);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    s[c] = (h * 32 + c < n_vis) ? fast_exp2(fmaf(s[c], p.scale_log2, -m_use)) : 0.f;
+                    ps4[c & 3] += s[c];
+                }
+#pragma unroll
+                for (int ck = 0; ck < 4; ++ck) {
+                    uint4 w4;
+                    w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
+                    w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
+                    w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
+                    w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
+                    *reinterpret_cast<uint4*>(prow + (((h * 4 + ck) ^ (row & 7)) << 4)) = w4;
+                }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_free[wg * 2 + bsel]);   // this S buffer may be overwritten (tile k + 2)
+            l_run = l_run * alpha + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
             // keys that do not exist must not poison P.V with whatever the page holds there
             if (n_valid < PG) {
                 uint8_t* dV = sKV + (size_t)st * KV_STAGE_BYTES + KV_STAGE_BYTES / 2;
@@ -375,7 +390,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const float w0 = (m_run > -CUDART_INF_F) ? fast_exp2(m_run - M) : 0.f;
             const float w1 = (ml1.x > -CUDART_INF_F) ? fast_exp2(ml1.x - M) : 0.f;
             const float l_tot = l_run * w0 + ml1.y * w1;
-            float acc[HD];
+            __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD;
+            const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+            const float f0 = (n_splits == 1) ? w0 * inv : w0, f1 = (n_splits == 1) ? w1 * inv : w1;
+            float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);     // this thread's own row
+            // 32 columns at a time: merged values go straight to the output (one range) or back into this
+            // thread's staging row (several ranges: unnormalised partial, copied out below)
 #pragma unroll
             for (int c4 = 0; c4 < HD / 32; ++c4) {
                 float o[32];
@@ -384,35 +404,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int d = 0; d < 32; d += 4) {
                     float4 o1 = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (w1 > 0.f) o1 = orow[(c4 * 32 + d) >> 2];
-                    acc[c4 * 32 + d + 0] = o[d + 0] * w0 + o1.x * w1;
-                    acc[c4 * 32 + d + 1] = o[d + 1] * w0 + o1.y * w1;
-                    acc[c4 * 32 + d + 2] = o[d + 2] * w0 + o1.z * w1;
-                    acc[c4 * 32 + d + 3] = o[d + 3] * w0 + o1.w * w1;
+                    o[d + 0] = o[d + 0] * f0 + o1.x * f1;
+                    o[d + 1] = o[d + 1] * f0 + o1.y * f1;
+                    o[d + 2] = o[d + 2] * f0 + o1.z * f1;
+                    o[d + 3] = o[d + 3] * f0 + o1.w * f1;
+                }
+                if (n_splits == 1) {
+                    if (row_valid) {
+#pragma unroll
+                        for (int d = 0; d < 32; d += 8) {
+                            uint4 w4;
+                            w4.x = pack_bf16(o[d], o[d + 1]);
+                            w4.y = pack_bf16(o[d + 2], o[d + 3]);
+                            w4.z = pack_bf16(o[d + 4], o[d + 5]);
+                            w4.w = pack_bf16(o[d + 6], o[d + 7]);
+                            *reinterpret_cast<uint4*>(dst + c4 * 32 + d) = w4;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int d = 0; d < 32; d += 4) srow[(c4 * 32 + d) >> 2] = make_float4(o[d], o[d + 1], o[d + 2], o[d + 3]);
                 }
             }
-            __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD;
-            if (n_splits == 1) {
-                if (row_valid) {
-                    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-#pragma unroll
-                    for (int d = 0; d < HD; d += 8) {
-                        uint4 w4;
-                        w4.x = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
-                        w4.y = pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv);
-                        w4.z = pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv);
-                        w4.w = pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv);
-                        *reinterpret_cast<uint4*>(dst + d) = w4;
-                    }
-                }
-            } else {
-                // partial result of this KV range: rows staged so that the global write is one contiguous copy
-                wg_bar(0);               // every row of the hand-over area has been read
-                if (row_valid) {
-                    float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);
-#pragma unroll
-                    for (int d = 0; d < HD; d += 4) srow[d >> 2] = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-                    srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
-                }
+            if (n_splits > 1) {
+                srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
                 wg_bar(0);
                 const int bg = b * p.Hkv + g;
                 float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * p.rows_valid * PART_LD);
