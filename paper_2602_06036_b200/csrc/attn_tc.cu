@@ -2,7 +2,7 @@
 //   every block row of a sequence attends over [paged context K/V ; the block's own K/V].
 // One CTA works on one (sequence, kv head, range of KV tiles). The queries of all block rows and of
 // the q heads that share the kv head (rows x group <= 128) are the 128-row "M" operand; a KV tile
-// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (5-deep K/V ring that
+// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (4-deep K/V ring that
 // runs ahead of the math) and TWO independent pipelines that take alternate tiles, each made of one
 // MMA-issuing warp and one softmax warpgroup with their own S buffers (two, so the next S is ready
 // before the current softmax ends), P buffer and output accumulator:
@@ -13,7 +13,10 @@
 //                        in TMEM is rescaled in place), P -> shared memory (bf16)
 //   O_w += P V           tcgen05.mma accumulating in TMEM, V as an MN-major operand straight from
 //                        the page layout
-// so the softmax of one tile overlaps the contractions of the next, and the output never leaves
+// When the query rows fill at most half of the 128-row operand (the draft block: 16 rows x 4 heads) they
+// are loaded twice; the threads of the second copy sit on the other two TMEM lane quadrants (hence the
+// other two warp schedulers) and take keys 32..63 of every tile, so no issue slot idles on padding.
+// So the softmax of one tile overlaps the contractions of the next, and the output never leaves
 // TMEM until the end, where the two accumulators are merged. Long contexts are split across CTAs;
 // each writes its partial (acc, max, sum) and a small second kernel merges them in range order
 // (bit-reproducible). DRAFT mode: no mask inside the block; VERIFY mode: block row r sees block
@@ -33,12 +36,12 @@ using namespace ptx;
 
 constexpr int HD = 128;          // head_dim
 constexpr int PG = 64;           // tokens per page = keys per tile
-constexpr int NS = 5;            // K/V ring depth
+constexpr int NS = 4;            // K/V ring depth
 constexpr int Q_BYTES = 128 * HD * 2;            // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
 constexpr int P_BYTES = 128 * PG * 2;            // 16 KiB per warpgroup
 constexpr int PART_LD = HD + 4;                  // acc[128], running max, running sum, 2 pad (16-byte rows)
-constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512;
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512 + 2 * 384 * 4;
 constexpr uint32_t TMEM_COLS = 512;              // S[w][2] (4 x 64) | O0 | O1 (128 each)
 constexpr int N_THREADS = 352;                   // producer, MMA issuer 0, 2 x 4 softmax warps, MMA issuer 1
 constexpr uint32_t TMEM_O = 256;                 // first column of the output accumulators
@@ -46,6 +49,7 @@ constexpr float RESCALE_GAP = 8.f;               // log2 units
 
 struct AParams {
     int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks, rows_valid;
+    int dup;     // rows_valid <= 64: the query rows are loaded twice and each copy handles 32 of a tile's 64 keys
     float scale_log2;
     const int32_t* ctx_len;
     const int32_t* page_table;
@@ -150,6 +154,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort
     volatile int* tile_ok = flags + 2;      // [NS] 0 if the ring stage holds a page that must be ignored
+    float* xchg = reinterpret_cast<float*>(const_cast<int*>(tile_ok) + 8);   // [2 pipelines][3][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -173,8 +178,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint64_t pol_kv = policy_evict_first(), pol_q = policy_evict_last();
             mbar_expect_tx(q_full, Q_BYTES);
             // q viewed as [S*R][Hkv][group][hd]: box = 64 x group x 1 x (128/group) -> rows ordered (r, j)
-            tma_load_4d(sQ, &tmQ, 0, 0, g, b * p.R, q_full, pol_q);
-            tma_load_4d(sQ + Q_BYTES / 2, &tmQ, 64, 0, g, b * p.R, q_full, pol_q);
+            if (p.dup) {     // box of 64 rows, placed at rows 0..63 and again at rows 64..127 of each K half
+                for (int hf = 0; hf < 2; ++hf)
+                    for (int cp = 0; cp < 2; ++cp)
+                        tma_load_4d(sQ + hf * (Q_BYTES / 2) + cp * (Q_BYTES / 4), &tmQ, hf * 64, 0, g, b * p.R, q_full, pol_q);
+            } else {
+                tma_load_4d(sQ, &tmQ, 0, 0, g, b * p.R, q_full, pol_q);
+                tma_load_4d(sQ + Q_BYTES / 2, &tmQ, 64, 0, g, b * p.R, q_full, pol_q);
+            }
             bool ok = true;
             for (int i = 0; i < n_tiles; ++i) {
                 const int st = i % NS;
@@ -262,11 +273,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // ---------------- softmax warpgroups: thread = query row ----------------
         const int wg = (warp - 2) >> 2;                     // 0: even tiles, 1: odd tiles
         const int ew = warp & 3;                            // TMEM lane quadrant of this warp
-        const int row = ew * 32 + lane;                     // query row = TMEM lane
-        const int r = row / p.group, j = row % p.group;     // block row, q head inside the group
+        const int row = ew * 32 + lane;                     // TMEM lane
+        const int dup = p.dup;
+        const int half = dup ? (row >> 6) : 0;              // dup: which 32 keys of a tile this thread takes
+        const int lrow = dup ? (row & 63) : row;            // query row
+        const int ncol = dup ? 32 : PG;                     // keys per thread and tile
+        const int r = lrow / p.group, j = lrow % p.group;   // block row, q head inside the group
         const uint32_t lane_sel = (uint32_t)(ew * 32) << 16;
         const uint32_t tmem_O = tmem_base + TMEM_O + wg * HD + lane_sel;
         uint8_t* myP = sP + wg * P_BYTES;
+        float* xch = xchg + wg * 384;                       // [3][128] exchange between the two copies of a row
         float m_run = -CUDART_INF_F, l_run = 0.f;           // log2-domain reference maximum, running sum
         bool ok = true;
         int k = 0;                                          // index of this warpgroup's tile
@@ -283,21 +299,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 n_vis = p.causal ? min(r + 1, p.R) : p.R;
             }
             const uint32_t bsel = k & 1;
-            const uint32_t tmem_S = tmem_base + (wg * 2 + bsel) * PG + lane_sel;
+            const uint32_t tmem_S = tmem_base + (wg * 2 + bsel) * PG + half * 32 + lane_sel;
             if (!mbar_wait(&s_full[wg * 2 + bsel], (k >> 1) & 1, &flags[0])) { ok = false; break; }
             tc_fence_after();
             if (t < n_ctx_tiles && !tile_ok[st]) { n_valid = 0; n_vis = 0; }   // written by the producer before the tile's copy
-            // pass 1 over the S row (32 columns at a time, straight from TMEM): the row maximum
+            const int vis_here = n_vis - half * 32;          // visible keys among this thread's columns
+            // pass 1 over this thread's part of the S row (32 columns at a time, straight from TMEM): the maximum
             float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h * 32 < ncol; ++h) {
                 float s[32];
                 tmem_ld32(tmem_S + h * 32, s);
+                if (vis_here >= (h + 1) * 32) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c)
-                    if (h * 32 + c < n_vis) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+                    for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (h * 32 + c < vis_here) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+                }
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;   // scale > 0
+            float mx_raw = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            if (dup) {       // the other copy of this row looked at the other 32 keys
+                xch[bsel * 128 + row] = mx_raw;
+                wg_bar(wg);
+                mx_raw = fmaxf(mx_raw, xch[bsel * 128 + (row ^ 64)]);
+            }
+            const float mx = mx_raw * p.scale_log2;          // scale > 0
             // raise the reference maximum only when this tile tops it by more than the gap
             const bool raise = mx > m_run + RESCALE_GAP || (m_run == -CUDART_INF_F && mx > -CUDART_INF_F);
             const float m_new = raise ? mx : m_run;
@@ -306,7 +333,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             m_run = m_new;
             // the previous P_w V of this warpgroup must be finished before P_w is rewritten or O_w rescaled
             if (!mbar_wait(&pv_done[wg], (k & 1) ^ 1, &flags[0])) { ok = false; break; }
-            if (k > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+            if (k > 0 && half == 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                 tc_fence_after();
 #pragma unroll
                 for (int c4 = 0; c4 < HD / 32; ++c4) {
@@ -321,15 +348,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             // pass 2: exponentials, row sum, P (bf16) into the swizzled K-major tile
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-            uint8_t* prow = myP + row * 128;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            uint8_t* prow = myP + lrow * 128;
+            for (int h = 0; h * 32 < ncol; ++h) {
                 float s[32];
                 tmem_ld32(tmem_S + h * 32, s);
+                if (vis_here >= (h + 1) * 32) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    s[c] = (h * 32 + c < n_vis) ? fast_exp2(fmaf(s[c], p.scale_log2, -m_use)) : 0.f;
-                    ps4[c & 3] += s[c];
+                    for (int c = 0; c < 32; ++c) {
+                        s[c] = fast_exp2(fmaf(s[c], p.scale_log2, -m_use));
+                        ps4[c & 3] += s[c];
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        s[c] = (h * 32 + c < vis_here) ? fast_exp2(fmaf(s[c], p.scale_log2, -m_use)) : 0.f;
+                        ps4[c & 3] += s[c];
+                    }
                 }
 #pragma unroll
                 for (int ck = 0; ck < 4; ++ck) {
@@ -338,7 +372,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
                     w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
                     w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
-                    *reinterpret_cast<uint4*>(prow + (((h * 4 + ck) ^ (row & 7)) << 4)) = w4;
+                    *reinterpret_cast<uint4*>(prow + ((((half + h) * 4 + ck) ^ (lrow & 7)) << 4)) = w4;
                 }
             }
             tc_fence_before();
@@ -365,11 +399,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (lane == 0 && p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
         }
         tc_fence_after();
+        if (dup) {               // whole-row sum: the two copies add their parts
+            xch[256 + row] = l_run;
+            wg_bar(wg);
+            l_run += xch[256 + (row ^ 64)];
+        }
         // ---- merge the two accumulators: warpgroup 1 hands (max, sum, O_1 row) over through the idle ring
         float* stage = reinterpret_cast<float*>(sKV);
         const bool row_valid = r < p.R;
         both_bar();              // every contraction of both warpgroups is complete: the ring is idle
-        if (wg == 1 && !flags[0]) {
+        if (wg == 1 && half == 0 && !flags[0]) {
             float4* srow = reinterpret_cast<float4*>(stage + row * PART_LD);
             if (k > 0) {
 #pragma unroll
@@ -383,7 +422,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             srow[HD >> 2] = make_float4(k > 0 ? m_run : -CUDART_INF_F, k > 0 ? l_run : 0.f, 0.f, 0.f);
         }
         both_bar();
-        if (wg == 0 && !flags[0]) {
+        if (wg == 0 && half == 0 && !flags[0]) {
             const float4* orow = reinterpret_cast<const float4*>(stage + row * PART_LD);
             const float4 ml1 = orow[HD >> 2];
             const float M = fmaxf(m_run, ml1.x);
@@ -426,14 +465,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     for (int d = 0; d < 32; d += 4) srow[(c4 * 32 + d) >> 2] = make_float4(o[d], o[d + 1], o[d + 2], o[d + 3]);
                 }
             }
-            if (n_splits > 1) {
-                srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
-                wg_bar(0);
-                const int bg = b * p.Hkv + g;
-                float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * p.rows_valid * PART_LD);
-                const float4* src4 = reinterpret_cast<const float4*>(stage);
-                for (int e = row; e < p.rows_valid * (PART_LD / 4); e += 128) dst4[e] = src4[e];
-            }
+            if (n_splits > 1) srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
+        }
+        if (wg == 0 && n_splits > 1 && !flags[0]) {
+            wg_bar(0);
+            const int bg = b * p.Hkv + g;
+            float4* dst4 = reinterpret_cast<float4*>(p.part + ((size_t)bg * p.n_chunks + chunk) * p.rows_valid * PART_LD);
+            const float4* src4 = reinterpret_cast<const float4*>(stage);
+            for (int e = row; e < p.rows_valid * (PART_LD / 4); e += 128) dst4[e] = src4[e];
         }
     }
 
@@ -557,6 +596,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.causal = a.mode == DFLASH_ATTN_CAUSAL ? 1 : 0;
     p.tiles_per_unit = tiles_per_unit(a.batch, c.n_kv_heads, a.max_ctx_len, L.h->sm_count);
     p.rows_valid = std::min(128, a.rows * p.group);
+    p.dup = (p.rows_valid <= 64 && 64 % p.group == 0) ? 1 : 0;
     const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
     p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
@@ -568,7 +608,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     {   // q as [S*R][Hkv][group][hd]
         const uint64_t dims[4] = {(uint64_t)HD, (uint64_t)p.group, (uint64_t)p.Hkv, (uint64_t)a.batch * a.rows};
         const uint64_t str[3] = {(uint64_t)HD * 2, (uint64_t)p.group * HD * 2, (uint64_t)p.Hq * HD * 2};
-        const uint32_t box[4] = {64, (uint32_t)p.group, 1, (uint32_t)(128 / p.group)};
+        const uint32_t box[4] = {64, (uint32_t)p.group, 1, (uint32_t)((p.dup ? 64 : 128) / p.group)};
         if (!tmap_encode_bf16(&tq, a.q, 4, dims, str, box)) return DFLASH_ERR_CUDA;
     }
     {   // the whole pool as rows of head_dim
