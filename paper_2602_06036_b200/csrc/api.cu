@@ -37,7 +37,7 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     int64_t part = 0, counters = 0;
     if (tc) {
         const int M = (int)R, sm = h->sm_count;
-        const int kv_groups = std::min(c.n_layers, GEMM_MAX_GROUPS);
+        const int kv_groups = std::min(c.n_layers, GEMM_MAX_GROUPS - 1);
         // order = Workspace::CNT_* : every contraction shape has its own ticket range
         const int shapes[Workspace::CNT_N][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
                                                  {c.d_model, c.d_ffn, 1},         {c.vocab, c.d_model, 1}, {c.d_model, feat, 1},
@@ -316,16 +316,27 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
         g.epilogue = EPI_STORE_F32; g.g_next = h->w.g_c; g.xn_out = (__nv_bfloat16*)ws.u; g.ssq_out = ws.ssq;
         g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_FUSE];
         int flag_set = 0;
-        RUN(FAM_CTX_FUSE, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
-        for (int i0 = 0; i0 < c.n_layers; i0 += GEMM_MAX_GROUPS) {
+        bool fused_done = false;
+        for (int i0 = 0; i0 < c.n_layers; i0 += GEMM_MAX_GROUPS - 1) {
             GemmArgs k{};
-            k.n_groups = std::min(GEMM_MAX_GROUPS, c.n_layers - i0);
+            k.n_groups = std::min(GEMM_MAX_GROUPS - 1, c.n_layers - i0);
             for (int j = 0; j < k.n_groups; ++j) k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
             k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
             k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part;
             k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV];
             if (flag_set >= ws.n_flag_sets - 1) return DFLASH_ERR_UNSUPPORTED;
-            RUN(FAM_CTX_KV, launch_gemm_tc(L, k, ws.flags + GEMM_MAX_PHASES * flag_set++));
+            if (!fused_done) {
+                // one launch: the fusion contraction, then the K/V contractions of the first layers as its second phase
+                GemmArgs ph[2] = {g, k};
+                unsigned long long* tr[2] = {trace_slot(h, FAM_CTX_FUSE), trace_slot(h, FAM_CTX_KV)};
+                prof_begin(L, FAM_GEMM_CHAIN);
+                const int rc = launch_gemm_chain(L, ph, 2, ws.flags + GEMM_MAX_PHASES * flag_set++, tr);
+                prof_end(L);
+                if (rc != DFLASH_OK) return rc;
+                fused_done = true;
+            } else {
+                RUN(FAM_CTX_KV, launch_gemm_tc(L, k, ws.flags + GEMM_MAX_PHASES * flag_set++));
+            }
         }
         return DFLASH_OK;
     }
