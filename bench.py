@@ -156,40 +156,50 @@ class Step:
         self.e_anchor = torch.empty_like(self.d_anchor)
         self.e_logits = torch.empty_like(self.d_logits)
         self.n_new = (planted + 1).to(torch.int32).to(device)      # rows committed by the previous cycle
-        self.draft_ids = torch.zeros((S, B), dtype=torch.int32, device=device)
-        self.tau = torch.zeros(S, dtype=torch.int32, device=device)
-        self.out_tokens = torch.zeros((S, g + 1), dtype=torch.int32, device=device)
-        self.bonus = torch.zeros(S, dtype=torch.int32, device=device)
-        self.new_len = torch.zeros(S, dtype=torch.int32, device=device)
-        self.h_out = torch.zeros((S, B + g + 1 + 3), dtype=torch.int32).pin_memory()
-        self.d_out = torch.zeros((S, B + g + 1 + 3), dtype=torch.int32, device=device)
+        # every result of a step lives in one flat int32 buffer, so the end-to-end run reads it back in one copy
+        n_out = S * B + S * (g + 1) + 3 * S
+        self.d_out = torch.zeros(n_out, dtype=torch.int32, device=device)
+        self.h_out = torch.zeros(n_out, dtype=torch.int32).pin_memory()
+        o = 0
+        self.draft_ids = self.d_out[o:o + S * B].view(S, B); o += S * B
+        self.out_tokens = self.d_out[o:o + S * (g + 1)].view(S, g + 1); o += S * (g + 1)
+        self.tau = self.d_out[o:o + S]; o += S
+        self.bonus = self.d_out[o:o + S]; o += S
+        self.new_len = self.d_out[o:o + S]
         self.max_ctx = max(wl.ctx_lens)
         self.rows_new = int(self.n_new.sum().item())
+        self.side = None
 
-    def run(self, feats, anchor, logits):
+    def run_draft(self, feats, anchor):
         lib = self.lib
         lib.dflash_ctx_project(feats, self.n_new, self.ctx_len, self.page_table, self.pool)
         lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids)
+
+    def run_verify(self, logits):
         # The target's verify pass is outside this library; its logits are an input. The drafts
         # verified are synthetic ones with a planted agreeing prefix (the random-init drafter would
         # never be accepted), so the accept kernel sees realistic accept lengths.
-        lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
-                                 self.out_tokens, self.bonus, self.new_len, logits=logits)
+        self.lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
+                                      self.out_tokens, self.bonus, self.new_len, logits=logits)
 
     def step_resident(self):
-        self.run(self.d_feats, self.d_anchor, self.d_logits)
+        self.run_draft(self.d_feats, self.d_anchor)
+        self.run_verify(self.d_logits)
 
     def step_e2e(self):
+        # The verify logits are only needed at the end of the step: their host-to-device copy runs on a
+        # side stream next to the context projection and the draft (a fork/join inside the captured graph).
+        cur = torch.cuda.current_stream()
+        if self.side is None:
+            self.side = torch.cuda.Stream()
+        self.side.wait_stream(cur)
+        with torch.cuda.stream(self.side):
+            self.e_logits.copy_(self.h_logits, non_blocking=True)
         self.e_feats.copy_(self.h_feats, non_blocking=True)
         self.e_anchor.copy_(self.h_anchor, non_blocking=True)
-        self.e_logits.copy_(self.h_logits, non_blocking=True)
-        self.run(self.e_feats, self.e_anchor, self.e_logits)
-        B, g = self.cfg.block_size, self.gamma
-        self.d_out[:, :B] = self.draft_ids
-        self.d_out[:, B:B + g + 1] = self.out_tokens
-        self.d_out[:, B + g + 1] = self.tau
-        self.d_out[:, B + g + 2] = self.bonus
-        self.d_out[:, B + g + 3] = self.new_len
+        self.run_draft(self.e_feats, self.e_anchor)
+        cur.wait_stream(self.side)
+        self.run_verify(self.e_logits)
         self.h_out.copy_(self.d_out, non_blocking=True)
 
     def e2e_bytes(self):
