@@ -323,7 +323,7 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
             for (int j = 0; j < k.n_groups; ++j) k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
             k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
             k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part;
-            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV];
+            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV]; k.epoch = i0 / (GEMM_MAX_GROUPS - 1) + 1;
             if (flag_set >= ws.n_flag_sets - 1) return DFLASH_ERR_UNSUPPORTED;
             if (!fused_done) {
                 // one launch: the fusion contraction, then the K/V contractions of the first layers as its second phase
@@ -388,7 +388,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             g.X = xn; g.W[0] = h->layers[i].W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model; g.ssq_in = ws.ssq;
             g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
             g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
-            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV];
+            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV]; g.epoch = i + 1;
             return g;
         };
         RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, ws.x, h->layers[0].g1, xn, ws.ssq));
@@ -409,20 +409,20 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             o.X = ws.attn; o.W[0] = lw.W_o; o.M = rows; o.N = c.d_model; o.K = qdim;
             o.epilogue = EPI_RESIDUAL; o.out_f32 = ws.x; o.ld_out = c.d_model; o.part = ws.part;
             o.counters = ws.counters + ws.cnt_off[Workspace::CNT_O];
-            o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq;
+            o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq; o.epoch = i + 1;
             fam[0] = FAM_GEMM_O;
             GemmArgs& u = ph[1];      // h = silu(W_gate u) * (W_up u)
             u = GemmArgs{};
             u.X = xn; u.W[0] = lw.W_gateup; u.M = rows; u.N = 2 * c.d_ffn; u.K = c.d_model; u.ssq_in = ws.ssq;
             u.epilogue = EPI_SWIGLU; u.h = (__nv_bfloat16*)ws.h; u.part = ws.part;
-            u.counters = ws.counters + ws.cnt_off[Workspace::CNT_GATEUP];
+            u.counters = ws.counters + ws.cnt_off[Workspace::CNT_GATEUP]; u.epoch = i + 1;
             fam[1] = FAM_GEMM_GATEUP;
             GemmArgs& d = ph[2];      // x += W_down h; emits the next layer's (or the final) norm inputs
             d = GemmArgs{};
             d.X = ws.h; d.W[0] = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
             d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part;
             d.counters = ws.counters + ws.cnt_off[Workspace::CNT_DOWN];
-            d.g_next = last ? h->w.g_f : h->layers[i + 1].g1; d.xn_out = xn; d.ssq_out = ws.ssq;
+            d.g_next = last ? h->w.g_f : h->layers[i + 1].g1; d.xn_out = xn; d.ssq_out = ws.ssq; d.epoch = i + 1;
             fam[2] = FAM_GEMM_DOWN;
             if (!last) {
                 ph[3] = qkv_args(i + 1);

@@ -7,9 +7,11 @@
 // buffers so the epilogue of one piece of work overlaps the main loop of the next. The work is the
 // sequence of all (output tile, K chunk) pairs, cut into one contiguous, equally long range per CTA
 // ("stream-K"): every SM streams the same number of weight bytes whatever the tile count. A range
-// that covers a whole output tile goes straight to the epilogue; tiles shared by several CTAs meet
-// in a fixed-order sum done by whichever CTA arrives last at a ticket counter (no waiting,
-// bit-reproducible). RMSNorm never runs as a kernel of its own: epilogues that produce residual
+// that covers a whole output tile goes straight to the epilogue; a tile shared by several CTAs is
+// finished at the end of the phase by ALL of them: each writes its partial sums and a ticket, waits
+// (bounded) until the tile's tickets are complete, and then sums the pieces in CTA order for its own
+// share of the tile's token passes (bit-reproducible, and the finishing work is spread over the CTAs
+// instead of piling up on one). RMSNorm never runs as a kernel of its own: epilogues that produce residual
 // rows also emit the gain-scaled bf16 operand and per-tile sums of squares, and the consuming
 // contraction scales its accumulator columns by the per-token rsqrt.
 // One launch runs a CHAIN of up to four such contractions ("phases": e.g. output projection ->
@@ -54,6 +56,7 @@ struct WMaps {
 
 struct KParams {
     int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, w_map0, x_map;
+    int epoch;                   // how many launches since the tickets were zeroed use this ticket range (>= 1)
     float* part;
     int32_t* counters;
     const float* ssq_in;
@@ -550,6 +553,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             const KParams& p = mp.ph[ph];
             const long long T = (long long)p.n_tiles * p.chunks_total;
             int rstd_tt = -1, info_tt = -1;
+            Unit pend[2];            // this CTA's pieces of shared tiles (at most its first and its last piece)
+            int n_pend = 0;
             for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
@@ -595,41 +600,60 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 if (!un.full) {
-                    // the tile is shared: ticket; the CTA that completes the set sums the pieces in CTA order
-                    const long long x0 = (long long)un.tile * p.chunks_total;
-                    const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
+                    // the tile is shared: publish the piece, take a ticket, finish the tile at the end of the phase
                     __threadfence();
                     epi_bar();
-                    if (row == 0) {
-                        const int old = atomicAdd(p.counters + un.tile, 1);
-                        flags[1] = (old == j1 - j0) ? 1 : 0;
-                        if (old == j1 - j0) p.counters[un.tile] = 0;   // ready for the next launch
+                    if (row == 0) atomicAdd(p.counters + un.tile, 1);
+                    pend[n_pend++] = un;
+                }
+            }
+            if (!alive) break;
+            // ---- shared tiles: wait for every contributor's piece, then do this CTA's share of the passes
+            for (int pi = 0; pi < n_pend && alive; ++pi) {
+                const Unit un = pend[pi];
+                const int tok_base = un.tt * NT;
+                const bool all_tok = p.M <= TOK_CACHE;
+                const int tok_off = all_tok ? tok_base : 0;
+                const long long x0 = (long long)un.tile * p.chunks_total;
+                const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
+                const int n_contrib = j1 - j0 + 1, my_q = (int)blockIdx.x - j0;
+                const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
+                if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
+                if (row == 0) {
+                    const long long t0 = clock64();
+                    bool ok = true;
+                    while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
+                        if (flags[0] || clock64() - t0 > SPIN_LIMIT) { ok = false; break; }
                     }
+                    if (!ok) flags[2] = 1;
+                }
+                epi_bar();
+                if (flags[2]) { alive = false; break; }
+                __threadfence();
+                if (!all_tok) {      // caches hold one token tile at a time
+                    if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && info_tt != un.tt) { token_info(p, tok_base, NT, row, sPos, sPage); info_tt = un.tt; }
+                    if (p.ssq_in && rstd_tt != un.tt) { token_rstd(p, tok_base, NT, row, sRstd); rstd_tt = un.tt; }
                     epi_bar();
-                    if (flags[1]) {
-                        __threadfence();
-                        for (int ch = 0; ch < n_ch; ++ch) {
-                            float acc[CH];
+                }
+                for (int ch = my_q; ch < n_ch; ch += n_contrib) {
+                    float acc[CH];
 #pragma unroll
-                            for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                            // pieces are summed in CTA order; the CH loads of a piece are all in flight together
-                            for (int j = j0; j <= j1; ++j) {
-                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
-                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
-                                float va[CH];
+                    for (int c = 0; c < CH; ++c) acc[c] = 0.f;
+                    // pieces are summed in CTA order; the CH loads of a piece are all in flight together
+                    for (int j = j0; j <= j1; ++j) {
+                        const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
+                        const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+                        float va[CH];
 #pragma unroll
-                                for (int c = 0; c < CH; ++c) va[c] = __ldcg(pa + (size_t)c * TILE_F);
+                        for (int c = 0; c < CH; ++c) va[c] = __ldcg(pa + (size_t)c * TILE_F);
 #pragma unroll
-                                for (int c = 0; c < CH; ++c) acc[c] += va[c];
-                            }
-#pragma unroll
-                            for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
-                            epi_bar();
-                            apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
-                            epi_bar();
-                        }
+                        for (int c = 0; c < CH; ++c) acc[c] += va[c];
                     }
-                    epi_bar();   // flags[1] is rewritten by the next piece
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
+                    epi_bar();
+                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
+                    epi_bar();
                 }
             }
             if (!alive) break;
@@ -791,6 +815,7 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, KParams& p) {
     }
     p.PG = c.page_size; p.first_layer = a.first_layer;
     p.status = L.status;
+    p.epoch = a.epoch > 0 ? a.epoch : 1;
     return DFLASH_OK;
 }
 
