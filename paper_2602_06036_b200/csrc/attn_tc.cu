@@ -122,10 +122,11 @@ __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPool,
                const __grid_constant__ CUtensorMap tmKb, const __grid_constant__ CUtensorMap tmVb, const AParams p) {
     // ---- which work unit ----
+    // Lengths and the page table are inputs of the call (no kernel writes them), so the work unit, the
+    // barriers, the TMEM allocation and the first page numbers are ready before the grid dependency
+    // (q and the block's k/v from the contraction before this kernel) resolves.
     if (threadIdx.x == 0) trace_min(p.trace, 0);
     pdl_trigger();
-    pdl_wait();      // lengths, page table, q and the block's k/v come from earlier kernels
-    if (threadIdx.x == 0) trace_min(p.trace, 1);
     const int chunk = blockIdx.x % p.n_chunks;
     const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
     const int b = blockIdx.x / (p.n_chunks * p.Hkv);
@@ -167,10 +168,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         fence_proxy_async();
     }
     if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);      // warp 1 owns the allocation
+    constexpr int PAGE_PRE = 4;                           // page numbers fetched ahead of the dependency
+    int page_pre[PAGE_PRE];
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < PAGE_PRE; ++i) {
+            const int t = t_lo + i;
+            page_pre[i] = (i < n_tiles && t < n_ctx_tiles && t < p.max_pages) ? __ldg(p.page_table + (size_t)b * p.max_pages + t) : -1;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+    if (threadIdx.x == 0) trace_min(p.trace, 1);
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -196,7 +208,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 mbar_expect_tx(&kv_full[st], KV_STAGE_BYTES);
                 const int t = t_lo + i;
                 if (t < n_ctx_tiles) {
-                    int page = t < p.max_pages ? p.page_table[(size_t)b * p.max_pages + t] : -1;
+                    int page;
+                    if (i < PAGE_PRE) {
+                        page = page_pre[0];
+#pragma unroll
+                        for (int q = 1; q < PAGE_PRE; ++q)
+                            if (i == q) page = page_pre[q];
+                    } else {
+                        page = t < p.max_pages ? __ldg(p.page_table + (size_t)b * p.max_pages + t) : -1;
+                    }
                     tile_ok[st] = 1;
                     if (page < 0 || page >= p.n_pages) {
                         if (p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
@@ -491,25 +511,34 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     unsigned long long* trace = p.trace ? p.trace + 4 : nullptr;   // the record after the main kernel's
     if (threadIdx.x == 0) trace_min(trace, 0);
     pdl_trigger();
-    pdl_wait();
-    if (threadIdx.x == 0) trace_min(trace, 1);
     const int rows_valid = p.rows_valid;
     const int row_blocks = (rows_valid + 3) / 4;
     const int bg = blockIdx.x / row_blocks;
     const int row = (blockIdx.x % row_blocks) * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int b = bg / p.Hkv, g = bg % p.Hkv;
-    const int L = max(p.ctx_len[b], 0);
+    const int L = max(__ldg(p.ctx_len + b), 0);      // an input of the call: no kernel writes it
     const int T = (L + PG - 1) / PG + 1;
     const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
+    pdl_wait();
+    if (threadIdx.x == 0) trace_min(trace, 1);
     if (n_splits <= 1 || row >= rows_valid) return;
     const float* base = p.part + ((size_t)bg * p.n_chunks * rows_valid + row) * PART_LD;
     const size_t unit_stride = (size_t)rows_valid * PART_LD;
+    // One round trip in the common case: the accumulator rows of the first KF ranges and every
+    // range's (max, sum) are requested together; the weights then travel by shuffle.
+    // More than 32 ranges: a first pass over (max, sum) finds the global maximum.
+    constexpr int KF = 20;
+    float4 a[KF];
+    auto fetch = [&](int s_first, int n) {
+#pragma unroll
+        for (int k = 0; k < KF; ++k)
+            a[k] = (k < n) ? __ldcg(reinterpret_cast<const float4*>(base + (size_t)(s_first + k) * unit_stride) + lane)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    fetch(0, min(KF, n_splits));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float Lsum = 0.f;
-    // Few dependent round trips: lane s fetches (max, sum) of range s (all ranges in flight at once),
-    // the weights travel by shuffle, and the accumulator rows are fetched sixteen at a time.
-    // More than 32 ranges: a first pass over (max, sum) finds the global maximum.
     float M = -CUDART_INF_F;
     float2 ml0 = make_float2(-CUDART_INF_F, 0.f);
     for (int s0 = 0; s0 < n_splits; s0 += 32) {
@@ -533,16 +562,12 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
         for (int o = 16; o > 0; o >>= 1) l_mine += __shfl_xor_sync(0xffffffffu, l_mine, o);
         Lsum += l_mine;
         const int n_here = min(32, n_splits - s0);
-        for (int k0 = 0; k0 < n_here; k0 += 16) {
-            float4 a[16];
+        for (int k0 = 0; k0 < n_here; k0 += KF) {
+            if (s0 + k0 > 0) fetch(s0 + k0, min(KF, n_here - k0));
 #pragma unroll
-            for (int k = 0; k < 16; ++k)
-                a[k] = (k0 + k < n_here) ? __ldcg(reinterpret_cast<const float4*>(base + (s0 + k0 + k) * unit_stride) + lane)
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
+            for (int k = 0; k < KF; ++k) {
                 const float w = __shfl_sync(0xffffffffu, w_mine, (k0 + k) & 31);
-                acc.x += a[k].x * w; acc.y += a[k].y * w; acc.z += a[k].z * w; acc.w += a[k].w * w;
+                if (k0 + k < n_here) { acc.x += a[k].x * w; acc.y += a[k].y * w; acc.z += a[k].z * w; acc.w += a[k].w * w; }
             }
         }
     }

@@ -153,10 +153,25 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
     else a.v2 = fmaxf(a.v2, v1);
 }
 
+// Residual rows of one pass (x += ...): loaded by the caller, ahead of whatever else it waits for.
+template <int CH>
+__device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, int tok0, int row, float (&xres)[CH]) {
+    const int f = un.ft * TILE_F + row;
+    const int n_tok = min(CH, p.M - tok0);
+#pragma unroll
+    for (int c = 0; c < CH; ++c) xres[c] = 0.f;
+    if (p.epi == EPI_RESIDUAL && f < p.N) {
+        const float* o = p.out_f32 + (size_t)tok0 * p.ld_out + f;
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+            if (c < n_tok) xres[c] = __ldcg(o + (size_t)c * p.ld_out);
+    }
+}
+
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
 template <int CH>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
-                                               int row, const int* tPos, const int* tPage) {
+                                               int row, const int* tPos, const int* tPage, const float (&xres)[CH]) {
     // tPos / tPage: position and physical page of the 16 tokens of this pass (-1 = skip the token)
     constexpr int ACC_LD = CH + 1;
     constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
@@ -167,15 +182,9 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
         case EPI_RESIDUAL: {
             float xv[CH];
 #pragma unroll
-            for (int c = 0; c < CH; ++c) xv[c] = 0.f;
+            for (int c = 0; c < CH; ++c) xv[c] = (p.epi == EPI_RESIDUAL) ? xres[c] : 0.f;
             if (f < p.N) {
                 float* o = p.out_f32 ? p.out_f32 + (size_t)tok0 * p.ld_out + f : nullptr;
-                // all loads first: they are independent and must not queue behind the stores
-                if (p.epi == EPI_RESIDUAL) {
-#pragma unroll
-                    for (int c = 0; c < CH; ++c)
-                        if (c < n_tok) xv[c] = __ldcg(o + (size_t)c * p.ld_out);
-                }
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
                     if (c < n_tok) {
@@ -346,25 +355,38 @@ __device__ __forceinline__ void token_info(const KParams& p, int tok_base, int n
 }
 
 // rsqrt(mean square) of operand rows tok_base .. tok_base+nt-1 from the per-tile sums of squares:
-// one thread per token, eight partial sums in flight.
+// eight threads per token, sixteen loads in flight per thread-group of a pass (64 tokens per pass).
 __device__ __forceinline__ void token_rstd(const KParams& p, int tok_base, int nt, int row, float* sRstd) {
-    for (int t = row; t < nt; t += 128) {
-        const int tok = tok_base + t;
-        float rs = 1.f;
-        if (tok < p.M) {
-            float s[8];
+    const int sub = row & 7, tl = row >> 3;
+    for (int t0 = 0; t0 < nt; t0 += 64) {
+        float s[4];
+        bool on[4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) s[k] = 0.f;
-            const float* src = p.ssq_in + tok;
-            for (int q = 0; q < p.n_parts_in; q += 8) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    if (q + k < p.n_parts_in) s[k] += __ldcg(src + (size_t)(q + k) * p.M);
-            }
-            const float sum = ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
-            rs = rsqrtf(sum * p.inv_dim_in + p.eps);
+        for (int u = 0; u < 4; ++u) {
+            s[u] = 0.f;
+            const int t = t0 + u * 16 + tl;
+            on[u] = t < nt && tok_base + t < p.M;
         }
-        sRstd[t] = rs;
+        for (int q0 = sub; q0 < p.n_parts_in; q0 += 32) {
+            float v[4][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int q = q0 + 8 * k;
+                    v[u][k] = (on[u] && q < p.n_parts_in) ? __ldcg(p.ssq_in + (size_t)q * p.M + tok_base + t0 + u * 16 + tl) : 0.f;
+                }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) s[u] += (v[u][0] + v[u][1]) + (v[u][2] + v[u][3]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            s[u] += __shfl_xor_sync(0xffffffffu, s[u], 1);
+            s[u] += __shfl_xor_sync(0xffffffffu, s[u], 2);
+            s[u] += __shfl_xor_sync(0xffffffffu, s[u], 4);
+            const int t = t0 + u * 16 + tl;
+            if (sub == 0 && t < nt) sRstd[t] = on[u] ? rsqrtf(s[u] * p.inv_dim_in + p.eps) : 1.f;
+        }
     }
 }
 
@@ -384,6 +406,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     constexpr int X_STAGE_BYTES = NT * BK * 2;
     constexpr int CH = pass_cols(NT);
     constexpr int ACC_LD = CH + 1;
+    constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 2 : 1));   // partial pieces fetched together when finishing
     constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
     const int stages = mp.stages;
     uint8_t* sW = smem;
@@ -552,21 +575,40 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
             const long long T = (long long)p.n_tiles * p.chunks_total;
+            const bool all_tok = p.M <= TOK_CACHE;   // per-token data cached for the whole phase (else per token tile)
+            const bool need_info = p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV;
             int rstd_tt = -1, info_tt = -1;
+            // token positions / pages do not depend on this chain: work them out while the main loop runs
+            if (need_info && all_tok) {
+                token_info(p, 0, p.M, row, sPos, sPage);
+                info_tt = 0;             // visible after the next barrier
+            }
+            // per-token scales: as soon as the previous phase is complete (its sums of squares are final),
+            // long before this phase's first accumulator
+            if (p.ssq_in && all_tok) {
+                if (ph > 0) {
+                    if (row == 0) {
+                        const long long t0 = clock64();
+                        while (ld_acquire(mp.phase_done + ph - 1) < G) {
+                            if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
+                        }
+                    }
+                    epi_bar();
+                    if (flags[2]) { alive = false; break; }
+                }
+                token_rstd(p, 0, p.M, row, sRstd);
+                rstd_tt = 0;
+            }
             Unit pend[2];            // this CTA's pieces of shared tiles (at most its first and its last piece)
             int n_pend = 0;
             for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
-                // Per-token data is cached for the whole phase when the rows fit (else per token tile).
-                const bool all_tok = p.M <= TOK_CACHE;
                 const int tok_off = all_tok ? tok_base : 0;          // index of this tile's first token in the caches
-                // token positions / pages do not depend on this chain: work them out while the main loop runs
-                if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && (all_tok ? info_tt < 0 : info_tt != un.tt)) {
-                    if (all_tok) token_info(p, 0, p.M, row, sPos, sPage);
-                    else token_info(p, tok_base, NT, row, sPos, sPage);
-                    info_tt = un.tt;     // visible after the barrier below
+                if (need_info && !all_tok && info_tt != un.tt) {
+                    token_info(p, tok_base, NT, row, sPos, sPage);
+                    info_tt = un.tt;
                 }
                 const bool got = mbar_wait(&acc_full[buf], aph, &flags[0]);
                 if (!got) flags[2] = 1;
@@ -574,9 +616,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 if (flags[2]) { alive = false; break; }   // uniform over the four warps
                 tc_fence_after();
                 // The accumulator exists, so the previous phase is complete and its sums of squares are final.
-                if (p.ssq_in && (all_tok ? rstd_tt < 0 : rstd_tt != un.tt)) {
-                    if (all_tok) token_rstd(p, 0, p.M, row, sRstd);
-                    else token_rstd(p, tok_base, NT, row, sRstd);
+                if (p.ssq_in && !all_tok && rstd_tt != un.tt) {
+                    token_rstd(p, tok_base, NT, row, sRstd);
                     rstd_tt = un.tt;
                     epi_bar();
                 }
@@ -591,8 +632,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     } else {
 #pragma unroll
                         for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[tok_off + ch * CH + c] : v[c];
+                        float xres[CH];
+                        residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
                         epi_bar();
-                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
+                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres);
                         epi_bar();
                     }
                 }
@@ -612,47 +655,61 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             for (int pi = 0; pi < n_pend && alive; ++pi) {
                 const Unit un = pend[pi];
                 const int tok_base = un.tt * NT;
-                const bool all_tok = p.M <= TOK_CACHE;
                 const int tok_off = all_tok ? tok_base : 0;
                 const long long x0 = (long long)un.tile * p.chunks_total;
                 const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
                 const int n_contrib = j1 - j0 + 1, my_q = (int)blockIdx.x - j0;
                 const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
                 if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
+                // residual rows of the first pass travel while the tickets are polled
+                float xres[CH];
+                if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres);
                 if (row == 0) {
                     const long long t0 = clock64();
-                    bool ok = true;
                     while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
-                        if (flags[0] || clock64() - t0 > SPIN_LIMIT) { ok = false; break; }
+                        if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
                     }
-                    if (!ok) flags[2] = 1;
                 }
-                epi_bar();
+                epi_bar();               // row 0's acquire, then the barrier: every piece is visible to all rows
                 if (flags[2]) { alive = false; break; }
-                __threadfence();
                 if (!all_tok) {      // caches hold one token tile at a time
-                    if ((p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV) && info_tt != un.tt) { token_info(p, tok_base, NT, row, sPos, sPage); info_tt = un.tt; }
+                    if (need_info && info_tt != un.tt) { token_info(p, tok_base, NT, row, sPos, sPage); info_tt = un.tt; }
                     if (p.ssq_in && rstd_tt != un.tt) { token_rstd(p, tok_base, NT, row, sRstd); rstd_tt = un.tt; }
                     epi_bar();
                 }
                 for (int ch = my_q; ch < n_ch; ch += n_contrib) {
+                    if constexpr (CH <= 32) {
+                        if (ch != my_q) residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
+                    }
                     float acc[CH];
 #pragma unroll
                     for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                    // pieces are summed in CTA order; the CH loads of a piece are all in flight together
-                    for (int j = j0; j <= j1; ++j) {
-                        const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
-                        const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
-                        float va[CH];
+                    // pieces are summed in CTA order; the loads of PF pieces are all in flight together
+                    for (int jb = j0; jb <= j1; jb += PF) {
+                        float va[PF][CH];
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) va[c] = __ldcg(pa + (size_t)c * TILE_F);
+                        for (int u = 0; u < PF; ++u) {
+                            const int j = jb + u;
+                            if (j <= j1) {
+                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
+                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) acc[c] += va[c];
+                                for (int c = 0; c < CH; ++c) va[u][c] = __ldcg(pa + (size_t)c * TILE_F);
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) va[u][c] = 0.f;
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < PF; ++u)
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) acc[c] += va[u][c];
                     }
 #pragma unroll
                     for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
+                    if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
                     epi_bar();
-                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH);
+                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres);
                     epi_bar();
                 }
             }
