@@ -468,6 +468,24 @@ def main():
                               "same weights and row count as in the step",
                     "in_step_us": kernels.get("lmhead_argmax", {}).get("us_per_launch")}
     step_bytes = alg["draft_block_total"] + alg["ctx_project_total"] + S * (B + 1) * cfg.vocab * 2
+    # lower bound of the step: its phases run one after the other, each bound by the slower of its
+    # HBM traffic and its dense bf16 contraction (2 x rows x weights; sustained tensor figure)
+    tensor = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    es = 4 if cfg.dtype == "fp32" else 2
+    bound_s, tensor_phases = 0.0, []
+    for fam, n_launch, rows in (("ctx_fuse", 1, step.rows_new), ("ctx_kv", 1, step.rows_new),
+                                ("gemm_qkv", cfg.n_layers, S * B), ("gemm_o", cfg.n_layers, S * B),
+                                ("gemm_gateup", cfg.n_layers, S * B), ("gemm_down", cfg.n_layers, S * B),
+                                ("lmhead_argmax", 1, S * B), ("attention", cfg.n_layers, 0)):
+        t_hbm = alg[fam] / (hbm * 1e9)
+        t_tc = 2.0 * rows * (alg[fam] / es) / tensor if cfg.dtype != "fp32" else 0.0
+        if t_tc > t_hbm:
+            tensor_phases.append(fam)
+        bound_s += n_launch * max(t_hbm, t_tc)
+        if fam in kernels:
+            kernels[fam]["us_at_peak"] = max(t_hbm, t_tc) * 1e6
+            kernels[fam]["bound"] = "tensor" if t_tc > t_hbm else "hbm"
+    bound_s += S * (B + 1) * cfg.vocab * 2 / (hbm * 1e9)      # verify reads the target logits once
     line = {
         "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": per_step_ms, "us_per_draft_block": per_step_ms * 1e3,
@@ -477,8 +495,10 @@ def main():
                    "l2": "per-step weight traffic (3.2 GB) exceeds the 126 MB L2; no flush",
                    "launch": "eager" if args.no_graph else "cuda graph replay of one step",
                    "parallelism": "replicas" if world > 1 else "single"},
-        "step_roofline": {"alg_bytes": step_bytes, "us_at_peak": step_bytes / (hbm * 1e9) * 1e6,
-                          "frac": step_bytes / (hbm * 1e9) / (per_step_ms * 1e-3)},
+        "step_roofline": {"alg_bytes": step_bytes, "us_at_hbm_peak": step_bytes / (hbm * 1e9) * 1e6,
+                          "us_at_peak": bound_s * 1e6, "frac": bound_s / (per_step_ms * 1e-3),
+                          "tensor_bound_phases": tensor_phases,
+                          "note": "sum over the step's phases of max(bytes / measured HBM, flops / measured sustained bf16)"},
         "roofline": roofline, "kernels": kernels,
         "kernels_note": "device-side timeline of one eager step: per phase, from inputs ready to last CTA done",
         "clocks": clocks, "gpu_launches": int(launches),
