@@ -38,8 +38,13 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_F = 128;                      // weight rows per tile = MMA M
-constexpr int BK = 64;                           // K elements per stage = one 128-byte swizzle row
-constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB
+constexpr int BK = 64;                           // K elements per slab = one 128-byte swizzle row
+constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB per slab
+// A ring stage holds SL slabs (SL * 64 K-elements) of both operands, each fetched by ONE copy:
+// with few tokens the tensor-core work per byte is tiny and the single issuing thread, not HBM,
+// limits the stream, so small token tiles take two slabs per copy (a 3-D view [64][rows][K/64] of
+// the row-major matrix lands as [slab][row][64], i.e. two canonical swizzled tiles back to back).
+constexpr int slabs_for(int nt, bool k_mult_64) { return (nt <= 32 && k_mult_64) ? 2 : 1; }
 constexpr int MAX_STAGES = 12;
 constexpr int TOK_CACHE = 1024;                  // per-token scale / position / page kept for this many rows
 // token columns handled per epilogue pass (each of the 128 epilogue threads holds CH accumulators)
@@ -153,11 +158,13 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
     else a.v2 = fmaxf(a.v2, v1);
 }
 
-// Residual rows of one pass (x += ...): loaded by the caller, ahead of whatever else it waits for.
+// Residual rows of one pass (x += ...) and the next norm's gain for this feature: loaded by the caller,
+// ahead of whatever else it waits for.
 template <int CH>
-__device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, int tok0, int row, float (&xres)[CH]) {
+__device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, int tok0, int row, float (&xres)[CH], float& gain) {
     const int f = un.ft * TILE_F + row;
     const int n_tok = min(CH, p.M - tok0);
+    gain = (p.g_next && (p.epi == EPI_RESIDUAL || p.epi == EPI_STORE_F32) && f < p.N) ? __bfloat162float(p.g_next[f]) : 0.f;
 #pragma unroll
     for (int c = 0; c < CH; ++c) xres[c] = 0.f;
     if (p.epi == EPI_RESIDUAL && f < p.N) {
@@ -171,7 +178,7 @@ __device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, 
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
 template <int CH>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
-                                               int row, const int* tPos, const int* tPage, const float (&xres)[CH]) {
+                                               int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain) {
     // tPos / tPage: position and physical page of the 16 tokens of this pass (-1 = skip the token)
     constexpr int ACC_LD = CH + 1;
     constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
@@ -193,7 +200,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                     }
                 }
                 if (p.g_next) {
-                    const float gv = __bfloat162float(p.g_next[f]);
+                    const float gv = gain;
 #pragma unroll
                     for (int c = 0; c < CH; ++c)
                         if (c < n_tok) p.xn_out[(size_t)(tok0 + c) * p.N + f] = __float2bfloat16_rn(gv * xv[c]);
@@ -397,21 +404,26 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     return v;
 }
 
-template <int NT>
+template <int NT, int SL>
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps tmX, const __grid_constant__ MParams mp) {
     if (threadIdx.x == 0) trace_min(mp.ph[0].trace, 0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    constexpr int X_STAGE_BYTES = NT * BK * 2;
+    constexpr int W_STAGE = W_STAGE_BYTES * SL;
+    constexpr int X_SLAB = NT * BK * 2;
+    constexpr int X_STAGE = X_SLAB * SL;
     constexpr int CH = pass_cols(NT);
     constexpr int ACC_LD = CH + 1;
-    constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 2 : 1));   // partial pieces fetched together when finishing
+    // partial pieces fetched together when finishing. More would shorten the tail further, but the register
+    // count must leave room for the CTAs of the next kernel to become resident beside this one: a
+    // dependent kernel that cannot start early was measured 30 us slower.
+    constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 2 : 1));
     constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
     const int stages = mp.stages;
     uint8_t* sW = smem;
-    uint8_t* sX = sW + (size_t)stages * W_STAGE_BYTES;
-    float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE_BYTES);
+    uint8_t* sX = sW + (size_t)stages * W_STAGE;
+    float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE);
     Top2Entry* sRed = reinterpret_cast<Top2Entry*>(sAcc + TILE_F * ACC_LD);
     float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [TOK_CACHE] per-token rsqrt(mean square)
     int* sPos = reinterpret_cast<int*>(sRstd + TOK_CACHE);        // [TOK_CACHE] per-token position (-1: skip)
@@ -451,6 +463,11 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         // queue is empty and both tiles are issued back to back.
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+            // chunk c of rows y.. : SL slabs of 64 K-elements
+            auto load = [&](void* dst, const CUtensorMap* m, int c, int y, uint64_t* bar, uint64_t pol) {
+                if constexpr (SL == 1) tma_load_2d(dst, m, c * BK, y, bar, pol);
+                else tma_load_3d(dst, m, 0, y, c * SL, bar, pol);
+            };
             int* q_ph = sPend;                      // queued slots: phase, chunk, token tile (ring order)
             int* q_c = sPend + MAX_STAGES;
             int* q_tt = sPend + 2 * MAX_STAGES;
@@ -475,8 +492,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         }
                         ready_ph = ph;
                     }
-                    tma_load_2d(sX + (size_t)q_head * X_STAGE_BYTES, &tmX.m[mp.ph[ph].x_map], q_c[q_head] * BK, q_tt[q_head] * NT,
-                                &full[q_head], pol_x);
+                    load(sX + (size_t)q_head * X_STAGE, &tmX.m[mp.ph[ph].x_map], q_c[q_head], q_tt[q_head] * NT, &full[q_head], pol_x);
                     q_head = (q_head + 1 == stages) ? 0 : q_head + 1;
                     --q_count;
                 }
@@ -497,10 +513,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                             }
                             if (!ok) break;
                         }
-                        mbar_expect_tx(&full[st], W_STAGE_BYTES + X_STAGE_BYTES);
-                        tma_load_2d(sW + (size_t)st * W_STAGE_BYTES, wm, c * BK, y_w, &full[st], pol_w);
+                        mbar_expect_tx(&full[st], W_STAGE + X_STAGE);
+                        load(sW + (size_t)st * W_STAGE, wm, c, y_w, &full[st], pol_w);
                         if (q_count == 0 && ph <= ready_ph) {
-                            tma_load_2d(sX + (size_t)st * X_STAGE_BYTES, xm, c * BK, y_x, &full[st], pol_x);
+                            load(sX + (size_t)st * X_STAGE, xm, c, y_x, &full[st], pol_x);
                         } else {
                             if (q_count == 0) q_head = st;
                             q_ph[st] = ph; q_c[st] = c; q_tt[st] = un.tt;
@@ -547,11 +563,12 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         const uint32_t phs = (it / stages) & 1;
                         if (!mbar_wait(&full[st], phs, &flags[0])) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t a_addr = smem_u32(sW + (size_t)st * W_STAGE_BYTES);
-                        const uint32_t b_addr = smem_u32(sX + (size_t)st * X_STAGE_BYTES);
+                        const uint32_t a_addr = smem_u32(sW + (size_t)st * W_STAGE);
+                        const uint32_t b_addr = smem_u32(sX + (size_t)st * X_STAGE);
 #pragma unroll
-                        for (int kk = 0; kk < BK / 16; ++kk)
-                            mma_bf16(d_tmem, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32), idesc,
+                        for (int kk = 0; kk < SL * (BK / 16); ++kk)
+                            mma_bf16(d_tmem, smem_desc_sw128(a_addr + (kk >> 2) * W_STAGE_BYTES + (kk & 3) * 32),
+                                     smem_desc_sw128(b_addr + (kk >> 2) * X_SLAB + (kk & 3) * 32), idesc,
                                      (c > un.c0 || kk > 0) ? 1u : 0u);
                         mma_commit(&empty[st]);
                     }
@@ -632,10 +649,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     } else {
 #pragma unroll
                         for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[tok_off + ch * CH + c] : v[c];
-                        float xres[CH];
-                        residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
+                        float xres[CH], gain;
+                        residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
                         epi_bar();
-                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres);
+                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
                         epi_bar();
                     }
                 }
@@ -662,8 +679,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
                 if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
                 // residual rows of the first pass travel while the tickets are polled
-                float xres[CH];
-                if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres);
+                float xres[CH], gain = 0.f;
+                if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres, gain);
                 if (row == 0) {
                     const long long t0 = clock64();
                     while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
@@ -679,7 +696,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 }
                 for (int ch = my_q; ch < n_ch; ch += n_contrib) {
                     if constexpr (CH <= 32) {
-                        if (ch != my_q) residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
+                        if (ch != my_q) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
                     }
                     float acc[CH];
 #pragma unroll
@@ -707,9 +724,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     }
 #pragma unroll
                     for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
-                    if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres);
+                    if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
                     epi_bar();
-                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres);
+                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
                     epi_bar();
                 }
             }
@@ -747,9 +764,17 @@ __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __r
     if (threadIdx.x == 0) trace_min(trace, 1);
     const int tok = blockIdx.x;
     T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-    for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
-        const Top2Entry e = top2[(size_t)i * M + tok];
-        t2_merge(t, e.v1, e.i1, e.v2);
+    constexpr int INFL = 12;             // entries requested together per thread
+    for (int i0 = threadIdx.x; i0 < n_tiles; i0 += INFL * blockDim.x) {
+        float4 e[INFL];
+#pragma unroll
+        for (int k = 0; k < INFL; ++k) {
+            const int i = i0 + k * blockDim.x;
+            e[k] = i < n_tiles ? __ldcg(reinterpret_cast<const float4*>(top2 + (size_t)i * M + tok))
+                               : make_float4(-CUDART_INF_F, __int_as_float(0x7fffffff), -CUDART_INF_F, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < INFL; ++k) t2_merge(t, e[k].x, __float_as_int(e[k].y), e[k].z);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -805,12 +830,19 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __
     if (threadIdx.x == 0) trace_max(trace, 3);
 }
 
-// [rows, K] bf16 row-major; box = 64 K-elements x box_rows rows
-bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
-    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)rows};
-    const uint64_t strides[1] = {(uint64_t)K * 2};
-    const uint32_t box[2] = {(uint32_t)BK, (uint32_t)box_rows};
-    return tmap_encode_bf16(m, base, 2, dims, strides, box);
+// [rows, K] bf16 row-major; box = 64 K-elements x box_rows rows (x `slabs` consecutive 64-element
+// column blocks, through the view [64][rows][K/64], when slabs > 1: K must be a multiple of 64)
+bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows, int slabs) {
+    if (slabs == 1) {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)rows};
+        const uint64_t strides[1] = {(uint64_t)K * 2};
+        const uint32_t box[2] = {(uint32_t)BK, (uint32_t)box_rows};
+        return tmap_encode_bf16(m, base, 2, dims, strides, box);
+    }
+    const uint64_t dims[3] = {(uint64_t)BK, (uint64_t)rows, (uint64_t)(K / BK)};
+    const uint64_t strides[2] = {(uint64_t)K * 2, (uint64_t)BK * 2};
+    const uint32_t box[3] = {(uint32_t)BK, (uint32_t)box_rows, (uint32_t)slabs};
+    return tmap_encode_bf16(m, base, 3, dims, strides, box);
 }
 
 int pick_nt(int M) {
@@ -818,16 +850,16 @@ int pick_nt(int M) {
     return 256;
 }
 
-template <int NT>
+template <int NT, int SL>
 int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
     static bool attr_set = false;
-    const int smem = 1024 + mp.stages * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
+    const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         attr_set = true;
     }
-    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
+    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT, SL>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
@@ -844,7 +876,7 @@ int64_t gemm_tc_counter_bytes(int M, int N, int n_groups) {
     return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt) * 4;
 }
 
-static int fill_phase(const Launch& L, const GemmArgs& a, int nt, KParams& p) {
+static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KParams& p) {
     if (a.K % 8 != 0) return DFLASH_ERR_UNSUPPORTED;
     const dflash_config& c = L.h->cfg;
     const int groups = std::max(a.n_groups, 1);
@@ -853,7 +885,7 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, KParams& p) {
     p.n_groups = groups;
     p.n_ftiles = (a.N + TILE_F - 1) / TILE_F;
     p.n_ttiles = (a.M + nt - 1) / nt;
-    p.chunks_total = (a.K + BK - 1) / BK;
+    p.chunks_total = (a.K + BK * slabs - 1) / (BK * slabs);
     p.n_tiles = groups * p.n_ftiles * p.n_ttiles;
     if (!a.part || !a.counters) return DFLASH_ERR_INVALID_ARG;
     p.part = a.part; p.counters = a.counters;
@@ -885,8 +917,11 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     MParams mp{};
     WMaps tw;
     XMaps tx;
+    bool k64 = true;
+    for (int i = 0; i < n_phases; ++i) k64 = k64 && phases[i].K % BK == 0;
+    const int slabs = slabs_for(nt, k64);
     mp.n_phases = n_phases;
-    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (W_STAGE_BYTES + nt * BK * 2));
+    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (slabs * (W_STAGE_BYTES + nt * BK * 2)));
     mp.phase_done = phase_done;
     mp.status = L.status;
 
@@ -895,29 +930,29 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     for (int i = 0; i < n_phases; ++i) {
         const GemmArgs& a = phases[i];
         if (a.M != M || a.N <= 0) return DFLASH_ERR_INVALID_ARG;
-        const int rc = fill_phase(L, a, nt, mp.ph[i]);
+        const int rc = fill_phase(L, a, nt, slabs, mp.ph[i]);
         if (rc != DFLASH_OK) return rc;
         KParams& p = mp.ph[i];
         p.trace = traces ? traces[i] : nullptr;
         if (n_maps + p.n_groups > GEMM_MAX_GROUPS) return DFLASH_ERR_UNSUPPORTED;
         p.w_map0 = n_maps;
         for (int g = 0; g < p.n_groups; ++g)
-            if (!make_map(&tw.m[n_maps++], a.W[g], a.N, a.K, TILE_F)) return DFLASH_ERR_CUDA;
+            if (!make_map(&tw.m[n_maps++], a.W[g], a.N, a.K, TILE_F, slabs)) return DFLASH_ERR_CUDA;
         p.x_map = i;
-        if (!make_map(&tx.m[i], a.X, a.M, a.K, nt)) return DFLASH_ERR_CUDA;
+        if (!make_map(&tx.m[i], a.X, a.M, a.K, nt, slabs)) return DFLASH_ERR_CUDA;
         const long long pairs = (long long)p.n_tiles * p.chunks_total;
         min_pairs = min_pairs < 0 ? pairs : std::min(min_pairs, pairs);
     }
     for (int g = n_maps; g < GEMM_MAX_GROUPS; ++g) tw.m[g] = tw.m[0];
     for (int i = n_phases; i < MAX_PHASES; ++i) tx.m[i] = tx.m[0];
-    // one CTA per SM unless the smallest phase would leave ranges under 4 chunks
-    const int grid = (int)std::max<long long>(1, std::min<long long>(L.h->sm_count, min_pairs / 4));
+    // one CTA per SM unless the smallest phase would leave ranges under 256 K-elements
+    const int grid = (int)std::max<long long>(1, std::min<long long>(L.h->sm_count, min_pairs * slabs / 4));
     switch (nt) {
-        case 16: return launch_nt<16>(L, tw, tx, mp, grid);
-        case 32: return launch_nt<32>(L, tw, tx, mp, grid);
-        case 64: return launch_nt<64>(L, tw, tx, mp, grid);
-        case 128: return launch_nt<128>(L, tw, tx, mp, grid);
-        default: return launch_nt<256>(L, tw, tx, mp, grid);
+        case 16: return slabs == 2 ? launch_nt<16, 2>(L, tw, tx, mp, grid) : launch_nt<16, 1>(L, tw, tx, mp, grid);
+        case 32: return slabs == 2 ? launch_nt<32, 2>(L, tw, tx, mp, grid) : launch_nt<32, 1>(L, tw, tx, mp, grid);
+        case 64: return launch_nt<64, 1>(L, tw, tx, mp, grid);
+        case 128: return launch_nt<128, 1>(L, tw, tx, mp, grid);
+        default: return launch_nt<256, 1>(L, tw, tx, mp, grid);
     }
 }
 
