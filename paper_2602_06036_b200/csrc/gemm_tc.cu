@@ -258,9 +258,13 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
         case EPI_SWIGLU: {
             if ((row & 1) == 0 && f + 1 < p.N) {
                 const int j = f >> 1;
-                for (int c = 0; c < n_tok; ++c) {
-                    const float g = sAcc[row * ACC_LD + c], u = sAcc[(row + 1) * ACC_LD + c];
-                    p.h[(size_t)(tok0 + c) * p.F + j] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+                __nv_bfloat16* dst = p.h + (size_t)tok0 * p.F + j;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {      // unrolled: independent iterations overlap their latencies
+                    if (c < n_tok) {
+                        const float g = sAcc[row * ACC_LD + c], u = sAcc[(row + 1) * ACC_LD + c];
+                        dst[(size_t)c * p.F] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+                    }
                 }
             }
         } break;
@@ -753,10 +757,59 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     }
 }
 
-// one CTA per token: merge the per-tile winners (index-aware, so order-independent)
-__global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __restrict__ top2, int n_tiles, int M,
-                                                            int32_t* __restrict__ ids, float* __restrict__ top1,
-                                                            float* __restrict__ margin, unsigned long long* trace) {
+// Merge of the per-tile winners (index-aware, so order-independent). The entries are laid out
+// [tile][token]: a CTA takes 8 consecutive tokens (one full 128-byte line per tile) and 64 interleaved
+// sub-sequences of the tiles, so every request is a whole line however few SMs the CTAs land on.
+constexpr int FIN_TOK = 8, FIN_SUB = 64;
+__global__ void __launch_bounds__(FIN_TOK * FIN_SUB) argmax_finish_kernel(const Top2Entry* __restrict__ top2, int n_tiles, int M,
+                                                                          int32_t* __restrict__ ids, float* __restrict__ top1,
+                                                                          float* __restrict__ margin, unsigned long long* trace) {
+    __shared__ Top2Entry sh[FIN_TOK * FIN_SUB / 32][FIN_TOK];
+    if (threadIdx.x == 0) trace_min(trace, 0);
+    pdl_trigger();
+    pdl_wait();
+    if (threadIdx.x == 0) trace_min(trace, 1);
+    const int tl = threadIdx.x & (FIN_TOK - 1), sub = threadIdx.x / FIN_TOK;
+    const int tok = blockIdx.x * FIN_TOK + tl;
+    T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
+    if (tok < M) {
+        constexpr int INFL = 8;             // entries requested together per thread
+        for (int i0 = sub; i0 < n_tiles; i0 += INFL * FIN_SUB) {
+            float4 e[INFL];
+#pragma unroll
+            for (int k = 0; k < INFL; ++k) {
+                const int i = i0 + k * FIN_SUB;
+                e[k] = i < n_tiles ? __ldcg(reinterpret_cast<const float4*>(top2 + (size_t)i * M + tok))
+                                   : make_float4(-CUDART_INF_F, __int_as_float(0x7fffffff), -CUDART_INF_F, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < INFL; ++k) t2_merge(t, e[k].x, __float_as_int(e[k].y), e[k].z);
+        }
+    }
+    // lanes tl, tl + 8, tl + 16, tl + 24 of a warp hold the same token
+#pragma unroll
+    for (int o = FIN_TOK; o < 32; o <<= 1) {
+        const float v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        const int i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        const float v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t2_merge(t, v1, i1, v2);
+    }
+    if ((threadIdx.x & 31) < FIN_TOK) sh[threadIdx.x >> 5][tl] = Top2Entry{t.v1, t.i1, t.v2, 0};
+    __syncthreads();
+    if (threadIdx.x < FIN_TOK && tok < M) {
+        T2 r{sh[0][tl].v1, sh[0][tl].i1, sh[0][tl].v2};
+        for (int w = 1; w < FIN_TOK * FIN_SUB / 32; ++w) t2_merge(r, sh[w][tl].v1, sh[w][tl].i1, sh[w][tl].v2);
+        ids[tok] = r.i1 == 0x7fffffff ? 0 : r.i1;
+        if (top1) top1[tok] = r.v1;
+        if (margin) margin[tok] = r.v1 - r.v2;
+    }
+    if (threadIdx.x == 0) trace_max(trace, 3);
+}
+
+// Few tokens: one CTA per token (more CTAs in flight matter more than whole-line requests).
+__global__ void __launch_bounds__(128) argmax_finish_rows_kernel(const Top2Entry* __restrict__ top2, int n_tiles, int M,
+                                                                 int32_t* __restrict__ ids, float* __restrict__ top1,
+                                                                 float* __restrict__ margin, unsigned long long* trace) {
     __shared__ Top2Entry sh[4];
     if (threadIdx.x == 0) trace_min(trace, 0);
     pdl_trigger();
@@ -764,7 +817,7 @@ __global__ void __launch_bounds__(128) argmax_finish_kernel(const Top2Entry* __r
     if (threadIdx.x == 0) trace_min(trace, 1);
     const int tok = blockIdx.x;
     T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-    constexpr int INFL = 12;             // entries requested together per thread
+    constexpr int INFL = 12;
     for (int i0 = threadIdx.x; i0 < n_tiles; i0 += INFL * blockDim.x) {
         float4 e[INFL];
 #pragma unroll
@@ -965,7 +1018,10 @@ int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done) {
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,
                          float* margin) {
     if (M <= 0) return DFLASH_OK;
-    const cudaError_t e = launch_pdl(argmax_finish_kernel, dim3(M), dim3(128), 0, L.st, top2, n_tiles, M, ids, top1, margin, L.trace);
+    const cudaError_t e =
+        M <= 32 ? launch_pdl(argmax_finish_rows_kernel, dim3(M), dim3(128), 0, L.st, top2, n_tiles, M, ids, top1, margin, L.trace)
+                : launch_pdl(argmax_finish_kernel, dim3((M + FIN_TOK - 1) / FIN_TOK), dim3(FIN_TOK * FIN_SUB), 0, L.st, top2,
+                             n_tiles, M, ids, top1, margin, L.trace);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
