@@ -461,7 +461,7 @@ def main():
                 if line.startswith("dram_bytes_per_launch:"):
                     traffic = int(line.split(":")[1].strip().split()[0])
         gbs = alg["lmhead_argmax"] / (lm_us * 1e-6) / 1e9
-        roofline = {"kernel": "gemm_tc_kernel<16> as LM head + argmax (V x D weights, 16 rows)", "bound": "hbm",
+        roofline = {"kernel": "gemm_tc_kernel<16, 2> as LM head + argmax (V x D weights, 16 rows)", "bound": "hbm",
                     "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm, "traffic": traffic,
                     "peak_source": peaks["_source"] + " (copy bandwidth)", "us_per_launch": lm_us,
                     "timing": "CUDA event pair around each launch of the kernel run alone (dflash_lmhead_argmax), "

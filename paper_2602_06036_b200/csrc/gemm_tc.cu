@@ -179,7 +179,7 @@ __device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, 
 template <int CH>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
                                                int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain) {
-    // tPos / tPage: position and physical page of the 16 tokens of this pass (-1 = skip the token)
+    // tPos / tPage: position and (context projection) pool row of the page slot of the tokens of this pass (-1 = skip)
     constexpr int ACC_LD = CH + 1;
     constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
     const int f = un.ft * TILE_F + row;
@@ -233,25 +233,37 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 const int partner = row ^ half;
                 const int qdim = p.Hq * hd, kdim = p.Hkv * hd;
                 const bool rot = p.use_rope && head < p.Hq + p.Hkv;
-                float cs[CH], sn[CH];
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int pos = tPos[c];
-                    const bool on = rot && c < n_tok && pos >= 0;
-                    cs[c] = on ? __ldg(p.cs + (size_t)pos * half + i) : 1.f;
-                    sn[c] = on ? __ldg(p.sn + (size_t)pos * half + i) : 0.f;
-                }
                 __nv_bfloat16* dst;
                 int ld;
                 if (head < p.Hq) { dst = p.q + f; ld = qdim; }
                 else if (head < p.Hq + p.Hkv) { dst = p.k + (f - qdim); ld = kdim; }
                 else { dst = p.v + (f - qdim - kdim); ld = kdim; }
+                constexpr int SB = CH <= 16 ? 8 : 16;        // tokens per sub-block: their table loads are in flight together
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    if (c >= n_tok) break;
-                    const float a = sAcc[row * ACC_LD + c], b = sAcc[partner * ACC_LD + c];
-                    const float val = hrow < half ? (a * cs[c] - b * sn[c]) : (a * cs[c] + b * sn[c]);
-                    dst[(size_t)(tok0 + c) * ld] = __float2bfloat16_rn(val);
+                for (int c0 = 0; c0 < CH; c0 += SB) {
+                    if (c0 >= n_tok) break;
+                    float cs[SB], sn[SB];
+#pragma unroll
+                    for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
+                    if (p.use_rope) {       // unconditional loads (table row 0 when the token is unused)
+#pragma unroll
+                        for (int c = 0; c < SB; ++c) {
+                            const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
+                            const size_t at = (size_t)max(pos, 0) * half + i;
+                            cs[c] = __ldg(p.cs + at);
+                            sn[c] = __ldg(p.sn + at);
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < SB; ++c) {
+                        if (c0 + c < n_tok) {
+                            const bool on = rot && tPos[c0 + c] >= 0;
+                            const float cc = on ? cs[c] : 1.f, ss = on ? sn[c] : 0.f;
+                            const float a = sAcc[row * ACC_LD + c0 + c], b = sAcc[partner * ACC_LD + c0 + c];
+                            const float val = hrow < half ? (a * cc - b * ss) : (a * cc + b * ss);
+                            dst[(size_t)(tok0 + c0 + c) * ld] = __float2bfloat16_rn(val);
+                        }
+                    }
                 }
             }
         } break;
@@ -296,26 +308,36 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 const int head = fh / hd, hrow = fh % hd, i = hrow % half;
                 const int partner = row ^ half;
                 const int layer = p.first_layer + un.g;
-                float cs[CH], sn[CH];
+                const bool rot = !is_v && p.use_rope;
+                // pool[layer][page][K|V][head][slot][hd]: tPage[c] = row of (page, K, head 0, slot)
+                __nv_bfloat16* base = p.pool + (((size_t)layer * p.n_pages * 2 + is_v) * p.Hkv + head) * p.PG * hd + hrow;
+                constexpr int SB = CH <= 16 ? 8 : 16;
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int pos = tPos[c];
-                    const bool on = !is_v && p.use_rope && c < n_tok && pos >= 0;
-                    cs[c] = on ? __ldg(p.cs + (size_t)pos * half + i) : 1.f;
-                    sn[c] = on ? __ldg(p.sn + (size_t)pos * half + i) : 0.f;
-                }
+                for (int c0 = 0; c0 < CH; c0 += SB) {
+                    if (c0 >= n_tok) break;
+                    float cs[SB], sn[SB];
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int pos = tPos[c], page = tPage[c];
-                    if (c < n_tok && pos >= 0 && page >= 0) {
-                        float val = sAcc[row * ACC_LD + c];
-                        if (!is_v && p.use_rope) {
-                            const float bb = sAcc[partner * ACC_LD + c];
-                            val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
+                    for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
+                    if (rot) {
+#pragma unroll
+                        for (int c = 0; c < SB; ++c) {
+                            const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
+                            const size_t at = (size_t)max(pos, 0) * half + i;
+                            cs[c] = __ldg(p.cs + at);
+                            sn[c] = __ldg(p.sn + at);
                         }
-                        const size_t dst = (((((size_t)layer * p.n_pages + page) * 2 + is_v) * p.Hkv + head) * p.PG +
-                                            (pos % p.PG)) * hd + hrow;
-                        p.pool[dst] = __float2bfloat16_rn(val);
+                    }
+#pragma unroll
+                    for (int c = 0; c < SB; ++c) {
+                        const int prow = (c0 + c < n_tok) ? tPage[c0 + c] : -1;
+                        if (prow >= 0) {
+                            float val = sAcc[row * ACC_LD + c0 + c];
+                            if (rot) {
+                                const float bb = sAcc[partner * ACC_LD + c0 + c];
+                                val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
+                            }
+                            base[(size_t)prow * hd] = __float2bfloat16_rn(val);
+                        }
                     }
                 }
             }
@@ -327,8 +349,10 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-// Position (and, for the context projection, physical page) of every token of a token tile, worked
-// out once per phase by the epilogue threads so that the per-pass epilogues carry no dependent loads.
+// Position (and, for the context projection, the pool row of its page slot) of every token of a token
+// tile, worked out once per phase by the epilogue threads: the per-pass epilogues then carry no
+// dependent loads and little address arithmetic (with one warp per scheduler every instruction of a
+// dependent chain costs its full latency).
 __device__ __forceinline__ void token_info(const KParams& p, int tok_base, int nt, int row, int* sPos, int* sPage) {
     for (int t = row; t < nt; t += 128) {      // sPos[t] describes token tok_base + t
         const int tok = tok_base + t;
@@ -355,6 +379,8 @@ __device__ __forceinline__ void token_info(const KParams& p, int tok_base, int n
                             if (p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
                             pos = -1;
                             page = -1;
+                        } else {
+                            page = page * 2 * p.Hkv * p.PG + pos % p.PG;     // row of (page, K, head 0, slot) in the layer's pool
                         }
                     }
                 }
@@ -422,7 +448,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     // partial pieces fetched together when finishing. More would shorten the tail further, but the register
     // count must leave room for the CTAs of the next kernel to become resident beside this one: a
     // dependent kernel that cannot start early was measured 30 us slower.
-    constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 2 : 1));
+    constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 3 : 1));
     constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
     const int stages = mp.stages;
     uint8_t* sW = smem;
