@@ -108,37 +108,65 @@ struct Unit {
     int full;      // covers every chunk of the tile
 };
 
-// Walks the pieces of CTA `cta` out of `n_ctas`: range [cta*T/G, (cta+1)*T/G) of the T = n_tiles *
-// chunks_total (tile, chunk) pairs, tiles ordered token-tile fastest so neighbours share weights.
+// Work of CTA `cta` out of `n_ctas` in one phase. With at least one tile per CTA the tiles are split
+// into a SHARED part (the first n_tiles % n_ctas tiles) and whole tiles, the same number per CTA:
+//   1. the (tile, chunk) pairs of the shared part are cut into one contiguous, equally long range per
+//      CTA ("stream-K"), processed FIRST: the cross-CTA reduction of those tiles then overlaps the
+//      streaming of the whole tiles instead of sitting at the end of the phase;
+//   2. whole tiles shared + k * n_ctas + cta, k = 0.., go straight from the accumulator to the epilogue.
+// Every CTA streams the same number of chunks (+-1). With fewer tiles than CTAs everything is shared.
+// Tiles are ordered token-tile fastest, so neighbouring CTAs share weight tiles through L2.
+// The shared part never leaves a CTA an empty range (every CTA between the first and the last
+// contributor of a tile publishes a piece): a remainder that small takes one more round of tiles with it.
+__device__ __forceinline__ int shared_tiles(const KParams& p, int n_ctas) {
+    if (p.n_tiles < n_ctas) return p.n_tiles;
+    const int r = p.n_tiles % n_ctas;
+    if (r == 0) return 0;
+    if ((long long)r * p.chunks_total >= 4LL * n_ctas) return r;
+    return p.n_tiles / n_ctas >= 2 ? r + n_ctas : p.n_tiles;
+}
 struct PieceWalk {
     long long cur, hi;
-    int first;
+    int first, n_shared, dp_next, dp_stride;
     __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas) {
-        const long long T = (long long)p.n_tiles * p.chunks_total;
+        n_shared = shared_tiles(p, n_ctas);
+        const long long T = (long long)n_shared * p.chunks_total;
         cur = (long long)cta * T / n_ctas;
         hi = (long long)(cta + 1) * T / n_ctas;
         first = 1;
+        dp_next = n_shared + cta;
+        dp_stride = n_ctas;
     }
-    __device__ __forceinline__ bool done() const { return cur >= hi; }
+    __device__ __forceinline__ bool shared_done() const { return cur >= hi; }
+    __device__ __forceinline__ bool done(const KParams& p) const { return cur >= hi && dp_next >= p.n_tiles; }
     __device__ __forceinline__ Unit next(const KParams& p) {
         Unit u;
-        u.tile = (int)(cur / p.chunks_total);
-        u.c0 = (int)(cur % p.chunks_total);
-        const long long left = hi - cur;
-        u.c1 = (int)min((long long)p.chunks_total, u.c0 + left);
-        u.full = (u.c0 == 0 && u.c1 == p.chunks_total) ? 1 : 0;
-        u.slot = first ? 0 : 1;
+        if (cur < hi) {
+            u.tile = (int)(cur / p.chunks_total);
+            u.c0 = (int)(cur % p.chunks_total);
+            const long long left = hi - cur;
+            u.c1 = (int)min((long long)p.chunks_total, u.c0 + left);
+            u.full = (u.c0 == 0 && u.c1 == p.chunks_total) ? 1 : 0;
+            u.slot = first ? 0 : 1;
+            cur += u.c1 - u.c0;
+            first = 0;
+        } else {
+            u.tile = dp_next;
+            u.c0 = 0;
+            u.c1 = p.chunks_total;
+            u.full = 1;
+            u.slot = 0;
+            dp_next += dp_stride;
+        }
         int t = u.tile;
         u.tt = t % p.n_ttiles;
         t /= p.n_ttiles;
         u.ft = t % p.n_ftiles;
         u.g = t / p.n_ftiles;
-        cur += u.c1 - u.c0;
-        first = 0;
         return u;
     }
 };
-// CTA that owns (tile, chunk) pair number x:  largest j with floor(j*T/G) <= x
+// CTA that owns pair number x of the shared part (T pairs):  largest j with floor(j*T/G) <= x
 __device__ __forceinline__ int cta_of_pair(long long x, long long T, int G) { return (int)(((x + 1) * G + T - 1) / T - 1); }
 
 // ---------------------------------------------------------------------------------------------
@@ -530,7 +558,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
                 const CUtensorMap* xm = &tmX.m[p.x_map];
-                for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok;) {
+                for (PieceWalk w(p, blockIdx.x, G); !w.done(p) && ok;) {
                     const Unit un = w.next(p);
                     const CUtensorMap* wm = &tmW.m[p.w_map0 + un.g];
                     const int y_w = un.ft * TILE_F, y_x = un.tt * NT;
@@ -582,7 +610,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             bool ok = true;
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
-                for (PieceWalk w(p, blockIdx.x, G); !w.done() && ok; ++ui) {
+                for (PieceWalk w(p, blockIdx.x, G); !w.done(p) && ok; ++ui) {
                     const Unit un = w.next(p);
                     const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
                     if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
@@ -621,7 +649,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         pdl_wait();      // lengths, page tables, residual rows ... come from earlier kernels
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
-            const long long T = (long long)p.n_tiles * p.chunks_total;
+            const long long T = (long long)shared_tiles(p, G) * p.chunks_total;      // pairs of the shared part
             const bool all_tok = p.M <= TOK_CACHE;   // per-token data cached for the whole phase (else per token tile)
             const bool need_info = p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV;
             int rstd_tt = -1, info_tt = -1;
@@ -648,7 +676,74 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             }
             Unit pend[2];            // this CTA's pieces of shared tiles (at most its first and its last piece)
             int n_pend = 0;
-            for (PieceWalk w(p, blockIdx.x, G); !w.done(); ++ui) {
+            // ---- shared tiles: wait for every contributor's piece, then do this CTA's share of the passes.
+            // Runs as soon as this CTA's shared pieces are published: while whole tiles remain, the
+            // reduction overlaps their streaming.
+            auto finish_shared = [&]() {
+                for (int pi = 0; pi < n_pend && alive; ++pi) {
+                    const Unit un = pend[pi];
+                    const int tok_base = un.tt * NT;
+                    const int tok_off = all_tok ? tok_base : 0;
+                    const long long x0 = (long long)un.tile * p.chunks_total;
+                    const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
+                    const int n_contrib = j1 - j0 + 1, my_q = (int)blockIdx.x - j0;
+                    const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
+                    if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
+                    // residual rows of the first pass travel while the tickets are polled
+                    float xres[CH], gain = 0.f;
+                    if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres, gain);
+                    if (row == 0) {
+                        const long long t0 = clock64();
+                        while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
+                            if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
+                        }
+                    }
+                    epi_bar();               // row 0's acquire, then the barrier: every piece is visible to all rows
+                    if (flags[2]) { alive = false; return; }
+                    if (!all_tok) {      // caches hold one token tile at a time
+                        if (need_info && info_tt != un.tt) { token_info(p, tok_base, NT, row, sPos, sPage); info_tt = un.tt; }
+                        if (p.ssq_in && rstd_tt != un.tt) { token_rstd(p, tok_base, NT, row, sRstd); rstd_tt = un.tt; }
+                        epi_bar();
+                    }
+                    for (int ch = my_q; ch < n_ch; ch += n_contrib) {
+                        if constexpr (CH <= 32) {
+                            if (ch != my_q) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
+                        }
+                        float acc[CH];
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) acc[c] = 0.f;
+                        // pieces are summed in CTA order; the loads of PF pieces are all in flight together
+                        for (int jb = j0; jb <= j1; jb += PF) {
+                            float va[PF][CH];
+#pragma unroll
+                            for (int u = 0; u < PF; ++u) {
+                                const int j = jb + u;
+                                if (j <= j1) {
+                                    const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
+                                    const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+#pragma unroll
+                                    for (int c = 0; c < CH; ++c) va[u][c] = __ldcg(pa + (size_t)c * TILE_F);
+                                } else {
+#pragma unroll
+                                    for (int c = 0; c < CH; ++c) va[u][c] = 0.f;
+                                }
+                            }
+#pragma unroll
+                            for (int u = 0; u < PF; ++u)
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) acc[c] += va[u][c];
+                        }
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
+                        if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
+                        epi_bar();
+                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
+                        epi_bar();
+                    }
+                }
+                n_pend = 0;
+            };
+            for (PieceWalk w(p, blockIdx.x, G); !w.done(p); ++ui) {
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
@@ -695,71 +790,14 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     epi_bar();
                     if (row == 0) atomicAdd(p.counters + un.tile, 1);
                     pend[n_pend++] = un;
+                    if (w.shared_done() && !w.done(p)) {      // whole tiles follow: reduce now, under their main loop
+                        finish_shared();
+                        if (!alive) break;
+                    }
                 }
             }
             if (!alive) break;
-            // ---- shared tiles: wait for every contributor's piece, then do this CTA's share of the passes
-            for (int pi = 0; pi < n_pend && alive; ++pi) {
-                const Unit un = pend[pi];
-                const int tok_base = un.tt * NT;
-                const int tok_off = all_tok ? tok_base : 0;
-                const long long x0 = (long long)un.tile * p.chunks_total;
-                const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
-                const int n_contrib = j1 - j0 + 1, my_q = (int)blockIdx.x - j0;
-                const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
-                if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
-                // residual rows of the first pass travel while the tickets are polled
-                float xres[CH], gain = 0.f;
-                if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres, gain);
-                if (row == 0) {
-                    const long long t0 = clock64();
-                    while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
-                        if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
-                    }
-                }
-                epi_bar();               // row 0's acquire, then the barrier: every piece is visible to all rows
-                if (flags[2]) { alive = false; break; }
-                if (!all_tok) {      // caches hold one token tile at a time
-                    if (need_info && info_tt != un.tt) { token_info(p, tok_base, NT, row, sPos, sPage); info_tt = un.tt; }
-                    if (p.ssq_in && rstd_tt != un.tt) { token_rstd(p, tok_base, NT, row, sRstd); rstd_tt = un.tt; }
-                    epi_bar();
-                }
-                for (int ch = my_q; ch < n_ch; ch += n_contrib) {
-                    if constexpr (CH <= 32) {
-                        if (ch != my_q) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
-                    }
-                    float acc[CH];
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-                    // pieces are summed in CTA order; the loads of PF pieces are all in flight together
-                    for (int jb = j0; jb <= j1; jb += PF) {
-                        float va[PF][CH];
-#pragma unroll
-                        for (int u = 0; u < PF; ++u) {
-                            const int j = jb + u;
-                            if (j <= j1) {
-                                const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
-                                const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) va[u][c] = __ldcg(pa + (size_t)c * TILE_F);
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) va[u][c] = 0.f;
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < PF; ++u)
-#pragma unroll
-                            for (int c = 0; c < CH; ++c) acc[c] += va[u][c];
-                    }
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
-                    if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
-                    epi_bar();
-                    apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
-                    epi_bar();
-                }
-            }
+            if (n_pend > 0) finish_shared();
             if (!alive) break;
             // this CTA's share of the phase is done and visible: tell the others
             __threadfence();
