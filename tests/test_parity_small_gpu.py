@@ -50,6 +50,19 @@ def test_tiny_without_rope_and_paper_block_sizes():
         case.check_draft(got)
 
 
+@pytest.mark.parametrize("B,k,layers,lens", [(8, 3, 2, (33, 150)), (10, 5, 3, (0, 64, 129)), (16, 5, 1, (257,))])
+def test_bf16_block_sizes_and_feature_counts(B, k, layers, lens):
+    # tensor-core path at the block sizes the paper runs (8, 10, 16: Sec. 5.3 and the LLaMA setting),
+    # with k = 5 tapped layers (App. A.1) and other layer counts; contexts end inside, at and past a page edge
+    cfg = dataclasses.replace(synth.MID, block_size=B, n_feat_layers=k, n_layers=layers)
+    case = Case(cfg, lens, seed=11)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    n_sure = case.check_draft(got)
+    assert n_sure >= case.S * B // 2
+
+
 def test_decode_step_appends_at_ctx_len():
     # second projection call with n_new < max_new appends rows at positions L..L+n-1 only
     cfg = synth.MID
