@@ -27,6 +27,20 @@ replicated MHA, causal last row = full last row), accept-rule enumeration of all
 and equality of speculative output with plain greedy decoding of a toy target.
 The composed forward `draft_block` has no external value to compare with: parity unpinned beyond
 its parts (each step above is pinned separately).
+
+Sampling (temperature > 0) verification, the setting of the paper's T = 1 results (Sec. 5.1, Table 2):
+the paper relies on standard speculative sampling (Sec. 2 related work) without restating it, so
+the rule is written out here                                     -> softmax_t, sample_cdf, verify_accept_sample
+  p_j = softmax(target_logits[j] / T),  q_j = softmax(draft_logits[j] / T);
+  draft d_{j+1} is kept while  u_j * q_j(d_{j+1}) < p_j(d_{j+1})   (probability min(1, p/q));
+  at the first rejection a the cycle emits one token drawn from max(p_a - q_a, 0) / sum (from p_a if
+  that sum is zero); with all gamma kept it emits one token drawn from p_gamma;  tau = a + 1.
+  Every draw maps a uniform u in [0, 1) to the first vocabulary index whose running sum of weights
+  reaches u * total (inverse CDF in vocabulary order). Uniforms are inputs.
+Pins (tests/test_oracle_sampling.py): the first emitted token is distributed exactly as p_0 (measure
+of the uniform cube, computed cell by cell on small vocabularies), a hand-worked two-token case,
+p = q keeps everything, T -> 0 reduces to the greedy rule, rejected positions only emit tokens
+with p > q.
 """
 from __future__ import annotations
 
@@ -252,6 +266,69 @@ def verify_accept_logits(draft_ids, target_logits, ctx_len):
     """Same, starting from the target's logits [gamma+1, V]."""
     p, _, _ = argmax_top2(target_logits)
     return verify_accept(draft_ids, p, ctx_len)
+
+
+# --------------------------------------------------------------------------------------------
+# sampling verify / accept (speculative sampling; the rule is stated in the header)
+# --------------------------------------------------------------------------------------------
+def softmax_t(logits, T):
+    """softmax(logits / T) along the last axis, T > 0."""
+    z = _f64(logits) / float(T)
+    z = z - z.max(axis=-1, keepdims=True)
+    e = np.exp(z)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def sample_cdf(w, u):
+    """Inverse-CDF draw from non-negative weights w (need not be normalised), u in [0, 1):
+    the first index i with w_0 + ... + w_i >= u * sum(w) among indices with w_i > 0.
+    Returns (index, margin): margin = distance of u * sum(w) to the nearest edge of that index's
+    interval, relative to sum(w) (how far u is from changing the answer)."""
+    w = _f64(w)
+    c = np.cumsum(w)
+    total = c[-1]
+    assert total > 0
+    x = float(u) * total
+    i = int(np.searchsorted(c, x, side="left"))
+    i = min(i, len(w) - 1)
+    while w[i] <= 0 and i + 1 < len(w):   # u * total landed exactly on an edge shared with empty entries
+        i += 1
+    while w[i] <= 0:                      # ... at the very end of the vocabulary
+        i -= 1
+    lo = c[i] - w[i]
+    return i, float(min(x - lo, c[i] - x) / total)
+
+
+def verify_accept_sample(draft_ids, draft_logits, target_logits, T, u_accept, u_final, ctx_len):
+    """Speculative-sampling verification of gamma drafts (rule in the header).
+    draft_ids [gamma]; draft_logits [gamma, V]; target_logits [gamma+1, V]; u_accept [gamma];
+    u_final scalar. Returns (tau, out_tokens [gamma+1] padded with -1, final token, new_ctx_len,
+    info) where info = dict(accept_margin=[...], final_margin=..., a=..., residual=bool)."""
+    gamma = len(draft_ids)
+    p = softmax_t(target_logits, T)
+    q = softmax_t(draft_logits, T) if gamma else np.zeros((0, p.shape[-1]))
+    assert p.shape[0] == gamma + 1
+    a = 0
+    margins = []
+    while a < gamma:
+        d = int(draft_ids[a])
+        lhs, rhs = float(u_accept[a]) * q[a, d], p[a, d]
+        margins.append(abs(rhs - lhs) / max(rhs, lhs, 1e-300))
+        if not lhs < rhs:
+            break
+        a += 1
+    residual = a < gamma
+    if residual:
+        w = np.maximum(p[a] - q[a], 0.0)
+        if w.sum() <= 0:
+            w = p[a]
+    else:
+        w = p[gamma]
+    tok, fm = sample_cdf(w, u_final)
+    out = np.full((gamma + 1,), -1, dtype=np.int64)
+    out[:a] = np.asarray(draft_ids[:a], dtype=np.int64)
+    out[a] = tok
+    return a + 1, out, tok, int(ctx_len) + a + 1, dict(accept_margin=margins, final_margin=fm, a=a, residual=residual)
 
 
 # --------------------------------------------------------------------------------------------
