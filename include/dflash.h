@@ -201,6 +201,63 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a /*[ho
 #define DFLASH_STATIC_MAX_ROWS 1088
 int32_t dflash_verify_accept_static(dflash_handle* h, const dflash_verify_args* a /*[host]*/, void* stream);
 
+/* ---- sampling (temperature > 0): drafting draws and speculative-sampling verification ----
+ * The paper reports T = 1 results (Sec. 5.1) and relies on standard speculative sampling (Sec. 2)
+ * without restating the rule; it is, with p_j = softmax(target_logits[b, j] / T) and
+ * q_j = softmax(draft_logits[b, j] / T):
+ *   draft j (j = 0..gamma-1, in order) is kept while  u_accept[b, j] * q_j(d_j) < p_j(d_j);
+ *   at the first rejection a:  one token drawn from max(p_a - q_a, 0) (from p_a if that is all zero);
+ *   with every draft kept (a = gamma): one token drawn from p_gamma;   tau = a + 1.
+ * A draw maps a uniform u in [0, 1) to the first vocabulary index (with non-zero weight) whose running
+ * sum of weights reaches u * total. The uniforms are INPUTS: the library draws no random numbers, so a
+ * caller (and the CPU oracle) reproduces a result from the same uniforms. Sums that decide an index are
+ * accumulated in double in a fixed order; against exact arithmetic a result can only differ when
+ * u * total lies within ~1e-6 (relative) of an interval edge.
+ * Scratch: `workspace` of dflash_sample_workspace_bytes(n_logit_rows, vocab) bytes, 256-byte aligned,
+ * n_logit_rows = n_rows (dflash_sample_rows) or batch * (2 * gamma + 1) (dflash_verify_accept_sample).
+ * Errors: DFLASH_ERR_INVALID_ARG (null pointer, T <= 0, bad dtype or sizes), DFLASH_ERR_WORKSPACE;
+ * a draft id outside [0, vocab) counts as rejected and sets DFLASH_DEV_BAD_TOKEN in *dev_status. */
+typedef struct {
+    const void*    logits;        /* [device] [n_rows, vocab]                                   */
+    int32_t        logits_dtype;  /* DFLASH_F32 | DFLASH_BF16                                   */
+    int64_t        row_stride;    /* elements between rows (0 = vocab)                          */
+    int32_t        n_rows, vocab;
+    float          temperature;   /* > 0                                                        */
+    const float*   u;             /* [device] [n_rows] uniforms in [0, 1)                       */
+    int32_t*       ids;           /* [device] out [n_rows] drawn index                          */
+    float*         prob;          /* [device] out [n_rows] its probability; may be NULL         */
+    void*          workspace;     /* [device]                                                   */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;    /* [device] may be NULL                                       */
+} dflash_sample_args;
+int32_t dflash_sample_rows(dflash_handle* h, const dflash_sample_args* a /*[host]*/, void* stream);
+
+typedef struct {
+    const void*    target_logits;      /* [device] [batch, gamma+1, vocab]                      */
+    int32_t        target_dtype;       /* DFLASH_F32 | DFLASH_BF16                              */
+    int64_t        target_row_stride;  /* elements (0 = vocab)                                  */
+    const void*    draft_logits;       /* [device] draft j of sequence b = row b*draft_rows_per_seq + j */
+    int32_t        draft_dtype;
+    int64_t        draft_row_stride;   /* elements (0 = vocab)                                  */
+    int32_t        draft_rows_per_seq; /* stored rows per sequence (>= gamma), e.g. the block size */
+    const int32_t* draft_ids;          /* [device] first draft of sequence b at draft_ids + b*draft_stride */
+    int32_t        draft_stride;
+    int32_t        batch, gamma, vocab;
+    float          temperature;        /* > 0, applied to both distributions                    */
+    const float*   u_accept;           /* [device] [batch, gamma] uniforms in [0, 1)            */
+    const float*   u_final;            /* [device] [batch] uniform of the emitted token         */
+    const int32_t* ctx_len;            /* [device] [batch]                                      */
+    int32_t*       accept_len;         /* [device] out [batch] tau                              */
+    int32_t*       out_tokens;         /* [device] out [batch, gamma+1]: kept drafts, the emitted token, then -1 */
+    int32_t*       bonus;              /* [device] out [batch] the emitted token (next anchor)  */
+    int32_t*       new_ctx_len;        /* [device] out [batch]; may alias ctx_len               */
+    void*          workspace;          /* [device]                                              */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;         /* [device] may be NULL                                  */
+} dflash_verify_sample_args;
+int32_t dflash_verify_accept_sample(dflash_handle* h, const dflash_verify_sample_args* a /*[host]*/, void* stream);
+int64_t dflash_sample_workspace_bytes(int32_t n_logit_rows, int32_t vocab);
+
 /* ---- building block: attention of `rows` block rows per sequence over paged context + the block
  * itself (App. A.3: K = [K_ctx ; K_block]_seq). FULL = draft mode, CAUSAL = the target's verify
  * pass over (gamma+1) rows. Head geometry and dtype come from the handle. q and k_blk must already

@@ -27,7 +27,8 @@ EXPORTS = (
     "dflash_ctx_project", "dflash_draft_block", "dflash_verify_accept", "dflash_block_attention",
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
-    "dflash_verify_accept_static",
+    "dflash_verify_accept_static", "dflash_sample_rows", "dflash_verify_accept_sample",
+    "dflash_sample_workspace_bytes",
 )
 N_FAMILIES = 15
 
@@ -74,6 +75,24 @@ class VerifyArgs(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p)]
 
 
+class SampleArgs(C.Structure):
+    _fields_ = [("logits", C.c_void_p), ("logits_dtype", C.c_int32), ("row_stride", C.c_int64),
+                ("n_rows", C.c_int32), ("vocab", C.c_int32), ("temperature", C.c_float), ("u", C.c_void_p),
+                ("ids", C.c_void_p), ("prob", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p)]
+
+
+class VerifySampleArgs(C.Structure):
+    _fields_ = [("target_logits", C.c_void_p), ("target_dtype", C.c_int32), ("target_row_stride", C.c_int64),
+                ("draft_logits", C.c_void_p), ("draft_dtype", C.c_int32), ("draft_row_stride", C.c_int64),
+                ("draft_rows_per_seq", C.c_int32), ("draft_ids", C.c_void_p), ("draft_stride", C.c_int32),
+                ("batch", C.c_int32), ("gamma", C.c_int32), ("vocab", C.c_int32), ("temperature", C.c_float),
+                ("u_accept", C.c_void_p), ("u_final", C.c_void_p), ("ctx_len", C.c_void_p),
+                ("accept_len", C.c_void_p), ("out_tokens", C.c_void_p), ("bonus", C.c_void_p),
+                ("new_ctx_len", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64),
+                ("dev_status", C.c_void_p)]
+
+
 class AttnArgs(C.Structure):
     _fields_ = [("mode", C.c_int32), ("q", C.c_void_p), ("k_blk", C.c_void_p), ("v_blk", C.c_void_p),
                 ("batch", C.c_int32), ("rows", C.c_int32), ("ctx_len", C.c_void_p), ("max_ctx_len", C.c_int32),
@@ -107,10 +126,13 @@ def load():
     lib.dflash_workspace_bytes.restype = C.c_int64
     for name, st in (("dflash_ctx_project", CtxArgs), ("dflash_draft_block", DraftArgs),
                      ("dflash_verify_accept", VerifyArgs), ("dflash_verify_accept_static", VerifyArgs), ("dflash_block_attention", AttnArgs),
-                     ("dflash_lmhead_argmax", LmHeadArgs)):
+                     ("dflash_lmhead_argmax", LmHeadArgs), ("dflash_sample_rows", SampleArgs),
+                     ("dflash_verify_accept_sample", VerifySampleArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(st), C.c_void_p]
         fn.restype = C.c_int32
+    lib.dflash_sample_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.dflash_sample_workspace_bytes.restype = C.c_int64
     lib.dflash_status_string.argtypes = [C.c_int32]
     lib.dflash_status_string.restype = C.c_char_p
     lib.dflash_launch_count.argtypes = []
@@ -306,6 +328,42 @@ class DFlash:
                        logits.shape[-1], _ptr(ctx_len), _ptr(accept_len), _ptr(out_tokens), _ptr(bonus),
                        _ptr(new_ctx_len), _ptr(target_ids_out), None, 0, _ptr(self.status))
         _check(self.lib.dflash_verify_accept_static(self.h, C.byref(a), _stream(stream)))
+
+    def _sample_ws(self, n_rows, vocab):
+        need = int(self.lib.dflash_sample_workspace_bytes(n_rows, vocab))
+        if need < 0:
+            raise DFlashError(-1)
+        ws = getattr(self, "_samp_ws", None)
+        if ws is None or ws.numel() < need:
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+            self._samp_ws = ws
+        return ws
+
+    def dflash_sample_rows(self, logits, temperature, u, ids, prob=None, stream=None):
+        """ids[m] = inverse-CDF draw from softmax(logits[m] / T) with the uniform u[m]."""
+        n, V = logits.shape[0], logits.shape[-1]
+        ws = self._sample_ws(n, V)
+        a = SampleArgs(_ptr(logits), F32 if logits.dtype == torch.float32 else BF16, logits.stride(0), n, V,
+                       float(temperature), _ptr(u), _ptr(ids), _ptr(prob), _ptr(ws), ws.numel(), _ptr(self.status))
+        _check(self.lib.dflash_sample_rows(self.h, C.byref(a), _stream(stream)))
+
+    def dflash_verify_accept_sample(self, target_logits, draft_logits, draft_rows_per_seq, draft_ids, draft_stride,
+                                    gamma, temperature, u_accept, u_final, ctx_len, accept_len, out_tokens, bonus,
+                                    new_ctx_len, draft_row_offset=0, draft_offset=0, stream=None):
+        """Speculative-sampling verification. target_logits [S, gamma+1, V]; draft_logits: 2-D [rows, V] with
+        draft j of sequence b at row draft_row_offset + b * draft_rows_per_seq + j."""
+        S, V = ctx_len.shape[0], target_logits.shape[-1]
+        ws = self._sample_ws(S * (2 * gamma + 1), V)
+        dl = draft_logits.reshape(-1, V) if draft_logits is not None else None
+        dl_ptr = C.c_void_p(dl.data_ptr() + draft_row_offset * dl.stride(0) * dl.element_size()) if dl is not None else None
+        a = VerifySampleArgs(_ptr(target_logits), F32 if target_logits.dtype == torch.float32 else BF16, 0, dl_ptr,
+                             (F32 if dl.dtype == torch.float32 else BF16) if dl is not None else F32,
+                             dl.stride(0) if dl is not None else 0, draft_rows_per_seq,
+                             C.c_void_p(draft_ids.data_ptr() + 4 * draft_offset) if draft_ids is not None else None,
+                             draft_stride, S, gamma, V, float(temperature), _ptr(u_accept), _ptr(u_final),
+                             _ptr(ctx_len), _ptr(accept_len), _ptr(out_tokens), _ptr(bonus), _ptr(new_ctx_len),
+                             _ptr(ws), ws.numel(), _ptr(self.status))
+        _check(self.lib.dflash_verify_accept_sample(self.h, C.byref(a), _stream(stream)))
 
     def dflash_block_attention(self, mode, q, k_blk, v_blk, ctx_len, max_ctx_len, page_table, kv_pool, layer,
                                out, stream=None):
