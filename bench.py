@@ -115,9 +115,10 @@ class ClockSampler:
 # the step
 # ------------------------------------------------------------------------------------------------
 class Step:
-    def __init__(self, wl, device, seed=0):
+    def __init__(self, wl, device, seed=0, temperature=0.0):
         from paper_2602_06036_b200 import binding
         cfg = wl.cfg
+        self.T = float(temperature)
         self.wl, self.cfg, self.dev = wl, cfg, device
         B, S = cfg.block_size, wl.batch
         self.gamma = B
@@ -169,16 +170,34 @@ class Step:
         self.max_ctx = max(wl.ctx_lens)
         self.rows_new = int(self.n_new.sum().item())
         self.side = None
+        if self.T > 0:
+            # sampling: the draft's logits are kept (fp32), drafts are drawn from them, and verification
+            # is speculative sampling; the uniforms are seeded inputs
+            gu = synth.substream(seed, "step.uniforms")
+            self.draft_logits = torch.empty((S * B, cfg.vocab), dtype=torch.float32, device=device)
+            self.u_draft = torch.rand((S * B,), generator=gu, dtype=torch.float32).to(device)
+            self.u_acc = torch.rand((S, g), generator=gu, dtype=torch.float32).to(device)
+            self.u_fin = torch.rand((S,), generator=gu, dtype=torch.float32).to(device)
 
     def run_draft(self, feats, anchor):
         lib = self.lib
         lib.dflash_ctx_project(feats, self.n_new, self.ctx_len, self.page_table, self.pool)
-        lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids)
+        if self.T > 0:
+            lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids,
+                                   logits_out=self.draft_logits)
+            lib.dflash_sample_rows(self.draft_logits, self.T, self.u_draft, self.draft_ids.view(-1))
+        else:
+            lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids)
 
     def run_verify(self, logits):
         # The target's verify pass is outside this library; its logits are an input. The drafts
         # verified are synthetic ones with a planted agreeing prefix (the random-init drafter would
         # never be accepted), so the accept kernel sees realistic accept lengths.
+        if self.T > 0:
+            self.lib.dflash_verify_accept_sample(logits, self.draft_logits, self.cfg.block_size, self.draft_ids,
+                                                 self.cfg.block_size, self.gamma, self.T, self.u_acc, self.u_fin,
+                                                 self.ctx_len, self.tau, self.out_tokens, self.bonus, self.new_len)
+            return
         self.lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
                                       self.out_tokens, self.bonus, self.new_len, logits=logits)
 
@@ -345,6 +364,8 @@ def main():
     ap.add_argument("--kernel", default=None, choices=["lmhead", "attention"],
                     help="run one building block alone (for profiler captures) instead of the step")
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="> 0: drafts are drawn from the draft's logits and verified by speculative sampling (default: greedy)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
@@ -369,7 +390,7 @@ def main():
     cfg = wl.cfg
     peaks = load_peaks()
     # replicas: every rank runs the same batch on its own GPU; there is no data-path collective
-    step = Step(wl, device, seed=0)
+    step = Step(wl, device, seed=0, temperature=args.temperature)
     S, B = wl.batch, cfg.block_size
 
     if args.kernel:
@@ -491,7 +512,8 @@ def main():
         "warmup": args.warmup, "ms_per_step": per_step_ms, "us_per_draft_block": per_step_ms * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "batch": S, "block_size": B, "ctx_lens": list(wl.ctx_lens)[:8],
-                   "step": "ctx_project(n_new=tau) + draft_block + verify_accept(logits)",
+                   "step": "ctx_project(n_new=tau) + draft_block + verify_accept(logits)" if args.temperature <= 0 else
+                           f"ctx_project(n_new=tau) + draft_block(logits kept) + sample_rows + verify_accept_sample, T={args.temperature}",
                    "l2": "per-step weight traffic (3.2 GB) exceeds the 126 MB L2; no flush",
                    "launch": "eager" if args.no_graph else "cuda graph replay of one step",
                    "parallelism": "replicas" if world > 1 else "single"},
