@@ -136,7 +136,7 @@ static int check_ws(const dflash_handle* h, void* ws, int64_t bytes, int batch, 
 
 static int zero_counters(const Launch& L, const Workspace& ws) {
     if (L.h->cfg.dtype != DFLASH_BF16) return DFLASH_OK;
-    return cudaMemsetAsync(ws.counters, 0, ws.counter_bytes, L.st) == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    return launch_zero(L, ws.counters, ws.counter_bytes);      // counter_bytes is a multiple of 256
 }
 
 // LM head + argmax over `rows` normalised rows z (config dtype)

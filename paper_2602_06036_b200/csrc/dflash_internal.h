@@ -109,5 +109,6 @@ int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t ro
                       int vocab, float4* seg_scratch, int32_t* ids, float* top1, float* margin);
 int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids);
 int launch_copy_f32(const Launch& L, const float* src, float* dst, int64_t n);
+int launch_zero(const Launch& L, void* dst, int64_t bytes);
 
 }  // namespace dflash

@@ -2,6 +2,7 @@
 // tiny configuration) and the small element-wise steps of the bf16 path; the bf16 contractions
 // and attention have tensor-core kernels of their own.
 #include "dflash_internal.h"
+#include "ptx_sm100.cuh"
 
 #include <math_constants.h>
 
@@ -466,6 +467,8 @@ __global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict
                                                              int vocab, int seg_len, float4* __restrict__ out) {
     __shared__ Top2 sh[8];
     constexpr int VEC = 16 / (int)sizeof(T);
+    ptx::pdl_trigger();
+    ptx::pdl_wait();      // the scratch written below may alias what the previous kernel still uses
     const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
     const T* src = logits + (size_t)row * row_stride;
     const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
@@ -509,6 +512,8 @@ __global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict
 __global__ void __launch_bounds__(256) row_argmax_merge_kernel(const float4* __restrict__ seg, int nseg, int rows,
                                                                int32_t* __restrict__ ids, float* __restrict__ top1,
                                                                float* __restrict__ margin) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -545,14 +550,20 @@ int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t ro
     const int nseg = row_argmax_segments(rows, vocab, L.h->sm_count);
     const int seg_len = ((vocab + nseg - 1) / nseg + 7) / 8 * 8;
     dim3 grid(nseg, rows);
+    // programmatic dependent launch: each kernel's blocks become resident while its predecessor drains
+    cudaError_t e;
     if (dtype == DFLASH_F32)
-        row_argmax_seg_kernel<float><<<grid, 256, 0, L.st>>>((const float*)logits, row_stride, vocab, seg_len, seg_scratch);
+        e = launch_pdl(row_argmax_seg_kernel<float>, grid, dim3(256), 0, L.st, (const float*)logits, row_stride, vocab, seg_len,
+                       seg_scratch);
     else
-        row_argmax_seg_kernel<__nv_bfloat16><<<grid, 256, 0, L.st>>>((const __nv_bfloat16*)logits, row_stride, vocab,
-                                                                     seg_len, seg_scratch);
-    DFLASH_CHECK_LAUNCH();
-    row_argmax_merge_kernel<<<(rows + 7) / 8, 256, 0, L.st>>>(seg_scratch, nseg, rows, ids, top1, margin);
-    DFLASH_CHECK_LAUNCH();
+        e = launch_pdl(row_argmax_seg_kernel<__nv_bfloat16>, grid, dim3(256), 0, L.st, (const __nv_bfloat16*)logits, row_stride,
+                       vocab, seg_len, seg_scratch);
+    ++g_launches;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
+    e = launch_pdl(row_argmax_merge_kernel, dim3((rows + 7) / 8), dim3(256), 0, L.st, (const float4*)seg_scratch, nseg, rows, ids,
+                   top1, margin);
+    ++g_launches;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
     return DFLASH_OK;
 }
 
@@ -564,6 +575,8 @@ __global__ void accept_kernel(const int32_t* __restrict__ target_ids, const int3
                               int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
                               int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx_len,
                               int32_t* __restrict__ target_ids_out) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int32_t* p = target_ids + (size_t)b * (gamma + 1);
@@ -582,11 +595,29 @@ __global__ void accept_kernel(const int32_t* __restrict__ target_ids, const int3
 
 int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids) {
     if (a.batch == 0) return DFLASH_OK;
-    accept_kernel<<<(a.batch + 127) / 128, 128, 0, L.st>>>(target_ids, a.draft_ids, a.draft_stride, a.batch,
-                                                           a.gamma, a.ctx_len, a.accept_len, a.out_tokens,
-                                                           a.bonus, a.new_ctx_len, a.target_ids_out);
-    DFLASH_CHECK_LAUNCH();
+    const cudaError_t e = launch_pdl(accept_kernel, dim3((a.batch + 127) / 128), dim3(128), 0, L.st, target_ids, a.draft_ids,
+                                     a.draft_stride, a.batch, a.gamma, a.ctx_len, a.accept_len, a.out_tokens, a.bonus,
+                                     a.new_ctx_len, a.target_ids_out);
+    ++g_launches;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
     return DFLASH_OK;
+}
+
+// Zeroing as a kernel (not a memset) so that it takes part in programmatic dependent launch: its
+// blocks are resident while the previous call's last kernel drains, and the kernel after it chains on.
+__global__ void __launch_bounds__(256) zero_kernel(uint4* __restrict__ dst, int64_t n16) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();          // the tickets may still be read by the previous kernel
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = make_uint4(0, 0, 0, 0);
+}
+int launch_zero(const Launch& L, void* dst, int64_t bytes) {      // dst 16-byte aligned, bytes a multiple of 16
+    if (bytes <= 0) return DFLASH_OK;
+    const int64_t n16 = bytes / 16;
+    const int grid = (int)std::min<int64_t>((n16 + 255) / 256, 64);
+    const cudaError_t e = launch_pdl(zero_kernel, dim3(grid), dim3(256), 0, L.st, reinterpret_cast<uint4*>(dst), n16);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 __global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
