@@ -16,6 +16,7 @@
 // Sums that decide an index are accumulated in double in a fixed order, so a result is reproducible
 // and differs from exact arithmetic only when u * total lies within ~1e-6 (relative) of an interval edge.
 #include "dflash_internal.h"
+#include "ptx_sm100.cuh"
 
 #include <math_constants.h>
 
@@ -64,6 +65,8 @@ __global__ void __launch_bounds__(256) softmax_stats_seg_kernel(const T* __restr
                                                                 int group_pitch, int vocab, int seg_len, float c,
                                                                 float2* __restrict__ out) {
     __shared__ float2 sh[8];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
     const T* src = logits + ((size_t)(row / group_rows) * group_pitch + row % group_rows) * row_stride;
     const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
@@ -108,6 +111,8 @@ __device__ __forceinline__ float2 row_stat(const float2* seg, int nseg, float c,
 __global__ void __launch_bounds__(32) rows_plan_kernel(const void* logits, int bf16, int64_t row_stride, int es, int n_rows,
                                                        int nseg, float c, const float2* __restrict__ stats,
                                                        const float* __restrict__ u, int32_t* ids, float* prob, Draw* draws) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const int row = blockIdx.x, lane = threadIdx.x;
     const float2 st = row_stat(stats + (size_t)row * nseg, nseg, c, lane);
     if (lane == 0) {
@@ -126,6 +131,8 @@ __global__ void __launch_bounds__(32) rows_plan_kernel(const void* logits, int b
 __global__ void __launch_bounds__(32) verify_plan_kernel(dflash_verify_sample_args a, int nseg, float c,
                                                          const float2* __restrict__ t_stats, const float2* __restrict__ d_stats,
                                                          Draw* draws) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const int b = blockIdx.x, lane = threadIdx.x;
     const int g = a.gamma, V = a.vocab;
     const int t_es = a.target_dtype == DFLASH_BF16 ? 2 : 4, d_es = a.draft_dtype == DFLASH_BF16 ? 2 : 4;
@@ -200,6 +207,8 @@ __device__ __forceinline__ void block_sum2(double& a, double& b, double* sh) {
 __global__ void __launch_bounds__(256) weights_seg_kernel(const Draw* __restrict__ draws, int vocab, int seg_len, float c,
                                                           double2* __restrict__ seg_w) {
     __shared__ double sh[16];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     const Draw d = draws[blockIdx.y];
     const int seg = blockIdx.x, nseg = gridDim.x;
     const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
@@ -220,6 +229,8 @@ __global__ void __launch_bounds__(256) weights_seg_kernel(const Draw* __restrict
 __global__ void __launch_bounds__(256) select_kernel(const Draw* __restrict__ draws, int vocab, int seg_len, int nseg, float c,
                                                      const double2* __restrict__ seg_w) {
     __shared__ double s_run[256];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
     __shared__ double s_x;
     __shared__ int s_seg, s_use_p, s_owner;
     const Draw d = draws[blockIdx.x];
@@ -334,21 +345,25 @@ int launch_stats(cudaStream_t st, const void* logits, int dtype, int64_t ld, int
                  int nseg, int seg_len, float c, float2* out) {
     if (rows == 0) return DFLASH_OK;
     dim3 grid(nseg, rows);
+    cudaError_t e;
     if (dtype == DFLASH_BF16)
-        softmax_stats_seg_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)logits, ld, group_rows, group_pitch, vocab,
-                                                                      seg_len, c, out);
+        e = launch_pdl(softmax_stats_seg_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (const __nv_bfloat16*)logits, ld, group_rows,
+                       group_pitch, vocab, seg_len, c, out);
     else
-        softmax_stats_seg_kernel<float><<<grid, 256, 0, st>>>((const float*)logits, ld, group_rows, group_pitch, vocab, seg_len, c, out);
+        e = launch_pdl(softmax_stats_seg_kernel<float>, grid, dim3(256), 0, st, (const float*)logits, ld, group_rows, group_pitch,
+                       vocab, seg_len, c, out);
     g_launches += 1;
-    return cudaGetLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 int launch_draws(cudaStream_t st, const Scratch& s, int n_draws, int vocab, int nseg, int seg_len, float c) {
     if (n_draws == 0) return DFLASH_OK;
-    weights_seg_kernel<<<dim3(nseg, n_draws), 256, 0, st>>>(s.draws, vocab, seg_len, c, s.seg_w);
-    select_kernel<<<n_draws, 256, 0, st>>>(s.draws, vocab, seg_len, nseg, c, s.seg_w);
+    const cudaError_t e1 = launch_pdl(weights_seg_kernel, dim3(nseg, n_draws), dim3(256), 0, st, (const Draw*)s.draws, vocab, seg_len, c,
+                                      s.seg_w);
+    const cudaError_t e2 = launch_pdl(select_kernel, dim3(n_draws), dim3(256), 0, st, (const Draw*)s.draws, vocab, seg_len, nseg, c,
+                                      (const double2*)s.seg_w);
     g_launches += 2;
-    return cudaGetLastError() == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    return (e1 == cudaSuccess && e2 == cudaSuccess) ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
 bool dtype_ok(int d) { return d == DFLASH_F32 || d == DFLASH_BF16; }
@@ -378,10 +393,11 @@ int32_t dflash_sample_rows(dflash_handle* h, const dflash_sample_args* a, void* 
     const float c = LOG2E / a->temperature;
     const int64_t ld = a->row_stride ? a->row_stride : a->vocab;
     SAMPLE_TRY(launch_stats(st, a->logits, a->logits_dtype, ld, a->n_rows, a->n_rows, a->n_rows, a->vocab, nseg, seg_len, c, s.stats));
-    rows_plan_kernel<<<a->n_rows, 32, 0, st>>>(a->logits, a->logits_dtype == DFLASH_BF16, ld, a->logits_dtype == DFLASH_BF16 ? 2 : 4,
-                                               a->n_rows, nseg, c, s.stats, a->u, a->ids, a->prob, s.draws);
+    const cudaError_t e = launch_pdl(rows_plan_kernel, dim3(a->n_rows), dim3(32), 0, st, a->logits, (int)(a->logits_dtype == DFLASH_BF16),
+                                     ld, a->logits_dtype == DFLASH_BF16 ? 2 : 4, a->n_rows, nseg, c, (const float2*)s.stats, a->u,
+                                     a->ids, a->prob, s.draws);
     g_launches += 1;
-    if (cudaGetLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
     return launch_draws(st, s, a->n_rows, a->vocab, nseg, seg_len, c);
 }
 
@@ -411,9 +427,10 @@ int32_t dflash_verify_accept_sample(dflash_handle* h, const dflash_verify_sample
     if (a->gamma > 0)      // the gamma draft rows of sequence b start at stored row b * draft_rows_per_seq
         SAMPLE_TRY(launch_stats(st, a->draft_logits, a->draft_dtype, d_ld, (int)d_rows, a->gamma, a->draft_rows_per_seq, a->vocab, nseg,
                                 seg_len, c, d_stats));
-    verify_plan_kernel<<<a->batch, 32, 0, st>>>(*a, nseg, c, s.stats, d_stats, s.draws);
+    const cudaError_t e = launch_pdl(verify_plan_kernel, dim3(a->batch), dim3(32), 0, st, *a, nseg, c, (const float2*)s.stats,
+                                     (const float2*)d_stats, s.draws);
     g_launches += 1;
-    if (cudaGetLastError() != cudaSuccess) return DFLASH_ERR_CUDA;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
     return launch_draws(st, s, a->batch, a->vocab, nseg, seg_len, c);
 }
 
