@@ -63,6 +63,18 @@ def test_bf16_block_sizes_and_feature_counts(B, k, layers, lens):
     assert n_sure >= case.S * B // 2
 
 
+def test_bf16_feature_dims_that_are_not_multiples_of_64():
+    # contraction lengths of 520 / 1544 / 1560 (multiples of 8 only): the one-slab ring stages with a
+    # zero-filled K tail, ragged 128-feature tiles in the folded norms, a ragged last weight tile
+    cfg = dataclasses.replace(synth.MID, d_model=520, d_ffn=1544, d_target=520, vocab=3001)
+    case = Case(cfg, (5, 140), seed=13)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    n_sure = case.check_draft(got)
+    assert n_sure >= case.S * cfg.block_size // 2
+
+
 def test_decode_step_appends_at_ctx_len():
     # second projection call with n_new < max_new appends rows at positions L..L+n-1 only
     cfg = synth.MID
