@@ -9,7 +9,8 @@ namespace dflash {
 bool attn_tc_supported(const dflash_config& c, int rows);
 int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count);
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
-// `part` / `counters`: split-KV scratch of the sizes above; counters must be zero on entry.
+// `part`: split-KV scratch of the size above. `counters` is not used by the current kernels (the
+// partials are merged by a second kernel, not by a last arriver).
 int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters);
 
 }  // namespace dflash

@@ -4,14 +4,19 @@
 // (16..256 columns), so the tensor core runs full-height instructions however few tokens there
 // are. A CTA is one TMA producer warp, one MMA-issuing warp and four epilogue warps; operands
 // stream through a ring of 128-byte-swizzled shared-memory stages, accumulators live in two TMEM
-// buffers so the epilogue of one piece of work overlaps the main loop of the next. The work is the
-// sequence of all (output tile, K chunk) pairs, cut into one contiguous, equally long range per CTA
-// ("stream-K"): every SM streams the same number of weight bytes whatever the tile count. A range
-// that covers a whole output tile goes straight to the epilogue; a tile shared by several CTAs is
-// finished at the end of the phase by ALL of them: each writes its partial sums and a ticket, waits
-// (bounded) until the tile's tickets are complete, and then sums the pieces in CTA order for its own
-// share of the tile's token passes (bit-reproducible, and the finishing work is spread over the CTAs
-// instead of piling up on one). RMSNorm never runs as a kernel of its own: epilogues that produce residual
+// buffers so the epilogue of one piece of work overlaps the main loop of the next.
+// Work split ("stream-K" remainder first, whole tiles last): with at least one output tile per CTA,
+// the n_tiles % n_ctas remainder tiles are cut into (tile, K chunk) pairs and shared out as one
+// contiguous, equally long range per CTA; the other tiles go whole, the same number to every CTA. So
+// every SM streams the same number of weight bytes whatever the tile count, the cross-CTA reduction
+// of the shared tiles runs under the main loop of the whole tiles, and a phase ends with direct
+// epilogues. With fewer tiles than CTAs all tiles are shared. A shared tile is finished by ALL of its
+// contributors: each writes its partial sums and takes a ticket, waits (bounded) until the tile's
+// tickets are complete, and then sums the pieces in CTA order for its own share of the tile's token
+// passes (bit-reproducible, and the finishing work is spread over the CTAs instead of piling up on
+// one). A ring stage holds one or two 64-element K slabs of both operands (two for small token tiles,
+// fetched by one 3-D copy each: the single issuing thread, not HBM, is the limit there).
+// RMSNorm never runs as a kernel of its own: epilogues that produce residual
 // rows also emit the gain-scaled bf16 operand and per-tile sums of squares, and the consuming
 // contraction scales its accumulator columns by the per-token rsqrt.
 // One launch runs a CHAIN of up to four such contractions ("phases": e.g. output projection ->
@@ -20,8 +25,10 @@
 // waits until every CTA has signalled the end of the previous phase (a counter in global memory,
 // polled with a bound), so the tail of one phase - partial sums, tickets, epilogues - overlaps the
 // weight stream of the next and HBM stays busy across the chain.
-// Launched with programmatic dependent launch: barrier set-up, TMEM allocation and the first ring
-// of WEIGHT tiles (which no earlier kernel writes) are issued before griddepcontrol.wait.
+// Launched with programmatic dependent launch: barrier set-up and TMEM allocation happen before
+// griddepcontrol.wait. (Filling the ring with weight tiles before that wait was measured slower: the
+// copy queue is in order, so CTAs that start after the dependency resolved had their first
+// activation tiles stuck behind a ring of HBM-bound weight copies.)
 // Every wait on an mbarrier is bounded; on expiry the kernel raises DFLASH_DEV_TIMEOUT, drains its
 // outstanding copies, frees its TMEM and returns.
 #include "gemm_tc.cuh"
@@ -491,7 +498,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
-    volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] last-arriver, [2] epilogue abort
+    volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [2] epilogue abort
     int* sPend = const_cast<int*>(flags) + 4;                               // [3 * MAX_STAGES] producer's queue
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -499,7 +506,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
-        flags[0] = 0; flags[1] = 0; flags[2] = 0;
+        flags[0] = 0; flags[2] = 0;
         fence_barrier_init();
         fence_proxy_async();
     }
