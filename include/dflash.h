@@ -156,6 +156,9 @@ typedef struct {
     float*         hidden_out;   /* [device] out [batch*B, D] fp32 residual stream after the last layer; may be NULL */
     float*         logits_out;   /* [device] out [batch*B, V] fp32; may be NULL (tests only)  */
     int32_t*       dev_status;   /* [device] may be NULL                                      */
+    int32_t        block_rows;   /* rows per sequence in THIS call: 0 = the handle's block_size B, else 1..B
+                                    (a drafter trained at B = 16 also runs blocks of 8 or 10, Sec. 5.3); every
+                                    [batch, B] / [batch*B, ...] shape above then uses block_rows in place of B */
 } dflash_draft_args;
 int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a /*[host]*/, void* stream);
 

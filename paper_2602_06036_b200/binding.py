@@ -63,7 +63,7 @@ class DraftArgs(C.Structure):
                 ("kv_pool", C.c_void_p), ("n_pool_pages", C.c_int32), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_int64), ("draft_ids", C.c_void_p), ("top1", C.c_void_p),
                 ("margin", C.c_void_p), ("hidden_out", C.c_void_p), ("logits_out", C.c_void_p),
-                ("dev_status", C.c_void_p)]
+                ("dev_status", C.c_void_p), ("block_rows", C.c_int32)]
 
 
 class VerifyArgs(C.Structure):
@@ -292,12 +292,13 @@ class DFlash:
         _check(self.lib.dflash_ctx_project(self.h, C.byref(a), _stream(stream)))
 
     def dflash_draft_block(self, anchor_ids, ctx_len, max_ctx_len, page_table, kv_pool, draft_ids,
-                           top1=None, margin=None, hidden_out=None, logits_out=None, stream=None):
+                           top1=None, margin=None, hidden_out=None, logits_out=None, stream=None, block_rows=0):
+        """block_rows: rows per sequence in this call (0 = the handle's block size)."""
         S = anchor_ids.shape[0]
         ws = self.workspace(S, S * self.cfg.block_size)
         a = DraftArgs(_ptr(anchor_ids), S, _ptr(ctx_len), int(max_ctx_len), _ptr(page_table), page_table.shape[1],
                       _ptr(kv_pool), kv_pool.shape[1], _ptr(ws), ws.numel(), _ptr(draft_ids), _ptr(top1),
-                      _ptr(margin), _ptr(hidden_out), _ptr(logits_out), _ptr(self.status))
+                      _ptr(margin), _ptr(hidden_out), _ptr(logits_out), _ptr(self.status), int(block_rows))
         _check(self.lib.dflash_draft_block(self.h, C.byref(a), _stream(stream)))
 
     def dflash_verify_accept(self, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus,

@@ -358,7 +358,8 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     if (!a->anchor_ids || !a->ctx_len || !a->page_table || !a->kv_pool || !a->draft_ids) return DFLASH_ERR_INVALID_ARG;
     const dflash_config& c = h->cfg;
     if ((int64_t)a->batch * c.block_size > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
-    const int B = c.block_size, rows = a->batch * B;
+    if (a->block_rows < 0 || a->block_rows > c.block_size) return DFLASH_ERR_INVALID_ARG;
+    const int B = a->block_rows > 0 ? a->block_rows : c.block_size, rows = a->batch * B;
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
     Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
@@ -391,7 +392,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV]; g.epoch = i + 1;
             return g;
         };
-        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, ws.x, h->layers[0].g1, xn, ws.ssq));
+        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, B, ws.x, h->layers[0].g1, xn, ws.ssq));
         {
             const GemmArgs g = qkv_args(0);
             RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
@@ -450,7 +451,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     }
 
     // fp32: CUDA-core kernels, one step per launch
-    RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, ws.x, a->batch));
+    RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, ws.x, a->batch, B));
     for (int i = 0; i < c.n_layers; ++i) {
         const dflash_layer_weights& lw = h->layers[i];
         // attention half: u = RMSNorm(x); q,k,v = W u (+RoPE); x += W_o attention(q, [K_ctx; k], [V_ctx; v])

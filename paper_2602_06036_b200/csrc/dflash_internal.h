@@ -94,7 +94,7 @@ struct Launch {
 };
 
 // ---- generic (any dtype) kernels: the whole fp32 path, and the small steps of the bf16 path ----
-int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch);
+int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch, int block_rows);
 int launch_rmsnorm(const Launch& L, const void* in, bool in_is_f32, const void* g, bool apply,
                    void* out, int rows, int dim);
 int launch_gemm_simt(const Launch& L, const void* X, const void* W, float* Y, int M, int N, int K,

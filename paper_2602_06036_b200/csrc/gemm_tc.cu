@@ -1097,14 +1097,14 @@ int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, in
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
-int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, float* x, const void* g, __nv_bfloat16* xn,
-                      float* ssq) {
+int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, int block_rows, float* x, const void* g,
+                      __nv_bfloat16* xn, float* ssq) {
     const dflash_config& c = L.h->cfg;
-    const int rows = batch * c.block_size;
+    const int rows = batch * block_rows;
     if (rows <= 0) return DFLASH_OK;
     const cudaError_t e = launch_pdl(embed_norm_kernel, dim3(rows), dim3(256), 0, L.st,
                                      (const __nv_bfloat16*)L.h->w.embed, anchor, x, (const __nv_bfloat16*)g, xn, ssq,
-                                     c.block_size, c.d_model, c.vocab, c.mask_token_id, rows, L.status, L.trace);
+                                     block_rows, c.d_model, c.vocab, c.mask_token_id, rows, L.status, L.trace);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }

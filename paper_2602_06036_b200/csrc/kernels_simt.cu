@@ -73,15 +73,15 @@ __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict_
     for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = to_f(src[d]);
 }
 
-int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch) {
+int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch, int block_rows) {
     const dflash_config& c = L.h->cfg;
-    const int rows = batch * c.block_size;
+    const int rows = batch * block_rows;
     if (c.dtype == DFLASH_F32)
-        embed_kernel<float><<<rows, 256, 0, L.st>>>((const float*)L.h->w.embed, anchor, x, c.block_size,
+        embed_kernel<float><<<rows, 256, 0, L.st>>>((const float*)L.h->w.embed, anchor, x, block_rows,
                                                     c.d_model, c.vocab, c.mask_token_id, L.status);
     else
         embed_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>((const __nv_bfloat16*)L.h->w.embed, anchor, x,
-                                                            c.block_size, c.d_model, c.vocab,
+                                                            block_rows, c.d_model, c.vocab,
                                                             c.mask_token_id, L.status);
     DFLASH_CHECK_LAUNCH();
     return DFLASH_OK;

@@ -63,6 +63,37 @@ def test_bf16_block_sizes_and_feature_counts(B, k, layers, lens):
     assert n_sure >= case.S * B // 2
 
 
+@pytest.mark.parametrize("name", ["cfg0", "mid"])
+def test_block_size_chosen_per_call(name):
+    # one handle (block size 8 or 16), blocks of fewer rows per call (Sec. 5.3: a drafter trained with a
+    # large block also drafts smaller ones); the oracle runs the same weights at that block size
+    wl = synth.workload(name)
+    case = Case(wl.cfg, wl.ctx_lens, seed=wl.seed)
+    case.project_prefill()
+    full = wl.cfg.block_size
+    for rows in sorted({1, full // 2, min(10, full), full}):
+        cfg_r = dataclasses.replace(wl.cfg, block_size=rows)
+        S, dev = case.S, case.device
+        ids = torch.full((S, rows), -7, dtype=torch.int32, device=dev)
+        margin = torch.zeros((S, rows), dtype=torch.float32, device=dev)
+        logits = torch.zeros((S * rows, wl.cfg.vocab), dtype=torch.float32, device=dev)
+        anchors = synth.make_anchors(wl.cfg, S, wl.seed)
+        case.lib.status.zero_()
+        case.lib.dflash_draft_block(anchors.to(dev), case.ctx_len, max(case.ctx_lens + [0]), case.page_table, case.pool, ids,
+                                    margin=margin, logits_out=logits, block_rows=rows)
+        torch.cuda.synchronize()
+        assert int(case.lib.status.item()) == 0
+        got_logits = logits.cpu().numpy().reshape(S, rows, -1)
+        for b in range(S):
+            Ks, Vs = case.oracle_ctx(b)
+            ref = orc.draft_block(int(anchors[b]), case.ctx_lens[b], Ks, Vs, case.w_np, cfg_r, return_logits=True)
+            assert_close(got_logits[b], ref["logits"], wl.cfg.dtype, f"logits rows={rows} seq {b}")
+            sure = ref["margin"] > (0.1 if wl.cfg.dtype == "bf16" else 1e-3)
+            assert (ids[b].cpu().numpy()[sure] == ref["ids"][sure]).all()
+    with pytest.raises(Exception):
+        case.lib.dflash_draft_block(anchors.to(dev), case.ctx_len, 0, case.page_table, case.pool, ids, block_rows=full + 1)
+
+
 def test_bf16_feature_dims_that_are_not_multiples_of_64():
     # contraction lengths of 520 / 1544 / 1560 (multiples of 8 only): the one-slab ring stages with a
     # zero-filled K tail, ragged 128-feature tiles in the folded norms, a ragged last weight tile
