@@ -15,7 +15,9 @@ Everything is float64 numpy, one sequence at a time, in the order and notation o
   Sec. 3.1 (Eq. 1 and the sentence after it): gamma drafts verified in parallel,
   tau in [1, gamma+1] including the bonus token; lossless under greedy decoding    -> verify_accept
 
-Readings taken where the paper is silent (each is listed in the design notes): pre-norm residual
+Readings taken where the paper is silent (each is listed in the design notes): optional per-head
+RMSNorm of q and k before the rotation (cfg.qk_norm; App. A.3 shows plain projections, the Qwen3 layers
+the draft shares its architecture with carry it); pre-norm residual
 layers; RMSNorm y * (mean(y^2)+eps)^-1/2 * g; no biases; SwiGLU FFN; rotary position encoding with
 rotate-half pairing (i, i + hd/2), context token p at position p and block row r at position L+r;
 softmax scale hd^-1/2; argmax takes the lowest index among equal maxima and NaN never wins.
@@ -120,11 +122,14 @@ def ctx_fuse(feats, W_c, g_c, eps):
     return rmsnorm(linear(feats, W_c), g_c, eps)
 
 
-def ctx_kv(H_t, W_k, W_v, pos, cfg):
-    """K^ctx = RoPE(W_i^K H_t), V^ctx = W_i^V H_t for one draft layer. Returns [T, Hkv, hd] each."""
+def ctx_kv(H_t, W_k, W_v, pos, cfg, g_k=None):
+    """K^ctx = RoPE(W_i^K H_t), V^ctx = W_i^V H_t for one draft layer. Returns [T, Hkv, hd] each.
+    With cfg.qk_norm, every key head is RMS-normalised with gain g_k before the rotation."""
     T = H_t.shape[0]
     k = linear(H_t, W_k).reshape(T, cfg.n_kv_heads, cfg.head_dim)
     v = linear(H_t, W_v).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    if getattr(cfg, "qk_norm", 0):
+        k = rmsnorm(k, g_k, cfg.rms_eps)
     if cfg.use_rope:
         k = rope(k, pos, cfg.rope_theta)
     return k, v
@@ -135,7 +140,7 @@ def ctx_project(feats, pos, weights, cfg):
     H_t = ctx_fuse(feats, weights["W_c"], weights["g_c"], cfg.rms_eps)
     Ks, Vs = [], []
     for lw in weights["layers"]:
-        k, v = ctx_kv(H_t, lw["W_k"], lw["W_v"], pos, cfg)
+        k, v = ctx_kv(H_t, lw["W_k"], lw["W_v"], pos, cfg, lw.get("g_k"))
         Ks.append(k)
         Vs.append(v)
     return np.stack(Ks), np.stack(Vs)
@@ -206,6 +211,9 @@ def draft_layer(x, lw, k_ctx, v_ctx, pos, cfg, causal=False):
     q = linear(u, lw["W_q"]).reshape(R, cfg.n_q_heads, cfg.head_dim)
     k = linear(u, lw["W_k"]).reshape(R, cfg.n_kv_heads, cfg.head_dim)
     v = linear(u, lw["W_v"]).reshape(R, cfg.n_kv_heads, cfg.head_dim)
+    if getattr(cfg, "qk_norm", 0):       # per-head RMSNorm over head_dim (the target family's attention variant)
+        q = rmsnorm(q, lw["g_q"], cfg.rms_eps)
+        k = rmsnorm(k, lw["g_k"], cfg.rms_eps)
     if cfg.use_rope:
         q = rope(q, pos, cfg.rope_theta)
         k = rope(k, pos, cfg.rope_theta)

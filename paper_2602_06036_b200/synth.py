@@ -47,6 +47,7 @@ class DFlashConfig:
     use_rope: int = 1
     rms_eps: float = 1e-6
     rope_theta: float = 1.0e6
+    qk_norm: int = 0       # 1: per-head RMSNorm of q and k (gains g_q, g_k of length hd) before the rotation
 
     @property
     def mask_token_id(self) -> int:
@@ -173,6 +174,9 @@ def make_weights(cfg: DFlashConfig, seed: int = 0) -> Dict:
             "W_up": lin(p + "W_up", F, D),
             "W_down": lin(p + "W_down", D, F),
         })
+        if cfg.qk_norm:
+            w["layers"][-1]["g_q"] = normal((cfg.head_dim,), 0.1, seed, p + "g_q", dt, mean=1.0)
+            w["layers"][-1]["g_k"] = normal((cfg.head_dim,), 0.1, seed, p + "g_k", dt, mean=1.0)
     return w
 
 
@@ -194,6 +198,9 @@ def pack_device_weights(cfg: DFlashConfig, w: Dict) -> Dict:
             "W_gateup": gu.contiguous(),
             "W_down": lw["W_down"],
         })
+        if cfg.qk_norm:
+            out["layers"][-1]["g_q"] = lw["g_q"]
+            out["layers"][-1]["g_k"] = lw["g_k"]
     return out
 
 

@@ -249,3 +249,34 @@ def test_pool_roundtrip_and_page_scatter():
         p = 131
         assert pool[0, table[p // 64], 0, 1, p % 64, 3] == K[0, p, 1, 3]
         assert pool[0, table[p // 64], 1, 0, p % 64, 5] == V[0, p, 0, 5]
+
+
+def test_qk_norm_is_a_per_head_rmsnorm_before_the_rotation():
+    # the optional attention variant (cfg.qk_norm): checked against explicit loops over heads, and through
+    # two properties: the layer's output does not change when W_q (or W_k) is scaled by a positive constant,
+    # and with it off the same scaling does change the output
+    import dataclasses
+    from paper_2602_06036_b200 import synth
+    cfg = dataclasses.replace(synth.TINY, qk_norm=1, block_size=4)
+    w = synth.weights_to_numpy(synth.make_weights(cfg, 21))
+    lw = w["layers"][0]
+    rng = np.random.default_rng(2)
+    x = rng.normal(size=(4, cfg.d_model))
+    kc = rng.normal(size=(9, cfg.n_kv_heads, cfg.head_dim))
+    vc = rng.normal(size=(9, cfg.n_kv_heads, cfg.head_dim))
+    pos = np.arange(9, 13)
+    base = orc.draft_layer(x, lw, kc, vc, pos, cfg)
+    scaled = dict(lw, W_q=lw["W_q"] * 3.7, W_k=lw["W_k"] * 0.21)
+    np.testing.assert_allclose(orc.draft_layer(x, scaled, kc, vc, pos, cfg), base, rtol=0, atol=1e-4)      # exact up to eps / mean square
+    off = dataclasses.replace(cfg, qk_norm=0)
+    assert np.abs(orc.draft_layer(x, scaled, kc, vc, pos, off) - orc.draft_layer(x, lw, kc, vc, pos, off)).max() > 1e-2
+    # context keys: loops over tokens and heads
+    H_t = rng.normal(size=(5, cfg.d_model))
+    K, V = orc.ctx_kv(H_t, lw["W_k"], lw["W_v"], np.arange(5), cfg, lw["g_k"])
+    raw = (H_t @ lw["W_k"].T).reshape(5, cfg.n_kv_heads, cfg.head_dim)
+    for t in range(5):
+        for h in range(cfg.n_kv_heads):
+            r = raw[t, h]
+            n = lw["g_k"] * r / np.sqrt(np.mean(r * r) + cfg.rms_eps)
+            np.testing.assert_allclose(K[t, h], orc.rope(n[None, None, :], np.array([t]), cfg.rope_theta)[0, 0], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(V, (H_t @ lw["W_v"].T).reshape(5, cfg.n_kv_heads, cfg.head_dim), rtol=1e-12)
