@@ -72,6 +72,10 @@ typedef struct {
     int32_t use_rope;       /* 1: rotary positions (rotate-half pairing) on q and k; 0: none */
     float   rms_eps;
     float   softmax_scale;  /* usually head_dim^-1/2 */
+    int32_t qk_norm;        /* 1: every q and k head is RMS-normalised over head_dim (gains g_q, g_k, same rms_eps)
+                               before the rotation, for block rows and for the injected context keys. The paper's
+                               App. A.3 shows plain projections; the Qwen3 layers the draft shares its
+                               architecture with carry this norm. 0: off. */
 } dflash_config;
 
 typedef struct {
@@ -81,6 +85,8 @@ typedef struct {
     const void* g2;        /* [device] [D]            pre-FFN norm gain                  */
     const void* W_gateup;  /* [device] [2F, D]        row 2j = gate_j, row 2j+1 = up_j   */
     const void* W_down;    /* [device] [D, F]                                             */
+    const void* g_q;       /* [device] [hd] gain of the q-head norm (qk_norm = 1, else ignored / NULL) */
+    const void* g_k;       /* [device] [hd] gain of the k-head norm (qk_norm = 1, else ignored / NULL) */
 } dflash_layer_weights;
 
 typedef struct {

@@ -37,11 +37,11 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "n_feat_layers",
         "d_target", "block_size", "page_size", "dtype", "mask_token_id", "use_rope")] + [
-        ("rms_eps", C.c_float), ("softmax_scale", C.c_float)]
+        ("rms_eps", C.c_float), ("softmax_scale", C.c_float), ("qk_norm", C.c_int32)]
 
 
 class LayerWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("g1", "W_qkv", "W_o", "g2", "W_gateup", "W_down")]
+    _fields_ = [(n, C.c_void_p) for n in ("g1", "W_qkv", "W_o", "g2", "W_gateup", "W_down", "g_q", "g_k")]
 
 
 class Weights(C.Structure):
@@ -188,7 +188,7 @@ class DFlash:
         self.ccfg = Config(cfg.n_layers, cfg.d_model, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ffn,
                            cfg.vocab, cfg.n_feat_layers, cfg.d_target, cfg.block_size, cfg.page_size,
                            F32 if cfg.dtype == "fp32" else BF16, cfg.mask_token_id, cfg.use_rope,
-                           cfg.rms_eps, cfg.softmax_scale)
+                           cfg.rms_eps, cfg.softmax_scale, int(getattr(cfg, "qk_norm", 0)))
         hp = C.c_void_p()
         _check(self.lib.dflash_create(C.byref(self.ccfg), C.byref(hp)))
         self.h = hp
@@ -217,7 +217,8 @@ class DFlash:
         keep["rope_sin"] = rope_sin.to(dev, torch.float32).contiguous()
         arr = (LayerWeights * self.cfg.n_layers)()
         for i, lw in enumerate(keep["layers"]):
-            arr[i] = LayerWeights(*(lw[k].data_ptr() for k in ("g1", "W_qkv", "W_o", "g2", "W_gateup", "W_down")))
+            arr[i] = LayerWeights(*(lw[k].data_ptr() for k in ("g1", "W_qkv", "W_o", "g2", "W_gateup", "W_down")),
+                                  *((lw[k].data_ptr() if k in lw else None) for k in ("g_q", "g_k")))
         w = Weights(keep["embed"].data_ptr(), keep["W_c"].data_ptr(), keep["g_c"].data_ptr(), arr,
                     keep["g_f"].data_ptr(), keep["W_lm"].data_ptr(), keep["rope_cos"].data_ptr(),
                     keep["rope_sin"].data_ptr(), keep["rope_cos"].shape[0])

@@ -192,6 +192,7 @@ int32_t dflash_create(const dflash_config* cfg, dflash_handle** out) {
         c.page_size < 1 || !(c.rms_eps >= 0.f) || !(c.softmax_scale > 0.f))
         return DFLASH_ERR_INVALID_ARG;
     if (c.mask_token_id < 0 || c.mask_token_id >= c.vocab) return DFLASH_ERR_INVALID_ARG;
+    if (c.qk_norm != 0 && c.qk_norm != 1) return DFLASH_ERR_INVALID_ARG;
     if (c.dtype != DFLASH_F32 && c.dtype != DFLASH_BF16) return DFLASH_ERR_UNSUPPORTED;
     if (c.n_layers > DFLASH_MAX_LAYERS) return DFLASH_ERR_UNSUPPORTED;
     if (c.head_dim != 64 && c.head_dim != 128) return DFLASH_ERR_UNSUPPORTED;
@@ -277,6 +278,7 @@ int32_t dflash_set_weights(dflash_handle* h, const dflash_weights* w) {
     for (int i = 0; i < h->cfg.n_layers; ++i) {
         const dflash_layer_weights& l = w->layers[i];
         if (!l.g1 || !l.W_qkv || !l.W_o || !l.g2 || !l.W_gateup || !l.W_down) return DFLASH_ERR_INVALID_ARG;
+        if (h->cfg.qk_norm && (!l.g_q || !l.g_k)) return DFLASH_ERR_INVALID_ARG;
         h->layers[i] = l;
     }
     h->w = *w;
@@ -320,7 +322,10 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
         for (int i0 = 0; i0 < c.n_layers; i0 += GEMM_MAX_GROUPS - 1) {
             GemmArgs k{};
             k.n_groups = std::min(GEMM_MAX_GROUPS - 1, c.n_layers - i0);
-            for (int j = 0; j < k.n_groups; ++j) k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
+            for (int j = 0; j < k.n_groups; ++j) {
+                k.W[j] = (const char*)h->layers[i0 + j].W_qkv + kv_off;
+                k.g_k_group[j] = c.qk_norm ? h->layers[i0 + j].g_k : nullptr;
+            }
             k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
             k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part;
             k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV]; k.epoch = i0 / (GEMM_MAX_GROUPS - 1) + 1;
@@ -345,7 +350,7 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
     for (int i = 0; i < c.n_layers; ++i) {
         const char* Wkv = (const char*)h->layers[i].W_qkv + kv_off;
         RUN(FAM_CTX_KV, launch_gemm_simt(L, ws.u, Wkv, ws.tmp, rows, 2 * kdim, c.d_model, false));
-        RUN(FAM_CTX_KV, launch_ctx_scatter(L, ws.tmp, *a, i));
+        RUN(FAM_CTX_KV, launch_ctx_scatter(L, ws.tmp, *a, i, c.qk_norm ? h->layers[i].g_k : nullptr));
     }
     return DFLASH_OK;
 }
@@ -389,6 +394,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             g.X = xn; g.W[0] = h->layers[i].W_qkv; g.M = rows; g.N = qdim + 2 * kdim; g.K = c.d_model; g.ssq_in = ws.ssq;
             g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
             g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
+            if (c.qk_norm) { g.g_q = h->layers[i].g_q; g.g_k = h->layers[i].g_k; }
             g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV]; g.epoch = i + 1;
             return g;
         };
@@ -457,7 +463,8 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
         // attention half: u = RMSNorm(x); q,k,v = W u (+RoPE); x += W_o attention(q, [K_ctx; k], [V_ctx; v])
         RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g1, true, ws.u, rows, c.d_model));
         RUN(FAM_GEMM_QKV, launch_gemm_simt(L, ws.u, lw.W_qkv, ws.tmp, rows, qdim + 2 * kdim, c.d_model, false));
-        RUN(FAM_GEMM_QKV, launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk));
+        RUN(FAM_GEMM_QKV, launch_rope_split(L, ws.tmp, a->ctx_len, B, rows, ws.q, ws.k_blk, ws.v_blk, c.qk_norm ? lw.g_q : nullptr,
+                                                c.qk_norm ? lw.g_k : nullptr));
         at.layer = i;
         RUN(FAM_ATTENTION, launch_attention_simt(L, at));
         RUN(FAM_GEMM_O, launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));

@@ -99,11 +99,12 @@ int launch_rmsnorm(const Launch& L, const void* in, bool in_is_f32, const void* 
                    void* out, int rows, int dim);
 int launch_gemm_simt(const Launch& L, const void* X, const void* W, float* Y, int M, int N, int K,
                      bool accumulate);
+// g_q / g_k: gains of the per-head q / k norm applied before the rotation, or nullptr
 int launch_rope_split(const Launch& L, const float* qkv, const int32_t* ctx_len, int rows_per_seq,
-                      int rows, void* q, void* k, void* v);
+                      int rows, void* q, void* k, void* v, const void* g_q, const void* g_k);
 int launch_swiglu(const Launch& L, const float* gu, void* h, int rows);
 int launch_attention_simt(const Launch& L, const dflash_attn_args& a);
-int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer);
+int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer, const void* g_k);
 // two-stage row argmax; seg_scratch holds rows * 64 float4 entries
 int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows,
                       int vocab, float4* seg_scratch, int32_t* ids, float* top1, float* margin);

@@ -80,6 +80,8 @@ struct KParams {
     float* out_f32;
     int ld_out;
     __nv_bfloat16 *q, *k, *v;
+    const __nv_bfloat16* gq;                          // per-head norm gains [hd] (nullptr: no head norm)
+    const __nv_bfloat16* gk[GEMM_MAX_GROUPS];         // QKV: [0]; context K/V: one per group (layer)
     const int32_t* ctx_len;
     int rows_per_seq, Hq, Hkv, hd, use_rope;
     const float *cs, *sn;
@@ -210,8 +212,40 @@ __device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, 
     }
 }
 
+// rn[c] = rsqrt(mean over this row's head of acc^2 + eps) for SB token columns of sAcc, all 128
+// threads together (two named barriers): a head is the tile's 128 rows (hd = 128) or its half (hd = 64).
+template <int SB>
+__device__ __forceinline__ void head_rnorm(const KParams& p, const float* sAcc, int acc_ld, float* red, int row, int c0, int n_tok,
+                                           bool active, float (&rn)[SB]) {
+    float sq[SB];
+#pragma unroll
+    for (int c = 0; c < SB; ++c) {
+        const float a = (active && c0 + c < n_tok) ? sAcc[row * acc_ld + c0 + c] : 0.f;
+        sq[c] = a * a;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int c = 0; c < SB; ++c) sq[c] += __shfl_xor_sync(0xffffffffu, sq[c], o);
+    if ((row & 31) == 0) {
+#pragma unroll
+        for (int c = 0; c < SB; ++c) red[(row >> 5) * SB + c] = sq[c];
+    }
+    epi_bar();
+    const int w0 = p.hd == 128 ? 0 : (row >> 6) * 2, nw = p.hd == 128 ? 4 : 2;
+    const float inv_hd = 1.f / (float)p.hd;
+#pragma unroll
+    for (int c = 0; c < SB; ++c) {
+        float t = 0.f;
+        for (int w = 0; w < nw; ++w) t += red[(w0 + w) * SB + c];
+        rn[c] = rsqrtf(t * inv_hd + p.eps);
+    }
+    epi_bar();
+}
+
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
-template <int CH>
+// QKN: the launch has per-head q/k norms (a separate instantiation keeps the common path's registers down).
+template <int CH, bool QKN>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
                                                int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain) {
     // tPos / tPage: position and (context projection) pool row of the page slot of the tokens of this pass (-1 = skip)
@@ -262,42 +296,56 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
             }
         } break;
         case EPI_QKV_ROPE: {
-            if (f < p.N) {
-                const int hd = p.hd, half = hd >> 1;
-                const int head = f / hd, hrow = f % hd, i = hrow % half;
-                const int partner = row ^ half;
-                const int qdim = p.Hq * hd, kdim = p.Hkv * hd;
-                const bool rot = p.use_rope && head < p.Hq + p.Hkv;
-                __nv_bfloat16* dst;
-                int ld;
-                if (head < p.Hq) { dst = p.q + f; ld = qdim; }
-                else if (head < p.Hq + p.Hkv) { dst = p.k + (f - qdim); ld = kdim; }
-                else { dst = p.v + (f - qdim - kdim); ld = kdim; }
-                constexpr int SB = CH <= 16 ? 8 : 16;        // tokens per sub-block: their table loads are in flight together
+            // N is a multiple of 128 on this path (whole heads per tile), so every row is a real feature
+            const int hd = p.hd, half = hd >> 1;
+            const int head = f / hd, hrow = f % hd, i = hrow % half;
+            const int partner = row ^ half;
+            const int qdim = p.Hq * hd, kdim = p.Hkv * hd;
+            const bool rot = p.use_rope && head < p.Hq + p.Hkv;
+            __nv_bfloat16* dst;
+            int ld;
+            if (head < p.Hq) { dst = p.q + f; ld = qdim; }
+            else if (head < p.Hq + p.Hkv) { dst = p.k + (f - qdim); ld = kdim; }
+            else { dst = p.v + (f - qdim - kdim); ld = kdim; }
+            // optional per-head RMSNorm of q and k before the rotation
+            const __nv_bfloat16* gain = (!QKN || !p.gq) ? nullptr : (head < p.Hq ? p.gq : (head < p.Hq + p.Hkv ? p.gk[0] : nullptr));
+            const float g_self = gain ? __bfloat162float(gain[hrow]) : 1.f;
+            const float g_part = gain ? __bfloat162float(gain[hrow ^ half]) : 1.f;
+            constexpr int SB = CH <= 16 ? 8 : 16;        // tokens per sub-block: their table loads are in flight together
 #pragma unroll
-                for (int c0 = 0; c0 < CH; c0 += SB) {
-                    if (c0 >= n_tok) break;
-                    float cs[SB], sn[SB];
+            for (int c0 = 0; c0 < CH; c0 += SB) {
+                if (c0 >= n_tok) break;
+                float cs[SB], sn[SB];
 #pragma unroll
-                    for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
-                    if (p.use_rope) {       // unconditional loads (table row 0 when the token is unused)
-#pragma unroll
-                        for (int c = 0; c < SB; ++c) {
-                            const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
-                            const size_t at = (size_t)max(pos, 0) * half + i;
-                            cs[c] = __ldg(p.cs + at);
-                            sn[c] = __ldg(p.sn + at);
-                        }
-                    }
+                for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
+                if (p.use_rope) {       // unconditional loads (table row 0 when the token is unused)
 #pragma unroll
                     for (int c = 0; c < SB; ++c) {
-                        if (c0 + c < n_tok) {
-                            const bool on = rot && tPos[c0 + c] >= 0;
-                            const float cc = on ? cs[c] : 1.f, ss = on ? sn[c] : 0.f;
-                            const float a = sAcc[row * ACC_LD + c0 + c], b = sAcc[partner * ACC_LD + c0 + c];
-                            const float val = hrow < half ? (a * cc - b * ss) : (a * cc + b * ss);
-                            dst[(size_t)(tok0 + c0 + c) * ld] = __float2bfloat16_rn(val);
-                        }
+                        const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
+                        const size_t at = (size_t)max(pos, 0) * half + i;
+                        cs[c] = __ldg(p.cs + at);
+                        sn[c] = __ldg(p.sn + at);
+                    }
+                }
+                float rn[SB];
+#pragma unroll
+                for (int c = 0; c < SB; ++c) rn[c] = 1.f;
+                if (QKN && p.gq) {      // uniform over the 128 threads
+                    head_rnorm<SB>(p, sAcc, ACC_LD, reinterpret_cast<float*>(sRed), row, c0, n_tok, gain != nullptr, rn);
+                    if (!gain) {
+#pragma unroll
+                        for (int c = 0; c < SB; ++c) rn[c] = 1.f;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < SB; ++c) {
+                    if (c0 + c < n_tok) {
+                        const bool on = rot && tPos[c0 + c] >= 0;
+                        const float cc = on ? cs[c] : 1.f, ss = on ? sn[c] : 0.f;
+                        const float a = sAcc[row * ACC_LD + c0 + c] * (rn[c] * g_self);
+                        const float b = sAcc[partner * ACC_LD + c0 + c] * (rn[c] * g_part);
+                        const float val = hrow < half ? (a * cc - b * ss) : (a * cc + b * ss);
+                        dst[(size_t)(tok0 + c0 + c) * ld] = __float2bfloat16_rn(val);
                     }
                 }
             }
@@ -335,44 +383,57 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
             }
         } break;
         case EPI_CTX_KV: {
-            if (f < p.N) {
-                const int hd = p.hd, half = hd >> 1;
-                const int kdim = p.Hkv * hd;
-                const int is_v = f >= kdim ? 1 : 0;
-                const int fh = f - is_v * kdim;
-                const int head = fh / hd, hrow = fh % hd, i = hrow % half;
-                const int partner = row ^ half;
-                const int layer = p.first_layer + un.g;
-                const bool rot = !is_v && p.use_rope;
-                // pool[layer][page][K|V][head][slot][hd]: tPage[c] = row of (page, K, head 0, slot)
-                __nv_bfloat16* base = p.pool + (((size_t)layer * p.n_pages * 2 + is_v) * p.Hkv + head) * p.PG * hd + hrow;
-                constexpr int SB = CH <= 16 ? 8 : 16;
+            // N = 2 * Hkv * hd is a multiple of 128 on this path
+            const int hd = p.hd, half = hd >> 1;
+            const int kdim = p.Hkv * hd;
+            const int is_v = f >= kdim ? 1 : 0;
+            const int fh = f - is_v * kdim;
+            const int head = fh / hd, hrow = fh % hd, i = hrow % half;
+            const int partner = row ^ half;
+            const int layer = p.first_layer + un.g;
+            const bool rot = !is_v && p.use_rope;
+            const __nv_bfloat16* gk = QKN ? p.gk[un.g] : nullptr;         // per-head norm of the keys, or nullptr
+            const __nv_bfloat16* gain = is_v ? nullptr : gk;
+            const float g_self = gain ? __bfloat162float(gain[hrow]) : 1.f;
+            const float g_part = gain ? __bfloat162float(gain[hrow ^ half]) : 1.f;
+            // pool[layer][page][K|V][head][slot][hd]: tPage[c] = row of (page, K, head 0, slot)
+            __nv_bfloat16* base = p.pool + (((size_t)layer * p.n_pages * 2 + is_v) * p.Hkv + head) * p.PG * hd + hrow;
+            constexpr int SB = CH <= 16 ? 8 : 16;
 #pragma unroll
-                for (int c0 = 0; c0 < CH; c0 += SB) {
-                    if (c0 >= n_tok) break;
-                    float cs[SB], sn[SB];
+            for (int c0 = 0; c0 < CH; c0 += SB) {
+                if (c0 >= n_tok) break;
+                float cs[SB], sn[SB];
 #pragma unroll
-                    for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
-                    if (rot) {
-#pragma unroll
-                        for (int c = 0; c < SB; ++c) {
-                            const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
-                            const size_t at = (size_t)max(pos, 0) * half + i;
-                            cs[c] = __ldg(p.cs + at);
-                            sn[c] = __ldg(p.sn + at);
-                        }
-                    }
+                for (int c = 0; c < SB; ++c) { cs[c] = 1.f; sn[c] = 0.f; }
+                if (rot) {
 #pragma unroll
                     for (int c = 0; c < SB; ++c) {
-                        const int prow = (c0 + c < n_tok) ? tPage[c0 + c] : -1;
-                        if (prow >= 0) {
-                            float val = sAcc[row * ACC_LD + c0 + c];
-                            if (rot) {
-                                const float bb = sAcc[partner * ACC_LD + c0 + c];
-                                val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
-                            }
-                            base[(size_t)prow * hd] = __float2bfloat16_rn(val);
+                        const int pos = (c0 + c < n_tok) ? tPos[c0 + c] : 0;      // entries past n_tok are not initialised
+                        const size_t at = (size_t)max(pos, 0) * half + i;
+                        cs[c] = __ldg(p.cs + at);
+                        sn[c] = __ldg(p.sn + at);
+                    }
+                }
+                float rn[SB];
+#pragma unroll
+                for (int c = 0; c < SB; ++c) rn[c] = 1.f;
+                if (QKN && gk) {        // uniform over the 128 threads
+                    head_rnorm<SB>(p, sAcc, ACC_LD, reinterpret_cast<float*>(sRed), row, c0, n_tok, gain != nullptr, rn);
+                    if (!gain) {
+#pragma unroll
+                        for (int c = 0; c < SB; ++c) rn[c] = 1.f;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < SB; ++c) {
+                    const int prow = (c0 + c < n_tok) ? tPage[c0 + c] : -1;
+                    if (prow >= 0) {
+                        float val = sAcc[row * ACC_LD + c0 + c] * (rn[c] * g_self);
+                        if (rot) {
+                            const float bb = sAcc[partner * ACC_LD + c0 + c] * (rn[c] * g_part);
+                            val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
                         }
+                        base[(size_t)prow * hd] = __float2bfloat16_rn(val);
                     }
                 }
             }
@@ -469,7 +530,7 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     return v;
 }
 
-template <int NT, int SL>
+template <int NT, int SL, bool QKN>
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps tmX, const __grid_constant__ MParams mp) {
     if (threadIdx.x == 0) trace_min(mp.ph[0].trace, 0);
@@ -744,7 +805,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
                         if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
                         epi_bar();
-                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
+                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
                         epi_bar();
                     }
                 }
@@ -784,7 +845,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         float xres[CH], gain;
                         residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
                         epi_bar();
-                        apply_epilogue<CH>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
+                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
                         epi_bar();
                     }
                 }
@@ -974,16 +1035,16 @@ int pick_nt(int M) {
     return 256;
 }
 
-template <int NT, int SL>
+template <int NT, int SL, bool QKN>
 int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
     static bool attr_set = false;
     const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL, QKN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         attr_set = true;
     }
-    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT, SL>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
+    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
@@ -1016,7 +1077,11 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KPa
     p.ssq_in = a.ssq_in; p.n_parts_in = (a.K + 127) / 128; p.inv_dim_in = 1.f / (float)a.K; p.eps = c.rms_eps;
     p.g_next = (const __nv_bfloat16*)a.g_next; p.xn_out = a.xn_out; p.ssq_out = a.ssq_out;
     p.out_f32 = a.out_f32; p.ld_out = a.ld_out;
-    p.q = a.q; p.k = a.k; p.v = a.v; p.ctx_len = a.ctx_len; p.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : 1;
+    p.q = a.q; p.k = a.k; p.v = a.v;
+    p.gq = (const __nv_bfloat16*)a.g_q;
+    p.gk[0] = (const __nv_bfloat16*)a.g_k;
+    if (a.epilogue == EPI_CTX_KV)
+        for (int g = 0; g < groups; ++g) p.gk[g] = (const __nv_bfloat16*)a.g_k_group[g]; p.ctx_len = a.ctx_len; p.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : 1;
     p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.hd = c.head_dim; p.use_rope = c.use_rope;
     p.cs = L.h->w.rope_cos; p.sn = L.h->w.rope_sin; p.max_pos = L.h->w.rope_max_pos;
     p.h = a.h; p.F = c.d_ffn;
@@ -1071,13 +1136,21 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     for (int i = n_phases; i < MAX_PHASES; ++i) tx.m[i] = tx.m[0];
     // one CTA per SM unless the smallest phase would leave ranges under 256 K-elements
     const int grid = (int)std::max<long long>(1, std::min<long long>(L.h->sm_count, min_pairs * slabs / 4));
-    switch (nt) {
-        case 16: return slabs == 2 ? launch_nt<16, 2>(L, tw, tx, mp, grid) : launch_nt<16, 1>(L, tw, tx, mp, grid);
-        case 32: return slabs == 2 ? launch_nt<32, 2>(L, tw, tx, mp, grid) : launch_nt<32, 1>(L, tw, tx, mp, grid);
-        case 64: return launch_nt<64, 1>(L, tw, tx, mp, grid);
-        case 128: return launch_nt<128, 1>(L, tw, tx, mp, grid);
-        default: return launch_nt<256, 1>(L, tw, tx, mp, grid);
+    bool qkn = false;
+    for (int i = 0; i < n_phases; ++i) {
+        qkn = qkn || mp.ph[i].gq != nullptr;
+        for (int g = 0; g < mp.ph[i].n_groups; ++g) qkn = qkn || mp.ph[i].gk[g] != nullptr;
     }
+#define DFLASH_GEMM_CASE(NT_, SL_) \
+    (qkn ? launch_nt<NT_, SL_, true>(L, tw, tx, mp, grid) : launch_nt<NT_, SL_, false>(L, tw, tx, mp, grid))
+    switch (nt) {
+        case 16: return slabs == 2 ? DFLASH_GEMM_CASE(16, 2) : DFLASH_GEMM_CASE(16, 1);
+        case 32: return slabs == 2 ? DFLASH_GEMM_CASE(32, 2) : DFLASH_GEMM_CASE(32, 1);
+        case 64: return DFLASH_GEMM_CASE(64, 1);
+        case 128: return DFLASH_GEMM_CASE(128, 1);
+        default: return DFLASH_GEMM_CASE(256, 1);
+    }
+#undef DFLASH_GEMM_CASE
 }
 
 int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done) {

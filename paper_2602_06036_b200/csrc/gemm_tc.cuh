@@ -50,7 +50,8 @@ struct GemmArgs {
     // EPI_STORE_F32 / EPI_RESIDUAL
     float* out_f32;        // may be nullptr for EPI_STORE_F32 with norm_out
     int ld_out;
-    // EPI_QKV_ROPE
+    // EPI_QKV_ROPE (g_q / g_k: gains of the per-head norm of q and k, or nullptr)
+    const void *g_q, *g_k;
     __nv_bfloat16 *q, *k, *v;
     const int32_t* ctx_len;
     int rows_per_seq;
@@ -59,9 +60,10 @@ struct GemmArgs {
     // EPI_ARGMAX
     Top2Entry* top2;    // [n_feature_tiles, M]
     float* logits_out;  // optional [M, N]
-    // EPI_CTX_KV (group g writes pool layer first_layer + g)
+    // EPI_CTX_KV (group g writes pool layer first_layer + g; g_k_group[g]: that layer's k-head norm gain or nullptr)
     const dflash_ctx_args* ctx;
     int first_layer;
+    const void* g_k_group[GEMM_MAX_GROUPS];
 };
 
 // Scratch the launcher needs: partial accumulators of tiles shared by several CTAs, and their tickets.

@@ -208,7 +208,8 @@ __global__ void rope_split_kernel(const float* __restrict__ qkv, const int32_t* 
                                   int rows_per_seq, T* __restrict__ q, T* __restrict__ k,
                                   T* __restrict__ v, int Hq, int Hkv, int hd, int use_rope,
                                   const float* __restrict__ cs, const float* __restrict__ sn, int max_pos,
-                                  int32_t* status) {
+                                  int32_t* status, const T* __restrict__ gq, const T* __restrict__ gk, float eps) {
+    __shared__ float rnorm[128];          // per (q or k) head: rsqrt(mean square + eps), 1 without the head norm
     const int row = blockIdx.x, b = row / rows_per_seq, r = row % rows_per_seq;
     const int half = hd / 2;
     int pos = ctx_len[b] + r;
@@ -218,10 +219,24 @@ __global__ void rope_split_kernel(const float* __restrict__ qkv, const int32_t* 
     }
     const int qdim = Hq * hd, kdim = Hkv * hd;
     const float* src = qkv + (size_t)row * (qdim + 2 * kdim);
+    for (int head = threadIdx.x >> 5; head < Hq + Hkv; head += blockDim.x >> 5) {     // one warp per head
+        float s = 0.f;
+        if (gq)
+            for (int i = threadIdx.x & 31; i < hd; i += 32) s += src[head * hd + i] * src[head * hd + i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((threadIdx.x & 31) == 0 && head < 128) rnorm[head] = gq ? rsqrtf(s / (float)hd + eps) : 1.f;
+    }
+    __syncthreads();
     // rotated part: q heads then k heads
     for (int e = threadIdx.x; e < (Hq + Hkv) * half; e += blockDim.x) {
         const int head = e / half, i = e % half;
-        const float a = src[head * hd + i], bb = src[head * hd + i + half];
+        float a = src[head * hd + i], bb = src[head * hd + i + half];
+        if (gq) {
+            const T* g = head < Hq ? gq : gk;
+            a *= rnorm[head] * to_f(g[i]);
+            bb *= rnorm[head] * to_f(g[i + half]);
+        }
         float c = 1.f, s = 0.f;
         if (use_rope) { c = cs[(size_t)pos * half + i]; s = sn[(size_t)pos * half + i]; }
         const float o1 = a * c - bb * s, o2 = bb * c + a * s;
@@ -239,19 +254,21 @@ __global__ void rope_split_kernel(const float* __restrict__ qkv, const int32_t* 
 }
 
 int launch_rope_split(const Launch& L, const float* qkv, const int32_t* ctx_len, int rows_per_seq, int rows,
-                      void* q, void* k, void* v) {
+                      void* q, void* k, void* v, const void* g_q, const void* g_k) {
     const dflash_config& c = L.h->cfg;
     if (rows == 0) return DFLASH_OK;
+    if (g_q && c.n_q_heads + c.n_kv_heads > 128) return DFLASH_ERR_UNSUPPORTED;
     if (c.dtype == DFLASH_F32)
         rope_split_kernel<float><<<rows, 256, 0, L.st>>>(qkv, ctx_len, rows_per_seq, (float*)q, (float*)k,
                                                          (float*)v, c.n_q_heads, c.n_kv_heads, c.head_dim,
                                                          c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin,
-                                                         L.h->w.rope_max_pos, L.status);
+                                                         L.h->w.rope_max_pos, L.status, (const float*)g_q, (const float*)g_k,
+                                                         c.rms_eps);
     else
         rope_split_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>(
             qkv, ctx_len, rows_per_seq, (__nv_bfloat16*)q, (__nv_bfloat16*)k, (__nv_bfloat16*)v, c.n_q_heads,
             c.n_kv_heads, c.head_dim, c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin, L.h->w.rope_max_pos,
-            L.status);
+            L.status, (const __nv_bfloat16*)g_q, (const __nv_bfloat16*)g_k, c.rms_eps);
     DFLASH_CHECK_LAUNCH();
     return DFLASH_OK;
 }
@@ -392,7 +409,9 @@ __global__ void ctx_scatter_kernel(const float* __restrict__ kv, const int32_t* 
                                    const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ page_table,
                                    T* __restrict__ pool, int max_new, int Hkv, int hd, int PG, int max_pages,
                                    int n_pages, int layer, int use_rope, const float* __restrict__ cs,
-                                   const float* __restrict__ sn, int max_pos, int32_t* status) {
+                                   const float* __restrict__ sn, int max_pos, int32_t* status,
+                                   const T* __restrict__ gk, float eps) {
+    __shared__ float rnorm[128];
     const int row = blockIdx.x, b = row / max_new, r = row % max_new;
     const int nn = n_new ? n_new[b] : max_new;
     if (r >= nn) return;
@@ -411,9 +430,22 @@ __global__ void ctx_scatter_kernel(const float* __restrict__ kv, const int32_t* 
     const float* src = kv + (size_t)row * 2 * kdim;
     T* kdst = pool + ((((size_t)layer * n_pages + page) * 2) * Hkv) * PG * hd + (size_t)(pos % PG) * hd;
     T* vdst = kdst + (size_t)Hkv * PG * hd;
+    for (int head = threadIdx.x >> 5; head < Hkv; head += blockDim.x >> 5) {          // one warp per key head
+        float s = 0.f;
+        if (gk)
+            for (int i = threadIdx.x & 31; i < hd; i += 32) s += src[head * hd + i] * src[head * hd + i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((threadIdx.x & 31) == 0 && head < 128) rnorm[head] = gk ? rsqrtf(s / (float)hd + eps) : 1.f;
+    }
+    __syncthreads();
     for (int e = threadIdx.x; e < Hkv * half; e += blockDim.x) {
         const int head = e / half, i = e % half;
-        const float a = src[head * hd + i], bb = src[head * hd + i + half];
+        float a = src[head * hd + i], bb = src[head * hd + i + half];
+        if (gk) {
+            a *= rnorm[head] * to_f(gk[i]);
+            bb *= rnorm[head] * to_f(gk[i + half]);
+        }
         float c = 1.f, s = 0.f;
         if (use_rope) { c = cs[(size_t)pos * half + i]; s = sn[(size_t)pos * half + i]; }
         kdst[(size_t)head * PG * hd + i] = from_f<T>(a * c - bb * s);
@@ -425,7 +457,7 @@ __global__ void ctx_scatter_kernel(const float* __restrict__ kv, const int32_t* 
     }
 }
 
-int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer) {
+int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& a, int layer, const void* g_k) {
     const dflash_config& c = L.h->cfg;
     const int rows = a.batch * a.max_new;
     if (rows == 0) return DFLASH_OK;
@@ -433,12 +465,12 @@ int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& 
         ctx_scatter_kernel<float><<<rows, 128, 0, L.st>>>(
             kv, a.n_new, a.ctx_len, a.page_table, (float*)a.kv_pool, a.max_new, c.n_kv_heads, c.head_dim,
             c.page_size, a.max_pages, a.n_pool_pages, layer, c.use_rope, L.h->w.rope_cos, L.h->w.rope_sin,
-            L.h->w.rope_max_pos, L.status);
+            L.h->w.rope_max_pos, L.status, (const float*)g_k, c.rms_eps);
     else
         ctx_scatter_kernel<__nv_bfloat16><<<rows, 128, 0, L.st>>>(
             kv, a.n_new, a.ctx_len, a.page_table, (__nv_bfloat16*)a.kv_pool, a.max_new, c.n_kv_heads,
             c.head_dim, c.page_size, a.max_pages, a.n_pool_pages, layer, c.use_rope, L.h->w.rope_cos,
-            L.h->w.rope_sin, L.h->w.rope_max_pos, L.status);
+            L.h->w.rope_sin, L.h->w.rope_max_pos, L.status, (const __nv_bfloat16*)g_k, c.rms_eps);
     DFLASH_CHECK_LAUNCH();
     return DFLASH_OK;
 }

@@ -64,7 +64,7 @@ def _cfg(**over):
     vals = dict(n_layers=c.n_layers, d_model=c.d_model, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
                 head_dim=c.head_dim, d_ffn=c.d_ffn, vocab=c.vocab, n_feat_layers=c.n_feat_layers,
                 d_target=c.d_target, block_size=c.block_size, page_size=64, dtype=0, mask_token_id=c.vocab - 1,
-                use_rope=1, rms_eps=1e-6, softmax_scale=0.125)
+                use_rope=1, rms_eps=1e-6, softmax_scale=0.125, qk_norm=0)
     vals.update(over)
     return binding.Config(**vals)
 

@@ -94,6 +94,25 @@ def test_block_size_chosen_per_call(name):
         case.lib.dflash_draft_block(anchors.to(dev), case.ctx_len, 0, case.page_table, case.pool, ids, block_rows=full + 1)
 
 
+@pytest.mark.parametrize("base,over", [("tiny", {}), ("mid", {}), ("mid", dict(head_dim=64, n_q_heads=8, n_kv_heads=2)),
+                                       ("mid", dict(block_size=10, n_layers=3))])
+def test_per_head_qk_norm(base, over):
+    # the optional attention variant: q and k heads RMS-normalised (own gains) before the rotation, for
+    # block rows and for the injected context keys; CUDA-core path (tiny), tensor-core path with one head
+    # per 128-row weight tile (hd = 128) and with two (hd = 64)
+    cfg = dataclasses.replace(synth.TINY if base == "tiny" else synth.MID, qk_norm=1, **over)
+    case = Case(cfg, (0, 70, 131) if base == "mid" else (65,), seed=23)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    n_sure = case.check_draft(got)
+    assert n_sure >= case.S * cfg.block_size // 2
+    # and it is not a no-op: the same inputs without the norm give other logits
+    off = Case(dataclasses.replace(cfg, qk_norm=0), case.ctx_lens, seed=23)
+    off.project_prefill()
+    assert np.abs(off.run_draft()["logits"] - got["logits"]).max() > 0.05
+
+
 def test_bf16_feature_dims_that_are_not_multiples_of_64():
     # contraction lengths of 520 / 1544 / 1560 (multiples of 8 only): the one-slab ring stages with a
     # zero-filled K tail, ragged 128-feature tiles in the folded norms, a ragged last weight tile
