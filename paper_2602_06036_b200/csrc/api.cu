@@ -37,7 +37,9 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     int64_t part = 0, counters = 0;
     if (tc) {
         const int M = (int)R, sm = h->sm_count;
-        const int kv_groups = std::min(c.n_layers, GEMM_MAX_GROUPS - 1);
+        // context K/V: one ticket range per layer (launches of up to GEMM_MAX_GROUPS - 1 layers each take their own
+        // slice: their tile decompositions differ, so they cannot share tickets through the epoch count)
+        const int kv_groups = c.n_layers;
         // order = Workspace::CNT_* : every contraction shape has its own ticket range
         const int shapes[Workspace::CNT_N][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
                                                  {c.d_model, c.d_ffn, 1},         {c.vocab, c.d_model, 1}, {c.d_model, feat, 1},
@@ -328,7 +330,7 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
             }
             k.X = ws.u; k.M = rows; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = ws.ssq;
             k.epilogue = EPI_CTX_KV; k.ctx = a; k.first_layer = i0; k.part = ws.part;
-            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV]; k.epoch = i0 / (GEMM_MAX_GROUPS - 1) + 1;
+            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV] + (int64_t)i0 * (gemm_tc_counter_bytes(rows, 2 * kdim, 1) / 4);
             if (flag_set >= ws.n_flag_sets - 1) return DFLASH_ERR_UNSUPPORTED;
             if (!fused_done) {
                 // one launch: the fusion contraction, then the K/V contractions of the first layers as its second phase

@@ -50,7 +50,8 @@ def test_tiny_without_rope_and_paper_block_sizes():
         case.check_draft(got)
 
 
-@pytest.mark.parametrize("B,k,layers,lens", [(8, 3, 2, (33, 150)), (10, 5, 3, (0, 64, 129)), (16, 5, 1, (257,))])
+@pytest.mark.parametrize("B,k,layers,lens", [(8, 3, 2, (33, 150)), (10, 5, 3, (0, 64, 129)), (16, 5, 1, (257,)),
+                                             (16, 3, 8, (40, 100))])     # 8 layers: the context K/V of layer 8 takes a second launch
 def test_bf16_block_sizes_and_feature_counts(B, k, layers, lens):
     # tensor-core path at the block sizes the paper runs (8, 10, 16: Sec. 5.3 and the LLaMA setting),
     # with k = 5 tapped layers (App. A.1) and other layer counts; contexts end inside, at and past a page edge
