@@ -38,16 +38,23 @@ Workspace carve(const dflash_handle* h, void* base, int batch, int rows) {
     if (tc) {
         const int M = (int)R, sm = h->sm_count;
         // context K/V: one ticket range per layer (launches of up to GEMM_MAX_GROUPS - 1 layers each take their own
-        // slice: their tile decompositions differ, so they cannot share tickets through the epoch count)
+        // slice)
         const int kv_groups = c.n_layers;
         // order = Workspace::CNT_* : every contraction shape has its own ticket range
         const int shapes[Workspace::CNT_N][3] = {{qdim + 2 * kdim, c.d_model, 1}, {c.d_model, qdim, 1}, {2 * c.d_ffn, c.d_model, 1},
                                                  {c.d_model, c.d_ffn, 1},         {c.vocab, c.d_model, 1}, {c.d_model, feat, 1},
                                                  {2 * kdim, c.d_model, kv_groups}};
+        // Every launch that uses a shape within one call takes its own slice of tickets (one per layer for
+        // the four per-layer contractions): tickets are zeroed once per call and never shared between
+        // launches, whose tile splits may differ (a chained launch and a single one size their grids apart).
         for (int i = 0; i < Workspace::CNT_N; ++i) {
             part = std::max(part, gemm_tc_part_bytes(M, shapes[i][0], shapes[i][1], shapes[i][2], sm));
+            const bool per_layer = i == Workspace::CNT_QKV || i == Workspace::CNT_O || i == Workspace::CNT_GATEUP ||
+                                   i == Workspace::CNT_DOWN;
+            const int64_t one = align_up(gemm_tc_counter_bytes(M, shapes[i][0], shapes[i][2]), 256);
             w.cnt_off[i] = (int)(counters / 4);
-            counters += align_up(gemm_tc_counter_bytes(M, shapes[i][0], shapes[i][2]), 256);
+            w.cnt_stride[i] = (int)(one / 4);
+            counters += one * (per_layer ? c.n_layers : 1);
         }
     }
     w.part = (float*)a.take(std::max<int64_t>(part, 256));
@@ -397,7 +404,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             g.epilogue = EPI_QKV_ROPE; g.q = (__nv_bfloat16*)ws.q; g.k = (__nv_bfloat16*)ws.k_blk;
             g.v = (__nv_bfloat16*)ws.v_blk; g.ctx_len = a->ctx_len; g.rows_per_seq = B;
             if (c.qk_norm) { g.g_q = h->layers[i].g_q; g.g_k = h->layers[i].g_k; }
-            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV]; g.epoch = i + 1;
+            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV] + i * ws.cnt_stride[Workspace::CNT_QKV];
             return g;
         };
         RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, B, ws.x, h->layers[0].g1, xn, ws.ssq));
@@ -417,21 +424,21 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             o = GemmArgs{};
             o.X = ws.attn; o.W[0] = lw.W_o; o.M = rows; o.N = c.d_model; o.K = qdim;
             o.epilogue = EPI_RESIDUAL; o.out_f32 = ws.x; o.ld_out = c.d_model; o.part = ws.part;
-            o.counters = ws.counters + ws.cnt_off[Workspace::CNT_O];
-            o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq; o.epoch = i + 1;
+            o.counters = ws.counters + ws.cnt_off[Workspace::CNT_O] + i * ws.cnt_stride[Workspace::CNT_O];
+            o.g_next = lw.g2; o.xn_out = xn; o.ssq_out = ws.ssq;
             fam[0] = FAM_GEMM_O;
             GemmArgs& u = ph[1];      // h = silu(W_gate u) * (W_up u)
             u = GemmArgs{};
             u.X = xn; u.W[0] = lw.W_gateup; u.M = rows; u.N = 2 * c.d_ffn; u.K = c.d_model; u.ssq_in = ws.ssq;
             u.epilogue = EPI_SWIGLU; u.h = (__nv_bfloat16*)ws.h; u.part = ws.part;
-            u.counters = ws.counters + ws.cnt_off[Workspace::CNT_GATEUP]; u.epoch = i + 1;
+            u.counters = ws.counters + ws.cnt_off[Workspace::CNT_GATEUP] + i * ws.cnt_stride[Workspace::CNT_GATEUP];
             fam[1] = FAM_GEMM_GATEUP;
             GemmArgs& d = ph[2];      // x += W_down h; emits the next layer's (or the final) norm inputs
             d = GemmArgs{};
             d.X = ws.h; d.W[0] = lw.W_down; d.M = rows; d.N = c.d_model; d.K = c.d_ffn;
             d.epilogue = EPI_RESIDUAL; d.out_f32 = ws.x; d.ld_out = c.d_model; d.part = ws.part;
-            d.counters = ws.counters + ws.cnt_off[Workspace::CNT_DOWN];
-            d.g_next = last ? h->w.g_f : h->layers[i + 1].g1; d.xn_out = xn; d.ssq_out = ws.ssq; d.epoch = i + 1;
+            d.counters = ws.counters + ws.cnt_off[Workspace::CNT_DOWN] + i * ws.cnt_stride[Workspace::CNT_DOWN];
+            d.g_next = last ? h->w.g_f : h->layers[i + 1].g1; d.xn_out = xn; d.ssq_out = ws.ssq;
             fam[2] = FAM_GEMM_DOWN;
             if (!last) {
                 ph[3] = qkv_args(i + 1);

@@ -72,6 +72,7 @@ struct Workspace {
     enum { CNT_QKV = 0, CNT_O, CNT_GATEUP, CNT_DOWN, CNT_LM, CNT_FUSE, CNT_KV, CNT_N };
     int32_t* counters;   // tickets of shared output tiles (zeroed at the start of each call)
     int cnt_off[CNT_N];  // first ticket of each contraction shape (int32 units)
+    int cnt_stride[CNT_N];   // tickets per use of that shape within one call (QKV / O / gate-up / down: one slice per layer)
     int32_t* flags;      // [n_flag_sets][4] phase-completion counters of chained launches
     int n_flag_sets;
     int64_t counter_bytes;

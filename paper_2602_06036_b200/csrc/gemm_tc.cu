@@ -68,7 +68,6 @@ struct WMaps {
 
 struct KParams {
     int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, w_map0, x_map;
-    int epoch;                   // how many launches since the tickets were zeroed use this ticket range (>= 1)
     float* part;
     int32_t* counters;
     const float* ssq_in;
@@ -762,7 +761,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres, gain);
                     if (row == 0) {
                         const long long t0 = clock64();
-                        while (ld_acquire(p.counters + un.tile) < n_contrib * p.epoch) {
+                        while (ld_acquire(p.counters + un.tile) < n_contrib) {
                             if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
                         }
                     }
@@ -1093,7 +1092,6 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KPa
     }
     p.PG = c.page_size; p.first_layer = a.first_layer;
     p.status = L.status;
-    p.epoch = a.epoch > 0 ? a.epoch : 1;
     return DFLASH_OK;
 }
 

@@ -40,7 +40,7 @@ struct GemmArgs {
     // split-K scratch (needed when the chooser returns more than one split)
     float* part;
     int32_t* counters;
-    int epoch;             // 1 for the first launch that uses this ticket range after it was zeroed, 2 for the next, ...
+                           // tickets: zero on entry, one slice per launch (the kernel leaves them non-zero)
     // norm_in
     const float* ssq_in;   // [ceil(K/128), M] or nullptr
     // norm_out (EPI_STORE_F32 / EPI_RESIDUAL)
