@@ -114,6 +114,26 @@ def test_per_head_qk_norm(base, over):
     assert np.abs(off.run_draft()["logits"] - got["logits"]).max() > 0.05
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_bf16_random_shapes(seed):
+    # seeded draws of widths, head counts, layer counts, block sizes and batch sizes: every token-tile size of
+    # the contraction kernel (16 ... 256 rows), shared and whole-tile schedules, chained and single launches
+    rng = np.random.default_rng(1000 + seed)
+    hq, hkv = [(2, 1), (4, 2), (8, 2), (8, 8), (4, 4)][rng.integers(5)]
+    cfg = dataclasses.replace(
+        synth.MID, d_model=int(rng.choice([256, 384, 512, 640, 1024])), d_ffn=int(rng.choice([512, 1024, 1536, 2048])),
+        n_q_heads=hq, n_kv_heads=hkv, vocab=int(rng.choice([1000, 3001, 8192, 20011])), n_layers=int(rng.integers(1, 5)),
+        block_size=int(rng.choice([4, 8, 10, 16])), n_feat_layers=int(rng.choice([1, 3, 5])), d_target=int(rng.choice([256, 512])),
+        qk_norm=int(rng.integers(2)))
+    S = int(rng.choice([1, 2, 3, 5, 9, 16]))
+    lens = tuple(int(x) for x in rng.integers(0, 260, size=S))
+    case = Case(cfg, lens, seed=seed)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    case.check_draft(got)
+
+
 def test_bf16_feature_dims_that_are_not_multiples_of_64():
     # contraction lengths of 520 / 1544 / 1560 (multiples of 8 only): the one-slab ring stages with a
     # zero-filled K tail, ragged 128-feature tiles in the folded norms, a ragged last weight tile
