@@ -333,7 +333,33 @@ def run_kernel_only(args, step, device):
     from paper_2602_06036_b200 import binding
     cfg, wl = step.cfg, step.wl
     S, B = wl.batch, cfg.block_size
-    if args.kernel == "lmhead":
+    if args.kernel == "target_verify":
+        # The target's verify pass over gamma + 1 rows with a target-sized stack (36 layers of the same
+        # shape; the weight tensors of the drafter's layers are reused round-robin: 1.9 GB of distinct
+        # weights per cycle of 5 layers, far beyond L2, so every layer streams from HBM).
+        import dataclasses
+        n_layers, rows = 36, B + 1
+        tcfg = dataclasses.replace(cfg, n_layers=n_layers)
+        tlib = binding.DFlash(tcfg, str(device))
+        w = synth.pack_device_weights(cfg, synth.make_weights(cfg, 1))
+        w["layers"] = [{k: v.to(device) for k, v in lw.items()} for lw in w["layers"]]
+        w["layers"] = [w["layers"][i % cfg.n_layers] for i in range(n_layers)]
+        cos, sin = synth.rope_tables(tcfg, max(wl.ctx_lens) + 4 * B + 8)
+        tlib.set_weights(w, cos, sin)
+        table, n_pages = synth.make_page_table(tcfg, [L + 2 * B + 2 for L in wl.ctx_lens], 1)
+        table = table.to(device)
+        pool = torch.randn(synth.kv_pool_shape(tcfg, n_pages), device=device).to(tcfg.torch_dtype)
+        tokens = torch.randint(0, cfg.vocab - 1, (S, rows), dtype=torch.int32, device=device)
+        taps = [1, 9, 17, 25, 33]
+        ids = torch.zeros((S, rows), dtype=torch.int32, device=device)
+        feats = torch.zeros((S, rows, len(taps) * cfg.d_model), dtype=cfg.torch_dtype, device=device)
+        logits = torch.zeros((S * rows, cfg.vocab), dtype=torch.float32, device=device)
+        fn = lambda: tlib.dflash_target_verify(tokens, step.ctx_len, step.max_ctx, table, pool, taps, ids, feats_out=feats,
+                                               logits_out=logits)
+        alg = algorithmic_bytes(cfg, wl.ctx_lens, 0)
+        nbytes = n_layers * (alg["gemm_qkv"] + alg["gemm_o"] + alg["gemm_gateup"] + alg["gemm_down"] + alg["attention"]) + \
+            alg["lmhead_argmax"]
+    elif args.kernel == "lmhead":
         hid = torch.randn(S * B, cfg.d_model, device=device).to(cfg.torch_dtype)
         ids = torch.zeros(S * B, dtype=torch.int32, device=device)
         fn = lambda: step.lib.dflash_lmhead_argmax(hid, 1, ids)
@@ -361,7 +387,7 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention"],
+    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify"],
                     help="run one building block alone (for profiler captures) instead of the step")
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
     ap.add_argument("--temperature", type=float, default=0.0,

@@ -168,6 +168,37 @@ typedef struct {
 } dflash_draft_args;
 int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a /*[host]*/, void* stream);
 
+/* ---- the target's verify pass over the same kernels (Sec. 3.1: the target scores all gamma drafts in
+ * one parallel pass; Sec. 4.1: hidden states of k of its layers are the drafter's context features) ----
+ * A handle created with the TARGET's shape runs its stack over `rows` given tokens per sequence
+ * (anchor, d_1 .. d_gamma) on top of the target's own paged KV cache (same pool layout): causal
+ * inside the block, full over the cached context. Outputs: logits and their row argmax (the p_j of
+ * the accept rule), the hidden rows after the layers listed in tap_layers laid out as
+ * [batch, rows, n_taps * D] = the operand of dflash_ctx_project (no concatenation pass), and the
+ * block's K/V of every layer written into the cache at positions ctx_len .. ctx_len + rows - 1:
+ * after the accept step the caller only raises ctx_len by tau (rows past it stay invisible and are
+ * overwritten by the next cycle). The handle's W_c / g_c / mask token are not used.
+ * rows <= 32 and rows * (Hq / Hkv) <= 128 on the bf16 path; tap_layers ascending. */
+typedef struct {
+    const int32_t* token_ids;    /* [device] [batch, rows]                                     */
+    int32_t        batch, rows;
+    const int32_t* ctx_len;      /* [device] [batch] committed length of every sequence        */
+    int32_t        max_ctx_len;  /* [host value] upper bound of ctx_len                        */
+    const int32_t* page_table;   /* [device] [batch, max_pages]; must cover ctx_len + rows     */
+    int32_t        max_pages;
+    void*          kv_pool;      /* [device] the target's pool; read, and written at the block's positions */
+    int32_t        n_pool_pages;
+    const int32_t* tap_layers;   /* [host] n_taps layer indices (0-based, ascending); may be NULL if n_taps = 0 */
+    int32_t        n_taps;
+    void*          feats_out;    /* [device] out [batch, rows, n_taps * D] config dtype; may be NULL if n_taps = 0 */
+    float*         logits_out;   /* [device] out [batch * rows, V] fp32; may be NULL           */
+    int32_t*       ids_out;      /* [device] out [batch, rows] argmax of every row             */
+    void*          workspace;    /* [device] >= dflash_workspace_bytes(h, batch, batch * rows)  */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;   /* [device] may be NULL                                       */
+} dflash_target_args;
+int32_t dflash_target_verify(dflash_handle* h, const dflash_target_args* a /*[host]*/, void* stream);
+
 /* ---- greedy verify / accept (Sec. 3.1: tau in [1, gamma+1] incl. the bonus token) ----
  * p_j = argmax_v logits[b, j, :] (mode LOGITS) or target_ids[b, j] (mode IDS), j = 0..gamma.
  * a = length of the longest prefix with draft[b, i] == p_i, i < a;  tau = a + 1;

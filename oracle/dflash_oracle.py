@@ -30,6 +30,11 @@ and equality of speculative output with plain greedy decoding of a toy target.
 The composed forward `draft_block` has no external value to compare with: parity unpinned beyond
 its parts (each step above is pinned separately).
 
+The target's side of a cycle (Sec. 3.1: one parallel pass scores all drafts; Sec. 4.1: hidden states of
+k target layers become the context features): a causal stack over [anchor, d_1 .. d_gamma] on top of
+its cached K/V, returning logits, tapped rows and the block's cache entries       -> target_verify
+(pinned by equality with the plain full-sequence causal forward, continued from its own cache).
+
 Sampling (temperature > 0) verification, the setting of the paper's T = 1 results (Sec. 5.1, Table 2):
 the paper relies on standard speculative sampling (Sec. 2 related work) without restating it, so
 the rule is written out here                                     -> softmax_t, sample_cdf, verify_accept_sample
@@ -204,8 +209,9 @@ def block_attention(q, k_ctx, v_ctx, k_blk, v_blk, scale, causal=False):
 # --------------------------------------------------------------------------------------------
 # draft forward
 # --------------------------------------------------------------------------------------------
-def draft_layer(x, lw, k_ctx, v_ctx, pos, cfg, causal=False):
-    """One pre-norm layer on the block hidden states x [R, D] (H_d = the normalised hidden)."""
+def draft_layer(x, lw, k_ctx, v_ctx, pos, cfg, causal=False, return_kv=False):
+    """One pre-norm layer on the block hidden states x [R, D] (H_d = the normalised hidden).
+    return_kv: also return the block's own (position-encoded) k and v [R, Hkv, hd]."""
     R = x.shape[0]
     u = rmsnorm(x, lw["g1"], cfg.rms_eps)
     q = linear(u, lw["W_q"]).reshape(R, cfg.n_q_heads, cfg.head_dim)
@@ -221,7 +227,8 @@ def draft_layer(x, lw, k_ctx, v_ctx, pos, cfg, causal=False):
     x = x + linear(a.reshape(R, cfg.q_dim), lw["W_o"])
     u2 = rmsnorm(x, lw["g2"], cfg.rms_eps)
     h = silu(linear(u2, lw["W_gate"])) * linear(u2, lw["W_up"])
-    return x + linear(h, lw["W_down"])
+    out = x + linear(h, lw["W_down"])
+    return (out, k, v) if return_kv else out
 
 
 def lm_head(x, g_f, W_lm, eps):
@@ -337,6 +344,31 @@ def verify_accept_sample(draft_ids, draft_logits, target_logits, T, u_accept, u_
     out[:a] = np.asarray(draft_ids[:a], dtype=np.int64)
     out[a] = tok
     return a + 1, out, tok, int(ctx_len) + a + 1, dict(accept_margin=margins, final_margin=fm, a=a, residual=residual)
+
+
+# --------------------------------------------------------------------------------------------
+# the target's verify pass (Sec. 3.1: all drafts scored in one parallel pass; Sec. 4.1: hidden states
+# of k target layers are the drafter's context features)
+# --------------------------------------------------------------------------------------------
+def target_verify(tokens, L, ctx_K, ctx_V, weights, cfg, tap_layers):
+    """A causal stack over the rows `tokens` (anchor, d_1 .. d_gamma) at positions L .. L+R-1, on top of
+    the cached context ctx_K / ctx_V ([N][L, Hkv, hd], position-encoded): causal inside the block,
+    full over the context. Returns dict(logits [R, V], ids, feats [R, len(tap_layers) * D] = hidden rows
+    after the tapped layers side by side, K / V [N][R, Hkv, hd] = the block's entries for the cache)."""
+    R = len(tokens)
+    x = _f64(weights["embed"][np.asarray(tokens, dtype=np.int64)])
+    pos = L + np.arange(R)
+    taps, Ks, Vs = [], [], []
+    for i, lw in enumerate(weights["layers"]):
+        x, k, v = draft_layer(x, lw, ctx_K[i], ctx_V[i], pos, cfg, causal=True, return_kv=True)
+        Ks.append(k)
+        Vs.append(v)
+        if i in tap_layers:
+            taps.append(x)
+    logits = lm_head(x, weights["g_f"], weights["W_lm"], cfg.rms_eps)
+    ids, top1, margin = argmax_top2(logits)
+    feats = np.concatenate(taps, axis=-1) if taps else np.zeros((R, 0))
+    return dict(logits=logits, ids=ids, margin=margin, feats=feats, K=Ks, V=Vs)
 
 
 # --------------------------------------------------------------------------------------------

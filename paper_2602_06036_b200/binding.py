@@ -28,7 +28,7 @@ EXPORTS = (
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
     "dflash_verify_accept_static", "dflash_sample_rows", "dflash_verify_accept_sample",
-    "dflash_sample_workspace_bytes",
+    "dflash_sample_workspace_bytes", "dflash_target_verify",
 )
 N_FAMILIES = 15
 
@@ -73,6 +73,15 @@ class VerifyArgs(C.Structure):
                 ("ctx_len", C.c_void_p), ("accept_len", C.c_void_p), ("out_tokens", C.c_void_p),
                 ("bonus", C.c_void_p), ("new_ctx_len", C.c_void_p), ("target_ids_out", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p)]
+
+
+class TargetArgs(C.Structure):
+    _fields_ = [("token_ids", C.c_void_p), ("batch", C.c_int32), ("rows", C.c_int32), ("ctx_len", C.c_void_p),
+                ("max_ctx_len", C.c_int32), ("page_table", C.c_void_p), ("max_pages", C.c_int32),
+                ("kv_pool", C.c_void_p), ("n_pool_pages", C.c_int32), ("tap_layers", C.POINTER(C.c_int32)),
+                ("n_taps", C.c_int32), ("feats_out", C.c_void_p), ("logits_out", C.c_void_p),
+                ("ids_out", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64),
+                ("dev_status", C.c_void_p)]
 
 
 class SampleArgs(C.Structure):
@@ -127,7 +136,7 @@ def load():
     for name, st in (("dflash_ctx_project", CtxArgs), ("dflash_draft_block", DraftArgs),
                      ("dflash_verify_accept", VerifyArgs), ("dflash_verify_accept_static", VerifyArgs), ("dflash_block_attention", AttnArgs),
                      ("dflash_lmhead_argmax", LmHeadArgs), ("dflash_sample_rows", SampleArgs),
-                     ("dflash_verify_accept_sample", VerifySampleArgs)):
+                     ("dflash_verify_accept_sample", VerifySampleArgs), ("dflash_target_verify", TargetArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(st), C.c_void_p]
         fn.restype = C.c_int32
@@ -330,6 +339,18 @@ class DFlash:
                        logits.shape[-1], _ptr(ctx_len), _ptr(accept_len), _ptr(out_tokens), _ptr(bonus),
                        _ptr(new_ctx_len), _ptr(target_ids_out), None, 0, _ptr(self.status))
         _check(self.lib.dflash_verify_accept_static(self.h, C.byref(a), _stream(stream)))
+
+    def dflash_target_verify(self, token_ids, ctx_len, max_ctx_len, page_table, kv_pool, tap_layers, ids_out,
+                             feats_out=None, logits_out=None, stream=None):
+        """The target's verify pass: token_ids [S, rows]; writes the block's K/V into kv_pool at positions
+        ctx_len .. ctx_len + rows - 1, the tapped hidden rows into feats_out [S, rows, len(tap_layers) * D]."""
+        S, rows = token_ids.shape
+        ws = self.workspace(S, S * rows)
+        taps = (C.c_int32 * max(len(tap_layers), 1))(*tap_layers)
+        a = TargetArgs(_ptr(token_ids), S, rows, _ptr(ctx_len), int(max_ctx_len), _ptr(page_table), page_table.shape[1],
+                       _ptr(kv_pool), kv_pool.shape[1], taps, len(tap_layers), _ptr(feats_out), _ptr(logits_out),
+                       _ptr(ids_out), _ptr(ws), ws.numel(), _ptr(self.status))
+        _check(self.lib.dflash_target_verify(self.h, C.byref(a), _stream(stream)))
 
     def _sample_ws(self, n_rows, vocab):
         need = int(self.lib.dflash_sample_workspace_bytes(n_rows, vocab))

@@ -364,25 +364,59 @@ int32_t dflash_ctx_project(dflash_handle* h, const dflash_ctx_args* a, void* str
     return DFLASH_OK;
 }
 
-int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* stream) {
-    if (!h || !a) return DFLASH_ERR_INVALID_ARG;
-    if (!h->has_weights) return DFLASH_ERR_NOT_READY;
-    if (a->batch < 0 || a->max_pages < 1 || a->n_pool_pages < 1 || a->max_ctx_len < 0) return DFLASH_ERR_INVALID_ARG;
-    if (a->batch == 0) return DFLASH_OK;
-    if (!a->anchor_ids || !a->ctx_len || !a->page_table || !a->kv_pool || !a->draft_ids) return DFLASH_ERR_INVALID_ARG;
+}  // extern "C"
+
+// One pass of a stack of pre-norm layers over `rows_per_seq` rows per sequence on top of a paged KV
+// cache: the draft block (row 0 = anchor, the rest mask tokens, no mask inside the block) and the
+// target's verify pass (given tokens, causal inside the block, block K/V written behind the committed
+// context, hidden states of chosen layers tapped) are the same launches with different options.
+struct BlockRun {
+    const int32_t* anchor_ids;   // draft: token of row 0 of each sequence (rows 1.. embed the mask token)
+    const int32_t* token_ids;    // verify: token of every row [batch * rows_per_seq]; overrides anchor_ids
+    int batch, rows_per_seq, causal;
+    const int32_t* ctx_len;
+    int max_ctx_len;
+    const int32_t* page_table;
+    int max_pages;
+    const void* kv_pool;
+    int n_pool_pages;
+    bool commit_kv;              // write the block's K/V of every layer at positions L .. L + rows_per_seq - 1
+    void* workspace;
+    int64_t workspace_bytes;
+    int32_t* ids;
+    float *top1, *margin, *hidden_out, *logits_out;
+    int32_t* dev_status;
+    const int32_t* tap_layers;   // [host] ascending layer indices whose output rows go to feats_out
+    int n_taps;
+    void* feats_out;             // [batch * rows_per_seq, n_taps * D] config dtype
+};
+
+static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
     const dflash_config& c = h->cfg;
-    if ((int64_t)a->batch * c.block_size > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
-    if (a->block_rows < 0 || a->block_rows > c.block_size) return DFLASH_ERR_INVALID_ARG;
-    const int B = a->block_rows > 0 ? a->block_rows : c.block_size, rows = a->batch * B;
+    const int B = a->rows_per_seq, rows = a->batch * B;
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
     Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const int qdim = c.n_q_heads * c.head_dim, kdim = c.n_kv_heads * c.head_dim;
     const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
+    // after layer i: tapped hidden rows, and (verify) the block's K/V into the cache
+    int next_tap = 0;
+    auto after_attention = [&](int i) -> int {
+        if (a->commit_kv) RUN(FAM_MISC, launch_kv_commit(L, ws.k_blk, ws.v_blk, a->batch, B, a->ctx_len, a->page_table, a->max_pages,
+                                                         const_cast<void*>(a->kv_pool), a->n_pool_pages, i));
+        return DFLASH_OK;
+    };
+    auto after_layer = [&](int i) -> int {
+        if (next_tap < a->n_taps && a->tap_layers[next_tap] == i) {
+            RUN(FAM_MISC, launch_tap_copy(L, ws.x, a->feats_out, rows, c.d_model, a->n_taps * c.d_model, next_tap * c.d_model));
+            ++next_tap;
+        }
+        return DFLASH_OK;
+    };
 
     dflash_attn_args at{};
-    at.mode = DFLASH_ATTN_FULL;
+    at.mode = a->causal ? DFLASH_ATTN_CAUSAL : DFLASH_ATTN_FULL;
     at.q = ws.q; at.k_blk = ws.k_blk; at.v_blk = ws.v_blk;
     at.batch = a->batch; at.rows = B;
     at.ctx_len = a->ctx_len; at.max_ctx_len = a->max_ctx_len;
@@ -407,7 +441,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_QKV] + i * ws.cnt_stride[Workspace::CNT_QKV];
             return g;
         };
-        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->batch, B, ws.x, h->layers[0].g1, xn, ws.ssq));
+        RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->token_ids, a->batch, B, ws.x, h->layers[0].g1, xn, ws.ssq));
         {
             const GemmArgs g = qkv_args(0);
             RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
@@ -418,6 +452,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             at.layer = i;
             if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
             else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+            DFLASH_TRY(after_attention(i));
             GemmArgs ph[4];
             int fam[4];
             GemmArgs& o = ph[0];      // x += W_o attn; emits the FFN norm inputs
@@ -458,15 +493,16 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
             const int rc = launch_gemm_chain(L, ph, 4, ws.flags + GEMM_MAX_PHASES * flag_set++, tr);
             prof_end(L);
             if (rc != DFLASH_OK) return rc;
+            DFLASH_TRY(after_layer(i));      // x is final for layer i after the chain's third phase; the fourth does not touch it
         }
-        RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, a->draft_ids,
+        RUN(FAM_ARGMAX_FINISH, launch_argmax_finish(L, (const Top2Entry*)ws.top2, (c.vocab + 127) / 128, rows, a->ids,
                                                     a->top1, a->margin));
         if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
         return DFLASH_OK;
     }
 
     // fp32: CUDA-core kernels, one step per launch
-    RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, ws.x, a->batch, B));
+    RUN(FAM_EMBED, launch_embed(L, a->anchor_ids, a->token_ids, ws.x, a->batch, B));
     for (int i = 0; i < c.n_layers; ++i) {
         const dflash_layer_weights& lw = h->layers[i];
         // attention half: u = RMSNorm(x); q,k,v = W u (+RoPE); x += W_o attention(q, [K_ctx; k], [V_ctx; v])
@@ -476,16 +512,64 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
                                                 c.qk_norm ? lw.g_k : nullptr));
         at.layer = i;
         RUN(FAM_ATTENTION, launch_attention_simt(L, at));
+        DFLASH_TRY(after_attention(i));
         RUN(FAM_GEMM_O, launch_gemm_simt(L, ws.attn, lw.W_o, ws.x, rows, c.d_model, qdim, true));
         // FFN half: u = RMSNorm(x); x += W_down (silu(W_gate u) * W_up u)
         RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, lw.g2, true, ws.u, rows, c.d_model));
         RUN(FAM_GEMM_GATEUP, launch_gemm_simt(L, ws.u, lw.W_gateup, ws.tmp, rows, 2 * c.d_ffn, c.d_model, false));
         RUN(FAM_GEMM_GATEUP, launch_swiglu(L, ws.tmp, ws.h, rows));
         RUN(FAM_GEMM_DOWN, launch_gemm_simt(L, ws.h, lw.W_down, ws.x, rows, c.d_model, c.d_ffn, true));
+        DFLASH_TRY(after_layer(i));
     }
     if (a->hidden_out) RUN(FAM_MISC, launch_copy_f32(L, ws.x, a->hidden_out, (int64_t)rows * c.d_model));
     RUN(FAM_RMSNORM, launch_rmsnorm(L, ws.x, true, h->w.g_f, true, ws.u, rows, c.d_model));
-    return lmhead_rows(L, ws, ws.u, nullptr, rows, a->draft_ids, a->top1, a->margin, a->logits_out);
+    return lmhead_rows(L, ws, ws.u, nullptr, rows, a->ids, a->top1, a->margin, a->logits_out);
+}
+
+extern "C" {
+
+int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* stream) {
+    if (!h || !a) return DFLASH_ERR_INVALID_ARG;
+    if (!h->has_weights) return DFLASH_ERR_NOT_READY;
+    if (a->batch < 0 || a->max_pages < 1 || a->n_pool_pages < 1 || a->max_ctx_len < 0) return DFLASH_ERR_INVALID_ARG;
+    if (a->batch == 0) return DFLASH_OK;
+    if (!a->anchor_ids || !a->ctx_len || !a->page_table || !a->kv_pool || !a->draft_ids) return DFLASH_ERR_INVALID_ARG;
+    const dflash_config& c = h->cfg;
+    if ((int64_t)a->batch * c.block_size > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
+    if (a->block_rows < 0 || a->block_rows > c.block_size) return DFLASH_ERR_INVALID_ARG;
+    BlockRun r{};
+    r.anchor_ids = a->anchor_ids;
+    r.batch = a->batch; r.rows_per_seq = a->block_rows > 0 ? a->block_rows : c.block_size; r.causal = 0;
+    r.ctx_len = a->ctx_len; r.max_ctx_len = a->max_ctx_len; r.page_table = a->page_table; r.max_pages = a->max_pages;
+    r.kv_pool = a->kv_pool; r.n_pool_pages = a->n_pool_pages;
+    r.workspace = a->workspace; r.workspace_bytes = a->workspace_bytes;
+    r.ids = a->draft_ids; r.top1 = a->top1; r.margin = a->margin; r.hidden_out = a->hidden_out; r.logits_out = a->logits_out;
+    r.dev_status = a->dev_status;
+    return block_forward(h, &r, stream);
+}
+
+int32_t dflash_target_verify(dflash_handle* h, const dflash_target_args* a, void* stream) {
+    if (!h || !a) return DFLASH_ERR_INVALID_ARG;
+    if (!h->has_weights) return DFLASH_ERR_NOT_READY;
+    if (a->batch < 0 || a->rows < 1 || a->rows > 32 || a->max_pages < 1 || a->n_pool_pages < 1 || a->max_ctx_len < 0 ||
+        a->n_taps < 0 || a->n_taps > DFLASH_MAX_LAYERS)
+        return DFLASH_ERR_INVALID_ARG;
+    if (a->batch == 0) return DFLASH_OK;
+    if (!a->token_ids || !a->ctx_len || !a->page_table || !a->kv_pool || !a->ids_out) return DFLASH_ERR_INVALID_ARG;
+    if (a->n_taps > 0 && (!a->tap_layers || !a->feats_out)) return DFLASH_ERR_INVALID_ARG;
+    for (int t = 0; t < a->n_taps; ++t)
+        if (a->tap_layers[t] < 0 || a->tap_layers[t] >= h->cfg.n_layers || (t > 0 && a->tap_layers[t] <= a->tap_layers[t - 1]))
+            return DFLASH_ERR_INVALID_ARG;
+    if ((int64_t)a->batch * a->rows > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
+    BlockRun r{};
+    r.token_ids = a->token_ids;
+    r.batch = a->batch; r.rows_per_seq = a->rows; r.causal = 1;
+    r.ctx_len = a->ctx_len; r.max_ctx_len = a->max_ctx_len; r.page_table = a->page_table; r.max_pages = a->max_pages;
+    r.kv_pool = a->kv_pool; r.n_pool_pages = a->n_pool_pages; r.commit_kv = true;
+    r.workspace = a->workspace; r.workspace_bytes = a->workspace_bytes;
+    r.ids = a->ids_out; r.logits_out = a->logits_out; r.dev_status = a->dev_status;
+    r.tap_layers = a->tap_layers; r.n_taps = a->n_taps; r.feats_out = a->feats_out;
+    return block_forward(h, &r, stream);
 }
 
 int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void* stream) {

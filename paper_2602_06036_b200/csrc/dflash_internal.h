@@ -95,7 +95,13 @@ struct Launch {
 };
 
 // ---- generic (any dtype) kernels: the whole fp32 path, and the small steps of the bf16 path ----
-int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch, int block_rows);
+// token of row r of sequence b: token_ids[b * block_rows + r] if token_ids, else anchor[b] (r = 0) or the mask token
+int launch_embed(const Launch& L, const int32_t* anchor, const int32_t* token_ids, float* x, int batch, int block_rows);
+// block rows' k / v [batch * rows_per_seq, Hkv * hd] -> pool layer `layer` at positions ctx_len[b] + r
+int launch_kv_commit(const Launch& L, const void* k_blk, const void* v_blk, int batch, int rows_per_seq, const int32_t* ctx_len,
+                     const int32_t* page_table, int max_pages, void* pool, int n_pages, int layer);
+// feats[row, off .. off + D) = x[row, :] in the config dtype
+int launch_tap_copy(const Launch& L, const float* x, void* feats, int rows, int D, int ld_out, int off);
 int launch_rmsnorm(const Launch& L, const void* in, bool in_is_f32, const void* g, bool apply,
                    void* out, int rows, int dim);
 int launch_gemm_simt(const Launch& L, const void* X, const void* W, float* Y, int M, int N, int K,

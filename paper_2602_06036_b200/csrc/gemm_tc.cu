@@ -981,7 +981,8 @@ __global__ void __launch_bounds__(128) argmax_finish_rows_kernel(const Top2Entry
 
 // block row 0 of each sequence = anchor, rows 1.. = mask token; also the first layer's norm inputs
 __global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __restrict__ E,
-                                                         const int32_t* __restrict__ anchor, float* __restrict__ x,
+                                                         const int32_t* __restrict__ anchor,
+                                                         const int32_t* __restrict__ token_ids, float* __restrict__ x,
                                                          const __nv_bfloat16* __restrict__ g,
                                                          __nv_bfloat16* __restrict__ xn, float* __restrict__ ssq, int B,
                                                          int D, int V, int mask_id, int M, int32_t* status,
@@ -991,7 +992,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const __nv_bfloat16* __
     pdl_wait();
     if (threadIdx.x == 0) trace_min(trace, 1);
     const int row = blockIdx.x, b = row / B, r = row % B;
-    int id = (r == 0) ? anchor[b] : mask_id;
+    int id = token_ids ? token_ids[row] : ((r == 0) ? anchor[b] : mask_id);
     if (id < 0 || id >= V) {
         if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_TOKEN);
         id = 0;
@@ -1168,13 +1169,13 @@ int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, in
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
 
-int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, int block_rows, float* x, const void* g,
-                      __nv_bfloat16* xn, float* ssq) {
+int launch_embed_norm(const Launch& L, const int32_t* anchor, const int32_t* token_ids, int batch, int block_rows, float* x,
+                      const void* g, __nv_bfloat16* xn, float* ssq) {
     const dflash_config& c = L.h->cfg;
     const int rows = batch * block_rows;
     if (rows <= 0) return DFLASH_OK;
     const cudaError_t e = launch_pdl(embed_norm_kernel, dim3(rows), dim3(256), 0, L.st,
-                                     (const __nv_bfloat16*)L.h->w.embed, anchor, x, (const __nv_bfloat16*)g, xn, ssq,
+                                     (const __nv_bfloat16*)L.h->w.embed, anchor, token_ids, x, (const __nv_bfloat16*)g, xn, ssq,
                                      block_rows, c.d_model, c.vocab, c.mask_token_id, rows, L.status, L.trace);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;

@@ -81,7 +81,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,
                          float* margin);
 // x[row] = E[id] (fp32), xn[row] = bf16(g * x[row]), ssq[tile][row] = sum over the tile of x^2
-int launch_embed_norm(const Launch& L, const int32_t* anchor, int batch, int block_rows, float* x, const void* g,
-                      __nv_bfloat16* xn, float* ssq);
+int launch_embed_norm(const Launch& L, const int32_t* anchor, const int32_t* token_ids, int batch, int block_rows, float* x,
+                      const void* g, __nv_bfloat16* xn, float* ssq);
 
 }  // namespace dflash

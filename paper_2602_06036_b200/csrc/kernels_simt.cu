@@ -61,9 +61,10 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 // ------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ anchor,
-                             float* __restrict__ x, int B, int D, int V, int mask_id, int32_t* status) {
+                             const int32_t* __restrict__ token_ids, float* __restrict__ x, int B, int D, int V,
+                             int mask_id, int32_t* status) {
     const int row = blockIdx.x, b = row / B, r = row % B;
-    int id = (r == 0) ? anchor[b] : mask_id;
+    int id = token_ids ? token_ids[row] : ((r == 0) ? anchor[b] : mask_id);
     if (id < 0 || id >= V) {
         if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_TOKEN);
         id = 0;
@@ -73,14 +74,14 @@ __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict_
     for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = to_f(src[d]);
 }
 
-int launch_embed(const Launch& L, const int32_t* anchor, float* x, int batch, int block_rows) {
+int launch_embed(const Launch& L, const int32_t* anchor, const int32_t* token_ids, float* x, int batch, int block_rows) {
     const dflash_config& c = L.h->cfg;
     const int rows = batch * block_rows;
     if (c.dtype == DFLASH_F32)
-        embed_kernel<float><<<rows, 256, 0, L.st>>>((const float*)L.h->w.embed, anchor, x, block_rows,
+        embed_kernel<float><<<rows, 256, 0, L.st>>>((const float*)L.h->w.embed, anchor, token_ids, x, block_rows,
                                                     c.d_model, c.vocab, c.mask_token_id, L.status);
     else
-        embed_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>((const __nv_bfloat16*)L.h->w.embed, anchor, x,
+        embed_kernel<__nv_bfloat16><<<rows, 256, 0, L.st>>>((const __nv_bfloat16*)L.h->w.embed, anchor, token_ids, x,
                                                             block_rows, c.d_model, c.vocab,
                                                             c.mask_token_id, L.status);
     DFLASH_CHECK_LAUNCH();
@@ -648,6 +649,72 @@ int launch_zero(const Launch& L, void* dst, int64_t bytes) {      // dst 16-byte
     const int64_t n16 = bytes / 16;
     const int grid = (int)std::min<int64_t>((n16 + 255) / 256, 64);
     const cudaError_t e = launch_pdl(zero_kernel, dim3(grid), dim3(256), 0, L.st, reinterpret_cast<uint4*>(dst), n16);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------
+// the target's verify pass: block K/V into its cache, tapped hidden rows into the drafter's operand
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) kv_commit_kernel(const T* __restrict__ k_blk, const T* __restrict__ v_blk, int rows_per_seq,
+                                                        const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ page_table,
+                                                        int max_pages, T* __restrict__ pool, int n_pages, int layer, int Hkv, int hd,
+                                                        int PG, int32_t* status) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
+    const int row = blockIdx.x, b = row / rows_per_seq, r = row % rows_per_seq;
+    const int pos = ctx_len[b] + r, pidx = pos / PG;
+    if (pos < 0 || pidx >= max_pages) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_CTX_OVERFLOW);
+        return;
+    }
+    const int page = page_table[(size_t)b * max_pages + pidx];
+    if (page < 0 || page >= n_pages) {
+        if (threadIdx.x == 0 && status) atomicOr(status, DFLASH_DEV_BAD_PAGE);
+        return;
+    }
+    const int kdim = Hkv * hd;
+    T* kdst = pool + ((((size_t)layer * n_pages + page) * 2) * Hkv) * PG * hd + (size_t)(pos % PG) * hd;
+    T* vdst = kdst + (size_t)Hkv * PG * hd;
+    for (int e = threadIdx.x; e < kdim; e += blockDim.x) {
+        const int head = e / hd, i = e % hd;
+        kdst[(size_t)head * PG * hd + i] = k_blk[(size_t)row * kdim + e];
+        vdst[(size_t)head * PG * hd + i] = v_blk[(size_t)row * kdim + e];
+    }
+}
+int launch_kv_commit(const Launch& L, const void* k_blk, const void* v_blk, int batch, int rows_per_seq, const int32_t* ctx_len,
+                     const int32_t* page_table, int max_pages, void* pool, int n_pages, int layer) {
+    const dflash_config& c = L.h->cfg;
+    const int rows = batch * rows_per_seq;
+    if (rows == 0) return DFLASH_OK;
+    cudaError_t e;
+    if (c.dtype == DFLASH_F32)
+        e = launch_pdl(kv_commit_kernel<float>, dim3(rows), dim3(128), 0, L.st, (const float*)k_blk, (const float*)v_blk, rows_per_seq,
+                       ctx_len, page_table, max_pages, (float*)pool, n_pages, layer, c.n_kv_heads, c.head_dim, c.page_size, L.status);
+    else
+        e = launch_pdl(kv_commit_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, L.st, (const __nv_bfloat16*)k_blk,
+                       (const __nv_bfloat16*)v_blk, rows_per_seq, ctx_len, page_table, max_pages, (__nv_bfloat16*)pool, n_pages,
+                       layer, c.n_kv_heads, c.head_dim, c.page_size, L.status);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) tap_copy_kernel(const float* __restrict__ x, T* __restrict__ feats, int D, int ld_out, int off) {
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
+    const float* src = x + (size_t)blockIdx.x * D;
+    T* dst = feats + (size_t)blockIdx.x * ld_out + off;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = from_f<T>(src[d]);
+}
+int launch_tap_copy(const Launch& L, const float* x, void* feats, int rows, int D, int ld_out, int off) {
+    if (rows == 0) return DFLASH_OK;
+    cudaError_t e;
+    if (L.h->cfg.dtype == DFLASH_F32)
+        e = launch_pdl(tap_copy_kernel<float>, dim3(rows), dim3(256), 0, L.st, x, (float*)feats, D, ld_out, off);
+    else
+        e = launch_pdl(tap_copy_kernel<__nv_bfloat16>, dim3(rows), dim3(256), 0, L.st, x, (__nv_bfloat16*)feats, D, ld_out, off);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }

@@ -280,3 +280,27 @@ def test_qk_norm_is_a_per_head_rmsnorm_before_the_rotation():
             n = lw["g_k"] * r / np.sqrt(np.mean(r * r) + cfg.rms_eps)
             np.testing.assert_allclose(K[t, h], orc.rope(n[None, None, :], np.array([t]), cfg.rope_theta)[0, 0], rtol=1e-12, atol=1e-12)
     np.testing.assert_allclose(V, (H_t @ lw["W_v"].T).reshape(5, cfg.n_kv_heads, cfg.head_dim), rtol=1e-12)
+
+
+def test_target_verify_continues_a_full_causal_forward():
+    # the verify pass over the last rows, on top of the K/V its own earlier pass cached, must equal
+    # the plain causal transformer run over the whole token list at once (logits and tapped features)
+    import dataclasses
+    from paper_2602_06036_b200 import synth
+    tcfg = dataclasses.replace(synth.TINY, n_layers=3, block_size=4)
+    tw = synth.weights_to_numpy(synth.make_weights(tcfg, 31))
+    rng = np.random.default_rng(4)
+    tokens = rng.integers(0, tcfg.vocab - 1, size=13).tolist()
+    taps = (0, 2)
+    full_logits, full_feats = orc.toy_target_forward(tokens, tw, tcfg, taps)
+    empty = [np.zeros((0, tcfg.n_kv_heads, tcfg.head_dim))] * tcfg.n_layers
+    Lp = 8
+    pre = orc.target_verify(tokens[:Lp], 0, empty, empty, tw, tcfg, taps)
+    np.testing.assert_allclose(pre["logits"], full_logits[:Lp], rtol=1e-9, atol=1e-9)
+    inc = orc.target_verify(tokens[Lp:], Lp, pre["K"], pre["V"], tw, tcfg, taps)
+    np.testing.assert_allclose(inc["logits"], full_logits[Lp:], rtol=1e-9, atol=1e-9)
+    np.testing.assert_allclose(inc["feats"], full_feats[Lp:], rtol=1e-9, atol=1e-9)
+    assert inc["feats"].shape == (5, 2 * tcfg.d_model) and len(inc["K"]) == 3 and inc["K"][0].shape == (5, tcfg.n_kv_heads, tcfg.head_dim)
+    # a later row never influences an earlier one: dropping the last token leaves the other rows unchanged
+    short = orc.target_verify(tokens[Lp:-1], Lp, pre["K"], pre["V"], tw, tcfg, taps)
+    np.testing.assert_allclose(short["logits"], inc["logits"][:-1], rtol=1e-12, atol=1e-12)
