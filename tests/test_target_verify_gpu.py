@@ -118,3 +118,80 @@ def test_one_speculative_cycle_on_the_gpu():
             gk, gv = orc.pool_read(got_pool, drf.page_table_cpu[b].numpy(), L + n, i, dcfg.page_size)
             assert_close(gk[L:], K[i], dcfg.dtype, f"injected K seq {b} layer {i}")
             assert_close(gv[L:], V[i], dcfg.dtype, f"injected V seq {b} layer {i}")
+
+
+def test_speculative_decoding_on_the_gpu_equals_greedy_decoding():
+    # fp32 target (2 layers) and drafter (1 layer); every kernel of the cycle runs on the GPU:
+    #   verify [anchor, drafts] -> accept -> commit length -> project the kept rows' taps -> draft.
+    # The emitted tokens must equal the target's own greedy decoding (one row per step through the same
+    # call), whatever the drafter proposes; planted correct drafts make some cycles keep several tokens.
+    tcfg = dataclasses.replace(synth.TINY, n_layers=2, block_size=8)
+    dcfg = dataclasses.replace(synth.TINY, n_layers=1, block_size=8, n_feat_layers=2, d_target=tcfg.d_model)
+    taps, gamma, P, n_out = (0, 1), 8, 11, 40
+    S = 2
+    room = P + n_out + 3 * gamma
+    dev = torch.device("cuda:0")
+    prompt = torch.randint(0, tcfg.vocab - 1, (S, P), generator=synth.substream(61, "prompt"), dtype=torch.int32)
+
+    def fresh(cfg, seed):
+        c = Case(cfg, (0,) * S, seed=seed, headroom=room)
+        return c
+
+    def prefill(tgt):
+        ids = torch.zeros((S, P), dtype=torch.int32, device=dev)
+        feats = torch.zeros((S, P, len(taps) * tcfg.d_model), dtype=tcfg.torch_dtype, device=dev)
+        tgt.lib.dflash_target_verify(prompt.to(dev), tgt.ctx_len, 0, tgt.page_table, tgt.pool, list(taps), ids, feats_out=feats)
+        tgt.ctx_len += P
+        return ids[:, -1].clone(), feats
+
+    # ---- plain greedy decoding with the target alone
+    tgt = fresh(tcfg, 61)
+    tok, _ = prefill(tgt)
+    greedy = [tok.cpu()]
+    one = torch.zeros((S, 1), dtype=torch.int32, device=dev)
+    for _ in range(n_out + gamma):
+        tgt.lib.dflash_target_verify(greedy[-1].view(S, 1).to(dev), tgt.ctx_len, P + n_out + gamma, tgt.page_table, tgt.pool, [], one)
+        tgt.ctx_len += 1
+        greedy.append(one[:, 0].cpu().clone())
+    greedy = torch.stack(greedy, dim=1)                    # [S, n_out + gamma + 1]: greedy[:, 0] follows the prompt
+
+    # ---- speculative decoding
+    tgt, drf = fresh(tcfg, 61), fresh(dcfg, 62)
+    anchor, feats = prefill(tgt)
+    drf.lib.dflash_ctx_project(feats, torch.full((S,), P, dtype=torch.int32, device=dev), drf.ctx_len, drf.page_table, drf.pool)
+    drf.ctx_len += P
+    emitted = [[int(anchor[b])] for b in range(S)]
+    acc = torch.zeros(S, dtype=torch.int32, device=dev)
+    out = torch.zeros((S, gamma + 1), dtype=torch.int32, device=dev)
+    bonus = torch.zeros(S, dtype=torch.int32, device=dev)
+    new_len = torch.zeros(S, dtype=torch.int32, device=dev)
+    drafts = torch.zeros((S, gamma), dtype=torch.int32, device=dev)
+    logits = torch.zeros((S * (gamma + 1), tcfg.vocab), dtype=torch.float32, device=dev)
+    vfeats = torch.zeros((S, gamma + 1, len(taps) * tcfg.d_model), dtype=tcfg.torch_dtype, device=dev)
+    vids = torch.zeros((S, gamma + 1), dtype=torch.int32, device=dev)
+    taus = []
+    cycle = 0
+    while min(len(e) for e in emitted) < n_out:
+        drf.lib.dflash_draft_block(anchor, drf.ctx_len, P + n_out + gamma, drf.page_table, drf.pool, drafts)
+        for b in range(S):                                  # plant a few correct drafts (known greedy continuation)
+            k = (cycle + b) % 5
+            n = len(emitted[b])
+            drafts[b, :k] = greedy[b, n:n + k].to(dev)
+        tokens = torch.cat([anchor.view(S, 1), drafts], dim=1).contiguous()
+        tgt.lib.dflash_target_verify(tokens, tgt.ctx_len, P + n_out + gamma, tgt.page_table, tgt.pool, list(taps), vids,
+                                     feats_out=vfeats, logits_out=logits)
+        tgt.lib.dflash_verify_accept(drafts, gamma, gamma, tgt.ctx_len, acc, out, bonus, new_len, logits=logits.view(S, gamma + 1, -1))
+        drf.lib.dflash_ctx_project(vfeats, acc, drf.ctx_len, drf.page_table, drf.pool)
+        torch.cuda.synchronize()
+        assert int(tgt.lib.status.item()) == 0 and int(drf.lib.status.item()) == 0
+        for b in range(S):
+            t = int(acc[b])
+            emitted[b] += out[b, :t].tolist()
+            taus.append(t)
+        tgt.ctx_len.copy_(new_len)
+        drf.ctx_len.copy_(new_len)
+        anchor = bonus.clone()
+        cycle += 1
+    for b in range(S):
+        assert emitted[b][:n_out] == greedy[b, :n_out].tolist(), b
+    assert max(taus) >= 4 and min(taus) == 1
