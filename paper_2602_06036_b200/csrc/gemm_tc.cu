@@ -55,7 +55,7 @@ constexpr int slabs_for(int nt, bool k_mult_64) { return (nt <= 32 && k_mult_64)
 constexpr int MAX_STAGES = 12;
 constexpr int TOK_CACHE = 1024;                  // per-token scale / position / page kept for this many rows
 // token columns handled per epilogue pass (each of the 128 epilogue threads holds CH accumulators)
-constexpr int pass_cols(int nt) { return nt < 64 ? nt : 32; }   // 32-column passes: short dependent chains when finishing, room for ring stages
+constexpr int pass_cols(int nt) { return nt <= 16 ? nt : (nt == 32 ? 16 : 32); }   // short passes: short dependent chains when finishing, fewer registers
 constexpr int smem_fixed(int nt) {
     return TILE_F * (pass_cols(nt) + 1) * 4 + 128 * 16 + 3 * TOK_CACHE * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
 }
