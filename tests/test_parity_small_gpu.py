@@ -134,6 +134,27 @@ def test_bf16_random_shapes(seed):
     case.check_draft(got)
 
 
+def test_largest_block_and_empty_calls():
+    # block size 32 (the largest the library takes): 32 rows x 4 q heads fill the 128-row attention operand
+    cfg = dataclasses.replace(synth.MID, block_size=32)
+    case = Case(cfg, (0, 63, 64, 200), seed=29)
+    case.project_prefill()
+    _check_pool(case)
+    got = case.run_draft()
+    assert case.check_draft(got) >= case.S * 16
+    # nothing to do: empty batch, zero new rows; the pool and the outputs stay as they were
+    dev = case.device
+    before = case.pool.clone()
+    none_i = torch.zeros((0,), dtype=torch.int32, device=dev)
+    case.lib.dflash_draft_block(none_i, none_i, 0, case.page_table[:0], case.pool, torch.zeros((0, 32), dtype=torch.int32, device=dev))
+    case.lib.dflash_ctx_project(torch.zeros((0, 4, cfg.feat_dim), dtype=cfg.torch_dtype, device=dev), none_i, none_i,
+                                case.page_table[:0], case.pool)
+    feats = synth.make_features(cfg, case.S * 3, 29, "none").reshape(case.S, 3, cfg.feat_dim).to(dev)
+    case.lib.dflash_ctx_project(feats, torch.zeros(case.S, dtype=torch.int32, device=dev), case.ctx_len, case.page_table, case.pool)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) == 0 and torch.equal(case.pool, before)
+
+
 def test_bf16_feature_dims_that_are_not_multiples_of_64():
     # contraction lengths of 520 / 1544 / 1560 (multiples of 8 only): the one-slab ring stages with a
     # zero-filled K tail, ragged 128-feature tiles in the folded norms, a ragged last weight tile
