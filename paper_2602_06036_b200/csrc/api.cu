@@ -450,7 +450,9 @@ static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
             const dflash_layer_weights& lw = h->layers[i];
             const bool last = i + 1 == c.n_layers;
             at.layer = i;
-            if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters));
+            // layers after the first: the cache they read was final before this call's first attention ran
+            // (not so in the verify pass, which writes the cache as it goes)
+            if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters, i > 0 && !a->commit_kv));
             else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
             DFLASH_TRY(after_attention(i));
             GemmArgs ph[4];

@@ -50,6 +50,8 @@ constexpr float RESCALE_GAP = 8.f;               // log2 units
 struct AParams {
     int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks, rows_valid;
     int dup;     // rows_valid <= 64: the query rows are loaded twice and each copy handles 32 of a tile's 64 keys
+    int early_kv;   // the cached context of this layer was written before the previous kernel's dependencies:
+                    // its first tiles may be requested before the grid dependency resolves
     float scale_log2;
     const int32_t* ctx_len;
     const int32_t* page_table;
@@ -181,6 +183,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Context K/V tiles of the first ring stages travel while the previous kernel (which produces q and
+    // the block's own k/v, not the cache) is still running.
+    int n_early = 0;
+    if (threadIdx.x == 0 && p.early_kv) {
+        const uint64_t pol_kv = policy_evict_first();
+#pragma unroll
+        for (int i = 0; i < PAGE_PRE; ++i) {
+            const int t = t_lo + i;
+            const int page = page_pre[i];
+            if (i == n_early && i < n_tiles && i < NS && t < n_ctx_tiles && page >= 0 && page < p.n_pages) {
+                uint8_t* dK = sKV + (size_t)i * KV_STAGE_BYTES;
+                uint8_t* dV = dK + KV_STAGE_BYTES / 2;
+                mbar_expect_tx(&kv_full[i], KV_STAGE_BYTES);
+                tile_ok[i] = 1;
+                const int rowK = ((((p.layer * p.n_pages + page) * 2 + 0) * p.Hkv + g) * PG);
+                const int rowV = rowK + p.Hkv * PG;
+                tma_load_2d(dK, &tmPool, 0, rowK, &kv_full[i], pol_kv);
+                tma_load_2d(dK + 8192, &tmPool, 64, rowK, &kv_full[i], pol_kv);
+                tma_load_2d(dV, &tmPool, 0, rowV, &kv_full[i], pol_kv);
+                tma_load_2d(dV + 8192, &tmPool, 64, rowV, &kv_full[i], pol_kv);
+                n_early = i + 1;
+            }
+        }
+    }
     pdl_wait();
     if (threadIdx.x == 0) trace_min(p.trace, 1);
 
@@ -199,7 +225,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 tma_load_4d(sQ + Q_BYTES / 2, &tmQ, 64, 0, g, b * p.R, q_full, pol_q);
             }
             bool ok = true;
-            for (int i = 0; i < n_tiles; ++i) {
+            for (int i = n_early; i < n_tiles; ++i) {      // the first n_early tiles are already on their way
                 const int st = i % NS;
                 const uint32_t ph = (i / NS) & 1;
                 if (!mbar_wait(&kv_empty[st], ph ^ 1, &flags[0])) { ok = false; break; }
@@ -612,7 +638,7 @@ int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_c
 }
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
 
-int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters) {
+int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv) {
     const dflash_config& c = L.h->cfg;
     if (a.batch == 0 || a.rows == 0) return DFLASH_OK;
     AParams p{};
@@ -622,6 +648,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.tiles_per_unit = tiles_per_unit(a.batch, c.n_kv_heads, a.max_ctx_len, L.h->sm_count);
     p.rows_valid = std::min(128, a.rows * p.group);
     p.dup = (p.rows_valid <= 64 && 64 % p.group == 0) ? 1 : 0;
+    p.early_kv = early_kv ? 1 : 0;
     const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
     p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;

@@ -11,6 +11,9 @@ int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_c
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
 // `part`: split-KV scratch of the size above. `counters` is not used by the current kernels (the
 // partials are merged by a second kernel, not by a last arriver).
-int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters);
+// `early_kv`: the layer's cached context was complete before the kernel preceding this one started waiting
+// (true for layers after the first of a draft block: the first layer's wait covered the context
+// projection); its first tiles are then requested before this kernel's own grid dependency resolves.
+int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv = false);
 
 }  // namespace dflash
