@@ -2,7 +2,7 @@
 //   every block row of a sequence attends over [paged context K/V ; the block's own K/V].
 // One CTA works on one (sequence, kv head, range of KV tiles). The queries of all block rows and of
 // the q heads that share the kv head (rows x group <= 128) are the 128-row "M" operand; a KV tile
-// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (4-deep K/V ring that
+// is one 64-token page (or the block's own rows). Roles: a TMA producer warp (5-deep K/V ring that
 // runs ahead of the math) and TWO independent pipelines that take alternate tiles, each made of one
 // MMA-issuing warp and one softmax warpgroup with their own S buffers (two, so the next S is ready
 // before the current softmax ends), P buffer and output accumulator:
@@ -36,12 +36,13 @@ using namespace ptx;
 
 constexpr int HD = 128;          // head_dim
 constexpr int PG = 64;           // tokens per page = keys per tile
-constexpr int NS = 4;            // K/V ring depth
+constexpr int NS = 5;            // K/V ring depth (the kernel is bound by the bytes it keeps in flight: 3 stages ran 1.37x slower than 4)
 constexpr int Q_BYTES = 128 * HD * 2;            // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
 constexpr int P_BYTES = 128 * PG * 2;            // 16 KiB per warpgroup
 constexpr int PART_LD = HD + 4;                  // acc[128], running max, running sum, 2 pad (16-byte rows)
-constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512 + 2 * 384 * 4;
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NS * KV_STAGE_BYTES + 2 * P_BYTES + 512;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 constexpr uint32_t TMEM_COLS = 512;              // S[w][2] (4 x 64) | O0 | O1 (128 each)
 constexpr int N_THREADS = 352;                   // producer, MMA issuer 0, 2 x 4 softmax warps, MMA issuer 1
 constexpr uint32_t TMEM_O = 256;                 // first column of the output accumulators
@@ -157,7 +158,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort
     volatile int* tile_ok = flags + 2;      // [NS] 0 if the ring stage holds a page that must be ignored
-    float* xchg = reinterpret_cast<float*>(const_cast<int*>(tile_ok) + 8);   // [2 pipelines][3][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -328,7 +328,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t lane_sel = (uint32_t)(ew * 32) << 16;
         const uint32_t tmem_O = tmem_base + TMEM_O + wg * HD + lane_sel;
         uint8_t* myP = sP + wg * P_BYTES;
-        float* xch = xchg + wg * 384;                       // [3][128] exchange between the two copies of a row
+        // [3][128] exchange between the two copies of a row (dup only): it lives in rows 64..127 of this
+        // pipeline's P tile, which in that mode hold nothing (their products land in ignored output rows)
+        float* xch = reinterpret_cast<float*>(myP + 64 * 128);
         float m_run = -CUDART_INF_F, l_run = 0.f;           // log2-domain reference maximum, running sum
         bool ok = true;
         int k = 0;                                          // index of this warpgroup's tile
