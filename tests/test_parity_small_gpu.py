@@ -219,6 +219,33 @@ def test_block_attention_building_block(dtype, mode):
         assert_close(out[b].float().cpu().numpy(), ref, dtype, f"attention seq {b} L={L}")
 
 
+def test_many_anchor_blocks_over_one_cached_sequence():
+    # the training-side layout (Sec. 4.2: many anchor blocks drawn from one sequence, each bidirectional
+    # inside and seeing only the injected features before its anchor) is, for the forward pass, a batch of
+    # blocks that share ONE page-table row and differ in ctx_len = anchor position
+    from paper_2602_06036_b200 import binding
+    cfg = synth.MID
+    one = Case(cfg, (330,), seed=17)
+    one.fill_pool_synthetic()
+    anchors = (0, 16, 64, 65, 200, 313)
+    S, R = len(anchors), cfg.block_size
+    table = one.page_table.repeat(S, 1).contiguous()
+    ctx = torch.tensor(anchors, dtype=torch.int32, device=one.device)
+    q = synth.normal((S, R, cfg.n_q_heads, cfg.head_dim), 1.0, 17, "tr.q", cfg.torch_dtype)
+    k = synth.normal((S, R, cfg.n_kv_heads, cfg.head_dim), 1.0, 17, "tr.k", cfg.torch_dtype)
+    v = synth.normal((S, R, cfg.n_kv_heads, cfg.head_dim), 1.0, 17, "tr.v", cfg.torch_dtype)
+    out = torch.zeros_like(q, device=one.device)
+    one.lib.dflash_block_attention(binding.ATTN_FULL, q.to(one.device), k.to(one.device), v.to(one.device), ctx, max(anchors),
+                                   table, one.pool, 1, out)
+    torch.cuda.synchronize()
+    assert int(one.lib.status.item()) == 0
+    for b, a in enumerate(anchors):
+        kc, vc = orc.pool_read(one.pool_np, one.page_table_cpu[0].numpy(), a, 1, cfg.page_size)
+        ref = orc.block_attention(synth.to_numpy_f32(q[b]), kc, vc, synth.to_numpy_f32(k[b]), synth.to_numpy_f32(v[b]),
+                                  cfg.softmax_scale, causal=False)
+        assert_close(out[b].float().cpu().numpy(), ref, cfg.dtype, f"block anchored at {a}")
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_lmhead_argmax_building_block(dtype):
     cfg = synth.TINY if dtype == "fp32" else synth.MID
