@@ -491,10 +491,10 @@ def main():
         e["launches_per_step"] += 1
     for fam, e in kernels.items():
         n = e["launches_per_step"]
+        if fam == "attention":               # one or two records (main kernel, merge kernel) make one attention per layer
+            n = cfg.n_layers
+            e["launches_per_step"] = n
         e["us_per_launch"] = e.pop("us_total") / n
-        if fam == "attention":
-            e["us_per_launch"] *= 2          # two records (main kernel + merge) make one attention
-            e["launches_per_step"] = n // 2
         if fam in alg and e["us_per_launch"] > 0:
             e["alg_bytes"] = alg[fam]
             e["gbs"] = alg[fam] / (e["us_per_launch"] * 1e-6) / 1e9

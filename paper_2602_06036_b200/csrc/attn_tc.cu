@@ -618,14 +618,16 @@ bool attn_tc_supported(const dflash_config& c, int rows) {
 }
 
 // Keys are split into ranges of `tiles_per_unit` 64-key tiles. One sequence: about one wave of equal
-// CTAs. A batch: lengths differ (shorter sequences leave empty units that exit at once), so ranges
-// of at least 8 tiles and enough of them for several waves.
+// CTAs. A batch: lengths differ (shorter sequences leave empty units that exit at once).
 static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
     const int Tmax = (max_ctx_len + PG - 1) / PG + 1;
     const int64_t bh = (int64_t)batch * Hkv;
     if (batch > 1) {
-        const int64_t c = (bh * Tmax + 8 * (int64_t)sm_count - 1) / (8 * (int64_t)sm_count);
-        return (int)std::min<int64_t>(std::max<int64_t>(8, c), std::max(2, Tmax));
+        // measured on the serving-mix shapes: with at least one (sequence, kv head) per SM, whole sequences per
+        // CTA win (no partials, no merge kernel); with fewer, ranges of >= 16 tiles sized for about two waves
+        if (bh >= sm_count) return std::max(2, Tmax);
+        const int64_t c = (bh * Tmax + 2 * (int64_t)sm_count - 1) / (2 * (int64_t)sm_count);
+        return (int)std::min<int64_t>(std::max<int64_t>(16, c), std::max(2, Tmax));
     }
     for (int c = 2; c < Tmax; ++c)
         if (bh * ((Tmax + c - 1) / c) <= sm_count) return c;
@@ -633,7 +635,7 @@ static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
 }
 
 int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count) {
-    // units: one sequence <= SMs (+ rounding); a batch <= 8*SMs + batch*Hkv (ranges of >= total/(8*SMs) tiles)
+    // units: one sequence <= SMs (+ rounding); a batch <= 2*SMs + 2*batch*Hkv (ranges of >= total/(2*SMs) tiles); kept generous
     const int64_t units = 8 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
     const int rows_valid = std::min(128, rows * (c.n_q_heads / c.n_kv_heads));
     return units * rows_valid * PART_LD * 4;
