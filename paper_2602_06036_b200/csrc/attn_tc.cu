@@ -625,7 +625,8 @@ static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
     if (batch > 1) {
         // measured on the serving-mix shapes: with at least one (sequence, kv head) per SM, whole sequences per
         // CTA win (no partials, no merge kernel); with fewer, ranges of >= 16 tiles sized for about two waves
-        if (bh >= sm_count) return std::max(2, Tmax);
+        // (ranges capped at 128 tiles so that one very long sequence among short ones cannot hold the tail)
+        if (bh >= sm_count) return std::min(std::max(2, Tmax), 128);
         const int64_t c = (bh * Tmax + 2 * (int64_t)sm_count - 1) / (2 * (int64_t)sm_count);
         return (int)std::min<int64_t>(std::max<int64_t>(16, c), std::max(2, Tmax));
     }
