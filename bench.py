@@ -115,10 +115,11 @@ class ClockSampler:
 # the step
 # ------------------------------------------------------------------------------------------------
 class Step:
-    def __init__(self, wl, device, seed=0, temperature=0.0):
+    def __init__(self, wl, device, seed=0, temperature=0.0, fuse_ctx=True):
         from paper_2602_06036_b200 import binding
         cfg = wl.cfg
         self.T = float(temperature)
+        self.fuse_ctx = bool(fuse_ctx)
         self.wl, self.cfg, self.dev = wl, cfg, device
         B, S = cfg.block_size, wl.batch
         self.gamma = B
@@ -157,6 +158,9 @@ class Step:
         self.e_anchor = torch.empty_like(self.d_anchor)
         self.e_logits = torch.empty_like(self.d_logits)
         self.n_new = (planted + 1).to(torch.int32).to(device)      # rows committed by the previous cycle
+        # those rows are the last n_new of the context the block attends over: the step projects them, then drafts
+        self.ctx_before = (self.ctx_len - self.n_new).clamp_(min=0).to(torch.int32)
+        self.n_new = (self.ctx_len - self.ctx_before).to(torch.int32)
         # every result of a step lives in one flat int32 buffer, so the end-to-end run reads it back in one copy
         n_out = S * B + S * (g + 1) + 3 * S
         self.d_out = torch.zeros(n_out, dtype=torch.int32, device=device)
@@ -181,13 +185,17 @@ class Step:
 
     def run_draft(self, feats, anchor):
         lib = self.lib
-        lib.dflash_ctx_project(feats, self.n_new, self.ctx_len, self.page_table, self.pool)
+        ctx = None
+        if self.fuse_ctx:       # the projection rides in the draft call (one chained launch with the first QKV)
+            ctx = (feats, self.n_new, self.ctx_before)
+        else:
+            lib.dflash_ctx_project(feats, self.n_new, self.ctx_before, self.page_table, self.pool)
         if self.T > 0:
             lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids,
-                                   logits_out=self.draft_logits)
+                                   logits_out=self.draft_logits, ctx=ctx)
             lib.dflash_sample_rows(self.draft_logits, self.T, self.u_draft, self.draft_ids.view(-1))
         else:
-            lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids)
+            lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids, ctx=ctx)
 
     def run_verify(self, logits):
         # The target's verify pass is outside this library; its logits are an input. The drafts
@@ -392,6 +400,8 @@ def main():
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="> 0: drafts are drawn from the draft's logits and verified by speculative sampling (default: greedy)")
+    ap.add_argument("--separate-ctx", action="store_true",
+                    help="run the context projection as its own call before the draft call instead of inside it")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
@@ -416,7 +426,7 @@ def main():
     cfg = wl.cfg
     peaks = load_peaks()
     # replicas: every rank runs the same batch on its own GPU; there is no data-path collective
-    step = Step(wl, device, seed=0, temperature=args.temperature)
+    step = Step(wl, device, seed=0, temperature=args.temperature, fuse_ctx=not args.separate_ctx)
     S, B = wl.batch, cfg.block_size
 
     if args.kernel:

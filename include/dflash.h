@@ -165,6 +165,14 @@ typedef struct {
     int32_t        block_rows;   /* rows per sequence in THIS call: 0 = the handle's block_size B, else 1..B
                                     (a drafter trained at B = 16 also runs blocks of 8 or 10, Sec. 5.3); every
                                     [batch, B] / [batch*B, ...] shape above then uses block_rows in place of B */
+    const dflash_ctx_args* ctx;  /* [host] may be NULL. When given, the context projection described by *ctx (same
+                                    result as dflash_ctx_project with these arguments; same batch and pool as this
+                                    call; its workspace fields are ignored, this call's workspace must hold
+                                    dflash_workspace_bytes(h, batch, max(batch*B, batch*max_new))) runs inside this
+                                    call, chained in ONE launch with the first layer's QKV contraction: the draft's
+                                    first weights stream while the projection's last tiles finish. The draft sees
+                                    ctx_len[b] cached entries: pass the lengths AFTER the projection there if the
+                                    new rows are to be visible (ctx->ctx_len holds the lengths before it). */
 } dflash_draft_args;
 int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a /*[host]*/, void* stream);
 

@@ -63,7 +63,7 @@ class DraftArgs(C.Structure):
                 ("kv_pool", C.c_void_p), ("n_pool_pages", C.c_int32), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_int64), ("draft_ids", C.c_void_p), ("top1", C.c_void_p),
                 ("margin", C.c_void_p), ("hidden_out", C.c_void_p), ("logits_out", C.c_void_p),
-                ("dev_status", C.c_void_p), ("block_rows", C.c_int32)]
+                ("dev_status", C.c_void_p), ("block_rows", C.c_int32), ("ctx", C.POINTER(CtxArgs))]
 
 
 class VerifyArgs(C.Structure):
@@ -302,13 +302,23 @@ class DFlash:
         _check(self.lib.dflash_ctx_project(self.h, C.byref(a), _stream(stream)))
 
     def dflash_draft_block(self, anchor_ids, ctx_len, max_ctx_len, page_table, kv_pool, draft_ids,
-                           top1=None, margin=None, hidden_out=None, logits_out=None, stream=None, block_rows=0):
-        """block_rows: rows per sequence in this call (0 = the handle's block size)."""
+                           top1=None, margin=None, hidden_out=None, logits_out=None, stream=None, block_rows=0, ctx=None):
+        """block_rows: rows per sequence in this call (0 = the handle's block size).
+        ctx = (feats [S, max_new, k*D_t], n_new or None, ctx_len_before): run that context projection inside
+        this call, chained with the first layer's QKV contraction."""
         S = anchor_ids.shape[0]
-        ws = self.workspace(S, S * self.cfg.block_size)
+        rows = S * self.cfg.block_size
+        cptr = None
+        if ctx is not None:
+            feats, n_new, len_before = ctx
+            rows = max(rows, S * feats.shape[1])
+            self._ctx_keep = CtxArgs(_ptr(feats), S, feats.shape[1], _ptr(n_new), _ptr(len_before), _ptr(page_table),
+                                     page_table.shape[1], _ptr(kv_pool), kv_pool.shape[1], None, 0, _ptr(self.status))
+            cptr = C.pointer(self._ctx_keep)
+        ws = self.workspace(S, rows)
         a = DraftArgs(_ptr(anchor_ids), S, _ptr(ctx_len), int(max_ctx_len), _ptr(page_table), page_table.shape[1],
                       _ptr(kv_pool), kv_pool.shape[1], _ptr(ws), ws.numel(), _ptr(draft_ids), _ptr(top1),
-                      _ptr(margin), _ptr(hidden_out), _ptr(logits_out), _ptr(self.status), int(block_rows))
+                      _ptr(margin), _ptr(hidden_out), _ptr(logits_out), _ptr(self.status), int(block_rows), cptr)
         _check(self.lib.dflash_draft_block(self.h, C.byref(a), _stream(stream)))
 
     def dflash_verify_accept(self, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus,

@@ -389,16 +389,31 @@ struct BlockRun {
     const int32_t* tap_layers;   // [host] ascending layer indices whose output rows go to feats_out
     int n_taps;
     void* feats_out;             // [batch * rows_per_seq, n_taps * D] config dtype
+    const dflash_ctx_args* ctx;  // draft: context projection to run inside this call (chained with the first QKV), or nullptr
 };
 
 static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
     const dflash_config& c = h->cfg;
     const int B = a->rows_per_seq, rows = a->batch * B;
+    const bool tc = c.dtype == DFLASH_BF16;
+    // A context projection handed in with the draft: fused into the first chained launch when its weight
+    // maps fit one launch (fusion + one K/V group per layer + QKV), else run first as its own launches.
+    const dflash_ctx_args* cx = a->ctx;
+    const int rows_ctx = cx ? cx->batch * cx->max_new : 0;
+    if (cx && rows_ctx > 0 && (!cx->feats || !cx->ctx_len || !cx->page_table || !cx->kv_pool || cx->batch != a->batch ||
+                               cx->max_pages < 1 || cx->n_pool_pages < 1))
+        return DFLASH_ERR_INVALID_ARG;
+    const bool fuse_ctx = tc && cx && rows_ctx > 0 && c.n_layers + 2 <= GEMM_MAX_GROUPS;
+    if (cx && rows_ctx > 0 && !fuse_ctx) {
+        dflash_ctx_args own = *cx;
+        own.workspace = a->workspace; own.workspace_bytes = a->workspace_bytes;
+        if (!own.dev_status) own.dev_status = a->dev_status;
+        DFLASH_TRY(dflash_ctx_project(h, &own, stream));
+    }
     Workspace ws;
-    DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
+    DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, fuse_ctx ? std::max(rows, rows_ctx) : rows, &ws));
     Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
     const int qdim = c.n_q_heads * c.head_dim, kdim = c.n_kv_heads * c.head_dim;
-    const bool tc = c.dtype == DFLASH_BF16;
     DFLASH_TRY(zero_counters(L, ws));
     // after layer i: tapped hidden rows, and (verify) the block's K/V into the cache
     int next_tap = 0;
@@ -442,7 +457,36 @@ static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
             return g;
         };
         RUN(FAM_EMBED, launch_embed_norm(L, a->anchor_ids, a->token_ids, a->batch, B, ws.x, h->layers[0].g1, xn, ws.ssq));
-        {
+        if (fuse_ctx) {
+            // [context fusion, context K/V of every layer, QKV of layer 0] in one launch. The projection's
+            // normalised operand and sums of squares live in buffers the draft only uses later (tmp, h).
+            __nv_bfloat16* cxn = (__nv_bfloat16*)ws.tmp;
+            float* cssq = (float*)ws.h;
+            const int feat = c.n_feat_layers * c.d_target;
+            const size_t kv_off = (size_t)qdim * c.d_model * elem_size(c.dtype);
+            GemmArgs ph[3];
+            GemmArgs& g = ph[0];
+            g = GemmArgs{};
+            g.X = cx->feats; g.W[0] = h->w.W_c; g.M = rows_ctx; g.N = c.d_model; g.K = feat;
+            g.epilogue = EPI_STORE_F32; g.g_next = h->w.g_c; g.xn_out = cxn; g.ssq_out = cssq;
+            g.part = ws.part; g.counters = ws.counters + ws.cnt_off[Workspace::CNT_FUSE];
+            GemmArgs& k = ph[1];
+            k = GemmArgs{};
+            k.n_groups = c.n_layers;
+            for (int j = 0; j < c.n_layers; ++j) {
+                k.W[j] = (const char*)h->layers[j].W_qkv + kv_off;
+                k.g_k_group[j] = c.qk_norm ? h->layers[j].g_k : nullptr;
+            }
+            k.X = cxn; k.M = rows_ctx; k.N = 2 * kdim; k.K = c.d_model; k.ssq_in = cssq;
+            k.epilogue = EPI_CTX_KV; k.ctx = cx; k.first_layer = 0; k.part = ws.part;
+            k.counters = ws.counters + ws.cnt_off[Workspace::CNT_KV];
+            ph[2] = qkv_args(0);
+            unsigned long long* tr[3] = {trace_slot(h, FAM_CTX_FUSE), trace_slot(h, FAM_CTX_KV), trace_slot(h, FAM_GEMM_QKV)};
+            prof_begin(L, FAM_GEMM_CHAIN);
+            const int rc = launch_gemm_chain(L, ph, 3, ws.flags + GEMM_MAX_PHASES * flag_set++, tr);
+            prof_end(L);
+            if (rc != DFLASH_OK) return rc;
+        } else {
             const GemmArgs g = qkv_args(0);
             RUN(FAM_GEMM_QKV, launch_gemm_tc(L, g, ws.flags + GEMM_MAX_PHASES * flag_set++));
         }
@@ -452,7 +496,8 @@ static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
             at.layer = i;
             // layers after the first: the cache they read was final before this call's first attention ran
             // (not so in the verify pass, which writes the cache as it goes)
-            if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters, i > 0 && !a->commit_kv));
+            if (attn_tc_supported(c, B)) RUN(FAM_ATTENTION, launch_attention_tc(L, at, ws.attn_part, ws.attn_counters, i > 0 && !a->commit_kv,
+                                                                              fuse_ctx ? cx->ctx_len : nullptr));
             else RUN(FAM_ATTENTION, launch_attention_simt(L, at));
             DFLASH_TRY(after_attention(i));
             GemmArgs ph[4];
@@ -547,6 +592,7 @@ int32_t dflash_draft_block(dflash_handle* h, const dflash_draft_args* a, void* s
     r.workspace = a->workspace; r.workspace_bytes = a->workspace_bytes;
     r.ids = a->draft_ids; r.top1 = a->top1; r.margin = a->margin; r.hidden_out = a->hidden_out; r.logits_out = a->logits_out;
     r.dev_status = a->dev_status;
+    r.ctx = a->ctx;
     return block_forward(h, &r, stream);
 }
 

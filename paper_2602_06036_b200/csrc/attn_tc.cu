@@ -55,6 +55,7 @@ struct AParams {
                     // its first tiles may be requested before the grid dependency resolves
     float scale_log2;
     const int32_t* ctx_len;
+    const int32_t* early_len;   // with early_kv: rows [0, early_len[b]) are the final ones (nullptr: all of ctx_len[b])
     const int32_t* page_table;
     __nv_bfloat16* out;
     float* part;
@@ -188,11 +189,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     int n_early = 0;
     if (threadIdx.x == 0 && p.early_kv) {
         const uint64_t pol_kv = policy_evict_first();
+        // only pages that lie wholly below the rows an earlier kernel of this call may still be writing
+        const int n_final_tiles = p.early_len ? min(__ldg(p.early_len + b), L) / PG : n_ctx_tiles;
 #pragma unroll
         for (int i = 0; i < PAGE_PRE; ++i) {
             const int t = t_lo + i;
             const int page = page_pre[i];
-            if (i == n_early && i < n_tiles && i < NS && t < n_ctx_tiles && page >= 0 && page < p.n_pages) {
+            if (i == n_early && i < n_tiles && i < NS && t < n_ctx_tiles && t < n_final_tiles && page >= 0 && page < p.n_pages) {
                 uint8_t* dK = sKV + (size_t)i * KV_STAGE_BYTES;
                 uint8_t* dV = dK + KV_STAGE_BYTES / 2;
                 mbar_expect_tx(&kv_full[i], KV_STAGE_BYTES);
@@ -643,7 +646,8 @@ int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_c
 }
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
 
-int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv) {
+int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv,
+                        const int32_t* early_len) {
     const dflash_config& c = L.h->cfg;
     if (a.batch == 0 || a.rows == 0) return DFLASH_OK;
     AParams p{};
@@ -654,6 +658,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.rows_valid = std::min(128, a.rows * p.group);
     p.dup = (p.rows_valid <= 64 && 64 % p.group == 0) ? 1 : 0;
     p.early_kv = early_kv ? 1 : 0;
+    p.early_len = early_len;
     const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
     p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;

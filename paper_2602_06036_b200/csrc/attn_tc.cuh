@@ -14,6 +14,10 @@ int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
 // `early_kv`: the layer's cached context was complete before the kernel preceding this one started waiting
 // (true for layers after the first of a draft block: the first layer's wait covered the context
 // projection); its first tiles are then requested before this kernel's own grid dependency resolves.
-int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv = false);
+// `early_len` [device, batch] or nullptr: with early_kv, only pages wholly below this many rows per sequence
+// are requested early (the rows from there on are written inside the same call, by a kernel whose end
+// only this kernel's grid dependency covers).
+int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv = false,
+                        const int32_t* early_len = nullptr);
 
 }  // namespace dflash

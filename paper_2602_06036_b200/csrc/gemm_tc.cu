@@ -1099,7 +1099,10 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KPa
 int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int32_t* phase_done,
                       unsigned long long* const* traces) {
     if (n_phases < 1 || n_phases > MAX_PHASES) return DFLASH_ERR_INVALID_ARG;
-    const int M = phases[0].M;
+    // phases may differ in their row count (the context projection's rows, then a draft block's); the
+    // token tile is sized for the largest
+    int M = 0;
+    for (int i = 0; i < n_phases; ++i) M = std::max(M, phases[i].M);
     if (M <= 0) return DFLASH_OK;
     const int nt = pick_nt(M);
     MParams mp{};
@@ -1117,7 +1120,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     long long min_pairs = -1;
     for (int i = 0; i < n_phases; ++i) {
         const GemmArgs& a = phases[i];
-        if (a.M != M || a.N <= 0) return DFLASH_ERR_INVALID_ARG;
+        if (a.M <= 0 || a.N <= 0) return DFLASH_ERR_INVALID_ARG;
         const int rc = fill_phase(L, a, nt, slabs, mp.ph[i]);
         if (rc != DFLASH_OK) return rc;
         KParams& p = mp.ph[i];

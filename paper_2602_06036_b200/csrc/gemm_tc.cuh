@@ -74,8 +74,8 @@ int64_t gemm_tc_counter_bytes(int M, int N, int n_groups);
 // them non-zero: one launch per zeroing).
 constexpr int GEMM_MAX_PHASES = 4;
 int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done);
-// A chain of contractions over the same rows in ONE launch: phase i+1 reads what phase i's
-// epilogues wrote. traces[i] (may be nullptr) = timeline record of phase i.
+// A chain of contractions in ONE launch: phase i+1 may read what phase i's epilogues wrote. The
+// phases share the token-tile size (chosen for the largest row count) but not the row count. traces[i] (may be nullptr) = timeline record of phase i.
 int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int32_t* phase_done,
                       unsigned long long* const* traces);
 int launch_argmax_finish(const Launch& L, const Top2Entry* top2, int n_tiles, int M, int32_t* ids, float* top1,

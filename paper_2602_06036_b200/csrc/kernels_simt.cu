@@ -638,9 +638,12 @@ int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* t
 
 // Zeroing as a kernel (not a memset) so that it takes part in programmatic dependent launch: its
 // blocks are resident while the previous call's last kernel drains, and the kernel after it chains on.
+// It releases its dependents only after its own wait: every kernel of this call therefore starts after
+// all work queued before the call has ended, which is what lets later kernels of the call read data of
+// earlier calls (the cached context) ahead of their own grid dependency.
 __global__ void __launch_bounds__(256) zero_kernel(uint4* __restrict__ dst, int64_t n16) {
-    ptx::pdl_trigger();
     ptx::pdl_wait();          // the tickets may still be read by the previous kernel
+    ptx::pdl_trigger();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x)
         dst[i] = make_uint4(0, 0, 0, 0);
 }

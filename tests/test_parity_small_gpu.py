@@ -9,7 +9,7 @@ import torch
 
 from oracle import dflash_oracle as orc
 from paper_2602_06036_b200 import synth
-from tests.harness import Case, assert_close, TOL
+from tests.harness import Case, assert_close, assert_ids_match, TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -132,6 +132,59 @@ def test_bf16_random_shapes(seed):
     _check_pool(case)
     got = case.run_draft()
     case.check_draft(got)
+
+
+@pytest.mark.parametrize("name,layers", [("mid", 2), ("mid", 6), ("mid", 7), ("cfg0", 1)])
+def test_context_projection_inside_the_draft_call(name, layers):
+    # draft_block with `ctx`: the projection of the newly committed rows runs inside the call (one chained
+    # launch with the first QKV on the tensor-core path when the layer count allows, separate launches
+    # otherwise). The pool must end up exactly as the separate call leaves it (same kernels, same split of
+    # the same sums) and the block must match the oracle run on the oracle's own updated cache.
+    wl = synth.workload(name)
+    cfg = dataclasses.replace(wl.cfg, n_layers=layers)
+    lens = (5, 70, 190) if name == "mid" else (100,)
+    S, B = len(lens), cfg.block_size
+    max_new = B + 1
+    n_new = torch.tensor([3, max_new, 1][:S], dtype=torch.int32)
+    feats = synth.make_features(cfg, S * max_new, 77, "fused.feats").reshape(S, max_new, cfg.feat_dim)
+    anchors = synth.make_anchors(cfg, S, 77)
+    results = []
+    for fused in (False, True):
+        case = Case(cfg, lens, seed=77)
+        case.project_prefill(oracle=fused)
+        dev = case.device
+        after = (case.ctx_len + n_new.to(dev)).to(torch.int32)
+        ids = torch.zeros((S, B), dtype=torch.int32, device=dev)
+        hidden = torch.zeros((S * B, cfg.d_model), dtype=torch.float32, device=dev)
+        logits = torch.zeros((S * B, cfg.vocab), dtype=torch.float32, device=dev)
+        case.lib.status.zero_()
+        if fused:
+            case.lib.dflash_draft_block(anchors.to(dev), after, max(lens) + max_new, case.page_table, case.pool, ids,
+                                        hidden_out=hidden, logits_out=logits, ctx=(feats.to(dev), n_new.to(dev), case.ctx_len))
+        else:
+            case.lib.dflash_ctx_project(feats.to(dev), n_new.to(dev), case.ctx_len, case.page_table, case.pool)
+            case.lib.dflash_draft_block(anchors.to(dev), after, max(lens) + max_new, case.page_table, case.pool, ids,
+                                        hidden_out=hidden, logits_out=logits)
+        torch.cuda.synchronize()
+        assert int(case.lib.status.item()) == 0
+        results.append((case.pool.float().cpu().numpy(), logits.cpu().numpy(), ids.cpu().numpy(), hidden.cpu().numpy()))
+    (pool_a, log_a, ids_a, hid_a), (pool_b, log_b, ids_b, hid_b) = results
+    assert np.array_equal(pool_a, pool_b)
+    # `case` is the fused one: bring the oracle's cache up to date and draft from it
+    for b in range(S):
+        n = int(n_new[b])
+        pos = np.arange(lens[b], lens[b] + n)
+        K, V = orc.ctx_project(synth.to_numpy_f32(feats[b, :n]), pos, case.w_np, cfg)
+        orc.pool_write(case.pool_np, case.page_table_cpu[b].numpy(), list(pos), K, V, cfg.page_size)
+        case.ctx_lens[b] += n
+    case.anchors_cpu = anchors
+    for b in range(S):
+        ref = case.oracle_draft(b)
+        sl = slice(b * B, (b + 1) * B)
+        for got_h, got_l, got_i, what in ((hid_b, log_b, ids_b, "inside the call"), (hid_a, log_a, ids_a, "separate calls")):
+            assert_close(got_h[sl], ref["hidden"], cfg.dtype, f"hidden seq {b}, {what}")
+            assert_close(got_l[sl], ref["logits"], cfg.dtype, f"logits seq {b}, {what}")
+            assert_ids_match(got_i[b], ref["ids"], ref["margin"], cfg.dtype, f"ids seq {b}, {what}")
 
 
 def test_largest_block_and_empty_calls():
