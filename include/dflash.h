@@ -263,6 +263,9 @@ int32_t dflash_verify_accept_static(dflash_handle* h, const dflash_verify_args* 
  * u * total lies within ~1e-6 (relative) of an interval edge.
  * Scratch: `workspace` of dflash_sample_workspace_bytes(n_logit_rows, vocab) bytes, 256-byte aligned,
  * n_logit_rows = n_rows (dflash_sample_rows) or batch * (2 * gamma + 1) (dflash_verify_accept_sample).
+ * Each call is two launches (segment statistics of every row; then per draw the weights of each segment,
+ * the last segment to finish drawing the index). At most 65535 logit rows per call and gamma <= 64,
+ * else DFLASH_ERR_UNSUPPORTED.
  * Errors: DFLASH_ERR_INVALID_ARG (null pointer, T <= 0, bad dtype or sizes), DFLASH_ERR_WORKSPACE;
  * a draft id outside [0, vocab) counts as rejected and sets DFLASH_DEV_BAD_TOKEN in *dev_status. */
 typedef struct {
@@ -290,7 +293,7 @@ typedef struct {
     int32_t        draft_rows_per_seq; /* stored rows per sequence (>= gamma), e.g. the block size */
     const int32_t* draft_ids;          /* [device] first draft of sequence b at draft_ids + b*draft_stride */
     int32_t        draft_stride;
-    int32_t        batch, gamma, vocab;
+    int32_t        batch, gamma, vocab; /* gamma <= 64, else DFLASH_ERR_UNSUPPORTED               */
     float          temperature;        /* > 0, applied to both distributions                    */
     const float*   u_accept;           /* [device] [batch, gamma] uniforms in [0, 1)            */
     const float*   u_final;            /* [device] [batch] uniform of the emitted token         */
