@@ -640,9 +640,7 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
     if (stride < a->vocab) return DFLASH_ERR_INVALID_ARG;
     Workspace ws;
     DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, rows, &ws));
-    int32_t* ids = a->target_ids_out ? a->target_ids_out : ws.ids;
-    RUN(FAM_ROW_ARGMAX, launch_row_argmax(L, a->logits, a->logits_dtype, stride, rows, a->vocab, ws.seg, ids, nullptr, nullptr));
-    RUN(FAM_ACCEPT, launch_accept(L, *a, ids));
+    RUN(FAM_ROW_ARGMAX, launch_verify_logits(L, *a, stride, ws.seg));
     return DFLASH_OK;
 }
 

@@ -116,6 +116,8 @@ int launch_ctx_scatter(const Launch& L, const float* kv, const dflash_ctx_args& 
 int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t row_stride, int rows,
                       int vocab, float4* seg_scratch, int32_t* ids, float* top1, float* margin);
 int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* target_ids);
+// greedy verification from logits: segment arg-max pass, then per sequence the row merge and the accept rule
+int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t row_stride, float4* seg_scratch);
 int launch_copy_f32(const Launch& L, const float* src, float* dst, int64_t n);
 int launch_zero(const Launch& L, void* dst, int64_t bytes);
 

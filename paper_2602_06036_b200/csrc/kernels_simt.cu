@@ -636,6 +636,73 @@ int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* t
     return DFLASH_OK;
 }
 
+// Greedy verification from logits in two launches: the segment pass above, then one CTA per sequence
+// that merges the segments of its gamma + 1 rows (a warp per row) and applies the accept rule.
+__global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __restrict__ seg, int nseg,
+                                                            const int32_t* __restrict__ draft_ids, int draft_stride, int gamma,
+                                                            const int32_t* __restrict__ ctx_len, int32_t* __restrict__ accept_len,
+                                                            int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
+                                                            int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ target_ids_out) {
+    __shared__ int32_t s_p[65];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
+    const int b = blockIdx.x, lane = threadIdx.x & 31;
+    for (int j = threadIdx.x >> 5; j <= gamma; j += blockDim.x >> 5) {
+        const size_t row = (size_t)b * (gamma + 1) + j;
+        Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
+        for (int i = lane; i < nseg; i += 32) {
+            const float4 e = seg[row * nseg + i];
+            t = top2_merge(t, Top2{e.x, __float_as_int(e.y), e.z});
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            Top2 u;
+            u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+            u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+            u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+            t = top2_merge(t, u);
+        }
+        if (lane == 0) {
+            const int32_t id = (t.i1 == 0x7fffffff) ? 0 : t.i1;      // nothing compared greater than -inf
+            s_p[j] = id;
+            if (target_ids_out) target_ids_out[row] = id;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int32_t* d = draft_ids + (size_t)b * draft_stride;
+        int a = 0;
+        while (a < gamma && d[a] == s_p[a]) ++a;
+        int32_t* o = out_tokens + (size_t)b * (gamma + 1);
+        for (int i = 0; i <= gamma; ++i) o[i] = i < a ? d[i] : (i == a ? s_p[a] : -1);
+        accept_len[b] = a + 1;
+        bonus[b] = s_p[a];
+        new_ctx_len[b] = ctx_len[b] + a + 1;
+    }
+}
+
+int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t row_stride, float4* seg_scratch) {
+    if (a.batch == 0) return DFLASH_OK;
+    if (a.gamma > 64) return DFLASH_ERR_INVALID_ARG;
+    const int rows = a.batch * (a.gamma + 1);
+    const int nseg = row_argmax_segments(rows, a.vocab, L.h->sm_count);
+    const int seg_len = ((a.vocab + nseg - 1) / nseg + 7) / 8 * 8;
+    dim3 grid(nseg, rows);
+    cudaError_t e;
+    if (a.logits_dtype == DFLASH_F32)
+        e = launch_pdl(row_argmax_seg_kernel<float>, grid, dim3(256), 0, L.st, (const float*)a.logits, row_stride, a.vocab, seg_len,
+                       seg_scratch);
+    else
+        e = launch_pdl(row_argmax_seg_kernel<__nv_bfloat16>, grid, dim3(256), 0, L.st, (const __nv_bfloat16*)a.logits, row_stride,
+                       a.vocab, seg_len, seg_scratch);
+    ++g_launches;
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
+    e = launch_pdl(argmax_accept_kernel, dim3(a.batch), dim3(256), 0, L.st, (const float4*)seg_scratch, nseg, a.draft_ids,
+                   a.draft_stride, a.gamma, a.ctx_len, a.accept_len, a.out_tokens, a.bonus, a.new_ctx_len, a.target_ids_out);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
 // Zeroing as a kernel (not a memset) so that it takes part in programmatic dependent launch: its
 // blocks are resident while the previous call's last kernel drains, and the kernel after it chains on.
 // It releases its dependents only after its own wait: every kernel of this call therefore starts after

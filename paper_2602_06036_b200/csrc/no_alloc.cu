@@ -1,7 +1,7 @@
 // Greedy verify/accept from logits for callers that must not allocate device memory.
 //
 // The ordinary entry point (dflash_verify_accept) takes its scratch - the per-segment winners of
-// the row-wise argmax and the row ids - from a workspace the caller allocated. Some callers cannot
+// the row-wise argmax - from a workspace the caller allocated. Some callers cannot
 // do that: a serving engine that has already handed every free byte of the GPU to its KV-cache
 // pool, a latency-critical thread for which cudaMalloc's device-wide synchronisation is off limits,
 // or code that is recording a stream into a CUDA graph. For them the same kernels run here on a
@@ -27,7 +27,6 @@ constexpr int kMaxDevices = 64;
 
 struct StaticScratch {
     float4 seg[kMaxRows * kSegPerRow];   // per-(row, segment) winners of the argmax scan
-    int32_t ids[kMaxRows];               // row-wise argmax of the target logits
 };
 // Device memory owned by the library image. In host code this name is only a handle for the
 // runtime's symbol queries - never a pointer a kernel may be given.
@@ -70,8 +69,5 @@ extern "C" int32_t dflash_verify_accept_static(dflash_handle* h, const dflash_ve
     const int rc = resolve(&s);
     if (rc != DFLASH_OK) return rc;
     Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
-    int32_t* ids = a->target_ids_out ? a->target_ids_out : s->ids;
-    const int r1 = launch_row_argmax(L, a->logits, a->logits_dtype, stride, (int)rows, a->vocab, s->seg, ids, nullptr, nullptr);
-    if (r1 != DFLASH_OK) return r1;
-    return launch_accept(L, *a, ids);
+    return launch_verify_logits(L, *a, stride, s->seg);
 }
