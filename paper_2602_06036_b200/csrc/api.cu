@@ -657,7 +657,7 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     if (attn_tc_supported(h->cfg, a->rows)) {
         Workspace ws;
         DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, a->batch * a->rows, &ws));
-        RUN(FAM_ATTENTION, launch_attention_tc(L, *a, ws.attn_part, ws.attn_counters));
+        RUN(FAM_ATTENTION, launch_attention_tc(L, *a, ws.attn_part, ws.attn_counters, false, nullptr, true));
     } else {
         RUN(FAM_ATTENTION, launch_attention_simt(L, *a));
     }

@@ -647,7 +647,7 @@ int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_c
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
 
 int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv,
-                        const int32_t* early_len) {
+                        const int32_t* early_len, bool first_of_call) {
     const dflash_config& c = L.h->cfg;
     if (a.batch == 0 || a.rows == 0) return DFLASH_OK;
     AParams p{};
@@ -694,8 +694,12 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
         attr_set = true;
     }
     const int grid = a.batch * p.Hkv * p.n_chunks;
-    if (launch_pdl(attn_tc_kernel, dim3(grid), dim3(N_THREADS), (size_t)SMEM_BYTES, L.st, tq, tpool, tkb, tvb, p) != cudaSuccess)
-        return DFLASH_ERR_CUDA;
+    // the kernel reads lengths and page numbers ahead of its grid dependency: as the first kernel of a call
+    // it therefore starts in plain stream order (the caller's previous call may have produced them)
+    const cudaError_t e = first_of_call
+        ? launch_ordered(attn_tc_kernel, dim3(grid), dim3(N_THREADS), (size_t)SMEM_BYTES, L.st, tq, tpool, tkb, tvb, p)
+        : launch_pdl(attn_tc_kernel, dim3(grid), dim3(N_THREADS), (size_t)SMEM_BYTES, L.st, tq, tpool, tkb, tvb, p);
+    if (e != cudaSuccess) return DFLASH_ERR_CUDA;
     ++g_launches;
     if (p.n_chunks > 1) {
         const int rows_valid = p.rows_valid;

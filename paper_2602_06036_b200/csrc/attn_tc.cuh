@@ -17,7 +17,9 @@ int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
 // `early_len` [device, batch] or nullptr: with early_kv, only pages wholly below this many rows per sequence
 // are requested early (the rows from there on are written inside the same call, by a kernel whose end
 // only this kernel's grid dependency covers).
+// `first_of_call`: no kernel of the same call precedes this one; it then starts in plain stream order,
+// because lengths and page numbers (possibly outputs of the caller's previous call) are read early.
 int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv = false,
-                        const int32_t* early_len = nullptr);
+                        const int32_t* early_len = nullptr, bool first_of_call = false);
 
 }  // namespace dflash
