@@ -48,6 +48,18 @@ Pins (tests/test_oracle_sampling.py): the first emitted token is distributed exa
 of the uniform cube, computed cell by cell on small vocabularies), a hand-worked two-token case,
 p = q keeps everything, T -> 0 reduces to the greedy rule, rejected positions only emit tokens
 with p > q.
+
+Training loss of a block (Sec. 4.2 "Loss weighting", Eq. 4; App. A.1 for gamma)   -> loss_weights, block_loss
+  position k = 1 .. B-1 of a block (k = 0 is the clean anchor and carries no loss) has weight
+  w_k = exp(-(k - 1) / gamma); the loss of a block is sum_k w_k CE(logits_k, target_k), CE the plain
+  cross entropy logsumexp(z) - z[target]; its gradient w.r.t. the logits is w_k (softmax(z) - onehot).
+  Readings: the anchor row is skipped (the paper trains the B - 1 masked positions); a negative target
+  marks a position to ignore (a block cut short by the end of the sequence); the normalisation of the
+  sum (by the number of positions or by the sum of weights) is left to the caller: the functions return
+  the weighted sum and the sum of weights.
+Pins (tests/test_oracle_loss.py): w_1 = 1 and the constant ratio exp(-1/gamma), the printed gamma of
+each block size, uniform logits -> ln V, a dominant logit -> 0, gradient rows summing to zero, central
+finite differences of the summed loss, gamma -> infinity = unweighted sum.
 """
 from __future__ import annotations
 
@@ -369,6 +381,42 @@ def target_verify(tokens, L, ctx_K, ctx_V, weights, cfg, tap_layers):
     ids, top1, margin = argmax_top2(logits)
     feats = np.concatenate(taps, axis=-1) if taps else np.zeros((R, 0))
     return dict(logits=logits, ids=ids, margin=margin, feats=feats, K=Ks, V=Vs)
+
+
+# --------------------------------------------------------------------------------------------
+# training loss of a block (Sec. 4.2 "Loss weighting", Eq. 4)
+# --------------------------------------------------------------------------------------------
+def loss_weights(B, gamma):
+    """w[k], k = 0 .. B-1: 0 for the anchor row, exp(-(k-1)/gamma) for the predicted positions (Eq. 4)."""
+    w = np.zeros((B,), dtype=F64)
+    for k in range(1, B):
+        w[k] = np.exp(-(k - 1) / F64(gamma))
+    return w
+
+
+def block_loss(logits, targets, gamma, want_grad=True):
+    """logits [B, V] of one block (row 0 = anchor), targets [B] (entry 0 unused; negative = ignore).
+    Returns dict(row_loss [B] = w_k * CE_k, loss = their sum, weight = sum of the weights that count,
+    grad [B, V] = d loss / d logits)."""
+    z = _f64(logits)
+    B, V = z.shape
+    w = loss_weights(B, gamma)
+    row_loss = np.zeros((B,), dtype=F64)
+    grad = np.zeros((B, V), dtype=F64) if want_grad else None
+    weight = 0.0
+    for k in range(1, B):
+        t = int(targets[k])
+        if t < 0:
+            continue
+        m = np.max(z[k])
+        e = np.exp(z[k] - m)
+        lse = m + np.log(np.sum(e))
+        row_loss[k] = w[k] * (lse - z[k, t])
+        weight += w[k]
+        if want_grad:
+            grad[k] = w[k] * (e / np.sum(e))
+            grad[k, t] -= w[k]
+    return dict(row_loss=row_loss, loss=float(np.sum(row_loss)), weight=float(weight), grad=grad)
 
 
 # --------------------------------------------------------------------------------------------
