@@ -367,6 +367,19 @@ def run_kernel_only(args, step, device):
         alg = algorithmic_bytes(cfg, wl.ctx_lens, 0)
         nbytes = n_layers * (alg["gemm_qkv"] + alg["gemm_o"] + alg["gemm_gateup"] + alg["gemm_down"] + alg["attention"]) + \
             alg["lmhead_argmax"]
+    elif args.kernel == "block_loss":
+        # Training side: the position-weighted cross entropy with its gradient over the blocks of one training
+        # sequence (512 anchors per sequence, App. A.1; --loss-blocks for a smaller capture), bf16 logits of the
+        # drafter's vocabulary in, bf16 gradient out. Algorithmic bytes: logits read once + gradient written once.
+        nb = args.loss_blocks
+        gamma = {16: 7.0, 10: 5.0, 8: 4.0}.get(B, 7.0)
+        z = torch.empty((nb, B, cfg.vocab), dtype=torch.bfloat16, device=device).normal_(0.0, 3.0)
+        t = torch.randint(0, cfg.vocab, (nb, B), dtype=torch.int32, device=device)
+        dz = torch.empty_like(z)
+        row_loss = torch.zeros(nb * B, dtype=torch.float32, device=device)
+        sums = torch.zeros(2, dtype=torch.float32, device=device)
+        fn = lambda: step.lib.dflash_block_loss(z, t, gamma, row_loss, sums, dz, grad_scale=1.0 / (nb * (B - 1)))
+        nbytes = 2 * z.numel() * 2
     elif args.kernel == "lmhead":
         hid = torch.randn(S * B, cfg.d_model, device=device).to(cfg.torch_dtype)
         ids = torch.zeros(S * B, dtype=torch.int32, device=device)
@@ -395,8 +408,9 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify"],
+    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify", "block_loss"],
                     help="run one building block alone (for profiler captures) instead of the step")
+    ap.add_argument("--loss-blocks", type=int, default=512, help="--kernel block_loss: blocks (of block_size rows) per call")
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="> 0: drafts are drawn from the draft's logits and verified by speculative sampling (default: greedy)")

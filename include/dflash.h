@@ -351,6 +351,36 @@ typedef struct {
 } dflash_lmhead_args;
 int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a /*[host]*/, void* stream);
 
+/* ---- training side: position-weighted cross entropy of draft blocks (Sec. 4.2 "Loss weighting", Eq. 4) ----
+ * Row k of a block (k = 0 .. block_rows-1) holds the logits of block position k; position 0 is the clean
+ * anchor and carries no loss, position k >= 1 has weight w_k = exp(-(k-1)/gamma) (gamma = 7 / 5 / 4 for
+ * blocks of 16 / 10 / 8, App. A.1). Per row:  row_loss = w_k * (logsumexp(z) - z[target]);  optionally the
+ * gradient  dlogits = grad_scale * w_k * (softmax(z) - onehot(target))  (zeros for rows without loss).
+ * A negative target marks a position without loss (a block cut short by the end of its sequence); a target
+ * >= vocab is treated the same and sets DFLASH_DEV_BAD_TOKEN. loss_sum = {sum of row_loss, sum of the w_k
+ * that count}, added in double in a fixed order: the caller divides by whichever normaliser it trains with
+ * (the paper does not state one) and passes the matching grad_scale.
+ * Arithmetic: fp32 per row (maximum, sum of exponentials, logarithm). A CTA reads its row twice in a row
+ * (statistics, then gradient), the second time from L2: HBM traffic is one read of the logits plus one
+ * write of the gradient. `dlogits` may alias `logits` when dtype and stride agree. No scratch memory.
+ * Errors: DFLASH_ERR_INVALID_ARG (null pointer, gamma <= 0, bad dtype or sizes). */
+typedef struct {
+    const void*    logits;             /* [device] [n_blocks * block_rows, vocab]                       */
+    int32_t        logits_dtype;       /* DFLASH_F32 | DFLASH_BF16                                      */
+    int64_t        row_stride;         /* elements (0 = vocab)                                          */
+    int32_t        n_blocks, block_rows, vocab;
+    const int32_t* targets;            /* [device] [n_blocks, block_rows]; entry 0 of a block is unused */
+    float          gamma;              /* > 0                                                           */
+    float*         row_loss;           /* [device] out [n_blocks * block_rows]                          */
+    float*         loss_sum;           /* [device] out [2]; may be NULL                                 */
+    void*          dlogits;            /* [device] out [n_blocks * block_rows, vocab]; may be NULL      */
+    int32_t        dlogits_dtype;      /* DFLASH_F32 | DFLASH_BF16                                      */
+    int64_t        dlogits_row_stride; /* elements (0 = vocab)                                          */
+    float          grad_scale;
+    int32_t*       dev_status;         /* [device] may be NULL                                          */
+} dflash_block_loss_args;
+int32_t dflash_block_loss(dflash_handle* h, const dflash_block_loss_args* a /*[host]*/, void* stream);
+
 /* ---- per-kernel-family timing (host-side CUDA events; off by default) ----
  * While enabled, every launch the library issues is bracketed by an event pair on the caller's
  * stream. dflash_profile_read synchronises on the last event, adds the elapsed milliseconds and the

@@ -28,7 +28,7 @@ EXPORTS = (
     "dflash_lmhead_argmax", "dflash_status_string", "dflash_launch_count", "dflash_profile_enable",
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
     "dflash_verify_accept_static", "dflash_sample_rows", "dflash_verify_accept_sample",
-    "dflash_sample_workspace_bytes", "dflash_target_verify",
+    "dflash_sample_workspace_bytes", "dflash_target_verify", "dflash_block_loss",
 )
 N_FAMILIES = 15
 
@@ -84,6 +84,14 @@ class TargetArgs(C.Structure):
                 ("dev_status", C.c_void_p)]
 
 
+class BlockLossArgs(C.Structure):
+    _fields_ = [("logits", C.c_void_p), ("logits_dtype", C.c_int32), ("row_stride", C.c_int64),
+                ("n_blocks", C.c_int32), ("block_rows", C.c_int32), ("vocab", C.c_int32), ("targets", C.c_void_p),
+                ("gamma", C.c_float), ("row_loss", C.c_void_p), ("loss_sum", C.c_void_p), ("dlogits", C.c_void_p),
+                ("dlogits_dtype", C.c_int32), ("dlogits_row_stride", C.c_int64), ("grad_scale", C.c_float),
+                ("dev_status", C.c_void_p)]
+
+
 class SampleArgs(C.Structure):
     _fields_ = [("logits", C.c_void_p), ("logits_dtype", C.c_int32), ("row_stride", C.c_int64),
                 ("n_rows", C.c_int32), ("vocab", C.c_int32), ("temperature", C.c_float), ("u", C.c_void_p),
@@ -136,7 +144,8 @@ def load():
     for name, st in (("dflash_ctx_project", CtxArgs), ("dflash_draft_block", DraftArgs),
                      ("dflash_verify_accept", VerifyArgs), ("dflash_verify_accept_static", VerifyArgs), ("dflash_block_attention", AttnArgs),
                      ("dflash_lmhead_argmax", LmHeadArgs), ("dflash_sample_rows", SampleArgs),
-                     ("dflash_verify_accept_sample", VerifySampleArgs), ("dflash_target_verify", TargetArgs)):
+                     ("dflash_verify_accept_sample", VerifySampleArgs), ("dflash_target_verify", TargetArgs),
+                     ("dflash_block_loss", BlockLossArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(st), C.c_void_p]
         fn.restype = C.c_int32
@@ -371,6 +380,17 @@ class DFlash:
             ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
             self._samp_ws = ws
         return ws
+
+    def dflash_block_loss(self, logits, targets, gamma, row_loss, loss_sum=None, dlogits=None, grad_scale=1.0, stream=None):
+        """Position-weighted cross entropy of draft blocks. logits [n_blocks, B, V] (row 0 of a block = anchor, no
+        loss), targets [n_blocks, B] int32 (< 0: ignored). row_loss [n_blocks * B] fp32; loss_sum [2] fp32;
+        dlogits like logits (fp32 or bf16) = grad_scale * w_k * (softmax - onehot)."""
+        nb, B, V = logits.shape
+        a = BlockLossArgs(_ptr(logits), F32 if logits.dtype == torch.float32 else BF16, logits.stride(1), nb, B, V,
+                          _ptr(targets), float(gamma), _ptr(row_loss), _ptr(loss_sum), _ptr(dlogits),
+                          (F32 if dlogits.dtype == torch.float32 else BF16) if dlogits is not None else F32,
+                          dlogits.stride(1) if dlogits is not None else 0, float(grad_scale), _ptr(self.status))
+        _check(self.lib.dflash_block_loss(self.h, C.byref(a), _stream(stream)))
 
     def dflash_sample_rows(self, logits, temperature, u, ids, prob=None, stream=None):
         """ids[m] = inverse-CDF draw from softmax(logits[m] / T) with the uniform u[m]."""
