@@ -106,6 +106,39 @@ def test_verify_args_validated_on_the_host(lib):
     lib.dflash_destroy(h)
 
 
+def test_sampling_and_loss_args_validated_on_the_host(lib):
+    # every refusal below happens before the first CUDA call
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_cfg()), C.byref(h)) == 0
+    s = binding.SampleArgs()
+    s.n_rows, s.vocab, s.temperature = 4, 1000, 0.0
+    assert lib.dflash_sample_rows(h, C.byref(s), None) == -1           # T must be > 0
+    s.temperature, s.n_rows = 1.0, 0
+    assert lib.dflash_sample_rows(h, C.byref(s), None) == 0            # nothing to do
+    s.n_rows = 70000
+    assert lib.dflash_sample_rows(h, C.byref(s), None) == -2           # more rows than one launch takes
+    assert lib.dflash_sample_workspace_bytes(16, 151936) % 256 == 0 and lib.dflash_sample_workspace_bytes(-1, 10) < 0
+    v = binding.VerifySampleArgs()
+    v.batch, v.gamma, v.vocab, v.temperature = 1, 65, 1000, 1.0
+    v.draft_rows_per_seq = v.draft_stride = 65
+    for name in ("target_logits", "draft_logits", "draft_ids", "u_accept", "u_final", "ctx_len", "accept_len", "out_tokens",
+                 "bonus", "new_ctx_len"):
+        setattr(v, name, 256)                                          # non-null; never dereferenced on the host
+    assert lib.dflash_verify_accept_sample(h, C.byref(v), None) == -2  # gamma above 64
+    v.batch = 0
+    assert lib.dflash_verify_accept_sample(h, C.byref(v), None) == 0
+    b = binding.BlockLossArgs()
+    b.n_blocks, b.block_rows, b.vocab, b.gamma = 2, 16, 1000, 0.0
+    assert lib.dflash_block_loss(h, C.byref(b), None) == -1            # gamma must be > 0
+    b.gamma, b.logits_dtype = 7.0, 5
+    assert lib.dflash_block_loss(h, C.byref(b), None) == -1            # unknown dtype
+    b.logits_dtype = 0
+    assert lib.dflash_block_loss(h, C.byref(b), None) == -1            # null pointers
+    b.n_blocks = 0
+    assert lib.dflash_block_loss(h, C.byref(b), None) == 0             # nothing to do
+    lib.dflash_destroy(h)
+
+
 def test_status_strings(lib):
     seen = {lib.dflash_status_string(c).decode() for c in (0, -1, -2, -3, -4, -5)}
     assert len(seen) == 6 and lib.dflash_status_string(-99).decode() == "unknown status"
