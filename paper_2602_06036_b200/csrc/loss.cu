@@ -326,9 +326,8 @@ cudaError_t launch_cluster(const LossParams& p, int part, int sm_count, cudaStre
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    const int n_clusters = std::max(1, std::min(p.n_rows, sm_count * CLU_CTAS_PER_SM / CS));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_clusters * CS);
+    cfg.gridDim = dim3(sm_count / CS * CS);
     cfg.blockDim = dim3(CLU_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -339,6 +338,16 @@ cudaError_t launch_cluster(const LossParams& p, int part, int sm_count, cudaStre
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // as many clusters as can be resident at once (an SM left over in a GPC cannot host half a cluster):
+    // the clusters are persistent, so one that had to wait for a free pair of SMs would run after all the others
+    static int resident = 0;
+    if (resident == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, block_loss_cluster_kernel<IN, CS>, &cfg) != cudaSuccess || n < 1) n = sm_count / CS;
+        resident = n;
+    }
+    const int n_clusters = std::max(1, std::min(p.n_rows, std::min(resident, sm_count * CLU_CTAS_PER_SM / CS)));
+    cfg.gridDim = dim3(n_clusters * CS);
     return cudaLaunchKernelEx(&cfg, block_loss_cluster_kernel<IN, CS>, p, part);
 }
 
