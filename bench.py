@@ -216,14 +216,16 @@ class Step:
     def step_e2e(self):
         # The verify logits are only needed at the end of the step: their host-to-device copy runs on a
         # side stream next to the context projection and the draft (a fork/join inside the captured graph).
+        # The small inputs the draft starts from go first; the logits follow on the side stream only after them, so
+        # the 5 MB copy cannot sit in front of the features on the host-to-device path.
         cur = torch.cuda.current_stream()
         if self.side is None:
             self.side = torch.cuda.Stream()
+        self.e_feats.copy_(self.h_feats, non_blocking=True)
+        self.e_anchor.copy_(self.h_anchor, non_blocking=True)
         self.side.wait_stream(cur)
         with torch.cuda.stream(self.side):
             self.e_logits.copy_(self.h_logits, non_blocking=True)
-        self.e_feats.copy_(self.h_feats, non_blocking=True)
-        self.e_anchor.copy_(self.h_anchor, non_blocking=True)
         self.run_draft(self.e_feats, self.e_anchor)
         cur.wait_stream(self.side)
         self.run_verify(self.e_logits)
