@@ -154,8 +154,15 @@ class Step:
         self.d_feats = self.h_feats.to(device)
         self.d_anchor = self.h_anchor.to(device)
         self.d_logits = self.h_logits.to(device)
-        self.e_feats = torch.empty_like(self.d_feats)
-        self.e_anchor = torch.empty_like(self.d_anchor)
+        # end-to-end staging: features and anchors share one pinned host buffer and one device buffer (one copy)
+        nf = self.h_feats.numel() * self.h_feats.element_size()
+        nf_pad = (nf + 255) // 256 * 256
+        self.h_in = torch.zeros(nf_pad + 4 * S, dtype=torch.uint8).pin_memory()
+        self.h_in[:nf].copy_(self.h_feats.view(torch.uint8).reshape(-1))
+        self.h_in[nf_pad:].copy_(self.h_anchor.view(torch.uint8).reshape(-1))
+        self.e_in = torch.empty(nf_pad + 4 * S, dtype=torch.uint8, device=device)
+        self.e_feats = self.e_in[:nf].view(cfg.torch_dtype).view(S, g + 1, cfg.feat_dim)
+        self.e_anchor = self.e_in[nf_pad:].view(torch.int32)
         self.e_logits = torch.empty_like(self.d_logits)
         self.n_new = (planted + 1).to(torch.int32).to(device)      # rows committed by the previous cycle
         # those rows are the last n_new of the context the block attends over: the step projects them, then drafts
@@ -221,8 +228,7 @@ class Step:
         cur = torch.cuda.current_stream()
         if self.side is None:
             self.side = torch.cuda.Stream()
-        self.e_feats.copy_(self.h_feats, non_blocking=True)
-        self.e_anchor.copy_(self.h_anchor, non_blocking=True)
+        self.e_in.copy_(self.h_in, non_blocking=True)
         self.side.wait_stream(cur)
         with torch.cuda.stream(self.side):
             self.e_logits.copy_(self.h_logits, non_blocking=True)
@@ -232,7 +238,7 @@ class Step:
         self.h_out.copy_(self.d_out, non_blocking=True)
 
     def e2e_bytes(self):
-        h2d = self.h_feats.numel() * self.h_feats.element_size() + self.h_anchor.numel() * 4 + \
+        h2d = self.h_in.numel() + \
             self.h_logits.numel() * self.h_logits.element_size()
         return h2d, self.h_out.numel() * 4
 
