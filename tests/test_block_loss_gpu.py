@@ -23,6 +23,9 @@ def _case(nb, B, V, seed, dtype, scale=3.0):
     (5, 8, 5003, 4.0, torch.bfloat16, torch.float32),          # odd vocabulary: rows lose 16-byte alignment
     (4, 16, 32000, 7.0, torch.float32, torch.bfloat16),
     (1, 1, 300, 7.0, torch.float32, torch.float32),            # a block of the anchor alone: no loss at all
+    (3, 4, 16, 4.0, torch.bfloat16, torch.float32),            # one 16-byte vector per CTA of the cluster
+    (2, 8, 8, 4.0, torch.bfloat16, torch.bfloat16),            # the second CTA of the cluster holds nothing
+    (200, 2, 4096, 4.0, torch.float32, torch.float32),         # more rows than clusters, every other row an anchor
 ])
 def test_block_loss_matches_oracle(nb, B, V, gamma, in_dtype, out_dtype):
     dev = torch.device("cuda:0")
