@@ -46,6 +46,42 @@ def test_cfg1_end_to_end(model):
     n_sure = case.check_draft(got)
     assert n_sure >= 4
 
+def test_cfg1_step_as_benchmarked(model):
+    # The step bench.py times: the rows the previous cycle committed (the last 17 of the 2048 the block attends
+    # over) are projected INSIDE the draft call (one chained launch with the first QKV), then the block is drafted.
+    wl = synth.workload("cfg1")
+    cfg = CFG
+    case = _case(model, wl.ctx_lens, seed=3)
+    case.project_prefill(oracle=True)
+    dev = case.device
+    B, n = cfg.block_size, cfg.block_size + 1
+    L = wl.ctx_lens[0]
+    feats = synth.make_features(cfg, n, 3, "step.feats").reshape(1, n, cfg.feat_dim)
+    anchors = synth.make_anchors(cfg, 1, 3)
+    ids = torch.zeros((1, B), dtype=torch.int32, device=dev)
+    hidden = torch.zeros((B, cfg.d_model), dtype=torch.float32, device=dev)
+    logits = torch.zeros((B, cfg.vocab), dtype=torch.float32, device=dev)
+    before = torch.tensor([L - n], dtype=torch.int32, device=dev)
+    case.lib.status.zero_()
+    case.lib.dflash_draft_block(anchors.to(dev), case.ctx_len, L, case.page_table, case.pool, ids, hidden_out=hidden,
+                                logits_out=logits, ctx=(feats.to(dev), torch.tensor([n], dtype=torch.int32, device=dev), before))
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) == 0
+    pos = np.arange(L - n, L)
+    K, V = orc.ctx_project(synth.to_numpy_f32(feats[0]), pos, case.w_np, cfg)
+    orc.pool_write(case.pool_np, case.page_table_cpu[0].numpy(), list(pos), K, V, cfg.page_size)
+    got_pool = case.pool.float().cpu().numpy()
+    for i in range(cfg.n_layers):
+        gk, gv = orc.pool_read(got_pool, case.page_table_cpu[0].numpy(), L, i, cfg.page_size)
+        rk, rv = orc.pool_read(case.pool_np, case.page_table_cpu[0].numpy(), L, i, cfg.page_size)
+        assert_close(gk[L - n:], rk[L - n:], "bf16", f"new ctx K layer {i}")
+        assert_close(gv[L - n:], rv[L - n:], "bf16", f"new ctx V layer {i}")
+    case.anchors_cpu = anchors
+    ref = case.oracle_draft(0)
+    assert_close(hidden.cpu().numpy(), ref["hidden"], "bf16", "hidden")
+    assert_close(logits.cpu().numpy(), ref["logits"], "bf16", "logits")
+    assert_ids_match(ids.cpu().numpy()[0], ref["ids"], ref["margin"], "bf16", "draft ids")
+
 
 def test_cfg2_ragged_batch_and_accept_from_logits(model):
     wl = synth.workload("cfg2")
