@@ -187,6 +187,59 @@ def test_context_projection_inside_the_draft_call(name, layers):
             assert_ids_match(got_i[b], ref["ids"], ref["margin"], cfg.dtype, f"ids seq {b}, {what}")
 
 
+def test_step_replayed_as_a_cuda_graph():
+    # The benchmark replays one captured step: context projection inside the draft call, then verification from
+    # logits. A replay must give, bit for bit, what the same calls give when launched one by one.
+    cfg = synth.MID
+    lens = (5, 70, 190)
+    S, B = len(lens), cfg.block_size
+    case = Case(cfg, lens, seed=41)
+    case.project_prefill(oracle=False)
+    dev = case.device
+    n_new = torch.tensor([3, B + 1, 1], dtype=torch.int32, device=dev)
+    feats = synth.make_features(cfg, S * (B + 1), 41, "graph.feats").reshape(S, B + 1, cfg.feat_dim).to(dev)
+    anchors = synth.make_anchors(cfg, S, 41).to(dev)
+    after = (case.ctx_len + n_new).to(torch.int32)
+    tlog, _, _ = synth.make_verify_case(S, B, cfg.vocab, 0.5, 41, cfg.torch_dtype)
+    tlog = tlog.to(dev)
+    ids = torch.zeros((S, B), dtype=torch.int32, device=dev)
+    logits = torch.zeros((S * B, cfg.vocab), dtype=torch.float32, device=dev)
+    tau = torch.zeros(S, dtype=torch.int32, device=dev)
+    out = torch.zeros((S, B + 1), dtype=torch.int32, device=dev)
+    bonus = torch.zeros(S, dtype=torch.int32, device=dev)
+    new_len = torch.zeros(S, dtype=torch.int32, device=dev)
+    pool0 = case.pool.clone()
+
+    def step():
+        case.lib.dflash_draft_block(anchors, after, max(lens) + B + 1, case.page_table, case.pool, ids, logits_out=logits,
+                                    ctx=(feats, n_new, case.ctx_len))
+        case.lib.dflash_verify_accept(ids, B, B, after, tau, out, bonus, new_len, logits=tlog)
+
+    def snapshot():
+        torch.cuda.synchronize()
+        assert int(case.lib.status.item()) == 0
+        return [t.clone() for t in (case.pool, ids, logits, tau, out, bonus, new_len)]
+
+    case.lib.status.zero_()
+    step()
+    eager = snapshot()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):          # capture on a side stream, after the eager run has sized every buffer
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        case.pool.copy_(pool0)
+        for t in (ids, logits, tau, out, bonus, new_len):
+            t.zero_()
+        g.replay()
+        got = snapshot()
+        for a, b in zip(eager, got):
+            assert torch.equal(a, b)
+
+
 def test_largest_block_and_empty_calls():
     # block size 32 (the largest the library takes): 32 rows x 4 q heads fill the 128-row attention operand
     cfg = dataclasses.replace(synth.MID, block_size=32)
