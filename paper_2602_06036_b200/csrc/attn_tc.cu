@@ -687,11 +687,12 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
         if (!tmap_encode_bf16(&tkb, a.k_blk, 2, dims, str, box)) return DFLASH_ERR_CUDA;
         if (!tmap_encode_bf16(&tvb, a.v_blk, 2, dims, str, box)) return DFLASH_ERR_CUDA;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = current_device_slot();
+    if (dev < 0 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return DFLASH_ERR_CUDA;
-        attr_set = true;
+        if (dev >= 0) attr_set[dev] = true;
     }
     const int grid = a.batch * p.Hkv * p.n_chunks;
     // the kernel reads lengths and page numbers ahead of its grid dependency: as the first kernel of a call

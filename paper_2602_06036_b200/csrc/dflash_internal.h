@@ -41,6 +41,15 @@ namespace dflash {
 // Counts kernel launches issued by the library (reported by dflash_launch_count).
 extern long long g_launches;
 
+// Per-device memo for settings a launcher makes once per (kernel, device): function attributes are per
+// device, so a process that drives several GPUs must make them on each. Indexed by the current device.
+constexpr int MAX_DEVICES = 64;
+inline int current_device_slot() {
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= MAX_DEVICES) return -1;
+    return d;
+}
+
 inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 inline int elem_size(int dtype) { return dtype == DFLASH_F32 ? 4 : 2; }
 

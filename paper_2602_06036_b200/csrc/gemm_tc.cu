@@ -1037,12 +1037,13 @@ int pick_nt(int M) {
 
 template <int NT, int SL, bool QKN>
 int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
-    static bool attr_set = false;
+    static bool attr_set[MAX_DEVICES] = {};
     const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
-    if (!attr_set) {
+    const int dev = current_device_slot();
+    if (dev < 0 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL, QKN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
-        attr_set = true;
+        if (dev >= 0) attr_set[dev] = true;
     }
     const cudaError_t e = launch_pdl(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
     ++g_launches;

@@ -319,12 +319,15 @@ int cluster_size_for(int vocab, int es) {
 template <typename IN, int CS>
 cudaError_t launch_cluster(const LossParams& p, int part, int sm_count, cudaStream_t st) {
     const size_t smem = (size_t)part * sizeof(IN);
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[MAX_DEVICES] = {};
+    static int resident[MAX_DEVICES] = {};
+    const int dev = current_device_slot();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         const cudaError_t e = cudaFuncSetAttribute(block_loss_cluster_kernel<IN, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    CLU_PART_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sm_count / CS * CS);
@@ -340,13 +343,12 @@ cudaError_t launch_cluster(const LossParams& p, int part, int sm_count, cudaStre
     cfg.numAttrs = 1;
     // as many clusters as can be resident at once (an SM left over in a GPC cannot host half a cluster):
     // the clusters are persistent, so one that had to wait for a free pair of SMs would run after all the others
-    static int resident = 0;
-    if (resident == 0) {
+    if (resident[dev] == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, block_loss_cluster_kernel<IN, CS>, &cfg) != cudaSuccess || n < 1) n = sm_count / CS;
-        resident = n;
+        resident[dev] = n;
     }
-    const int n_clusters = std::max(1, std::min(p.n_rows, std::min(resident, sm_count * CLU_CTAS_PER_SM / CS)));
+    const int n_clusters = std::max(1, std::min(p.n_rows, std::min(resident[dev], sm_count * CLU_CTAS_PER_SM / CS)));
     cfg.gridDim = dim3(n_clusters * CS);
     return cudaLaunchKernelEx(&cfg, block_loss_cluster_kernel<IN, CS>, p, part);
 }
