@@ -187,6 +187,54 @@ def test_context_projection_inside_the_draft_call(name, layers):
             assert_ids_match(got_i[b], ref["ids"], ref["margin"], cfg.dtype, f"ids seq {b}, {what}")
 
 
+@pytest.mark.parametrize("S", [9, 33])
+def test_context_projection_inside_the_draft_call_for_batches(S):
+    # 9 sequences: 153 projected rows and 144 block rows in one 256-column token tile; 33 sequences: 561 and 528
+    # rows over three and two token tiles. Pool against the separate call (bit-equal), sampled blocks against the oracle.
+    cfg = synth.MID
+    B = cfg.block_size
+    g = synth.substream(53, "fusedbatch.lens")
+    lens = [int(v) for v in torch.randint(0, 200, (S,), generator=g)]
+    n_new = torch.randint(0, B + 2, (S,), generator=g, dtype=torch.int32)
+    n_new[0], n_new[1] = B + 1, 0
+    feats = synth.make_features(cfg, S * (B + 1), 53, "fusedbatch.feats").reshape(S, B + 1, cfg.feat_dim)
+    anchors = synth.make_anchors(cfg, S, 53)
+    results = []
+    for fused in (False, True):
+        case = Case(cfg, lens, seed=53)
+        case.project_prefill(oracle=fused)
+        dev = case.device
+        after = (case.ctx_len + n_new.to(dev)).to(torch.int32)
+        ids = torch.zeros((S, B), dtype=torch.int32, device=dev)
+        hidden = torch.zeros((S * B, cfg.d_model), dtype=torch.float32, device=dev)
+        case.lib.status.zero_()
+        if fused:
+            case.lib.dflash_draft_block(anchors.to(dev), after, max(lens) + B + 1, case.page_table, case.pool, ids, hidden_out=hidden,
+                                        ctx=(feats.to(dev), n_new.to(dev), case.ctx_len))
+        else:
+            case.lib.dflash_ctx_project(feats.to(dev), n_new.to(dev), case.ctx_len, case.page_table, case.pool)
+            case.lib.dflash_draft_block(anchors.to(dev), after, max(lens) + B + 1, case.page_table, case.pool, ids, hidden_out=hidden)
+        torch.cuda.synchronize()
+        assert int(case.lib.status.item()) == 0
+        results.append((case.pool.float().cpu().numpy(), ids.cpu().numpy(), hidden.cpu().numpy()))
+    (pool_a, ids_a, hid_a), (pool_b, ids_b, hid_b) = results
+    assert np.array_equal(pool_a, pool_b)
+    for b in range(S):
+        n = int(n_new[b])
+        pos = np.arange(lens[b], lens[b] + n)
+        if n:
+            K, V = orc.ctx_project(synth.to_numpy_f32(feats[b, :n]), pos, case.w_np, cfg)
+            orc.pool_write(case.pool_np, case.page_table_cpu[b].numpy(), list(pos), K, V, cfg.page_size)
+        case.ctx_lens[b] += n
+    case.anchors_cpu = anchors
+    for b in (0, 1, S // 2, S - 1):
+        ref = case.oracle_draft(b)
+        sl = slice(b * B, (b + 1) * B)
+        assert_close(hid_b[sl], ref["hidden"], cfg.dtype, f"hidden seq {b}, inside the call")
+        assert_close(hid_a[sl], ref["hidden"], cfg.dtype, f"hidden seq {b}, separate calls")
+        assert_ids_match(ids_b[b], ref["ids"], ref["margin"], cfg.dtype, f"ids seq {b}")
+
+
 def test_step_replayed_as_a_cuda_graph():
     # The benchmark replays one captured step: context projection inside the draft call, then verification from
     # logits. A replay must give, bit for bit, what the same calls give when launched one by one.
