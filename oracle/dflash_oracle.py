@@ -26,7 +26,10 @@ Pins (tests/test_oracle_*.py): closed forms for RMSNorm / SiLU / RoPE, the App. 
 figures for the layouts, brute-force loops for attention and matmul on tiny inputs, attention
 special cases (uniform keys -> mean of V, dominant key -> its V, permutation invariance, GQA =
 replicated MHA, causal last row = full last row), accept-rule enumeration of all match patterns,
-and equality of speculative output with plain greedy decoding of a toy target.
+equality of speculative output with plain greedy decoding of a toy target, and for one layer
+(tests/test_oracle_draft_block.py) the SwiGLU half written out with scalar loops (SiLU on the gate
+branch, gate 0 closes a unit, a large gate passes the up value), the first norm feeding q, k, v and
+the second norm reading the hidden after the attention residual with its own gain.
 The composed forward `draft_block` has no external value to compare with: parity unpinned beyond
 its parts (each step above is pinned separately).
 

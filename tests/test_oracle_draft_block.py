@@ -68,3 +68,175 @@ def test_empty_context_is_allowed():
     empty = [np.zeros((0, cfg.n_kv_heads, cfg.head_dim))] * cfg.n_layers
     out = orc.draft_block(0, 0, empty, empty, w, cfg)
     assert out["ids"].shape == (cfg.block_size,) and np.all(np.isfinite(out["hidden"]))
+
+
+# ---------------------------------------------------------------------------------------------
+# one layer: which normalised hidden feeds what, and the SwiGLU feed-forward half
+# ---------------------------------------------------------------------------------------------
+class _LayerShape:
+    """A layer small enough to write out by hand: no rotation, no per-head norm."""
+    n_q_heads, n_kv_heads, head_dim = 2, 1, 2
+    q_dim = 4
+    use_rope, qk_norm, rope_theta = 0, 0, 1.0e6
+    rms_eps = 1e-6
+    softmax_scale = 2 ** -0.5
+
+
+def _blank_layer(D, F, rng=None):
+    cfg = _LayerShape()
+    z = lambda *s: np.zeros(s) if rng is None else rng.standard_normal(s)
+    lw = {"g1": np.ones(D), "g2": np.ones(D), "W_q": z(cfg.q_dim, D), "W_k": z(2, D), "W_v": z(2, D),
+          "W_o": np.zeros((D, cfg.q_dim)), "W_gate": np.zeros((F, D)), "W_up": np.zeros((F, D)),
+          "W_down": np.zeros((D, F))}
+    return cfg, lw
+
+
+def _no_ctx():
+    return np.zeros((0, 1, 2)), np.zeros((0, 1, 2))
+
+
+def test_feed_forward_half_gates_the_up_branch_with_silu_of_the_gate_branch():
+    # W_o = 0 removes the attention half. One FFN unit j reads normalised feature 0 through its gate
+    # and normalised feature 1 through its up projection and writes to output feature 2; eps = 0 and a
+    # row of mean square 1 make the normalised hidden equal to the row itself.
+    D, F = 4, 3
+    cfg, lw = _blank_layer(D, F)
+    cfg.rms_eps = 0.0
+    lw["W_gate"][1, 0] = 1.0
+    lw["W_up"][1, 1] = 1.0
+    lw["W_down"][2, 1] = 1.0
+    kc, vc = _no_ctx()
+
+    def run(gate_in, up_in):
+        # remaining two features chosen so that the mean square is exactly 1
+        rest = 4.0 - gate_in ** 2 - up_in ** 2
+        x = np.array([[gate_in, up_in, 0.0, np.sqrt(rest)]])
+        out = orc.draft_layer(x, lw, kc, vc, np.zeros(1), cfg)
+        return (out - x)[0]
+
+    d = run(0.0, 1.25)                      # gate pre-activation 0 -> silu(0) = 0 closes the unit
+    np.testing.assert_array_equal(d, np.zeros(4))
+    d = run(1.5, 0.0)                       # up branch 0 -> nothing passes, whatever the gate
+    np.testing.assert_array_equal(d, np.zeros(4))
+    # a large positive gate lets the up value through unchanged (silu(g) -> g, so scale the up weight by 1/g)
+    lw["W_gate"][1, 0] = 40.0
+    lw["W_up"][1, 1] = 1.0 / 60.0           # gate pre-activation = 40 * 1.5 = 60
+    d = run(1.5, 0.7)
+    np.testing.assert_allclose(d, [0.0, 0.0, 0.7, 0.0], rtol=1e-12, atol=1e-15)
+    # the SiLU sits on the GATE branch: a large negative gate closes the unit, a large negative up does not
+    lw["W_gate"][1, 0] = -40.0
+    assert abs(run(1.5, 0.7)[2]) < 1e-20
+    lw["W_gate"][1, 0] = 1.0
+    lw["W_up"][1, 1] = -40.0
+    g = 1.5
+    np.testing.assert_allclose(run(1.5, 0.7)[2], g / (1.0 + np.exp(-g)) * (-40.0 * 0.7), rtol=1e-13)
+
+
+def test_feed_forward_half_matches_scalar_loops_with_its_own_gain():
+    # float64 closed form of x + W_down (silu(W_gate u2) * (W_up u2)), u2 = g2 * x / rms(x), written
+    # with scalar loops; g1 differs from g2 and must not enter (W_o = 0 silences the attention half).
+    rng = np.random.default_rng(11)
+    D, F, R = 6, 5, 3
+    cfg, lw = _blank_layer(D, F, rng)
+    lw["g1"] = 1.0 + 0.3 * rng.standard_normal(D)
+    lw["g2"] = 1.0 + 0.3 * rng.standard_normal(D)
+    lw["W_gate"] = rng.standard_normal((F, D))
+    lw["W_up"] = rng.standard_normal((F, D))
+    lw["W_down"] = rng.standard_normal((D, F))
+    x = rng.standard_normal((R, D))
+    kc, vc = _no_ctx()
+    out = orc.draft_layer(x, lw, kc, vc, np.zeros(R), cfg)
+    for r in range(R):
+        ms = 0.0
+        for d in range(D):
+            ms += x[r, d] * x[r, d]
+        rs = 1.0 / np.sqrt(ms / D + cfg.rms_eps)
+        h = []
+        for j in range(F):
+            gate = up = 0.0
+            for d in range(D):
+                u2 = lw["g2"][d] * x[r, d] * rs
+                gate += lw["W_gate"][j, d] * u2
+                up += lw["W_up"][j, d] * u2
+            h.append(gate / (1.0 + np.exp(-gate)) * up)
+        for d in range(D):
+            y = x[r, d]
+            for j in range(F):
+                y += lw["W_down"][d, j] * h[j]
+            assert abs(out[r, d] - y) < 1e-12
+    # a different g1 changes nothing here, a different g2 does
+    lw2 = dict(lw, g1=2.0 * lw["g1"])
+    np.testing.assert_array_equal(orc.draft_layer(x, lw2, kc, vc, np.zeros(R), cfg), out)
+    lw3 = dict(lw, g2=2.0 * lw["g2"])
+    assert np.max(np.abs(orc.draft_layer(x, lw3, kc, vc, np.zeros(R), cfg) - out)) > 1e-3
+
+
+def test_second_norm_sees_the_hidden_after_the_attention_residual():
+    # With a non-zero W_o the FFN must normalise x' = x + W_o a, not x: rebuild x' from the attention
+    # of a single-row block (softmax over one key = 1, so a = v) and feed it to the scalar FFN.
+    rng = np.random.default_rng(12)
+    D, F = 4, 3
+    cfg, lw = _blank_layer(D, F, rng)
+    lw["g1"] = 1.0 + 0.3 * rng.standard_normal(D)
+    lw["g2"] = 1.0 + 0.3 * rng.standard_normal(D)
+    lw["W_o"] = rng.standard_normal((D, cfg.q_dim))
+    lw["W_gate"] = rng.standard_normal((F, D))
+    lw["W_up"] = rng.standard_normal((F, D))
+    lw["W_down"] = rng.standard_normal((D, F))
+    x = rng.standard_normal((1, D))
+    kc, vc = _no_ctx()
+    out = orc.draft_layer(x, lw, kc, vc, np.zeros(1), cfg)[0]
+    u = lw["g1"] * x[0] / np.sqrt(np.mean(x[0] ** 2) + cfg.rms_eps)
+    v = lw["W_v"] @ u                                    # the one kv head; both q heads attend to it alone
+    a = np.concatenate((v, v))
+    x1 = x[0] + lw["W_o"] @ a
+    u2 = lw["g2"] * x1 / np.sqrt(np.mean(x1 ** 2) + cfg.rms_eps)
+    gate, up = lw["W_gate"] @ u2, lw["W_up"] @ u2
+    ref = x1 + lw["W_down"] @ (gate / (1.0 + np.exp(-gate)) * up)
+    np.testing.assert_allclose(out, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_projections_read_the_first_norm_of_the_hidden():
+    # q, k, v come from u = RMSNorm(x; g1): rescaling x leaves the block's k and v unchanged (the norm
+    # removes the scale), doubling g1 doubles them, g2 does not reach them; and with W_o = W_down = 0
+    # the layer output is x itself.
+    rng = np.random.default_rng(13)
+    D, F, R = 6, 4, 3
+    cfg, lw = _blank_layer(D, F, rng)
+    cfg.rms_eps = 0.0
+    lw["g1"] = 1.0 + 0.3 * rng.standard_normal(D)
+    lw["g2"] = 1.0 + 0.3 * rng.standard_normal(D)
+    x = rng.standard_normal((R, D))
+    kc, vc = _no_ctx()
+    out, k, v = orc.draft_layer(x, lw, kc, vc, np.zeros(R), cfg, return_kv=True)
+    np.testing.assert_array_equal(out, x)
+    out7, k7, v7 = orc.draft_layer(7.5 * x, lw, kc, vc, np.zeros(R), cfg, return_kv=True)
+    np.testing.assert_allclose(k7, k, rtol=1e-13)
+    np.testing.assert_allclose(v7, v, rtol=1e-13)
+    _, k2, v2 = orc.draft_layer(x, dict(lw, g1=2.0 * lw["g1"]), kc, vc, np.zeros(R), cfg, return_kv=True)
+    np.testing.assert_allclose(k2, 2.0 * k, rtol=1e-13)
+    np.testing.assert_allclose(v2, 2.0 * v, rtol=1e-13)
+    _, k3, v3 = orc.draft_layer(x, dict(lw, g2=2.0 * lw["g2"]), kc, vc, np.zeros(R), cfg, return_kv=True)
+    np.testing.assert_array_equal(k3, k)
+    np.testing.assert_array_equal(v3, v)
+    # the values themselves: v[r] = W_v (g1 * x[r] / rms(x[r]))
+    for r in range(R):
+        u = lw["g1"] * x[r] / np.sqrt(np.mean(x[r] ** 2))
+        np.testing.assert_allclose(v[r, 0], lw["W_v"] @ u, rtol=1e-13)
+        np.testing.assert_allclose(k[r, 0], lw["W_k"] @ u, rtol=1e-13)
+    # q reads the same u: a single-row block attends to itself only, so the output projection sees v;
+    # to see q, use two rows and check the attention weights through the output
+    lwq = dict(lw, W_o=rng.standard_normal((D, cfg.q_dim)))
+    o1 = orc.draft_layer(x, lwq, kc, vc, np.zeros(R), cfg)
+    o2 = orc.draft_layer(7.5 * x, lwq, kc, vc, np.zeros(R), cfg)
+    np.testing.assert_allclose(o2 - 7.5 * x, o1 - x, rtol=1e-11, atol=1e-13)   # q, k, v all scale-free in x
+    for r in range(R):       # attention of row r over the block written out: scores q.k * scale, softmax, mix of v
+        u_all = lw["g1"] * x / np.sqrt(np.mean(x ** 2, axis=-1, keepdims=True))
+        acc = np.zeros(cfg.q_dim)
+        for h in range(2):
+            qh = lw["W_q"][2 * h:2 * h + 2] @ u_all[r]
+            s = np.array([qh @ (lw["W_k"] @ u_all[t]) for t in range(R)]) * cfg.softmax_scale
+            p = np.exp(s - s.max())
+            p /= p.sum()
+            acc[2 * h:2 * h + 2] = sum(p[t] * (lw["W_v"] @ u_all[t]) for t in range(R))
+        np.testing.assert_allclose(o1[r] - x[r], lwq["W_o"] @ acc, rtol=1e-11, atol=1e-13)
