@@ -104,7 +104,15 @@ typedef struct {
 /* ---- life cycle (host only, no CUDA work) ---- */
 
 /* Validates the configuration and builds a handle. Returns DFLASH_ERR_UNSUPPORTED for shapes the
- * kernels do not cover (head_dim not in {64,128}, Hq % Hkv != 0, block_size > 32, ...). */
+ * kernels do not cover (head_dim not in {64,128}, Hq % Hkv != 0, block_size > 32, ...).
+ * The handle remembers the SM count of the device that is current at this call (148 when the host has no
+ * GPU): grids, work splits and workspace sizes follow it, so use the handle on that device (or an equal one).
+ * bf16 attention runs on the tensor cores for head_dim = 128 with 64-token pages; head_dim = 64 (and other
+ * page sizes) take a CUDA-core kernel, as does everything in fp32.
+ * The chained contraction kernels run one CTA per SM and their CTAs wait for each other (bounded): two
+ * library calls must not overlap in time on one GPU (issue them on one stream, or order them with
+ * events), and the GPU's SMs must all be available to the process (no MPS / green-context SM limit);
+ * otherwise waits expire after ~1.5 s, DFLASH_DEV_TIMEOUT is set and the output is invalid. */
 int32_t dflash_create(const dflash_config* cfg /*[host]*/, dflash_handle** out /*[host]*/);
 void    dflash_destroy(dflash_handle* h);
 
@@ -360,9 +368,10 @@ int32_t dflash_lmhead_argmax(dflash_handle* h, const dflash_lmhead_args* a /*[ho
  * >= vocab is treated the same and sets DFLASH_DEV_BAD_TOKEN. loss_sum = {sum of row_loss, sum of the w_k
  * that count}, added in double in a fixed order: the caller divides by whichever normaliser it trains with
  * (the paper does not state one) and passes the matching grad_scale.
- * Arithmetic: fp32 per row (maximum, sum of exponentials, logarithm). A CTA reads its row twice in a row
- * (statistics, then gradient), the second time from L2: HBM traffic is one read of the logits plus one
- * write of the gradient. `dlogits` may alias `logits` when dtype and stride agree. No scratch memory.
+ * Arithmetic: fp32 per row (maximum, sum of exponentials, logarithm). A row is held in the shared memory of a
+ * small thread-block cluster between the statistics and the gradient pass (rows that do not allow 16-byte
+ * accesses are instead read twice by one CTA): HBM traffic is one read of the logits plus one write of the
+ * gradient. `dlogits` may alias `logits` when dtype and stride agree. No scratch memory.
  * Errors: DFLASH_ERR_INVALID_ARG (null pointer, gamma <= 0, bad dtype or sizes). */
 typedef struct {
     const void*    logits;             /* [device] [n_blocks * block_rows, vocab]                       */
@@ -401,6 +410,14 @@ const char* dflash_family_name(int32_t family);
  * the kernel family that wrote it, and rewinds. Passing NULL switches tracing off. */
 int32_t dflash_trace_enable(dflash_handle* h, uint64_t* dev_buf /*[device]*/, int32_t capacity_records);
 int32_t dflash_trace_read(dflash_handle* h, int32_t* families /*[host] capacity entries*/, int32_t* n_records /*[host]*/);
+
+/* How dflash_block_attention / the draft and verify passes split the keys of a call on the bf16 tensor-core
+ * path (host arithmetic only, no CUDA work): out[0] = 64-key tiles per range, out[1] = ranges per (sequence,
+ * kv head) at max_ctx_len, out[2] = partial-result slots the kernels index (batch * Hkv * ranges), out[3] =
+ * slots the workspace of dflash_workspace_bytes(h, batch, ...) provides. out[2] <= out[3] for every input:
+ * when many long sequences would need more, the ranges get longer instead. A ctx_len[b] above max_ctx_len is
+ * clamped to it by the kernels and sets DFLASH_DEV_CTX_OVERFLOW. */
+int32_t dflash_attention_plan(const dflash_handle* h, int32_t batch, int32_t max_ctx_len, int64_t* out /*[host] [4]*/);
 
 /* Static description of a return code. */
 const char* dflash_status_string(int32_t code);

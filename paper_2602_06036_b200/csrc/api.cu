@@ -216,7 +216,17 @@ int32_t dflash_create(const dflash_config* cfg, dflash_handle** out) {
     if (!h) return DFLASH_ERR_INVALID_ARG;
     h->cfg = c;
     h->has_weights = false;
+    // SMs of the current device (grids of one CTA per SM, split heuristics and the partial-tile workspace follow
+    // it); without a device - sizing queries on a host with no GPU - the B200's count
     h->sm_count = 148;
+    {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            h->sm_count = n;
+        else
+            (void)cudaGetLastError();
+    }
     h->prof_on = false;
     h->prof = nullptr;
     h->prof_cap = h->prof_used = 0;
@@ -399,6 +409,7 @@ static int block_forward(dflash_handle* h, const BlockRun* a, void* stream) {
     // A context projection handed in with the draft: fused into the first chained launch when its weight
     // maps fit one launch (fusion + one K/V group per layer + QKV), else run first as its own launches.
     const dflash_ctx_args* cx = a->ctx;
+    if (cx && (cx->batch < 0 || cx->max_new < 0)) return DFLASH_ERR_INVALID_ARG;
     const int rows_ctx = cx ? cx->batch * cx->max_new : 0;
     if (cx && rows_ctx > 0 && (!cx->feats || !cx->ctx_len || !cx->page_table || !cx->kv_pool || cx->batch != a->batch ||
                                cx->max_pages < 1 || cx->n_pool_pages < 1))
@@ -647,7 +658,7 @@ int32_t dflash_verify_accept(dflash_handle* h, const dflash_verify_args* a, void
 int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void* stream) {
     if (!h || !a) return DFLASH_ERR_INVALID_ARG;
     if (a->batch < 0 || a->rows < 0 || a->rows > 32 || a->max_pages < 1 || a->n_pool_pages < 1 ||
-        a->layer < 0 || a->max_ctx_len < 0)
+        a->layer < 0 || a->layer >= h->cfg.n_layers || a->max_ctx_len < 0)
         return DFLASH_ERR_INVALID_ARG;
     if (a->mode != DFLASH_ATTN_FULL && a->mode != DFLASH_ATTN_CAUSAL) return DFLASH_ERR_INVALID_ARG;
     if (a->batch == 0 || a->rows == 0) return DFLASH_OK;
@@ -661,6 +672,13 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     } else {
         RUN(FAM_ATTENTION, launch_attention_simt(L, *a));
     }
+    return DFLASH_OK;
+}
+
+int32_t dflash_attention_plan(const dflash_handle* h, int32_t batch, int32_t max_ctx_len, int64_t* out) {
+    if (!h || !out || batch < 1 || max_ctx_len < 0) return DFLASH_ERR_INVALID_ARG;
+    const AttnPlan pl = attn_tc_plan(h->cfg, batch, max_ctx_len, h->sm_count);
+    out[0] = pl.tiles_per_unit; out[1] = pl.n_chunks; out[2] = pl.units; out[3] = pl.capacity_units;
     return DFLASH_OK;
 }
 

@@ -50,6 +50,7 @@ constexpr float RESCALE_GAP = 8.f;               // log2 units
 
 struct AParams {
     int S, R, Hq, Hkv, group, max_pages, n_pages, layer, causal, tiles_per_unit, n_chunks, rows_valid;
+    int max_ctx_len;   // the caller's bound the KV split was sized for: longer lengths are clamped to it and flagged
     int dup;     // rows_valid <= 64: the query rows are loaded twice and each copy handles 32 of a tile's 64 keys
     int early_kv;   // the cached context of this layer was written before the previous kernel's dependencies:
                     // its first tiles may be requested before the grid dependency resolves
@@ -134,7 +135,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int chunk = blockIdx.x % p.n_chunks;
     const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
     const int b = blockIdx.x / (p.n_chunks * p.Hkv);
-    const int L = max(p.ctx_len[b], 0);
+    const int L_given = p.ctx_len[b];
+    const int L = min(max(L_given, 0), p.max_ctx_len);   // the ranges (and the partials buffer) cover max_ctx_len keys
+    if (L_given > p.max_ctx_len && threadIdx.x == 0 && chunk == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
     const int n_ctx_tiles = (L + PG - 1) / PG;
     const int T = n_ctx_tiles + 1;                       // + the block's own rows
     const int t_lo = chunk * p.tiles_per_unit;
@@ -548,7 +551,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     const int row = (blockIdx.x % row_blocks) * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int b = bg / p.Hkv, g = bg % p.Hkv;
-    const int L = max(__ldg(p.ctx_len + b), 0);      // an input of the call: no kernel writes it
+    const int L = min(max(__ldg(p.ctx_len + b), 0), p.max_ctx_len);      // an input of the call: no kernel writes it
     const int T = (L + PG - 1) / PG + 1;
     const int n_splits = (T + p.tiles_per_unit - 1) / p.tiles_per_unit;
     pdl_wait();
@@ -638,11 +641,29 @@ static int tiles_per_unit(int batch, int Hkv, int max_ctx_len, int sm_count) {
     return std::max(2, Tmax);
 }
 
+// Partials the workspace holds: one per (sequence, kv head, range). One sequence: <= SMs (+ rounding); a batch:
+// <= 2*SMs + 2*batch*Hkv (ranges of >= total/(2*SMs) tiles); kept generous. attn_tc_plan never exceeds it.
+static int64_t part_units(const dflash_config& c, int batch, int sm_count) {
+    return 8 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
+}
 int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count) {
-    // units: one sequence <= SMs (+ rounding); a batch <= 2*SMs + 2*batch*Hkv (ranges of >= total/(2*SMs) tiles); kept generous
-    const int64_t units = 8 * (int64_t)sm_count + 2 * (int64_t)batch * c.n_kv_heads;
     const int rows_valid = std::min(128, rows * (c.n_q_heads / c.n_kv_heads));
-    return units * rows_valid * PART_LD * 4;
+    return part_units(c, batch, sm_count) * rows_valid * PART_LD * 4;
+}
+AttnPlan attn_tc_plan(const dflash_config& c, int batch, int max_ctx_len, int sm_count) {
+    AttnPlan pl{};
+    const int Tmax = (max_ctx_len + PG - 1) / PG + 1;
+    pl.tiles_per_unit = tiles_per_unit(batch, c.n_kv_heads, max_ctx_len, sm_count);
+    pl.capacity_units = part_units(c, batch, sm_count);
+    const int64_t bh = (int64_t)batch * c.n_kv_heads;
+    // The heuristic caps a range at 128 tiles; a large batch of very long contexts would then need more
+    // partials than the workspace holds. Longer ranges instead: two per (sequence, kv head) always fit.
+    const int64_t max_chunks = std::max<int64_t>(1, pl.capacity_units / std::max<int64_t>(bh, 1));
+    if ((Tmax + pl.tiles_per_unit - 1) / pl.tiles_per_unit > max_chunks)
+        pl.tiles_per_unit = (int)((Tmax + max_chunks - 1) / max_chunks);
+    pl.n_chunks = (Tmax + pl.tiles_per_unit - 1) / pl.tiles_per_unit;
+    pl.units = bh * pl.n_chunks;
+    return pl;
 }
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch) { return (int64_t)batch * c.n_kv_heads * 4; }
 
@@ -654,13 +675,15 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.S = a.batch; p.R = a.rows; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.group = c.n_q_heads / c.n_kv_heads;
     p.max_pages = a.max_pages; p.n_pages = a.n_pool_pages; p.layer = a.layer;
     p.causal = a.mode == DFLASH_ATTN_CAUSAL ? 1 : 0;
-    p.tiles_per_unit = tiles_per_unit(a.batch, c.n_kv_heads, a.max_ctx_len, L.h->sm_count);
+    const AttnPlan plan = attn_tc_plan(c, a.batch, a.max_ctx_len, L.h->sm_count);
+    if (plan.units > plan.capacity_units) return DFLASH_ERR_WORKSPACE;      // cannot happen: the plan lengthens the ranges
+    p.tiles_per_unit = plan.tiles_per_unit;
+    p.max_ctx_len = a.max_ctx_len;
     p.rows_valid = std::min(128, a.rows * p.group);
     p.dup = (p.rows_valid <= 64 && 64 % p.group == 0) ? 1 : 0;
     p.early_kv = early_kv ? 1 : 0;
     p.early_len = early_len;
-    const int Tmax = (a.max_ctx_len + PG - 1) / PG + 1;
-    p.n_chunks = (Tmax + p.tiles_per_unit - 1) / p.tiles_per_unit;
+    p.n_chunks = plan.n_chunks;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
     p.ctx_len = a.ctx_len; p.page_table = a.page_table;
     p.out = (__nv_bfloat16*)a.out; p.part = part; p.status = L.status; p.trace = L.trace;

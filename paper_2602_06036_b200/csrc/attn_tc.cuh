@@ -9,6 +9,14 @@ namespace dflash {
 bool attn_tc_supported(const dflash_config& c, int rows);
 int64_t attn_tc_part_bytes(const dflash_config& c, int batch, int rows, int sm_count);
 int64_t attn_tc_counter_bytes(const dflash_config& c, int batch);
+// How the keys of a call are split into ranges, and what that needs of the partials buffer (host arithmetic only).
+struct AttnPlan {
+    int tiles_per_unit;        // 64-key tiles per range
+    int n_chunks;              // ranges per (sequence, kv head) at max_ctx_len
+    int64_t units;             // partial slots the kernels index: batch * Hkv * n_chunks
+    int64_t capacity_units;    // slots attn_tc_part_bytes provides for this batch (units never exceeds it)
+};
+AttnPlan attn_tc_plan(const dflash_config& c, int batch, int max_ctx_len, int sm_count);
 // `part`: split-KV scratch of the size above. `counters` is not used by the current kernels (the
 // partials are merged by a second kernel, not by a last arriver).
 // `early_kv`: the layer's cached context was complete before the kernel preceding this one started waiting

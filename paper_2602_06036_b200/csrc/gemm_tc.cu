@@ -1081,8 +1081,11 @@ static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KPa
     p.q = a.q; p.k = a.k; p.v = a.v;
     p.gq = (const __nv_bfloat16*)a.g_q;
     p.gk[0] = (const __nv_bfloat16*)a.g_k;
-    if (a.epilogue == EPI_CTX_KV)
-        for (int g = 0; g < groups; ++g) p.gk[g] = (const __nv_bfloat16*)a.g_k_group[g]; p.ctx_len = a.ctx_len; p.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : 1;
+    if (a.epilogue == EPI_CTX_KV) {
+        for (int g = 0; g < groups; ++g) p.gk[g] = (const __nv_bfloat16*)a.g_k_group[g];
+    }
+    p.ctx_len = a.ctx_len;
+    p.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : 1;
     p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads; p.hd = c.head_dim; p.use_rope = c.use_rope;
     p.cs = L.h->w.rope_cos; p.sn = L.h->w.rope_sin; p.max_pos = L.h->w.rope_max_pos;
     p.h = a.h; p.F = c.d_ffn;

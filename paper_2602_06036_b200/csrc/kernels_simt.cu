@@ -604,10 +604,10 @@ int launch_row_argmax(const Launch& L, const void* logits, int dtype, int64_t ro
 // accept rule (Sec. 3.1): longest agreeing prefix + bonus token, one thread per sequence
 // ------------------------------------------------------------------------------------------
 __global__ void accept_kernel(const int32_t* __restrict__ target_ids, const int32_t* __restrict__ draft_ids,
-                              int draft_stride, int batch, int gamma, const int32_t* __restrict__ ctx_len,
+                              int draft_stride, int batch, int gamma, const int32_t* ctx_len,
                               int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
-                              int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx_len,
-                              int32_t* __restrict__ target_ids_out) {
+                              int32_t* __restrict__ bonus, int32_t* new_ctx_len,
+                              int32_t* __restrict__ target_ids_out) {      // new_ctx_len may alias ctx_len: neither is restrict
     ptx::pdl_trigger();
     ptx::pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -640,9 +640,10 @@ int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* t
 // that merges the segments of its gamma + 1 rows (a warp per row) and applies the accept rule.
 __global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __restrict__ seg, int nseg,
                                                             const int32_t* __restrict__ draft_ids, int draft_stride, int gamma,
-                                                            const int32_t* __restrict__ ctx_len, int32_t* __restrict__ accept_len,
+                                                            const int32_t* ctx_len, int32_t* __restrict__ accept_len,
                                                             int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
-                                                            int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ target_ids_out) {
+                                                            int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out) {
+    // new_ctx_len may alias ctx_len: neither is restrict, and the length is read before anything is written
     __shared__ int32_t s_p[65];
     ptx::pdl_trigger();
     ptx::pdl_wait();
@@ -671,13 +672,14 @@ __global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __rest
     __syncthreads();
     if (threadIdx.x == 0) {
         const int32_t* d = draft_ids + (size_t)b * draft_stride;
+        const int32_t len = ctx_len[b];
         int a = 0;
         while (a < gamma && d[a] == s_p[a]) ++a;
         int32_t* o = out_tokens + (size_t)b * (gamma + 1);
         for (int i = 0; i <= gamma; ++i) o[i] = i < a ? d[i] : (i == a ? s_p[a] : -1);
         accept_len[b] = a + 1;
         bonus[b] = s_p[a];
-        new_ctx_len[b] = ctx_len[b] + a + 1;
+        new_ctx_len[b] = len + a + 1;
     }
 }
 

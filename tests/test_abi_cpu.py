@@ -139,6 +139,71 @@ def test_sampling_and_loss_args_validated_on_the_host(lib):
     lib.dflash_destroy(h)
 
 
+def _qwen_cfg():
+    c = synth.QWEN3_8B
+    return _cfg(n_layers=c.n_layers, d_model=c.d_model, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads, head_dim=c.head_dim,
+                d_ffn=c.d_ffn, vocab=c.vocab, n_feat_layers=c.n_feat_layers, d_target=c.d_target, block_size=c.block_size,
+                dtype=1, mask_token_id=c.vocab - 1, softmax_scale=c.softmax_scale)
+
+
+def test_attention_split_never_outgrows_its_partials_buffer(lib):
+    # host arithmetic only: for every (batch, kv heads, context bound) the partial slots the kernels index
+    # stay inside what the workspace provides, and every range covers the whole context
+    for hkv, hq in ((8, 32), (1, 8), (2, 8), (32, 32)):
+        h = C.c_void_p()
+        cfg = _qwen_cfg()
+        cfg.n_kv_heads, cfg.n_q_heads = hkv, hq
+        assert lib.dflash_create(C.byref(cfg), C.byref(h)) == 0
+        out = (C.c_int64 * 4)()
+        for batch in (1, 2, 3, 8, 17, 18, 19, 32, 37, 64, 148, 149, 256, 1024):
+            for L in (0, 1, 63, 64, 65, 2048, 8191, 8192, 32768, 40000, 65536, 131072, 1 << 20):
+                assert lib.dflash_attention_plan(h, batch, L, out) == 0
+                tiles_per_unit, n_chunks, units, capacity = out[0], out[1], out[2], out[3]
+                T = (L + 63) // 64 + 1
+                assert tiles_per_unit >= 1 and n_chunks >= 1
+                assert n_chunks * tiles_per_unit >= T, (batch, hkv, L)
+                assert (n_chunks - 1) * tiles_per_unit < T, (batch, hkv, L)       # no empty trailing range
+                assert units == batch * hkv * n_chunks
+                assert units <= capacity, (batch, hkv, L, units, capacity)
+        assert lib.dflash_attention_plan(h, 0, 10, out) == -1 and lib.dflash_attention_plan(h, 1, -1, out) == -1
+        lib.dflash_destroy(h)
+    # the example that used to overflow: 32 sequences x 8 kv heads at 65536 tokens
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_qwen_cfg()), C.byref(h)) == 0
+    out = (C.c_int64 * 4)()
+    assert lib.dflash_attention_plan(h, 32, 65536, out) == 0 and out[2] <= out[3] and out[0] > 128
+    lib.dflash_destroy(h)
+
+
+def test_attention_and_fused_projection_arguments_validated_on_the_host(lib):
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_cfg()), C.byref(h)) == 0
+    a = binding.AttnArgs()
+    a.batch, a.rows, a.max_pages, a.n_pool_pages, a.max_ctx_len = 1, 8, 4, 4, 128
+    for name in ("q", "k_blk", "v_blk", "ctx_len", "page_table", "kv_pool", "out"):
+        setattr(a, name, 256)                                          # non-null; never dereferenced on the host
+    a.layer = 1                                                        # the tiny shape has one layer
+    assert lib.dflash_block_attention(h, C.byref(a), None) == -1
+    a.layer = -1
+    assert lib.dflash_block_attention(h, C.byref(a), None) == -1
+    a.layer, a.batch = 0, 0
+    assert lib.dflash_block_attention(h, C.byref(a), None) == 0        # nothing to do
+    # a projection handed in with the draft call: a negative row count is refused like dflash_ctx_project refuses it
+    lw = (binding.LayerWeights * 1)(binding.LayerWeights(*([256] * 8)))
+    w = binding.Weights(256, 256, 256, lw, 256, 256, 256, 256, 1024)
+    assert lib.dflash_set_weights(h, C.byref(w)) == 0                   # borrowed pointers only, nothing is read
+    cx = binding.CtxArgs()
+    cx.batch, cx.max_new, cx.max_pages, cx.n_pool_pages = 1, -1, 4, 4
+    assert lib.dflash_ctx_project(h, C.byref(cx), None) == -1
+    d = binding.DraftArgs()
+    d.batch, d.max_pages, d.n_pool_pages, d.max_ctx_len = 1, 4, 4, 128
+    for name in ("anchor_ids", "ctx_len", "page_table", "kv_pool", "draft_ids"):
+        setattr(d, name, 256)
+    d.ctx = C.pointer(cx)
+    assert lib.dflash_draft_block(h, C.byref(d), None) == -1
+    lib.dflash_destroy(h)
+
+
 def test_status_strings(lib):
     seen = {lib.dflash_status_string(c).decode() for c in (0, -1, -2, -3, -4, -5)}
     assert len(seen) == 6 and lib.dflash_status_string(-99).decode() == "unknown status"
