@@ -53,11 +53,18 @@ constexpr int W_STAGE_BYTES = TILE_F * BK * 2;   // 16 KiB per slab
 // the row-major matrix lands as [slab][row][64], i.e. two canonical swizzled tiles back to back).
 constexpr int slabs_for(int nt, bool k_mult_64) { return (nt <= 32 && k_mult_64) ? 2 : 1; }
 constexpr int MAX_STAGES = 12;
-constexpr int TOK_CACHE = 1024;                  // per-token scale / position / page kept for this many rows
+// per-token scale / position / page kept for this many rows (token tiles of up to 32 rows only run with <= 32 rows)
+constexpr int tok_cache(int nt) { return nt <= 32 ? 32 : 1024; }
+// Thread-block clusters (token tiles of up to 32 rows): the CS CTAs of a cluster split the K range of one
+// weight tile and exchange their partial sums through distributed shared memory. Every CTA finishes NT / CS
+// token columns of the tile: it receives those columns from its CS - 1 peers into one of two buffers.
+constexpr int CS = 4;
+constexpr int xch_bytes(int nt) { return nt <= 32 ? 2 * (CS - 1) * (nt / CS) * TILE_F * 4 : 0; }
 // token columns handled per epilogue pass (each of the 128 epilogue threads holds CH accumulators)
 constexpr int pass_cols(int nt) { return nt <= 16 ? nt : (nt == 32 ? 16 : 32); }   // short passes: short dependent chains when finishing, fewer registers
 constexpr int smem_fixed(int nt) {
-    return TILE_F * (pass_cols(nt) + 1) * 4 + 128 * 16 + 3 * TOK_CACHE * 4 + (2 * MAX_STAGES + 4) * 8 + 64 + 3 * MAX_STAGES * 4;
+    return TILE_F * (pass_cols(nt) + 1) * 4 + 128 * 16 + 3 * tok_cache(nt) * 4 + xch_bytes(nt) + (2 * MAX_STAGES + 6) * 8 + 64 +
+           3 * MAX_STAGES * 4;
 }
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int N_THREADS = 192;
@@ -68,6 +75,7 @@ struct WMaps {
 
 struct KParams {
     int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, w_map0, x_map;
+    int cluster_k;     // the phase splits every tile's K range over the CTAs of a cluster (partial sums through their shared memory)
     float* part;
     int32_t* counters;
     const float* ssq_in;
@@ -104,6 +112,7 @@ struct XMaps {
 // A launch = a chain of phases that share the token tile size and the ring.
 struct MParams {
     int n_phases, stages;
+    int cs;                      // CTAs per cluster (1: launched without clusters)
     int32_t* phase_done;         // [MAX_PHASES] CTAs that finished each phase (zero on entry)
     int32_t* status;
     KParams ph[MAX_PHASES];
@@ -114,6 +123,7 @@ struct Unit {
     int tile, g, ft, tt, c0, c1;
     int slot;      // 0 = first piece of this CTA's range, 1 = a later one (partial pieces only: first or last)
     int full;      // covers every chunk of the tile
+    int cl;        // this CTA's K share of a tile that its cluster finishes together
 };
 
 // Work of CTA `cta` out of `n_ctas` in one phase. With at least one tile per CTA the tiles are split
@@ -127,6 +137,7 @@ struct Unit {
 // The shared part never leaves a CTA an empty range (every CTA between the first and the last
 // contributor of a tile publishes a piece): a remainder that small takes one more round of tiles with it.
 __device__ __forceinline__ int shared_tiles(const KParams& p, int n_ctas) {
+    if (p.cluster_k) return 0;      // every tile is finished inside a cluster
     if (p.n_tiles < n_ctas) return p.n_tiles;
     const int r = p.n_tiles % n_ctas;
     if (r == 0) return 0;
@@ -136,19 +147,32 @@ __device__ __forceinline__ int shared_tiles(const KParams& p, int n_ctas) {
 struct PieceWalk {
     long long cur, hi;
     int first, n_shared, dp_next, dp_stride;
-    __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas) {
+    int cl_c0, cl_c1;      // cluster mode: this CTA's chunk range of every tile its cluster takes (cl_c1 = 0: not cluster mode)
+    // cs: CTAs per cluster. A cluster-mode phase gives its tiles to the clusters in turn; rank r of a cluster
+    // streams chunks [r * C / cs, (r + 1) * C / cs) of each of its tiles.
+    __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas, int cs) {
+        first = 1;
         n_shared = shared_tiles(p, n_ctas);
         const long long T = (long long)n_shared * p.chunks_total;
         cur = (long long)cta * T / n_ctas;
         hi = (long long)(cta + 1) * T / n_ctas;
-        first = 1;
-        dp_next = n_shared + cta;
-        dp_stride = n_ctas;
+        if (p.cluster_k) {
+            const int rank = cta % cs;
+            dp_next = n_shared + cta / cs;
+            dp_stride = n_ctas / cs;
+            cl_c0 = rank * p.chunks_total / cs;
+            cl_c1 = (rank + 1) * p.chunks_total / cs;
+        } else {
+            cl_c0 = cl_c1 = 0;
+            dp_next = n_shared + cta;
+            dp_stride = n_ctas;
+        }
     }
     __device__ __forceinline__ bool shared_done() const { return cur >= hi; }
     __device__ __forceinline__ bool done(const KParams& p) const { return cur >= hi && dp_next >= p.n_tiles; }
     __device__ __forceinline__ Unit next(const KParams& p) {
         Unit u;
+        u.cl = 0;
         if (cur < hi) {
             u.tile = (int)(cur / p.chunks_total);
             u.c0 = (int)(cur % p.chunks_total);
@@ -164,6 +188,7 @@ struct PieceWalk {
             u.c1 = p.chunks_total;
             u.full = 1;
             u.slot = 0;
+            if (cl_c1 > 0) { u.c0 = cl_c0; u.c1 = cl_c1; u.full = 0; u.cl = 1; }
             dp_next += dp_stride;
         }
         int t = u.tile;
@@ -196,10 +221,12 @@ __device__ __forceinline__ void t2_merge(T2& a, float v1, int i1, float v2) {
 
 // Residual rows of one pass (x += ...) and the next norm's gain for this feature: loaded by the caller,
 // ahead of whatever else it waits for.
+// lim: token columns of this pass (<= CH)
 template <int CH>
-__device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, int tok0, int row, float (&xres)[CH], float& gain) {
+__device__ __forceinline__ void residual_load(const KParams& p, const Unit& un, int tok0, int row, float (&xres)[CH], float& gain,
+                                              int lim = CH) {
     const int f = un.ft * TILE_F + row;
-    const int n_tok = min(CH, p.M - tok0);
+    const int n_tok = min(lim, p.M - tok0);
     gain = (p.g_next && (p.epi == EPI_RESIDUAL || p.epi == EPI_STORE_F32) && f < p.N) ? __bfloat162float(p.g_next[f]) : 0.f;
 #pragma unroll
     for (int c = 0; c < CH; ++c) xres[c] = 0.f;
@@ -244,14 +271,16 @@ __device__ __forceinline__ void head_rnorm(const KParams& p, const float* sAcc, 
 
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
 // QKN: the launch has per-head q/k norms (a separate instantiation keeps the common path's registers down).
+// lim: token columns of this pass (<= CH; columns from lim on hold nothing and produce nothing)
 template <int CH, bool QKN>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
-                                               int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain) {
+                                               int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain,
+                                               int lim = CH) {
     // tPos / tPage: position and (context projection) pool row of the page slot of the tokens of this pass (-1 = skip)
     constexpr int ACC_LD = CH + 1;
     constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
     const int f = un.ft * TILE_F + row;
-    const int n_tok = min(CH, p.M - tok0);
+    const int n_tok = min(lim, p.M - tok0);
     switch (p.epi) {
         case EPI_STORE_F32:
         case EPI_RESIDUAL: {
@@ -529,8 +558,11 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     return v;
 }
 
+// Register cap: with small token tiles the kernel is kept at 232 registers, so that a warp of a small dependent
+// kernel (merge, finish) still fits into the register file partition that holds two of this CTA's six warps and
+// can become resident before this grid has drained.
 template <int NT, int SL, bool QKN>
-__global__ void __launch_bounds__(N_THREADS, 1)
+__global__ void __maxnreg__(NT <= 32 ? 232 : 255)
 gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps tmX, const __grid_constant__ MParams mp) {
     if (threadIdx.x == 0) trace_min(mp.ph[0].trace, 0);
     extern __shared__ uint8_t smem_raw[];
@@ -550,14 +582,17 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     uint8_t* sX = sW + (size_t)stages * W_STAGE;
     float* sAcc = reinterpret_cast<float*>(sX + (size_t)stages * X_STAGE);
     Top2Entry* sRed = reinterpret_cast<Top2Entry*>(sAcc + TILE_F * ACC_LD);
+    constexpr int TOK_CACHE = tok_cache(NT);
     float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [TOK_CACHE] per-token rsqrt(mean square)
     int* sPos = reinterpret_cast<int*>(sRstd + TOK_CACHE);        // [TOK_CACHE] per-token position (-1: skip)
     int* sPage = sPos + TOK_CACHE;                                // [TOK_CACHE] per-token physical page
-    uint64_t* full = reinterpret_cast<uint64_t*>(sPage + TOK_CACHE);
+    float* sXch = reinterpret_cast<float*>(sPage + TOK_CACHE);    // [2][CS - 1][NT / CS][128] columns received from cluster peers
+    uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(sXch) + xch_bytes(NT));
     uint64_t* empty = full + MAX_STAGES;
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* xch_bar = acc_empty + 2;                            // [2] one per receive buffer: (CS - 1) peers x 4 warps arrive
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(xch_bar + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [2] epilogue abort
     int* sPend = const_cast<int*>(flags) + 4;                               // [3 * MAX_STAGES] producer's queue
 
@@ -565,7 +600,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); mbar_init(&xch_bar[b], (CS - 1) * 4); }
         flags[0] = 0; flags[2] = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -576,6 +611,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     pdl_trigger();
+    // peers must not write into this CTA's receive buffers or arrive on its barriers before they exist
+    if (mp.cs > 1) cluster_sync_all();
 
     const int G = gridDim.x;
 
@@ -625,7 +662,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
                 const CUtensorMap* xm = &tmX.m[p.x_map];
-                for (PieceWalk w(p, blockIdx.x, G); !w.done(p) && ok;) {
+                for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p) && ok;) {
                     const Unit un = w.next(p);
                     const CUtensorMap* wm = &tmW.m[p.w_map0 + un.g];
                     const int y_w = un.ft * TILE_F, y_x = un.tt * NT;
@@ -677,7 +714,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             bool ok = true;
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
-                for (PieceWalk w(p, blockIdx.x, G); !w.done(p) && ok; ++ui) {
+                for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p) && ok; ++ui) {
                     const Unit un = w.next(p);
                     const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
                     if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
@@ -713,6 +750,15 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         const int row = ew * 32 + lane;
         uint32_t ui = 0;
         bool alive = true;
+        // cluster exchange: this CTA's rank, the peers' views of the receive buffers and of their barriers
+        const int rank = mp.cs > 1 ? (int)cluster_ctarank() : 0;
+        uint32_t xch_remote[CS], xbar_remote[CS];
+#pragma unroll
+        for (int q = 0; q < CS; ++q) {
+            xch_remote[q] = mp.cs > 1 ? mapa_shared(smem_u32(sXch), (uint32_t)q) : 0u;
+            xbar_remote[q] = mp.cs > 1 ? mapa_shared(smem_u32(xch_bar), (uint32_t)q) : 0u;
+        }
+        uint32_t cl_units = 0;       // cluster-shared tiles finished so far (the same number in every CTA of the cluster)
         pdl_wait();      // lengths, page tables, residual rows ... come from earlier kernels
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
@@ -810,7 +856,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 }
                 n_pend = 0;
             };
-            for (PieceWalk w(p, blockIdx.x, G); !w.done(p); ++ui) {
+            for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p); ++ui) {
                 const Unit un = w.next(p);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
@@ -829,6 +875,68 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     token_rstd(p, tok_base, NT, row, sRstd);
                     rstd_tt = un.tt;
                     epi_bar();
+                }
+                if constexpr (NT <= 32) {
+                    if (un.cl) {
+                        // ---- the tile is shared by the CTAs of this cluster, each holding the sums over its K share.
+                        // Rank q finishes token columns [q * GC, (q + 1) * GC): every CTA sends those columns of its
+                        // accumulator into rank q's receive buffer (distributed shared memory) and arrives on q's
+                        // barrier; q adds the four pieces in rank order (bit-reproducible) and runs the epilogue.
+                        // Two buffers suffice: a peer sends its (i+2)-th tile only after it has received this CTA's
+                        // (i+1)-th, which is sent after the i-th was read; phases are separated by the phase counter.
+                        constexpr int GC = NT / CS;
+                        const uint32_t xb = cl_units & 1, xpar = (cl_units >> 1) & 1;
+                        ++cl_units;
+                        const int tok0 = tok_base + rank * GC;
+                        float own[GC];
+#pragma unroll
+                        for (int c = 0; c < GC; ++c) own[c] = 0.f;
+#pragma unroll
+                        for (int ch = 0; ch < NT / CH; ++ch) {
+                            float v[CH];
+                            tmem_ld_cols<CH>(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) {
+                                const int col = ch * CH + c, q = col / GC, lc = col % GC;      // compile-time after unrolling
+                                if (q == rank) own[lc] = v[c];
+                                else if (tok_base + col < p.M) {
+                                    const int slot = rank - (rank > q ? 1 : 0);
+                                    st_cluster_f32(xch_remote[q] + (uint32_t)((((xb * (CS - 1) + slot) * GC + lc) * TILE_F + row) * 4), v[c]);
+                                }
+                            }
+                        }
+                        tc_fence_before();
+                        fence_acq_rel_cluster();
+                        __syncwarp();
+                        if (lane == 0) {
+                            mbar_arrive(&acc_empty[buf]);
+#pragma unroll
+                            for (int q = 0; q < CS; ++q)
+                                if (q != rank) mbar_arrive_cluster(xbar_remote[q] + xb * 8);
+                        }
+                        // residual rows travel while the peers' columns arrive
+                        float xres[CH], gain = 0.f;
+                        residual_load<CH>(p, un, tok0, row, xres, gain, GC);
+                        if (!mbar_wait_cluster(&xch_bar[xb], xpar, &flags[0])) flags[2] = 1;
+                        epi_bar();
+                        if (flags[2]) { alive = false; break; }
+                        if (tok0 < p.M) {
+                            const float* rx = sXch + (size_t)xb * (CS - 1) * GC * TILE_F + row;
+#pragma unroll
+                            for (int lc = 0; lc < GC; ++lc) {
+                                float a = 0.f;
+#pragma unroll
+                                for (int j = 0; j < CS; ++j)
+                                    a += (j == rank) ? own[lc] : rx[((j - (j > rank ? 1 : 0)) * GC + lc) * TILE_F];
+                                sAcc[row * ACC_LD + lc] = p.ssq_in ? a * sRstd[tok_off + rank * GC + lc] : a;
+                            }
+                            epi_bar();
+                            apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok0, row, sPos + tok_off + rank * GC, sPage + tok_off + rank * GC,
+                                                    xres, gain, GC);
+                            epi_bar();
+                        }
+                        continue;
+                    }
                 }
                 const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
                 for (int ch = 0; ch < n_ch; ++ch) {
@@ -886,6 +994,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    // no CTA of a cluster may go away while a peer can still write into its shared memory; every wait above is
+    // bounded, so every CTA gets here
+    if (mp.cs > 1) cluster_sync_all();
 }
 
 // Merge of the per-tile winners (index-aware, so order-independent). The entries are laid out
@@ -1035,17 +1146,77 @@ int pick_nt(int M) {
     return 256;
 }
 
+// Largest grid of clusters of CS CTAs whose CTAs are all resident at once (the CTAs of a launch wait for each
+// other), asked of the runtime once per device and kernel; 0 = run without clusters. Capped at 32 clusters: with
+// one CTA per SM the B200 co-schedules 32 clusters of 4 (its GPCs hold 16 to 20 usable SMs), and 128 CTAs
+// already draw the full HBM bandwidth (measured: a plain streaming kernel reads at the same rate with 74 CTAs
+// as with 148).
+constexpr int MAX_CLUSTERS = 32, MIN_CLUSTERS = 16;
 template <int NT, int SL, bool QKN>
-int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, const MParams& mp, int grid) {
+int cluster_capacity(int stages) {
+    static int memo[MAX_DEVICES];
+    static bool known[MAX_DEVICES] = {};
+    const int dev = current_device_slot();
+    if (dev >= 0 && known[dev]) return memo[dev];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CS * MAX_CLUSTERS);
+    cfg.blockDim = dim3(N_THREADS);
+    cfg.dynamicSmemBytes = (size_t)(1024 + stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT));
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CS;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<NT, SL, QKN>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    n = std::min(n, MAX_CLUSTERS);
+    if (n < MIN_CLUSTERS) n = 0;
+    if (dev >= 0) { memo[dev] = n; known[dev] = true; }
+    return n;
+}
+
+template <int NT, int SL, bool QKN>
+int set_attr() {
     static bool attr_set[MAX_DEVICES] = {};
-    const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
     const int dev = current_device_slot();
     if (dev < 0 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL, QKN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         if (dev >= 0) attr_set[dev] = true;
     }
-    const cudaError_t e = launch_pdl(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
+    return DFLASH_OK;
+}
+
+// `grid_free`: CTAs the work itself asks for (one per SM, fewer for tiny problems). With token tiles of up to
+// 32 rows the launch runs in clusters of CS CTAs when the device co-schedules enough of them: phases with fewer
+// tiles than CTAs then split each tile's K range inside a cluster instead of through global memory.
+template <int NT, int SL, bool QKN>
+int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, MParams& mp, int grid_free) {
+    if (set_attr<NT, SL, QKN>() != DFLASH_OK) return DFLASH_ERR_CUDA;
+    const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
+    int grid = grid_free;
+    mp.cs = 1;
+    if (NT <= 32 && grid_free >= CS) {
+        const int n_cl = std::min(cluster_capacity<NT, SL, QKN>(mp.stages), grid_free / CS);
+        if (n_cl >= 1) { mp.cs = CS; grid = n_cl * CS; }
+    }
+    // Cluster mode for the phases whose tiles fill whole rounds of one tile per cluster (or less than one round):
+    // every CTA then streams the same bytes. Other tile counts (48 QKV tiles over 32 clusters) would leave some
+    // CTAs twice the bytes of others, and a lone CTA cannot draw much more than its even share of HBM bandwidth
+    // through a ring of this depth (measured: the phase took as long as with the split through global memory).
+    for (int i = 0; i < mp.n_phases; ++i) {
+        const KParams& p = mp.ph[i];
+        const int n_cl = grid / CS;
+        mp.ph[i].cluster_k = (mp.cs > 1 && p.n_tiles < grid && p.chunks_total >= CS && (p.n_tiles <= n_cl || p.n_tiles % n_cl == 0)) ? 1 : 0;
+    }
+    const cudaError_t e =
+        mp.cs > 1 ? launch_pdl_cluster(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, CS, tw, tx, mp)
+                  : launch_pdl(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
