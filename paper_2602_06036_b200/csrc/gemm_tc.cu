@@ -551,6 +551,12 @@ __device__ __forceinline__ void token_rstd(const KParams& p, int tok_base, int n
     }
 }
 
+// Counter increment that publishes what this CTA wrote: the CTA's threads meet at a barrier, then ONE thread adds
+// with release semantics at GPU scope (cumulative over the writes ordered before it by the barrier); readers poll
+// with ld_acquire. Cheaper than a fence by each of the 128 threads.
+__device__ __forceinline__ void red_release_add(int32_t* p, int v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 // Bounded poll of a global counter written by other CTAs (release/acquire through L2).
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     int v;
@@ -586,12 +592,12 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     float* sRstd = reinterpret_cast<float*>(sRed + 128);          // [TOK_CACHE] per-token rsqrt(mean square)
     int* sPos = reinterpret_cast<int*>(sRstd + TOK_CACHE);        // [TOK_CACHE] per-token position (-1: skip)
     int* sPage = sPos + TOK_CACHE;                                // [TOK_CACHE] per-token physical page
-    float* sXch = reinterpret_cast<float*>(sPage + TOK_CACHE);    // [2][CS - 1][NT / CS][128] columns received from cluster peers
+    float* sXch = reinterpret_cast<float*>(sPage + TOK_CACHE);    // [2][CS - 1][128][NT / CS] columns received from cluster peers
     uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(sXch) + xch_bytes(NT));
     uint64_t* empty = full + MAX_STAGES;
     uint64_t* acc_full = empty + MAX_STAGES;
     uint64_t* acc_empty = acc_full + 2;
-    uint64_t* xch_bar = acc_empty + 2;                            // [2] one per receive buffer: (CS - 1) peers x 4 warps arrive
+    uint64_t* xch_bar = acc_empty + 2;                            // [2] one per receive buffer: counts the bytes the peers' stores deliver
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(xch_bar + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [2] epilogue abort
     int* sPend = const_cast<int*>(flags) + 4;                               // [3 * MAX_STAGES] producer's queue
@@ -600,7 +606,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); mbar_init(&xch_bar[b], (CS - 1) * 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); mbar_init(&xch_bar[b], 1); }
         flags[0] = 0; flags[2] = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -611,8 +617,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     pdl_trigger();
-    // peers must not write into this CTA's receive buffers or arrive on its barriers before they exist
-    if (mp.cs > 1) cluster_sync_all();
+    // Peers must not write into this CTA's receive buffers or count bytes on its barriers before they exist: every
+    // thread arrives on the cluster barrier here and waits on it later, where its role has nothing better to do (the
+    // epilogue warps before their first tile, the two single-thread roles at their end).
+    if (mp.cs > 1) cluster_arrive();
 
     const int G = gridDim.x;
 
@@ -706,6 +714,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             }
         }
         __syncwarp();     // the whole warp must reach the closing barrier together
+        if (mp.cs > 1) cluster_wait();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
@@ -744,6 +753,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             }
         }
         __syncwarp();
+        if (mp.cs > 1) cluster_wait();
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quadrant = warp % 4 ----------------
         const int ew = warp & 3;
@@ -760,6 +770,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         }
         uint32_t cl_units = 0;       // cluster-shared tiles finished so far (the same number in every CTA of the cluster)
         pdl_wait();      // lengths, page tables, residual rows ... come from earlier kernels
+        if (mp.cs > 1) cluster_wait();      // every peer has set up its barriers (they arrived after doing so)
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
             const long long T = (long long)shared_tiles(p, G) * p.chunks_total;      // pairs of the shared part
@@ -880,14 +891,18 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     if (un.cl) {
                         // ---- the tile is shared by the CTAs of this cluster, each holding the sums over its K share.
                         // Rank q finishes token columns [q * GC, (q + 1) * GC): every CTA sends those columns of its
-                        // accumulator into rank q's receive buffer (distributed shared memory) and arrives on q's
-                        // barrier; q adds the four pieces in rank order (bit-reproducible) and runs the epilogue.
-                        // Two buffers suffice: a peer sends its (i+2)-th tile only after it has received this CTA's
-                        // (i+1)-th, which is sent after the i-th was read; phases are separated by the phase counter.
+                        // accumulator into rank q's receive buffer with asynchronous stores into distributed shared
+                        // memory that count as transactions on q's barrier; q adds the four pieces in rank order
+                        // (bit-reproducible) and runs the epilogue. Every CTA sends every column and waits for all its
+                        // peers whether or not its columns hold tokens, which keeps the cluster in step: a peer sends
+                        // its (i+2)-th tile only after it has received this CTA's (i+1)-th, which is sent after the
+                        // i-th was read, so two buffers suffice; phases are separated by the phase counter.
                         constexpr int GC = NT / CS;
+                        static_assert(GC % 4 == 0, "columns per rank travel as groups of four floats");
                         const uint32_t xb = cl_units & 1, xpar = (cl_units >> 1) & 1;
                         ++cl_units;
                         const int tok0 = tok_base + rank * GC;
+                        if (row == 0) mbar_expect_tx(&xch_bar[xb], (uint32_t)((CS - 1) * GC * TILE_F * 4));
                         float own[GC];
 #pragma unroll
                         for (int c = 0; c < GC; ++c) own[c] = 0.f;
@@ -896,24 +911,21 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                             float v[CH];
                             tmem_ld_cols<CH>(tmem_base + buf * NT + ch * CH + ((uint32_t)(ew * 32) << 16), v);
 #pragma unroll
-                            for (int c = 0; c < CH; ++c) {
-                                const int col = ch * CH + c, q = col / GC, lc = col % GC;      // compile-time after unrolling
-                                if (q == rank) own[lc] = v[c];
-                                else if (tok_base + col < p.M) {
+                            for (int c4 = 0; c4 < CH; c4 += 4) {
+                                const int col = ch * CH + c4, q = col / GC, lc = col % GC;      // compile-time after unrolling
+                                if (q == rank) {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) own[lc + e] = v[c4 + e];
+                                } else {
                                     const int slot = rank - (rank > q ? 1 : 0);
-                                    st_cluster_f32(xch_remote[q] + (uint32_t)((((xb * (CS - 1) + slot) * GC + lc) * TILE_F + row) * 4), v[c]);
+                                    st_async_f32x4(xch_remote[q] + (uint32_t)((((xb * (CS - 1) + slot) * TILE_F + row) * GC + lc) * 4), v[c4],
+                                                   v[c4 + 1], v[c4 + 2], v[c4 + 3], xbar_remote[q] + xb * 8);
                                 }
                             }
                         }
                         tc_fence_before();
-                        fence_acq_rel_cluster();
                         __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(&acc_empty[buf]);
-#pragma unroll
-                            for (int q = 0; q < CS; ++q)
-                                if (q != rank) mbar_arrive_cluster(xbar_remote[q] + xb * 8);
-                        }
+                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
                         // residual rows travel while the peers' columns arrive
                         float xres[CH], gain = 0.f;
                         residual_load<CH>(p, un, tok0, row, xres, gain, GC);
@@ -921,14 +933,20 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         epi_bar();
                         if (flags[2]) { alive = false; break; }
                         if (tok0 < p.M) {
-                            const float* rx = sXch + (size_t)xb * (CS - 1) * GC * TILE_F + row;
+                            const float* rx = sXch + ((size_t)xb * (CS - 1) * TILE_F + row) * GC;
 #pragma unroll
-                            for (int lc = 0; lc < GC; ++lc) {
-                                float a = 0.f;
+                            for (int l4 = 0; l4 < GC; l4 += 4) {
+                                float a[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                                for (int j = 0; j < CS; ++j)
-                                    a += (j == rank) ? own[lc] : rx[((j - (j > rank ? 1 : 0)) * GC + lc) * TILE_F];
-                                sAcc[row * ACC_LD + lc] = p.ssq_in ? a * sRstd[tok_off + rank * GC + lc] : a;
+                                for (int j = 0; j < CS; ++j) {
+                                    float4 t;
+                                    if (j == rank) t = make_float4(own[l4], own[l4 + 1], own[l4 + 2], own[l4 + 3]);
+                                    else t = *reinterpret_cast<const float4*>(rx + (size_t)(j - (j > rank ? 1 : 0)) * TILE_F * GC + l4);
+                                    a[0] += t.x; a[1] += t.y; a[2] += t.z; a[3] += t.w;
+                                }
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    sAcc[row * ACC_LD + l4 + e] = p.ssq_in ? a[e] * sRstd[tok_off + rank * GC + l4 + e] : a[e];
                             }
                             epi_bar();
                             apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok0, row, sPos + tok_off + rank * GC, sPage + tok_off + rank * GC,
@@ -961,9 +979,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 if (!un.full) {
                     // the tile is shared: publish the piece, take a ticket, finish the tile at the end of the phase
-                    __threadfence();
                     epi_bar();
-                    if (row == 0) atomicAdd(p.counters + un.tile, 1);
+                    if (row == 0) red_release_add(p.counters + un.tile, 1);
                     pend[n_pend++] = un;
                     if (w.shared_done() && !w.done(p)) {      // whole tiles follow: reduce now, under their main loop
                         finish_shared();
@@ -975,11 +992,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             if (n_pend > 0) finish_shared();
             if (!alive) break;
             // this CTA's share of the phase is done and visible: tell the others
-            __threadfence();
             epi_bar();
             if (row == 0) {
                 trace_max(p.trace, 3);
-                atomicAdd(mp.phase_done + ph, 1);
+                red_release_add(mp.phase_done + ph, 1);
             }
         }
         if (flags[2] && row == 0) {
