@@ -114,8 +114,23 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # the step
 # ------------------------------------------------------------------------------------------------
+def make_lib(cfg, device, max_ctx, seed=0):
+    """A library handle holding the seeded random-init weights, with rotary tables long enough for max_ctx."""
+    from paper_2602_06036_b200 import binding
+    lib = binding.DFlash(cfg, str(device))
+    w = synth.make_weights(cfg, seed)
+    cos, sin = synth.rope_tables(cfg, max_ctx + 4 * cfg.block_size + 8)
+    lib.set_weights(synth.pack_device_weights(cfg, w), cos, sin)
+    return lib
+
+
 class Step:
-    def __init__(self, wl, device, seed=0, temperature=0.0, fuse_ctx=True):
+    """One workload's buffers and its step. `full_verify` (the serving-mix workload): the verify side of the step is
+    the target-shaped (B+1)-row causal verify attention of one layer over a paged target cache + the LM head with
+    row argmax on the [S * (B+1), D] target-shaped hidden + the accept rule on those ids, as the benchmark
+    definition words it; otherwise (and as a separately timed figure) verify/accept starts from given target logits."""
+
+    def __init__(self, wl, device, seed=0, temperature=0.0, fuse_ctx=True, lib=None, full_verify=None):
         from paper_2602_06036_b200 import binding
         cfg = wl.cfg
         self.T = float(temperature)
@@ -123,11 +138,8 @@ class Step:
         self.wl, self.cfg, self.dev = wl, cfg, device
         B, S = cfg.block_size, wl.batch
         self.gamma = B
-        self.lib = binding.DFlash(cfg, str(device))
-        w = synth.make_weights(cfg, seed)
-        cos, sin = synth.rope_tables(cfg, max(wl.ctx_lens) + 4 * B + 8)
-        self.lib.set_weights(synth.pack_device_weights(cfg, w), cos, sin)
-        del w
+        self.full_verify = (wl.name == "cfg4" and self.T <= 0) if full_verify is None else bool(full_verify)
+        self.lib = lib if lib is not None else make_lib(cfg, device, max(wl.ctx_lens), seed)
         caps = [L + 2 * B + 2 for L in wl.ctx_lens]
         table, n_pages = synth.make_page_table(cfg, caps, seed)
         self.page_table = table.to(device)
@@ -181,6 +193,26 @@ class Step:
         self.max_ctx = max(wl.ctx_lens)
         self.rows_new = int(self.n_new.sum().item())
         self.side = None
+        self.vlib = None
+        if self.full_verify:
+            # the target's side of the cycle, one target-shaped layer (same head geometry as the drafter's layers):
+            # its own paged cache over the same page table, the rotated queries and tail keys/values of the gamma+1
+            # verify rows, and the hidden rows its LM head reads; all N(0,1), seeded
+            import dataclasses
+            tcfg = dataclasses.replace(cfg, n_layers=1)
+            self.vlib = binding.DFlash(tcfg, str(device))
+            R = g + 1
+            self.t_pool = torch.empty(synth.kv_pool_shape(tcfg, n_pages), dtype=cfg.torch_dtype, device=device)
+            gen = torch.Generator(device=device)
+            gen.manual_seed(1234 + seed)
+            self.t_pool.normal_(0.0, 1.0, generator=gen)
+            mk = lambda *shape: torch.empty(shape, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen).to(cfg.torch_dtype)
+            self.t_q = mk(S, R, cfg.n_q_heads, cfg.head_dim)
+            self.t_k = mk(S, R, cfg.n_kv_heads, cfg.head_dim)
+            self.t_v = mk(S, R, cfg.n_kv_heads, cfg.head_dim)
+            self.t_attn = torch.zeros_like(self.t_q)
+            self.t_hidden = mk(S * R, cfg.d_model)
+            self.t_ids = torch.zeros(S * R, dtype=torch.int32, device=device)
         if self.T > 0:
             # sampling: the draft's logits are kept (fp32), drafts are drawn from them, and verification
             # is speculative sampling; the uniforms are seeded inputs
@@ -204,10 +236,23 @@ class Step:
         else:
             lib.dflash_draft_block(anchor, self.ctx_len, self.max_ctx, self.page_table, self.pool, self.draft_ids, ctx=ctx)
 
+    def run_verify_full(self):
+        # causal verify attention of one target-shaped layer, LM head + row argmax over the gamma+1 rows of every
+        # sequence, accept rule on the resulting ids (the drafter's own block is what gets verified)
+        from paper_2602_06036_b200 import binding
+        self.vlib.dflash_block_attention(binding.ATTN_CAUSAL, self.t_q, self.t_k, self.t_v, self.ctx_len, self.max_ctx,
+                                         self.page_table, self.t_pool, 0, self.t_attn)
+        self.lib.dflash_lmhead_argmax(self.t_hidden, 1, self.t_ids)
+        self.lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
+                                      self.out_tokens, self.bonus, self.new_len,
+                                      target_ids=self.t_ids.view(self.wl.batch, self.gamma + 1))
+
     def run_verify(self, logits):
-        # The target's verify pass is outside this library; its logits are an input. The drafts
-        # verified are synthetic ones with a planted agreeing prefix (the random-init drafter would
-        # never be accepted), so the accept kernel sees realistic accept lengths.
+        # The target's forward is outside this step: its logits are an input. What is verified is the drafter's own
+        # block of this step (random-init weights, so tau = 1 nearly always; the kernels' cost does not depend on
+        # tau). The planted-prefix drafts of the synthetic verify case are exercised by the parity tests.
+        if self.full_verify:
+            return self.run_verify_full()
         if self.T > 0:
             self.lib.dflash_verify_accept_sample(logits, self.draft_logits, self.cfg.block_size, self.draft_ids,
                                                  self.cfg.block_size, self.gamma, self.T, self.u_acc, self.u_fin,
@@ -220,6 +265,16 @@ class Step:
         self.run_draft(self.d_feats, self.d_anchor)
         self.run_verify(self.d_logits)
 
+    def verify_from_logits(self):
+        self.lib.dflash_verify_accept(self.draft_ids, self.cfg.block_size, self.gamma, self.ctx_len, self.tau,
+                                      self.out_tokens, self.bonus, self.new_len, logits=self.d_logits)
+
+    def dev_status(self):
+        st = int(self.lib.status.item())
+        if self.vlib is not None:
+            st |= int(self.vlib.status.item())
+        return st
+
     def step_e2e(self):
         # The verify logits are only needed at the end of the step: their host-to-device copy runs on a
         # side stream next to the context projection and the draft (a fork/join inside the captured graph).
@@ -229,6 +284,11 @@ class Step:
         if self.side is None:
             self.side = torch.cuda.Stream()
         self.e_in.copy_(self.h_in, non_blocking=True)
+        if self.full_verify:       # the verify side's inputs are produced on the device by the target: nothing to copy
+            self.run_draft(self.e_feats, self.e_anchor)
+            self.run_verify_full()
+            self.h_out.copy_(self.d_out, non_blocking=True)
+            return
         self.side.wait_stream(cur)
         with torch.cuda.stream(self.side):
             self.e_logits.copy_(self.h_logits, non_blocking=True)
@@ -238,8 +298,9 @@ class Step:
         self.h_out.copy_(self.d_out, non_blocking=True)
 
     def e2e_bytes(self):
-        h2d = self.h_in.numel() + \
-            self.h_logits.numel() * self.h_logits.element_size()
+        h2d = self.h_in.numel()
+        if not self.full_verify:
+            h2d += self.h_logits.numel() * self.h_logits.element_size()
         return h2d, self.h_out.numel() * 4
 
 
@@ -258,23 +319,29 @@ def max_over_ranks(ms, device):
     return float(t.item())
 
 
-def timed(fn, steps, warmup, dist_on):
+def timed(fn, steps, warmup, dist_on, repeats=1):
+    """`repeats` timed regions of exactly `steps` calls each, every region bracketed by a barrier (N > 1) and a
+    device synchronisation on both sides and timed with a CUDA event pair on the launching stream; per region the
+    maximum over ranks. Returns the list of region times in ms."""
     for _ in range(warmup):
         fn()
-    torch.cuda.synchronize()
-    if dist_on:
-        torch.distributed.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        fn()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        ms = max_over_ranks(ms, "cuda")
-    return ms
+    out = []
+    for _ in range(max(repeats, 1)):
+        torch.cuda.synchronize()
+        if dist_on:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist_on:
+            ms = max_over_ranks(ms, "cuda")
+        out.append(ms)
+    return out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -401,61 +468,50 @@ def run_kernel_only(args, step, device):
         fn = lambda: step.lib.dflash_block_attention(binding.ATTN_FULL, q, k, v, step.ctx_len, step.max_ctx,
                                                      step.page_table, step.pool, 0, out)
         nbytes = algorithmic_bytes(cfg, wl.ctx_lens, 0)["attention"]
-    ms = timed(fn, args.steps, args.warmup, False)
+    ms = timed(fn, args.steps, args.warmup, False)[0]
     us = ms / args.steps * 1e3
     print(json.dumps({"kernel": args.kernel, "workload": wl.name, "us_per_call": us, "alg_bytes": nbytes,
                       "gbs": nbytes / (us * 1e-6) / 1e9}))
 
 
 # ------------------------------------------------------------------------------------------------
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg1")
-    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify", "block_loss"],
-                    help="run one building block alone (for profiler captures) instead of the step")
-    ap.add_argument("--loss-blocks", type=int, default=512, help="--kernel block_loss: blocks (of block_size rows) per call")
-    ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
-    ap.add_argument("--temperature", type=float, default=0.0,
-                    help="> 0: drafts are drawn from the draft's logits and verified by speculative sampling (default: greedy)")
-    ap.add_argument("--separate-ctx", action="store_true",
-                    help="run the context projection as its own call before the draft call instead of inside it")
-    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
+def phase_table(trace_rows, cfg, alg, hbm, prefix=""):
+    """Per kernel family: microseconds per launch from a device-side timeline (a phase's interval runs from
+    max(its inputs ready, previous record's end) to the moment its last CTA signalled completion)."""
+    kernels = {}
+    prev_end = None
+    for fam, t_start, t_dep, t_loop, t_end in trace_rows:
+        if t_end is None:
+            continue
+        cands = [v for v in (t_dep, prev_end) if v is not None]
+        begin = max(cands) if cands else t_start
+        dur = max(t_end - begin, 0) / 1e3
+        prev_end = t_end if prev_end is None else max(prev_end, t_end)
+        e = kernels.setdefault(prefix + fam, {"us_total": 0.0, "launches_per_step": 0})
+        e["us_total"] += dur
+        e["launches_per_step"] += 1
+    for fam, e in kernels.items():
+        n = e["launches_per_step"]
+        if fam == "attention":               # one or two records (main kernel, merge kernel) make one attention per layer
+            n = cfg.n_layers
+            e["launches_per_step"] = n
+        if fam == "verify_attention":
+            n = 1
+            e["launches_per_step"] = n
+        e["us_per_launch"] = e.pop("us_total") / n
+        if fam in alg and e["us_per_launch"] > 0:
+            e["alg_bytes"] = alg[fam]
+            e["gbs"] = alg[fam] / (e["us_per_launch"] * 1e-6) / 1e9
+            e["frac_hbm"] = e["gbs"] / hbm
+    return kernels
 
-    if args.impl == "reference":
-        run_reference(args)
-        return
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dist_on = world > 1
-    torch.cuda.set_device(local)
-    device = torch.device(f"cuda:{local}")
-    if dist_on:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.distributed.init_process_group("nccl", device_id=device)
-
-    from paper_2602_06036_b200 import binding, build
-    build.build()
-    wl = synth.workload(args.workload)
-    cfg = wl.cfg
-    peaks = load_peaks()
-    # replicas: every rank runs the same batch on its own GPU; there is no data-path collective
-    step = Step(wl, device, seed=0, temperature=args.temperature, fuse_ctx=not args.separate_ctx)
+def measure(step, args, peaks, dist_on, rank, sampler=None, repeats=7, e2e_repeats=3):
+    """Times one workload's step (resident: CUDA-graph replay unless --no-graph; end to end: host buffers through
+    the C ABI), checks the timed step's outputs, and reads the device-side timeline of one eager step."""
+    from paper_2602_06036_b200 import binding
+    wl, cfg = step.wl, step.cfg
     S, B = wl.batch, cfg.block_size
-
-    if args.kernel:
-        run_kernel_only(args, step, device)
-        return
-
-    sampler = ClockSampler(local)
     run_resident, run_e2e = step.step_resident, step.step_e2e
     for _ in range(2):           # eager warm-up: sizes the workspace, sets kernel attributes
         run_resident()
@@ -467,18 +523,181 @@ def main():
     if not args.no_graph:
         run_resident = capture(step.step_resident)
         run_e2e = capture(step.step_e2e)
-    if rank == 0:
+    step.lib.status.zero_()
+    if step.vlib is not None:
+        step.vlib.status.zero_()
+    if sampler is not None:
         sampler.start()
-    ms = timed(run_resident, args.steps, args.warmup, dist_on)
-    launches = launches_per_step * args.steps
-    clocks = sampler.stop() if rank == 0 else None
-    ms_e2e = timed(run_e2e, args.steps, args.warmup, dist_on)
+    regions = timed(run_resident, args.steps, args.warmup, dist_on, repeats)
+    clocks = sampler.stop() if sampler is not None else None
+    out_resident = step.d_out.clone()
+    regions_e2e = timed(run_e2e, args.steps, args.warmup, dist_on, e2e_repeats)
+    torch.cuda.synchronize()
+    # the timed steps' results: no device-detected problem (bad id / page, expired wait), the end-to-end run's
+    # outputs equal the resident run's (same inputs), and what came back to the host is what the device holds
+    status = step.dev_status()
+    same = bool(torch.equal(step.d_out, out_resident)) and bool(torch.equal(step.h_out, step.d_out.cpu()))
+    in_range = bool(((step.draft_ids >= 0) & (step.draft_ids < cfg.vocab)).all().item()) and \
+        bool(((step.tau >= 1) & (step.tau <= step.gamma + 1)).all().item())
+    checked = status == 0 and same and in_range
+    if not checked:
+        raise RuntimeError(f"bench self-check failed on {wl.name}: dev_status={status} outputs_equal={same} in_range={in_range}")
 
-    # Per-kernel figures. Chained launches hide their phases from CUDA events, so the library's
-    # device-side timeline (global-timer stamps written by the kernels themselves) is read for one
-    # extra, eager step: a phase's interval runs from max(its inputs ready, previous record's end) to
-    # the moment its last CTA signalled completion.
-    trace_rows = step.lib.trace(step.step_resident) if rank == 0 else []
+    per = sorted(ms / args.steps for ms in regions)
+    per_step_ms = statistics.median(per)
+    per_e2e = statistics.median(ms / args.steps for ms in regions_e2e)
+    res = {"ms_per_step": per_step_ms, "ms_per_step_min": per[0], "ms_per_step_max": per[-1], "regions": len(per),
+           "ms_per_step_e2e": per_e2e, "launches_per_step": int(launches_per_step), "clocks": clocks, "checked": True}
+    if rank != 0:
+        return res
+    alg = algorithmic_bytes(cfg, wl.ctx_lens, step.rows_new)
+    hbm = peaks["hbm_gbs"]
+    es = 4 if cfg.dtype == "fp32" else 2
+    # device-side timeline of one extra eager step; the verify side of the serving-mix step runs on a second
+    # handle (the target-shaped layer) and on the LM head of this one: traced separately and prefixed
+    if step.full_verify:
+        kernels = phase_table(step.lib.trace(lambda: step.run_draft(step.d_feats, step.d_anchor)), cfg, alg, hbm)
+        alg_v = {"verify_attention": 2 * cfg.kv_dim * es * sum(wl.ctx_lens), "verify_lmhead_argmax": alg["lmhead_argmax"]}
+        from paper_2602_06036_b200 import binding as bnd
+        tr_a = step.vlib.trace(lambda: step.vlib.dflash_block_attention(bnd.ATTN_CAUSAL, step.t_q, step.t_k, step.t_v, step.ctx_len,
+                                                                         step.max_ctx, step.page_table, step.t_pool, 0, step.t_attn))
+        kernels.update(phase_table(tr_a, cfg, alg_v, hbm, prefix="verify_"))
+        tr_l = step.lib.trace(lambda: step.lib.dflash_lmhead_argmax(step.t_hidden, 1, step.t_ids))
+        kernels.update(phase_table(tr_l, cfg, alg_v, hbm, prefix="verify_"))
+        res["trace_rows"] = []
+    else:
+        rows = step.lib.trace(step.step_resident)
+        kernels = phase_table(rows, cfg, alg, hbm)
+        res["trace_rows"] = rows
+    # lower bound of the step: its phases run one after the other, each bound by the slower of its
+    # HBM traffic and its dense bf16 contraction (2 x rows x weights; sustained tensor figure)
+    tensor = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    bound_s, tensor_phases = 0.0, []
+    phases = [("ctx_fuse", 1, step.rows_new, alg["ctx_fuse"]), ("ctx_kv", 1, step.rows_new, alg["ctx_kv"]),
+              ("gemm_qkv", cfg.n_layers, S * B, alg["gemm_qkv"]), ("gemm_o", cfg.n_layers, S * B, alg["gemm_o"]),
+              ("gemm_gateup", cfg.n_layers, S * B, alg["gemm_gateup"]), ("gemm_down", cfg.n_layers, S * B, alg["gemm_down"]),
+              ("lmhead_argmax", 1, S * B, alg["lmhead_argmax"]), ("attention", cfg.n_layers, 0, alg["attention"])]
+    step_bytes = alg["draft_block_total"] + alg["ctx_project_total"]
+    if step.full_verify:
+        phases += [("verify_attention", 1, 0, alg_v["verify_attention"]),
+                   ("verify_lmhead_argmax", 1, S * (B + 1), alg_v["verify_lmhead_argmax"])]
+        step_bytes += alg_v["verify_attention"] + alg_v["verify_lmhead_argmax"]
+    else:
+        step_bytes += S * (B + 1) * cfg.vocab * 2
+        bound_s += S * (B + 1) * cfg.vocab * 2 / (hbm * 1e9)      # verify reads the target logits once
+    for fam, n_launch, rows_, nbytes in phases:
+        t_hbm = nbytes / (hbm * 1e9)
+        t_tc = 2.0 * rows_ * (nbytes / es) / tensor if cfg.dtype != "fp32" else 0.0
+        if t_tc > t_hbm:
+            tensor_phases.append(fam)
+        bound_s += n_launch * max(t_hbm, t_tc)
+        if fam in kernels:
+            kernels[fam]["us_at_peak"] = max(t_hbm, t_tc) * 1e6
+            kernels[fam]["bound"] = "tensor" if t_tc > t_hbm else "hbm"
+            kernels[fam]["frac_of_bound"] = kernels[fam]["us_at_peak"] / kernels[fam]["us_per_launch"]
+    res.update({"alg": alg, "kernels": kernels, "step_bytes": step_bytes,
+                "step_roofline": {"alg_bytes": step_bytes, "us_at_hbm_peak": step_bytes / (hbm * 1e9) * 1e6,
+                                  "us_at_peak": bound_s * 1e6, "frac": bound_s / (per_step_ms * 1e-3),
+                                  "tensor_bound_phases": tensor_phases,
+                                  "note": "sum over the step's phases of max(bytes / measured HBM, flops / measured sustained bf16)"}})
+    if step.full_verify:
+        # the same step's verify side from given target logits instead (the logits cross HBM once), timed alone
+        fn = step.verify_from_logits
+        fn()
+        fn = fn if args.no_graph else capture(fn)
+        ms = statistics.median(timed(fn, args.steps, 3, False, 3)) / args.steps
+        nb = S * (B + 1) * cfg.vocab * 2
+        res["accept_from_logits"] = {"us_per_call": ms * 1e3, "alg_bytes": nb, "gbs": nb / (ms * 1e-3) / 1e9,
+                                     "frac_hbm": nb / (ms * 1e-3) / 1e9 / hbm}
+    return res
+
+
+def step_text(step, args):
+    if args.temperature > 0:
+        return f"ctx_project(n_new=tau) + draft_block(logits kept) + sample_rows + verify_accept_sample, T={args.temperature}"
+    if step.full_verify:
+        return ("ctx_project(n_new=tau) + draft_block + causal verify attention of one target-shaped layer over (B+1) rows + "
+                "LM head with row argmax on [S*(B+1), D] + verify_accept(ids)")
+    return "ctx_project(n_new=tau) + draft_block + verify_accept(logits)"
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` started without a launcher: start the N ranks ourselves (one process per GPU,
+    the same command line torch.distributed.run would be given) and pass their output through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.exit(subprocess.call(cmd))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify", "block_loss", "attention_bwd"],
+                    help="run one building block alone (for profiler captures) instead of the step")
+    ap.add_argument("--loss-blocks", type=int, default=512, help="--kernel block_loss: blocks (of block_size rows) per call")
+    ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="> 0: drafts are drawn from the draft's logits and verified by speculative sampling (default: greedy)")
+    ap.add_argument("--separate-ctx", action="store_true",
+                    help="run the context projection as its own call before the draft call instead of inside it")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--repeats", type=int, default=7, help="timed regions of --steps steps each; ms_per_step is their median")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the extra key with the other benchmark configurations (cfg2, cfg3, cfg4) measured in the same run")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world == 1 and "RANK" not in os.environ:
+        spawn_ranks(args.gpus)
+    if world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); start one rank per GPU "
+                 f"(python -m torch.distributed.run --nproc-per-node {args.gpus} ...) or run plain `python bench.py --gpus {args.gpus}`")
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    if dist_on:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+
+    from paper_2602_06036_b200 import build
+    build.build()
+    wl = synth.workload(args.workload)
+    cfg = wl.cfg
+    peaks = load_peaks()
+    hbm = peaks["hbm_gbs"]
+    others = [] if (args.no_other_workloads or args.kernel or args.temperature > 0 or cfg.dtype == "fp32") else \
+        [n for n in ("cfg1", "cfg2", "cfg3", "cfg4") if n != wl.name]
+    if not others or args.workload == "cfg0":
+        others = []
+    # replicas: every rank runs the same batch on its own GPU; there is no data-path collective.
+    # One handle (one copy of the weights) serves every workload of the run.
+    max_ctx = max([max(wl.ctx_lens)] + [max(synth.workload(n).ctx_lens) for n in others])
+    lib = make_lib(cfg, device, max_ctx, seed=0)
+    step = Step(wl, device, seed=0, temperature=args.temperature, fuse_ctx=not args.separate_ctx, lib=lib)
+    S, B = wl.batch, cfg.block_size
+
+    if args.kernel:
+        run_kernel_only(args, step, device)
+        return
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    m = measure(step, args, peaks, dist_on, rank, sampler, repeats=args.repeats)
     # The dominant kernel alone, timed with CUDA event pairs around each of its launches.
     lm_us = None
     if rank == 0:
@@ -490,47 +709,43 @@ def main():
         prof_lm = step.lib.profile(lm_call, max(args.steps, 10))
         lm_us = prof_lm.get("lmhead_argmax", (None, 0))[0]
     if args.trace and rank == 0:
-        rows = trace_rows
         with open(args.trace, "w") as f:
             f.write("# kernel family, first CTA start, dependency resolved, main loop end, last CTA exit (us since first start)\n")
-            for fam, a, b, c, d in rows:
+            for fam, a, b, c, d in m.get("trace_rows", []):
                 us = lambda v: "      -" if v is None else f"{v / 1e3:8.2f}"
                 f.write(f"{fam:16s} {us(a)} {us(b)} {us(c)} {us(d)}\n")
+
+    h2d, d2h = step.e2e_bytes()
+    main_step_text = step_text(step, args)
+    # the other benchmark configurations, same process and weights (every rank runs them: the regions hold barriers)
+    extra = {}
+    del step
+    for name in others:
+        torch.cuda.empty_cache()
+        st2 = Step(synth.workload(name), device, seed=0, fuse_ctx=not args.separate_ctx, lib=lib)
+        r = measure(st2, args, peaks, dist_on, rank, None, repeats=3, e2e_repeats=1)
+        if rank == 0:
+            S2 = st2.wl.batch
+            e = {"ms_per_step": r["ms_per_step"], "ms_per_step_min": r["ms_per_step_min"], "ms_per_step_max": r["ms_per_step_max"],
+                 "us_per_draft_block": r["ms_per_step"] * 1e3, "draft_tokens_per_s": S2 * B * world / (r["ms_per_step"] * 1e-3),
+                 "ms_per_step_e2e": r["ms_per_step_e2e"], "batch": S2, "ctx_tokens": int(sum(st2.wl.ctx_lens)),
+                 "step": step_text(st2, args), "step_roofline": r["step_roofline"], "kernels": r["kernels"],
+                 "gpu_launches_per_step": r["launches_per_step"], "checked": r["checked"]}
+            if "accept_from_logits" in r:
+                e["accept_from_logits"] = r["accept_from_logits"]
+            extra[name] = e
+        del st2
 
     if rank != 0:
         if dist_on:
             torch.distributed.destroy_process_group()
         return
 
-    per_step_ms = ms / args.steps
+    per_step_ms = m["ms_per_step"]
     tokens = S * B * world
     value = tokens / (per_step_ms * 1e-3)
-    e2e_value = tokens / (ms_e2e / args.steps * 1e-3)
-    h2d, d2h = step.e2e_bytes()
-    alg = algorithmic_bytes(cfg, wl.ctx_lens, step.rows_new)
-    hbm = peaks["hbm_gbs"]
-    kernels = {}
-    prev_end = None
-    for fam, t_start, t_dep, t_loop, t_end in trace_rows:
-        if t_end is None:
-            continue
-        cands = [v for v in (t_dep, prev_end) if v is not None]
-        begin = max(cands) if cands else t_start
-        dur = max(t_end - begin, 0) / 1e3
-        prev_end = t_end if prev_end is None else max(prev_end, t_end)
-        e = kernels.setdefault(fam, {"us_total": 0.0, "launches_per_step": 0})
-        e["us_total"] += dur
-        e["launches_per_step"] += 1
-    for fam, e in kernels.items():
-        n = e["launches_per_step"]
-        if fam == "attention":               # one or two records (main kernel, merge kernel) make one attention per layer
-            n = cfg.n_layers
-            e["launches_per_step"] = n
-        e["us_per_launch"] = e.pop("us_total") / n
-        if fam in alg and e["us_per_launch"] > 0:
-            e["alg_bytes"] = alg[fam]
-            e["gbs"] = alg[fam] / (e["us_per_launch"] * 1e-6) / 1e9
-            e["frac_hbm"] = e["gbs"] / hbm
+    e2e_value = tokens / (m["ms_per_step_e2e"] * 1e-3)
+    alg, kernels = m["alg"], m["kernels"]
     roofline = None
     if lm_us:
         traffic = None
@@ -546,45 +761,30 @@ def main():
                     "timing": "CUDA event pair around each launch of the kernel run alone (dflash_lmhead_argmax), "
                               "same weights and row count as in the step",
                     "in_step_us": kernels.get("lmhead_argmax", {}).get("us_per_launch")}
-    step_bytes = alg["draft_block_total"] + alg["ctx_project_total"] + S * (B + 1) * cfg.vocab * 2
-    # lower bound of the step: its phases run one after the other, each bound by the slower of its
-    # HBM traffic and its dense bf16 contraction (2 x rows x weights; sustained tensor figure)
-    tensor = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
-    es = 4 if cfg.dtype == "fp32" else 2
-    bound_s, tensor_phases = 0.0, []
-    for fam, n_launch, rows in (("ctx_fuse", 1, step.rows_new), ("ctx_kv", 1, step.rows_new),
-                                ("gemm_qkv", cfg.n_layers, S * B), ("gemm_o", cfg.n_layers, S * B),
-                                ("gemm_gateup", cfg.n_layers, S * B), ("gemm_down", cfg.n_layers, S * B),
-                                ("lmhead_argmax", 1, S * B), ("attention", cfg.n_layers, 0)):
-        t_hbm = alg[fam] / (hbm * 1e9)
-        t_tc = 2.0 * rows * (alg[fam] / es) / tensor if cfg.dtype != "fp32" else 0.0
-        if t_tc > t_hbm:
-            tensor_phases.append(fam)
-        bound_s += n_launch * max(t_hbm, t_tc)
-        if fam in kernels:
-            kernels[fam]["us_at_peak"] = max(t_hbm, t_tc) * 1e6
-            kernels[fam]["bound"] = "tensor" if t_tc > t_hbm else "hbm"
-    bound_s += S * (B + 1) * cfg.vocab * 2 / (hbm * 1e9)      # verify reads the target logits once
     line = {
         "metric": "draft_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": per_step_ms, "us_per_draft_block": per_step_ms * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "batch": S, "block_size": B, "ctx_lens": list(wl.ctx_lens)[:8],
-                   "step": "ctx_project(n_new=tau) + draft_block + verify_accept(logits)" if args.temperature <= 0 else
-                           f"ctx_project(n_new=tau) + draft_block(logits kept) + sample_rows + verify_accept_sample, T={args.temperature}",
+                   "step": main_step_text,
                    "l2": "per-step weight traffic (3.2 GB) exceeds the 126 MB L2; no flush",
                    "launch": "eager" if args.no_graph else "cuda graph replay of one step",
                    "parallelism": "replicas" if world > 1 else "single"},
-        "step_roofline": {"alg_bytes": step_bytes, "us_at_hbm_peak": step_bytes / (hbm * 1e9) * 1e6,
-                          "us_at_peak": bound_s * 1e6, "frac": bound_s / (per_step_ms * 1e-3),
-                          "tensor_bound_phases": tensor_phases,
-                          "note": "sum over the step's phases of max(bytes / measured HBM, flops / measured sustained bf16)"},
+        "timing": {"regions": m["regions"], "steps_per_region": args.steps, "ms_per_step_median": per_step_ms,
+                   "ms_per_step_min": m["ms_per_step_min"], "ms_per_step_max": m["ms_per_step_max"],
+                   "note": "ms_per_step is the median over the timed regions; each region is exactly `steps` steps between "
+                           "synchronisations, timed by a CUDA event pair, maximum over ranks"},
+        "checked": m["checked"],
+        "checked_note": "after timing: device status word 0, the end-to-end run's outputs equal the resident run's and the host copy, ids and accept lengths in range",
+        "step_roofline": m["step_roofline"],
         "roofline": roofline, "kernels": kernels,
         "kernels_note": "device-side timeline of one eager step: per phase, from inputs ready to last CTA done",
-        "clocks": clocks, "gpu_launches": int(launches),
+        "clocks": m["clocks"], "gpu_launches": int(m["launches_per_step"] * args.steps * m["regions"]),
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / args.steps},
+                "ms_per_step": m["ms_per_step_e2e"]},
     }
+    if extra:
+        line["workloads"] = extra
     if not args.no_cpu_baseline:
         # the whole step (all layers, full vocabulary) for one sequence: about 10-30 s of host work
         reps, spent = [], 0.0

@@ -514,7 +514,23 @@ __global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict
         const int body = (hi - lo - head) / VEC;
         for (int i = threadIdx.x; i < head; i += blockDim.x) top2_push(t, to_f(src[lo + i]), lo + i);
         const uint4* v = reinterpret_cast<const uint4*>(src + lo + head);
-        for (int i = threadIdx.x; i < body; i += blockDim.x) {
+        // four 16-byte loads in flight per thread: a long segment (few segments per row when there are many rows) is
+        // otherwise one dependent load after the other
+        constexpr int INFL = 4;
+        int i = threadIdx.x;
+        for (; i + (INFL - 1) * (int)blockDim.x < body; i += INFL * blockDim.x) {
+            uint4 w[INFL];
+#pragma unroll
+            for (int u = 0; u < INFL; ++u) w[u] = __ldg(v + i + u * blockDim.x);
+#pragma unroll
+            for (int u = 0; u < INFL; ++u) {
+                const T* e = reinterpret_cast<const T*>(&w[u]);
+                const int base = lo + head + (i + u * (int)blockDim.x) * VEC;
+#pragma unroll
+                for (int k = 0; k < VEC; ++k) top2_push(t, to_f(e[k]), base + k);
+            }
+        }
+        for (; i < body; i += blockDim.x) {
             const uint4 w = __ldg(v + i);
             const T* e = reinterpret_cast<const T*>(&w);
             const int base = lo + head + i * VEC;
