@@ -63,6 +63,16 @@ Training loss of a block (Sec. 4.2 "Loss weighting", Eq. 4; App. A.1 for gamma) 
 Pins (tests/test_oracle_loss.py): w_1 = 1 and the constant ratio exp(-1/gamma), the printed gamma of
 each block size, uniform logits -> ln V, a dominant logit -> 0, gradient rows summing to zero, central
 finite differences of the summed loss, gamma -> infinity = unweighted sum.
+
+Training-side attention of anchor blocks (Sec. 4.2 "Random sampling of masked blocks": all blocks of a sequence
+in one forward and backward pass under a mask that is bidirectional inside a block, open towards the injected
+context before the block's anchor and closed between blocks)      -> block_attention_lse, block_attention_backward
+  The forward of that mask is block_attention per block with L = the anchor's position; the backward is the
+  plain softmax-attention gradient; context gradients of the blocks add up per position.
+Pins (tests/test_oracle_attention_bwd.py): central finite differences of block_attention in every input,
+torch autograd of an independently written attention, sum over keys of dV = sum over rows of dout, key
+gradients of a kv head summing to zero, a lone key passes dout straight to its value, exp(lse) = sum of exp,
+context gradients of two blocks over one sequence against finite differences of the joint loss.
 """
 from __future__ import annotations
 
@@ -219,6 +229,66 @@ def block_attention(q, k_ctx, v_ctx, k_blk, v_blk, scale, causal=False):
         p = p / np.sum(p, axis=-1, keepdims=True)
         out[:, h] = p @ vals
     return out
+
+
+def block_attention_lse(q, k_ctx, v_ctx, k_blk, v_blk, scale, causal=False):
+    """The log-sum-exp of every query row's scaled scores, [R, Hq] (natural logarithm): what a backward pass
+    keeps from the forward instead of the probabilities."""
+    q = _f64(q)
+    R, Hq, hd = q.shape
+    group = Hq // k_blk.shape[1]
+    L = k_ctx.shape[0]
+    lse = np.empty((R, Hq), dtype=F64)
+    for h in range(Hq):
+        kv = h // group
+        keys = np.concatenate((_f64(k_ctx[:, kv]), _f64(k_blk[:, kv])), axis=0)
+        s = (q[:, h] @ keys.T) * scale
+        if causal:
+            r = np.arange(R)
+            s[:, L:][r[None, :] > r[:, None]] = -np.inf
+        m = np.max(s, axis=-1)
+        lse[:, h] = m + np.log(np.sum(np.exp(s - m[:, None]), axis=-1))
+    return lse
+
+
+def block_attention_backward(q, k_ctx, v_ctx, k_blk, v_blk, dout, scale, causal=False):
+    """Gradient of block_attention for one block (training side, Sec. 4.2: many anchor blocks of one sequence are
+    trained in a single forward and backward pass; a block attends to the injected context before its anchor and,
+    in both directions, to itself). Given dout = d loss / d out [R, Hq, hd], returns
+    (dq [R, Hq, hd], dk_ctx [L, Hkv, hd], dv_ctx [L, Hkv, hd], dk_blk [R, Hkv, hd], dv_blk [R, Hkv, hd]).
+
+    Plain softmax-attention calculus per query head h (kv head h // group), keys = [context ; block]:
+      P = softmax(scale * q K^T)            dV  = P^T dout
+      dP = dout V^T                         dS  = P * (dP - rowsum(dP * P))
+      dq = scale * dS K                     dK  = scale * dS^T q
+    The gradients of a kv head add up over the query heads of its group. With many blocks over one cached
+    sequence the context gradients of the blocks add up position by position (the caller sums them)."""
+    q = _f64(q)
+    dout = _f64(dout)
+    R, Hq, hd = q.shape
+    Hkv = k_blk.shape[1]
+    group = Hq // Hkv
+    L = k_ctx.shape[0]
+    dq = np.zeros((R, Hq, hd), dtype=F64)
+    dk = np.zeros((L + R, Hkv, hd), dtype=F64)
+    dv = np.zeros((L + R, Hkv, hd), dtype=F64)
+    for h in range(Hq):
+        kv = h // group
+        keys = np.concatenate((_f64(k_ctx[:, kv]), _f64(k_blk[:, kv])), axis=0)   # [L+R, hd]
+        vals = np.concatenate((_f64(v_ctx[:, kv]), _f64(v_blk[:, kv])), axis=0)
+        s = (q[:, h] @ keys.T) * scale
+        if causal:
+            r = np.arange(R)
+            s[:, L:][r[None, :] > r[:, None]] = -np.inf
+        s = s - np.max(s, axis=-1, keepdims=True)
+        p = np.exp(s)
+        p = p / np.sum(p, axis=-1, keepdims=True)                                  # [R, L+R]
+        dv[:, kv] += p.T @ dout[:, h]
+        dp = dout[:, h] @ vals.T
+        ds = p * (dp - np.sum(dp * p, axis=-1, keepdims=True))
+        dq[:, h] = (ds @ keys) * scale
+        dk[:, kv] += (ds.T @ q[:, h]) * scale
+    return dq, dk[:L], dv[:L], dk[L:], dv[L:]
 
 
 # --------------------------------------------------------------------------------------------
