@@ -455,6 +455,41 @@ def run_kernel_only(args, step, device):
         sums = torch.zeros(2, dtype=torch.float32, device=device)
         fn = lambda: step.lib.dflash_block_loss(z, t, gamma, row_loss, sums, dz, grad_scale=1.0 / (nb * (B - 1)))
         nbytes = 2 * z.numel() * 2
+    elif args.kernel == "attention_bwd":
+        # Training side: backward of the block attention over one training sequence (App. A.1: 3072 tokens, 512
+        # anchor blocks of 16 rows; --loss-blocks for a smaller capture), one layer of the drafter's head geometry.
+        # Bound: the five contractions of the softmax-attention gradient, 2 flops per multiply-add, over the keys
+        # each block sees (context before its anchor + itself) against the sustained bf16 tensor figure; the
+        # operands stay in L2 (the sequence's K/V of one layer is 12.6 MB), so HBM only sees q, k, v, out, dout
+        # and the gradients once.
+        nb, Lseq = args.loss_blocks, 3072
+        table, n_pages = synth.make_page_table(cfg, [Lseq], 2)
+        table = table.to(device).repeat(nb, 1).contiguous()
+        pool = torch.randn(synth.kv_pool_shape(cfg, n_pages), device=device).to(cfg.torch_dtype)
+        gen = torch.Generator().manual_seed(5)
+        anchors = torch.randint(1, Lseq - B, (nb,), generator=gen, dtype=torch.int32).to(device)
+        mk = lambda *shape: torch.randn(*shape, device=device).to(cfg.torch_dtype)
+        q, k, v = mk(nb, B, cfg.n_q_heads, cfg.head_dim), mk(nb, B, cfg.n_kv_heads, cfg.head_dim), mk(nb, B, cfg.n_kv_heads, cfg.head_dim)
+        dout, out = mk(nb, B, cfg.n_q_heads, cfg.head_dim), torch.zeros(nb, B, cfg.n_q_heads, cfg.head_dim, device=device, dtype=cfg.torch_dtype)
+        lse = torch.zeros(nb, B, cfg.n_q_heads, dtype=torch.float32, device=device)
+        max_a = int(anchors.max().item())
+        step.lib.dflash_block_attention(binding.ATTN_FULL, q, k, v, anchors, max_a, table, pool, 0, out, lse_out=lse)
+        dq, dk, dv = torch.zeros_like(q), torch.zeros_like(k), torch.zeros_like(v)
+        dkv = torch.zeros((n_pages, 2, cfg.n_kv_heads, cfg.page_size, cfg.head_dim), dtype=torch.float32, device=device)
+        fn = lambda: step.lib.dflash_block_attention_bwd(binding.ATTN_FULL, q, k, v, out, lse, dout, anchors, max_a, table, pool, 0,
+                                                         dq, dk, dv, dkv, shared_page_row=True)
+        keys = float((anchors.float() + B).sum().item())
+        flops = 5 * 2.0 * (B * cfg.n_q_heads) * cfg.head_dim * keys
+        nbytes = (3 * q.numel() + 2 * q.numel() + 4 * k.numel()) * 2 + 2 * cfg.kv_dim * 2 * Lseq + dkv.numel() * 4 * Lseq // (n_pages * cfg.page_size)
+        ms = timed(fn, args.steps, args.warmup, False)[0]
+        us = ms / args.steps * 1e3
+        peaks = load_peaks()
+        tf = flops / (us * 1e-6) / 1e12
+        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        print(json.dumps({"kernel": "attention_bwd", "blocks": nb, "seq_len": Lseq, "us_per_call": us, "flops": flops, "tflops": tf,
+                          "bound": "tensor", "peak_tflops": peak, "frac": tf / peak, "hbm_bytes": nbytes,
+                          "us_at_tensor_peak": flops / (peak * 1e12) * 1e6, "us_at_hbm_peak": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6}))
+        return
     elif args.kernel == "lmhead":
         hid = torch.randn(S * B, cfg.d_model, device=device).to(cfg.torch_dtype)
         ids = torch.zeros(S * B, dtype=torch.int32, device=device)

@@ -338,8 +338,55 @@ typedef struct {
     void*          workspace;
     int64_t        workspace_bytes;
     int32_t*       dev_status;
+    float*         lse_out;      /* [device] out [batch, rows, Hq] fp32; may be NULL. Natural-log sum of exponentials
+                                    of every row's scaled scores (what dflash_block_attention_bwd takes back)  */
 } dflash_attn_args;
 int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a /*[host]*/, void* stream);
+
+/* ---- training side: backward pass of the block attention (Sec. 4.2: all anchor blocks of a sequence are trained
+ * in one forward and one backward pass; a block attends in both directions to itself and to the injected context
+ * before its anchor, never to another block) ----
+ * The forward of that mask is dflash_block_attention over a batch of blocks with ctx_len[b] = position of block
+ * b's anchor (mode FULL), all blocks sharing one page-table row. Given dout = d loss / d out, per query head h
+ * (kv head h / (Hq/Hkv)), with P the forward's probabilities over keys = [context ; block]:
+ *     dV = P^T dout     dP = dout V^T     dS = P * (dP - rowsum(dout * out))     dq = scale dS K     dK = scale dS^T q
+ * P is recomputed from q, the keys and the forward's log-sum-exp (lse_out of dflash_block_attention); no
+ * probability matrix is stored. Gradients of a kv head add up over the q heads of its group.
+ * dkv_ctx receives the context gradients of ONE layer in the pool's own layout, fp32:
+ *     dkv_ctx[page][K=0|V=1][kv_head][slot][head_dim]
+ * for every page that holds positions below max_ctx_len of a page-table row in use (whole pages are written,
+ * zeros where no block sees a key); other pages are not touched. shared_page_row = 1 (the training layout): every
+ * block reads page-table row 0 and the gradients of a position add up over all blocks that see it, in batch order
+ * (bit-reproducible, no atomics). shared_page_row = 0: block b uses row b and owns its pages.
+ * bf16 handles with head_dim 128, 64-token pages and rows * (Hq/Hkv) <= 64 only (DFLASH_ERR_UNSUPPORTED else).
+ * Workspace as for dflash_block_attention. Errors as there; a ctx_len above max_ctx_len is clamped and flagged. */
+typedef struct {
+    int32_t        mode;          /* DFLASH_ATTN_FULL | DFLASH_ATTN_CAUSAL (as in the forward)          */
+    const void*    q;             /* [device] [batch, rows, Hq, hd]                                    */
+    const void*    k_blk;         /* [device] [batch, rows, Hkv, hd]                                   */
+    const void*    v_blk;         /* [device] [batch, rows, Hkv, hd]                                   */
+    const void*    out;           /* [device] [batch, rows, Hq, hd] the forward's output               */
+    const float*   lse;           /* [device] [batch, rows, Hq] the forward's lse_out                  */
+    const void*    dout;          /* [device] [batch, rows, Hq, hd] gradient of the loss w.r.t. out    */
+    int32_t        batch, rows;
+    const int32_t* ctx_len;       /* [device] [batch]                                                  */
+    int32_t        max_ctx_len;   /* [host value] upper bound of ctx_len                               */
+    const int32_t* page_table;    /* [device] [batch, max_pages] (row 0 only if shared_page_row)       */
+    int32_t        max_pages;
+    const void*    kv_pool;       /* [device] pool, layout at the top of this file                     */
+    int32_t        n_pool_pages;
+    int32_t        layer;
+    int32_t        shared_page_row;
+    void*          dq;            /* [device] out [batch, rows, Hq, hd] config dtype                   */
+    void*          dk_blk;        /* [device] out [batch, rows, Hkv, hd]                               */
+    void*          dv_blk;        /* [device] out [batch, rows, Hkv, hd]                               */
+    float*         dkv_ctx;       /* [device] out fp32 [n_pool_pages, 2, Hkv, page_size, hd]; may be NULL (then the
+                                     context gradients are not computed)                               */
+    void*          workspace;     /* [device] >= dflash_workspace_bytes(h, batch, batch * rows)        */
+    int64_t        workspace_bytes;
+    int32_t*       dev_status;    /* [device] may be NULL                                              */
+} dflash_attn_bwd_args;
+int32_t dflash_block_attention_bwd(dflash_handle* h, const dflash_attn_bwd_args* a /*[host]*/, void* stream);
 
 /* ---- building block: LM head fused with row-wise argmax (Sec. 4.2: LM head shared with the
  * target). ids[m] = argmax_v (W_lm z_m)_v with z = hidden (apply_norm = 0) or

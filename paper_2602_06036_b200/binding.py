@@ -29,6 +29,7 @@ EXPORTS = (
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
     "dflash_verify_accept_static", "dflash_sample_rows", "dflash_verify_accept_sample",
     "dflash_sample_workspace_bytes", "dflash_target_verify", "dflash_block_loss", "dflash_attention_plan",
+    "dflash_block_attention_bwd",
 )
 N_FAMILIES = 15
 
@@ -115,7 +116,17 @@ class AttnArgs(C.Structure):
                 ("batch", C.c_int32), ("rows", C.c_int32), ("ctx_len", C.c_void_p), ("max_ctx_len", C.c_int32),
                 ("page_table", C.c_void_p), ("max_pages", C.c_int32), ("kv_pool", C.c_void_p),
                 ("n_pool_pages", C.c_int32), ("layer", C.c_int32), ("out", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p),
+                ("lse_out", C.c_void_p)]
+
+
+class AttnBwdArgs(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("q", C.c_void_p), ("k_blk", C.c_void_p), ("v_blk", C.c_void_p), ("out", C.c_void_p),
+                ("lse", C.c_void_p), ("dout", C.c_void_p), ("batch", C.c_int32), ("rows", C.c_int32), ("ctx_len", C.c_void_p),
+                ("max_ctx_len", C.c_int32), ("page_table", C.c_void_p), ("max_pages", C.c_int32), ("kv_pool", C.c_void_p),
+                ("n_pool_pages", C.c_int32), ("layer", C.c_int32), ("shared_page_row", C.c_int32), ("dq", C.c_void_p),
+                ("dk_blk", C.c_void_p), ("dv_blk", C.c_void_p), ("dkv_ctx", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_int64), ("dev_status", C.c_void_p)]
 
 
 class LmHeadArgs(C.Structure):
@@ -145,7 +156,7 @@ def load():
                      ("dflash_verify_accept", VerifyArgs), ("dflash_verify_accept_static", VerifyArgs), ("dflash_block_attention", AttnArgs),
                      ("dflash_lmhead_argmax", LmHeadArgs), ("dflash_sample_rows", SampleArgs),
                      ("dflash_verify_accept_sample", VerifySampleArgs), ("dflash_target_verify", TargetArgs),
-                     ("dflash_block_loss", BlockLossArgs)):
+                     ("dflash_block_loss", BlockLossArgs), ("dflash_block_attention_bwd", AttnBwdArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(st), C.c_void_p]
         fn.restype = C.c_int32
@@ -421,13 +432,25 @@ class DFlash:
         _check(self.lib.dflash_verify_accept_sample(self.h, C.byref(a), _stream(stream)))
 
     def dflash_block_attention(self, mode, q, k_blk, v_blk, ctx_len, max_ctx_len, page_table, kv_pool, layer,
-                               out, stream=None):
+                               out, stream=None, lse_out=None):
         S, R = q.shape[0], q.shape[1]
         ws = self.workspace(S, S * R)
         a = AttnArgs(mode, _ptr(q), _ptr(k_blk), _ptr(v_blk), S, R, _ptr(ctx_len), int(max_ctx_len),
                      _ptr(page_table), page_table.shape[1], _ptr(kv_pool), kv_pool.shape[1], layer, _ptr(out),
-                     _ptr(ws), ws.numel(), _ptr(self.status))
+                     _ptr(ws), ws.numel(), _ptr(self.status), _ptr(lse_out))
         _check(self.lib.dflash_block_attention(self.h, C.byref(a), _stream(stream)))
+
+    def dflash_block_attention_bwd(self, mode, q, k_blk, v_blk, out, lse, dout, ctx_len, max_ctx_len, page_table, kv_pool, layer,
+                                   dq, dk_blk, dv_blk, dkv_ctx=None, shared_page_row=False, stream=None):
+        """Gradients of dflash_block_attention: dq / dk_blk / dv_blk like q / k_blk / v_blk; dkv_ctx fp32
+        [n_pool_pages, 2, Hkv, page_size, hd] (one layer, the pool's layout) or None."""
+        S, R = q.shape[0], q.shape[1]
+        ws = self.workspace(S, S * R)
+        a = AttnBwdArgs(mode, _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out), _ptr(lse), _ptr(dout), S, R, _ptr(ctx_len),
+                        int(max_ctx_len), _ptr(page_table), page_table.shape[1], _ptr(kv_pool), kv_pool.shape[1], layer,
+                        1 if shared_page_row else 0, _ptr(dq), _ptr(dk_blk), _ptr(dv_blk), _ptr(dkv_ctx), _ptr(ws), ws.numel(),
+                        _ptr(self.status))
+        _check(self.lib.dflash_block_attention_bwd(self.h, C.byref(a), _stream(stream)))
 
     def dflash_lmhead_argmax(self, hidden, apply_norm, ids, top1=None, margin=None, logits_out=None, stream=None):
         M = hidden.shape[0]

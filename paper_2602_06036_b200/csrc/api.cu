@@ -675,6 +675,26 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a, void
     return DFLASH_OK;
 }
 
+int32_t dflash_block_attention_bwd(dflash_handle* h, const dflash_attn_bwd_args* a, void* stream) {
+    if (!h || !a) return DFLASH_ERR_INVALID_ARG;
+    if (a->batch < 0 || a->rows < 0 || a->rows > 32 || a->max_pages < 1 || a->n_pool_pages < 1 || a->layer < 0 ||
+        a->layer >= h->cfg.n_layers || a->max_ctx_len < 0)
+        return DFLASH_ERR_INVALID_ARG;
+    if (a->mode != DFLASH_ATTN_FULL && a->mode != DFLASH_ATTN_CAUSAL) return DFLASH_ERR_INVALID_ARG;
+    if (a->batch == 0 || a->rows == 0) return DFLASH_OK;
+    if (!a->q || !a->k_blk || !a->v_blk || !a->out || !a->lse || !a->dout || !a->ctx_len || !a->page_table || !a->kv_pool ||
+        !a->dq || !a->dk_blk || !a->dv_blk)
+        return DFLASH_ERR_INVALID_ARG;
+    if ((int64_t)a->batch * a->rows > (1 << 20)) return DFLASH_ERR_UNSUPPORTED;
+    if (!attn_bwd_supported(h->cfg, a->rows)) return DFLASH_ERR_UNSUPPORTED;
+    Workspace ws;
+    DFLASH_TRY(check_ws(h, a->workspace, a->workspace_bytes, a->batch, a->batch * a->rows, &ws));
+    Launch L{h, (cudaStream_t)stream, a->dev_status, nullptr};
+    // ws.tmp holds rows * d_model floats: room for one float per (row, q head)
+    RUN(FAM_ATTENTION, launch_attention_bwd(L, *a, ws.tmp));
+    return DFLASH_OK;
+}
+
 int32_t dflash_attention_plan(const dflash_handle* h, int32_t batch, int32_t max_ctx_len, int64_t* out) {
     if (!h || !out || batch < 1 || max_ctx_len < 0) return DFLASH_ERR_INVALID_ARG;
     const AttnPlan pl = attn_tc_plan(h->cfg, batch, max_ctx_len, h->sm_count);

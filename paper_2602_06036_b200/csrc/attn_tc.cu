@@ -59,6 +59,7 @@ struct AParams {
     const int32_t* early_len;   // with early_kv: rows [0, early_len[b]) are the final ones (nullptr: all of ctx_len[b])
     const int32_t* page_table;
     __nv_bfloat16* out;
+    float* lse;       // [S, R, Hq] natural-log sum of exponentials per query row, or nullptr
     float* part;
     int32_t* status;
     unsigned long long* trace;
@@ -520,6 +521,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
             }
             if (n_splits > 1) srow[HD >> 2] = make_float4(M, l_tot, 0.f, 0.f);
+            else if (p.lse && row_valid)      // M and the sum are in the log2 domain
+                p.lse[((size_t)b * p.R + r) * p.Hq + g * p.group + j] = (l_tot > 0.f) ? (M + log2f(l_tot)) * 0.6931471805599453f : -CUDART_INF_F;
         }
         if (wg == 0 && n_splits > 1 && !flags[0]) {
             wg_bar(0);
@@ -607,6 +610,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AParams p) {
     }
     const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
     const int r = row / p.group, j = row % p.group;
+    if (p.lse && lane == 0) p.lse[((size_t)b * p.R + r) * p.Hq + g * p.group + j] = (Lsum > 0.f) ? (M + log2f(Lsum)) * 0.6931471805599453f : -CUDART_INF_F;
     __nv_bfloat16* dst = p.out + (((size_t)b * p.R + r) * p.Hq + g * p.group + j) * HD + lane * 4;
     uint2 w2;
     w2.x = pack_bf16(acc.x * inv, acc.y * inv);
@@ -686,7 +690,7 @@ int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part,
     p.n_chunks = plan.n_chunks;
     p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
     p.ctx_len = a.ctx_len; p.page_table = a.page_table;
-    p.out = (__nv_bfloat16*)a.out; p.part = part; p.status = L.status; p.trace = L.trace;
+    p.out = (__nv_bfloat16*)a.out; p.lse = a.lse_out; p.part = part; p.status = L.status; p.trace = L.trace;
     (void)counters;
 
     CUtensorMap tq, tpool, tkb, tvb;

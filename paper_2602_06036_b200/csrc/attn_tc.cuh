@@ -30,4 +30,9 @@ AttnPlan attn_tc_plan(const dflash_config& c, int batch, int max_ctx_len, int sm
 int launch_attention_tc(const Launch& L, const dflash_attn_args& a, float* part, int32_t* counters, bool early_kv = false,
                         const int32_t* early_len = nullptr, bool first_of_call = false);
 
+// Backward of the block attention (tensor-core path): rows * (Hq/Hkv) <= 64, head_dim 128, 64-token pages.
+// `D`: fp32 scratch [batch * rows * Hq] (rowsum(dO * O), handed from the first kernel to the second).
+bool attn_bwd_supported(const dflash_config& c, int rows);
+int launch_attention_bwd(const Launch& L, const dflash_attn_bwd_args& a, float* D);
+
 }  // namespace dflash

@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(
     const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
     const T* __restrict__ pool, const int32_t* __restrict__ page_table, const int32_t* __restrict__ ctx_len,
     T* __restrict__ out, int R, int Hq, int Hkv, int hd, int PG, int max_pages, int n_pages, int layer,
-    float scale, int causal, int32_t* status) {
+    float scale, int causal, int32_t* status, float* __restrict__ lse) {
     __shared__ float sq[128];
     __shared__ float sp[128];
     __shared__ float red[32];
@@ -379,6 +379,7 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(
         __syncthreads();
     }
     if (tid < hd) out[(row * Hq + h) * hd + tid] = from_f<T>(l > 0.f ? acc / l : 0.f);
+    if (lse && tid == 0) lse[row * Hq + h] = l > 0.f ? m + logf(l) : -CUDART_INF_F;
 }
 
 int launch_attention_simt(const Launch& L, const dflash_attn_args& a) {
@@ -390,13 +391,13 @@ int launch_attention_simt(const Launch& L, const dflash_attn_args& a) {
         attention_simt_kernel<float><<<grid, 128, 0, L.st>>>(
             (const float*)a.q, (const float*)a.k_blk, (const float*)a.v_blk, (const float*)a.kv_pool,
             a.page_table, a.ctx_len, (float*)a.out, a.rows, c.n_q_heads, c.n_kv_heads, c.head_dim, c.page_size,
-            a.max_pages, a.n_pool_pages, a.layer, c.softmax_scale, causal, L.status);
+            a.max_pages, a.n_pool_pages, a.layer, c.softmax_scale, causal, L.status, a.lse_out);
     else
         attention_simt_kernel<__nv_bfloat16><<<grid, 128, 0, L.st>>>(
             (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k_blk, (const __nv_bfloat16*)a.v_blk,
             (const __nv_bfloat16*)a.kv_pool, a.page_table, a.ctx_len, (__nv_bfloat16*)a.out, a.rows,
             c.n_q_heads, c.n_kv_heads, c.head_dim, c.page_size, a.max_pages, a.n_pool_pages, a.layer,
-            c.softmax_scale, causal, L.status);
+            c.softmax_scale, causal, L.status, a.lse_out);
     DFLASH_CHECK_LAUNCH();
     return DFLASH_OK;
 }

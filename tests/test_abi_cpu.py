@@ -40,7 +40,8 @@ def test_struct_layouts_match_the_header():
                "dflash_draft_args": binding.DraftArgs, "dflash_verify_args": binding.VerifyArgs,
                "dflash_attn_args": binding.AttnArgs, "dflash_lmhead_args": binding.LmHeadArgs,
                "dflash_sample_args": binding.SampleArgs, "dflash_verify_sample_args": binding.VerifySampleArgs,
-               "dflash_target_args": binding.TargetArgs, "dflash_block_loss_args": binding.BlockLossArgs}
+               "dflash_target_args": binding.TargetArgs, "dflash_block_loss_args": binding.BlockLossArgs,
+               "dflash_attn_bwd_args": binding.AttnBwdArgs}
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "dflash.h"', "int main(void){"]
     for cname, st in structs.items():
         lines.append(f'printf("{cname} %zu\\n", sizeof({cname}));')

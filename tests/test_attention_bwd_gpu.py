@@ -1,0 +1,174 @@
+"""GPU parity of the training-side attention backward (dflash_block_attention_bwd) and of the forward's
+log-sum-exp output against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dflash_oracle as orc
+from paper_2602_06036_b200 import synth
+from tests.harness import Case
+
+pytestmark = pytest.mark.gpu
+
+# Gradients come out of bf16 tensor-core products of recomputed probabilities: P and dS are rounded to bf16
+# (relative 2^-9 each) before the contractions that add up 64..10^4 of them, accumulation is fp32. The
+# relative-L2 bound is the benchmark definition's for bf16 values; the absolute bound scales with the size of
+# the reference values (context gradients are sums over hundreds of blocks and grow like sqrt of their count).
+REL_L2 = 1e-2
+
+
+def close(got, ref, what):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.all(np.isfinite(got)), what
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    mx = float(np.max(np.abs(got - ref))) if got.size else 0.0
+    bound = 5e-2 * max(1.0, float(np.sqrt(np.mean(ref * ref)))) if ref.size else 0.0
+    assert rel <= REL_L2 and mx <= bound, f"{what}: rel_l2={rel:.3e} max_abs={mx:.3e} (bound {bound:.3e})"
+
+
+def _run(case, mode, q, k, v, dout, ctx, table, max_ctx, layer, shared):
+    from paper_2602_06036_b200 import binding
+    cfg, dev = case.cfg, case.device
+    S, R = q.shape[0], q.shape[1]
+    m = binding.ATTN_CAUSAL if mode == "causal" else binding.ATTN_FULL
+    d = lambda t: t.to(dev)
+    qd, kd, vd, dod = d(q), d(k), d(v), d(dout)
+    out = torch.zeros_like(qd)
+    lse = torch.zeros((S, R, cfg.n_q_heads), dtype=torch.float32, device=dev)
+    case.lib.status.zero_()
+    case.lib.dflash_block_attention(m, qd, kd, vd, ctx, max_ctx, table, case.pool, layer, out, lse_out=lse)
+    dq, dk, dv = torch.zeros_like(qd), torch.zeros_like(kd), torch.zeros_like(vd)
+    dkv = torch.full((case.n_pages, 2, cfg.n_kv_heads, cfg.page_size, cfg.head_dim), float("nan"), dtype=torch.float32, device=dev)
+    case.lib.dflash_block_attention_bwd(m, qd, kd, vd, out, lse, dod, ctx, max_ctx, table, case.pool, layer, dq, dk, dv, dkv,
+                                        shared_page_row=shared)
+    torch.cuda.synchronize()
+    assert int(case.lib.status.item()) == 0
+    f = lambda t: t.float().cpu().numpy()
+    return f(out), f(lse), f(dq), f(dk), f(dv), dkv.cpu().numpy()
+
+
+def _gather_ctx_grad(dkv, table_row, L, cfg):
+    """dK, dV [L, Hkv, hd] of logical positions 0..L-1 from the pool-shaped gradient."""
+    dK = np.zeros((L, cfg.n_kv_heads, cfg.head_dim))
+    dV = np.zeros_like(dK)
+    for p0 in range(0, L, cfg.page_size):
+        n = min(cfg.page_size, L - p0)
+        page = int(table_row[p0 // cfg.page_size])
+        dK[p0:p0 + n] = np.transpose(dkv[page, 0, :, :n, :], (1, 0, 2))
+        dV[p0:p0 + n] = np.transpose(dkv[page, 1, :, :n, :], (1, 0, 2))
+    return dK, dV
+
+
+@pytest.mark.parametrize("mode,R", [("full", 16), ("causal", 9), ("full", 5)])
+def test_backward_of_separate_sequences(mode, R):
+    cfg = synth.MID
+    lens = (0, 1, 63, 64, 65, 300)
+    case = Case(cfg, lens, seed=23)
+    case.fill_pool_synthetic()
+    S, layer = len(lens), 1
+    mk = lambda name, *shape: synth.normal(shape, 1.0, 23, name, cfg.torch_dtype)
+    q, k, v = mk("b.q", S, R, cfg.n_q_heads, cfg.head_dim), mk("b.k", S, R, cfg.n_kv_heads, cfg.head_dim), mk("b.v", S, R, cfg.n_kv_heads, cfg.head_dim)
+    dout = mk("b.do", S, R, cfg.n_q_heads, cfg.head_dim)
+    out, lse, dq, dk, dv, dkv = _run(case, mode, q, k, v, dout, case.ctx_len, case.page_table, max(lens), layer, shared=False)
+    n32 = synth.to_numpy_f32
+    for b, L in enumerate(lens):
+        kc, vc = orc.pool_read(case.pool_np, case.page_table_cpu[b].numpy(), L, layer, cfg.page_size)
+        args = (n32(q[b]), kc, vc, n32(k[b]), n32(v[b]))
+        causal = mode == "causal"
+        np.testing.assert_allclose(lse[b], orc.block_attention_lse(*args, cfg.softmax_scale, causal=causal), atol=2e-2, rtol=0)
+        rdq, rdkc, rdvc, rdkb, rdvb = orc.block_attention_backward(*args, n32(dout[b]), cfg.softmax_scale, causal=causal)
+        close(dq[b], rdq, f"dq seq {b} L={L}")
+        close(dk[b], rdkb, f"dk_blk seq {b}")
+        close(dv[b], rdvb, f"dv_blk seq {b}")
+        if L:
+            gK, gV = _gather_ctx_grad(dkv, case.page_table_cpu[b].numpy(), L, cfg)
+            close(gK, rdkc, f"dK_ctx seq {b}")
+            close(gV, rdvc, f"dV_ctx seq {b}")
+            # slots of the last page beyond the context hold exact zeros (whole pages are written)
+            last = int(case.page_table_cpu[b, (L - 1) // cfg.page_size])
+            n = L - (L - 1) // cfg.page_size * cfg.page_size
+            assert np.all(dkv[last, :, :, n:, :] == 0)
+
+
+def test_backward_of_anchor_blocks_over_one_sequence_adds_context_gradients_in_order():
+    cfg = synth.MID
+    one = Case(cfg, (330,), seed=29)
+    one.fill_pool_synthetic()
+    anchors = (0, 16, 64, 65, 200, 313, 17, 130)
+    S, R, layer = len(anchors), cfg.block_size, 0
+    table = one.page_table.repeat(S, 1).contiguous()
+    ctx = torch.tensor(anchors, dtype=torch.int32, device=one.device)
+    mk = lambda name, *shape: synth.normal(shape, 1.0, 29, name, cfg.torch_dtype)
+    q, k, v = mk("t.q", S, R, cfg.n_q_heads, cfg.head_dim), mk("t.k", S, R, cfg.n_kv_heads, cfg.head_dim), mk("t.v", S, R, cfg.n_kv_heads, cfg.head_dim)
+    dout = mk("t.do", S, R, cfg.n_q_heads, cfg.head_dim)
+    res = _run(one, "full", q, k, v, dout, ctx, table, max(anchors), layer, shared=True)
+    out, lse, dq, dk, dv, dkv = res
+    n32 = synth.to_numpy_f32
+    Lmax = max(anchors)
+    sumK = np.zeros((Lmax, cfg.n_kv_heads, cfg.head_dim))
+    sumV = np.zeros_like(sumK)
+    for b, a in enumerate(anchors):
+        kc, vc = orc.pool_read(one.pool_np, one.page_table_cpu[0].numpy(), a, layer, cfg.page_size)
+        rdq, rdkc, rdvc, rdkb, rdvb = orc.block_attention_backward(n32(q[b]), kc, vc, n32(k[b]), n32(v[b]), n32(dout[b]), cfg.softmax_scale)
+        close(dq[b], rdq, f"dq block at {a}")
+        close(dk[b], rdkb, f"dk_blk block at {a}")
+        close(dv[b], rdvb, f"dv_blk block at {a}")
+        sumK[:a] += rdkc
+        sumV[:a] += rdvc
+    gK, gV = _gather_ctx_grad(dkv, one.page_table_cpu[0].numpy(), Lmax, cfg)
+    close(gK, sumK, "dK_ctx summed over the blocks")
+    close(gV, sumV, "dV_ctx summed over the blocks")
+    # fixed accumulation order: a second run gives the same bits
+    res2 = _run(one, "full", q, k, v, dout, ctx, table, max(anchors), layer, shared=True)
+    for a_, b_ in zip(res[2:], res2[2:]):
+        assert np.array_equal(a_, b_, equal_nan=True)
+
+
+def test_backward_at_the_training_shape():
+    # one training sequence as the paper sets it up (App. A.1): 3072 tokens, 512 anchor positions, blocks of 16,
+    # at the Qwen3-8B-shaped head geometry (32 q / 8 kv heads of 128). The oracle checks sampled blocks for dq and
+    # the block gradients, and two kv heads of the context gradients (which add up over all 512 blocks).
+    import dataclasses
+    cfg = dataclasses.replace(synth.QWEN3_8B, n_layers=1, d_model=512, d_ffn=512, vocab=1024, d_target=512)
+    Lseq, NB, R = 3072, 512, 16
+    one = Case(cfg, (Lseq,), seed=31, headroom=0)
+    one.fill_pool_synthetic()
+    g = synth.substream(31, "anchors.train")
+    anchors = torch.randint(1, Lseq - R, (NB,), generator=g, dtype=torch.int32)
+    table = one.page_table.repeat(NB, 1).contiguous()
+    ctx = anchors.to(one.device)
+    mk = lambda name, *shape: synth.normal(shape, 1.0, 31, name, cfg.torch_dtype)
+    q, k, v = mk("f.q", NB, R, cfg.n_q_heads, cfg.head_dim), mk("f.k", NB, R, cfg.n_kv_heads, cfg.head_dim), mk("f.v", NB, R, cfg.n_kv_heads, cfg.head_dim)
+    dout = mk("f.do", NB, R, cfg.n_q_heads, cfg.head_dim)
+    out, lse, dq, dk, dv, dkv = _run(one, "full", q, k, v, dout, ctx, table, int(anchors.max()), 0, shared=True)
+    n32 = synth.to_numpy_f32
+    Kall, Vall = orc.pool_read(one.pool_np, one.page_table_cpu[0].numpy(), Lseq, 0, cfg.page_size)
+    order = np.argsort(anchors.numpy())
+    picks = sorted(set([int(order[0]), int(order[-1])] + [int(x) for x in np.random.default_rng(1).choice(NB, 10, replace=False)]))
+    for b in picks:
+        a = int(anchors[b])
+        rdq, _, _, rdkb, rdvb = orc.block_attention_backward(n32(q[b]), Kall[:a], Vall[:a], n32(k[b]), n32(v[b]), n32(dout[b]), cfg.softmax_scale)
+        close(dq[b], rdq, f"dq block {b} at {a}")
+        close(dk[b], rdkb, f"dk_blk block {b}")
+        close(dv[b], rdvb, f"dv_blk block {b}")
+        ref = orc.block_attention(n32(q[b]), Kall[:a], Vall[:a], n32(k[b]), n32(v[b]), cfg.softmax_scale)
+        close(out[b], ref, f"forward block {b}")
+    # context gradients of kv heads 0 and 5: every block contributes to the positions before its anchor
+    group = cfg.n_q_heads // cfg.n_kv_heads
+    Lmax = int(anchors.max())
+    for kvh in (0, 5):
+        hs = slice(kvh * group, (kvh + 1) * group)
+        sumK = np.zeros((Lmax, cfg.head_dim))
+        sumV = np.zeros_like(sumK)
+        for b in range(NB):
+            a = int(anchors[b])
+            _, rdkc, rdvc, _, _ = orc.block_attention_backward(n32(q[b][:, hs]), Kall[:a, kvh:kvh + 1], Vall[:a, kvh:kvh + 1],
+                                                               n32(k[b][:, kvh:kvh + 1]), n32(v[b][:, kvh:kvh + 1]),
+                                                               n32(dout[b][:, hs]), cfg.softmax_scale)
+            sumK[:a] += rdkc[:, 0]
+            sumV[:a] += rdvc[:, 0]
+        gK, gV = _gather_ctx_grad(dkv, one.page_table_cpu[0].numpy(), Lmax, cfg)
+        close(gK[:, kvh], sumK, f"dK_ctx kv head {kvh} over {NB} blocks")
+        close(gV[:, kvh], sumV, f"dV_ctx kv head {kvh} over {NB} blocks")
