@@ -411,11 +411,34 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+class _LibOnly:
+    """What the single-kernel runs that need no cached context take in place of a Step."""
+
+    def __init__(self, wl, lib, device):
+        self.wl, self.cfg, self.lib = wl, wl.cfg, lib
+        self.ctx_len = torch.tensor(wl.ctx_lens, dtype=torch.int32, device=device)
+        self.max_ctx = max(wl.ctx_lens)
+
+
 def run_kernel_only(args, step, device):
     """One building block alone, launched eagerly `steps` times after `warmup` (profiler captures)."""
     from paper_2602_06036_b200 import binding
     cfg, wl = step.cfg, step.wl
     S, B = wl.batch, cfg.block_size
+    if args.kernel == "verify":
+        # greedy verify/accept from bf16 target logits [S, B+1, V] (each logit crosses HBM once)
+        logits, drafts, planted = synth.make_verify_case(S, B, cfg.vocab, wl.accept_p, 0, cfg.torch_dtype)
+        logits, drafts = logits.to(device), drafts.to(device)
+        tau = torch.zeros(S, dtype=torch.int32, device=device)
+        toks = torch.zeros((S, B + 1), dtype=torch.int32, device=device)
+        bonus, new_len = torch.zeros_like(tau), torch.zeros_like(tau)
+        fn = lambda: step.lib.dflash_verify_accept(drafts, B, B, step.ctx_len, tau, toks, bonus, new_len, logits=logits)
+        nbytes = logits.numel() * 2
+        ms = timed(fn, args.steps, args.warmup, False)[0]
+        assert torch.equal(tau.cpu(), (planted + 1).to(torch.int32))
+        us = ms / args.steps * 1e3
+        print(json.dumps({"kernel": "verify", "workload": wl.name, "us_per_call": us, "alg_bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9}))
+        return
     if args.kernel == "target_verify":
         # The target's verify pass over gamma + 1 rows with a target-sized stack (36 layers of the same
         # shape; the weight tensors of the drafter's layers are reused round-robin: 1.9 GB of distinct
@@ -676,7 +699,7 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify", "block_loss", "attention_bwd"],
+    ap.add_argument("--kernel", default=None, choices=["lmhead", "attention", "target_verify", "block_loss", "attention_bwd", "verify"],
                     help="run one building block alone (for profiler captures) instead of the step")
     ap.add_argument("--loss-blocks", type=int, default=512, help="--kernel block_loss: blocks (of block_size rows) per call")
     ap.add_argument("--trace", default=None, help="write a device-side timeline of one step to this file")
@@ -724,6 +747,9 @@ def main():
     # One handle (one copy of the weights) serves every workload of the run.
     max_ctx = max([max(wl.ctx_lens)] + [max(synth.workload(n).ctx_lens) for n in others])
     lib = make_lib(cfg, device, max_ctx, seed=0)
+    if args.kernel in ("verify", "lmhead", "block_loss", "attention_bwd"):      # no cached context needed
+        run_kernel_only(args, _LibOnly(wl, lib, device), device)
+        return
     step = Step(wl, device, seed=0, temperature=args.temperature, fuse_ctx=not args.separate_ctx, lib=lib)
     S, B = wl.batch, cfg.block_size
 

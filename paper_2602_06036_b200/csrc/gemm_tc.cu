@@ -271,57 +271,83 @@ __device__ __forceinline__ void head_rnorm(const KParams& p, const float* sAcc, 
 
 // Every one of the 128 epilogue threads calls this (it contains named barriers).
 // QKN: the launch has per-head q/k norms (a separate instantiation keeps the common path's registers down).
+// val: this thread's accumulator row of the pass (already scaled by the per-token rsqrt of a folded norm). It goes
+// through shared memory (sAcc) only where an epilogue needs other rows' values (rotation partners, per-tile
+// reductions); the element-wise epilogues work from registers, with a lane exchange for the gate/up pairs.
 // lim: token columns of this pass (<= CH; columns from lim on hold nothing and produce nothing)
 template <int CH, bool QKN>
 __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, Top2Entry* sRed, const Unit& un, int tok0,
                                                int row, const int* tPos, const int* tPage, const float (&xres)[CH], float gain,
-                                               int lim = CH) {
+                                               const float (&val)[CH], int lim = CH) {
     // tPos / tPage: position and (context projection) pool row of the page slot of the tokens of this pass (-1 = skip)
     constexpr int ACC_LD = CH + 1;
     constexpr int GROUPS = 128 / CH;     // threads per token column in the cross-row reductions
     const int f = un.ft * TILE_F + row;
     const int n_tok = min(lim, p.M - tok0);
+    if (p.epi == EPI_QKV_ROPE || p.epi == EPI_ARGMAX || p.epi == EPI_CTX_KV) {      // other rows read this one's values
+#pragma unroll
+        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = val[c];
+        epi_bar();
+    }
     switch (p.epi) {
         case EPI_STORE_F32:
         case EPI_RESIDUAL: {
-            float xv[CH];
+            // New rows x (+)= acc go through a shared-memory tile [token][128 features], so that the global side is
+            // 16-byte accesses of whole 128-byte lines: the number of memory requests a CTA has in flight, not
+            // bytes, limits these epilogues (one 4-byte store per thread and token was measured several times slower).
+            // A warp writes out whole tokens: lane l holds features 4l .. 4l+3 of the tile, also scales them into
+            // the next contraction's bf16 operand and adds up the token's sum of squares by lane exchange.
+            float* sOut = sAcc;                         // CH x 128 floats (<= 128 x (CH + 1))
 #pragma unroll
-            for (int c = 0; c < CH; ++c) xv[c] = (p.epi == EPI_RESIDUAL) ? xres[c] : 0.f;
-            if (f < p.N) {
-                float* o = p.out_f32 ? p.out_f32 + (size_t)tok0 * p.ld_out + f : nullptr;
+            for (int c = 0; c < CH; ++c) {
+                float x = (p.epi == EPI_RESIDUAL) ? xres[c] : 0.f;
+                if (c < n_tok && f < p.N) x += val[c];
+                sOut[c * TILE_F + row] = x;
+            }
+            epi_bar();
+            const int we = row >> 5, ln = row & 31;
+            const int f4 = un.ft * TILE_F + ln * 4;
+            const bool vec = f4 + 3 < p.N;
+            float g4[4] = {0.f, 0.f, 0.f, 0.f};
+            if (p.g_next) {
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    if (c < n_tok) {
-                        xv[c] += sAcc[row * ACC_LD + c];
-                        if (o) o[(size_t)c * p.ld_out] = xv[c];
+                for (int e = 0; e < 4; ++e)
+                    if (f4 + e < p.N) g4[e] = __bfloat162float(p.g_next[f4 + e]);
+            }
+#pragma unroll
+            for (int t = we; t < CH; t += 4) {
+                if (t < n_tok) {                        // uniform over the warp
+                    const float4 x4 = *reinterpret_cast<const float4*>(sOut + t * TILE_F + ln * 4);
+                    const float xe[4] = {x4.x, x4.y, x4.z, x4.w};
+                    const size_t tok = (size_t)(tok0 + t);
+                    if (vec) {
+                        if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + tok * p.ld_out + f4) = x4;
+                        if (p.g_next) {
+                            __nv_bfloat162 lo = __floats2bfloat162_rn(g4[0] * xe[0], g4[1] * xe[1]);
+                            __nv_bfloat162 hi = __floats2bfloat162_rn(g4[2] * xe[2], g4[3] * xe[3]);
+                            uint2 w2;
+                            w2.x = *reinterpret_cast<uint32_t*>(&lo);
+                            w2.y = *reinterpret_cast<uint32_t*>(&hi);
+                            *reinterpret_cast<uint2*>(p.xn_out + tok * p.N + f4) = w2;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (f4 + e < p.N) {
+                                if (p.out_f32) p.out_f32[tok * p.ld_out + f4 + e] = xe[e];
+                                if (p.g_next) p.xn_out[tok * p.N + f4 + e] = __float2bfloat16_rn(g4[e] * xe[e]);
+                            }
+                        }
+                    }
+                    if (p.ssq_out) {                    // features past N hold zeros
+                        float sq = (xe[0] * xe[0] + xe[1] * xe[1]) + (xe[2] * xe[2] + xe[3] * xe[3]);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                        if (ln == 0) p.ssq_out[(size_t)un.ft * p.M + tok0 + t] = sq;
                     }
                 }
-                if (p.g_next) {
-                    const float gv = gain;
-#pragma unroll
-                    for (int c = 0; c < CH; ++c)
-                        if (c < n_tok) p.xn_out[(size_t)(tok0 + c) * p.N + f] = __float2bfloat16_rn(gv * xv[c]);
-                }
             }
-            if (p.ssq_out) {
-                // per-token sum of squares over this tile's 128 features
-#pragma unroll
-                for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = xv[c] * xv[c];
-                epi_bar();
-                const int c = row % CH, g8 = row / CH;
-                float s = 0.f;
-#pragma unroll
-                for (int r = 0; r < CH; ++r) s += sAcc[(g8 * CH + r) * ACC_LD + c];
-                float* red = reinterpret_cast<float*>(sRed);
-                red[g8 * CH + c] = s;
-                epi_bar();
-                if (row < n_tok) {
-                    float t = 0.f;
-#pragma unroll
-                    for (int gg = 0; gg < GROUPS; ++gg) t += red[gg * CH + row];
-                    p.ssq_out[(size_t)un.ft * p.M + tok0 + row] = t;
-                }
-            }
+            epi_bar();      // the next pass overwrites the tile
         } break;
         case EPI_QKV_ROPE: {
             // N is a multiple of 128 on this path (whole heads per tile), so every row is a real feature
@@ -330,11 +356,16 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
             const int partner = row ^ half;
             const int qdim = p.Hq * hd, kdim = p.Hkv * hd;
             const bool rot = p.use_rope && head < p.Hq + p.Hkv;
-            __nv_bfloat16* dst;
+            // the tile's 128 features lie in one of q / k / v (their widths are multiples of 128)
+            const int f0 = un.ft * TILE_F;
+            __nv_bfloat16* dst0;
             int ld;
-            if (head < p.Hq) { dst = p.q + f; ld = qdim; }
-            else if (head < p.Hq + p.Hkv) { dst = p.k + (f - qdim); ld = kdim; }
-            else { dst = p.v + (f - qdim - kdim); ld = kdim; }
+            if (f0 < qdim) { dst0 = p.q + f0; ld = qdim; }
+            else if (f0 < qdim + kdim) { dst0 = p.k + (f0 - qdim); ld = kdim; }
+            else { dst0 = p.v + (f0 - qdim - kdim); ld = kdim; }
+            float rot_out[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) rot_out[c] = 0.f;
             // optional per-head RMSNorm of q and k before the rotation
             const __nv_bfloat16* gain = (!QKN || !p.gq) ? nullptr : (head < p.Hq ? p.gq : (head < p.Hq + p.Hkv ? p.gk[0] : nullptr));
             const float g_self = gain ? __bfloat162float(gain[hrow]) : 1.f;
@@ -372,24 +403,54 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                         const float cc = on ? cs[c] : 1.f, ss = on ? sn[c] : 0.f;
                         const float a = sAcc[row * ACC_LD + c0 + c] * (rn[c] * g_self);
                         const float b = sAcc[partner * ACC_LD + c0 + c] * (rn[c] * g_part);
-                        const float val = hrow < half ? (a * cc - b * ss) : (a * cc + b * ss);
-                        dst[(size_t)(tok0 + c0 + c) * ld] = __float2bfloat16_rn(val);
+                        rot_out[c0 + c] = hrow < half ? (a * cc - b * ss) : (a * cc + b * ss);
                     }
                 }
             }
+            // out through a shared-memory tile [token][128] as 16-byte stores of whole lines (see the residual epilogue)
+            epi_bar();                                  // every row has read its partner's accumulators
+            __nv_bfloat16* sOut = reinterpret_cast<__nv_bfloat16*>(sAcc);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) sOut[c * TILE_F + row] = __float2bfloat16_rn(rot_out[c]);
+            epi_bar();
+            for (int q = row; q < CH * 16; q += 128) {
+                const int t = q >> 4, part = q & 15;
+                if (t < n_tok)
+                    *reinterpret_cast<uint4*>(dst0 + (size_t)(tok0 + t) * ld + part * 8) = *reinterpret_cast<const uint4*>(sOut + t * TILE_F + part * 8);
+            }
+            epi_bar();
         } break;
         case EPI_SWIGLU: {
-            if ((row & 1) == 0 && f + 1 < p.N) {
-                const int j = f >> 1;
-                __nv_bfloat16* dst = p.h + (size_t)tok0 * p.F + j;
+            // rows 2j / 2j+1 hold gate_j / up_j. The even lane finishes token columns [0, CH/2), the odd lane
+            // [CH/2, CH): each sends its partner the half it does not finish itself (one lane exchange per column
+            // pair). The 64 outputs per token go through a shared-memory tile [token][64] and leave as 16-byte
+            // stores of whole lines (see the residual epilogue).
+            const bool odd = (row & 1) != 0;
+            constexpr int HC = CH / 2;
+            const int c_base = odd ? HC : 0;
+            __nv_bfloat16* sOut = reinterpret_cast<__nv_bfloat16*>(sAcc);      // CH x 64 bf16
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {      // unrolled: independent iterations overlap their latencies
-                    if (c < n_tok) {
-                        const float g = sAcc[row * ACC_LD + c], u = sAcc[(row + 1) * ACC_LD + c];
-                        dst[(size_t)c * p.F] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+            for (int k = 0; k < HC; ++k) {
+                const float other = __shfl_xor_sync(0xffffffffu, odd ? val[k] : val[k + HC], 1);
+                const float g = odd ? other : val[k], u = odd ? val[k + HC] : other;
+                sOut[(c_base + k) * 64 + (row >> 1)] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+            }
+            epi_bar();
+            const int j_tile = un.ft * 64;              // first FFN unit of this tile
+            for (int q = row; q < CH * 8; q += 128) {
+                const int t = q >> 3, part = q & 7;
+                if (t < n_tok) {
+                    const int j0 = j_tile + part * 8;
+                    __nv_bfloat16* dst = p.h + (size_t)(tok0 + t) * p.F + j0;
+                    if (j0 + 8 <= p.F) {
+                        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(sOut + t * 64 + part * 8);
+                    } else {
+                        for (int e = 0; e < 8; ++e)
+                            if (j0 + e < p.F) dst[e] = sOut[t * 64 + part * 8 + e];
                     }
                 }
             }
+            epi_bar();
         } break;
         case EPI_ARGMAX: {
             if (p.logits_out && f < p.N)
@@ -409,6 +470,7 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 for (int gg = 1; gg < GROUPS; ++gg) t2_merge(m, sRed[gg * CH + row].v1, sRed[gg * CH + row].i1, sRed[gg * CH + row].v2);
                 p.top2[(size_t)un.ft * p.M + tok0 + row] = Top2Entry{m.v1, m.i1, m.v2, 0};
             }
+            epi_bar();
         } break;
         case EPI_CTX_KV: {
             // N = 2 * Hkv * hd is a multiple of 128 on this path
@@ -456,15 +518,16 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
                 for (int c = 0; c < SB; ++c) {
                     const int prow = (c0 + c < n_tok) ? tPage[c0 + c] : -1;
                     if (prow >= 0) {
-                        float val = sAcc[row * ACC_LD + c0 + c] * (rn[c] * g_self);
+                        float kv_v = sAcc[row * ACC_LD + c0 + c] * (rn[c] * g_self);
                         if (rot) {
                             const float bb = sAcc[partner * ACC_LD + c0 + c] * (rn[c] * g_part);
-                            val = hrow < half ? (val * cs[c] - bb * sn[c]) : (val * cs[c] + bb * sn[c]);
+                            kv_v = hrow < half ? (kv_v * cs[c] - bb * sn[c]) : (kv_v * cs[c] + bb * sn[c]);
                         }
-                        base[(size_t)prow * hd] = __float2bfloat16_rn(val);
+                        base[(size_t)prow * hd] = __float2bfloat16_rn(kv_v);
                     }
                 }
             }
+            epi_bar();
         } break;
         default: break;
     }
@@ -857,12 +920,12 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 #pragma unroll
                                 for (int c = 0; c < CH; ++c) acc[c] += va[u][c];
                         }
+                        if (p.ssq_in) {
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? acc[c] * sRstd[tok_off + ch * CH + c] : acc[c];
+                            for (int c = 0; c < CH; ++c) acc[c] *= sRstd[tok_off + ch * CH + c];
+                        }
                         if constexpr (CH > 32) residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
-                        epi_bar();
-                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
-                        epi_bar();
+                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain, acc);
                     }
                 }
                 n_pend = 0;
@@ -934,6 +997,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         if (flags[2]) { alive = false; break; }
                         if (tok0 < p.M) {
                             const float* rx = sXch + ((size_t)xb * (CS - 1) * TILE_F + row) * GC;
+                            float val[CH];
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) val[c] = 0.f;
 #pragma unroll
                             for (int l4 = 0; l4 < GC; l4 += 4) {
                                 float a[4] = {0.f, 0.f, 0.f, 0.f};
@@ -945,13 +1011,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                                     a[0] += t.x; a[1] += t.y; a[2] += t.z; a[3] += t.w;
                                 }
 #pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    sAcc[row * ACC_LD + l4 + e] = p.ssq_in ? a[e] * sRstd[tok_off + rank * GC + l4 + e] : a[e];
+                                for (int e = 0; e < 4; ++e) val[l4 + e] = p.ssq_in ? a[e] * sRstd[tok_off + rank * GC + l4 + e] : a[e];
                             }
-                            epi_bar();
                             apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok0, row, sPos + tok_off + rank * GC, sPage + tok_off + rank * GC,
-                                                    xres, gain, GC);
-                            epi_bar();
+                                                    xres, gain, val, GC);
                         }
                         continue;
                     }
@@ -965,13 +1028,13 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 #pragma unroll
                         for (int c = 0; c < CH; ++c) dst[(size_t)c * TILE_F] = v[c];
                     } else {
+                        if (p.ssq_in) {
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) sAcc[row * ACC_LD + c] = p.ssq_in ? v[c] * sRstd[tok_off + ch * CH + c] : v[c];
+                            for (int c = 0; c < CH; ++c) v[c] *= sRstd[tok_off + ch * CH + c];
+                        }
                         float xres[CH], gain;
                         residual_load<CH>(p, un, tok_base + ch * CH, row, xres, gain);
-                        epi_bar();
-                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain);
-                        epi_bar();
+                        apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain, v);
                     }
                 }
                 tc_fence_before();
