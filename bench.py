@@ -575,6 +575,8 @@ def measure(step, args, peaks, dist_on, rank, sampler=None, repeats=7, e2e_repea
         run_resident()
         run_e2e()
     torch.cuda.synchronize()
+    if step.dev_status() != 0:       # e.g. a bounded wait that ran out: do not go on to time a broken step
+        raise RuntimeError(f"bench: device status {step.dev_status()} after the warm-up steps of {wl.name}")
     n0 = binding.launch_count()
     run_resident()
     launches_per_step = binding.launch_count() - n0

@@ -645,7 +645,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     // count must leave room for the CTAs of the next kernel to become resident beside this one: a
     // dependent kernel that cannot start early was measured 30 us slower.
     constexpr int PF = (NT == 256) ? 1 : (CH <= 16 ? 4 : (CH <= 32 ? 3 : 1));
-    constexpr uint32_t TMEM_COLS = (2 * NT < 32) ? 32u : (uint32_t)(2 * NT);
+    constexpr uint32_t TMEM_COLS = (2 * NT <= 32) ? 32u : (2 * NT <= 64) ? 64u : (2 * NT <= 128) ? 128u : (2 * NT <= 256) ? 256u : 512u;   // a power of two
     const int stages = mp.stages;
     uint8_t* sW = smem;
     uint8_t* sX = sW + (size_t)stages * W_STAGE;
@@ -1220,9 +1220,18 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows, i
     return tmap_encode_bf16(m, base, 3, dims, strides, box);
 }
 
+// Token-tile width: up to 128 rows the smallest width that holds them; beyond that the width (a multiple of 32 up
+// to 256) that pads the fewest token columns over all token tiles, the widest among equals (fewer token tiles =
+// fewer passes over the weights through L2): 136 rows -> 160, 544 -> 3 x 192, 512 -> 2 x 256.
 int pick_nt(int M) {
     for (int nt : {16, 32, 64, 128}) if (M <= nt) return nt;
-    return 256;
+    int best = 256;
+    long long best_cols = (long long)((M + 255) / 256) * 256;
+    for (int nt : {192, 160}) {
+        const long long cols = (long long)((M + nt - 1) / nt) * nt;
+        if (cols < best_cols) { best = nt; best_cols = cols; }
+    }
+    return best;
 }
 
 // Largest grid of clusters of CS CTAs whose CTAs are all resident at once (the CTAs of a launch wait for each
@@ -1302,14 +1311,19 @@ int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, MParams& mp, in
 
 }  // namespace
 
+// A workspace sized for M rows also serves launches with fewer rows, whose token tile may be WIDER than the one M
+// rows get (520 rows take tiles of 192 columns, 640 rows tiles of 160): both sizes below are upper bounds over
+// every row count up to M.
 int64_t gemm_tc_part_bytes(int M, int N, int K, int n_groups, int sm_count) {
     (void)N; (void)K; (void)n_groups;
-    return (int64_t)sm_count * 2 * pick_nt(M) * TILE_F * 4;    // two partial pieces per CTA at most
+    const int nt_max = M > 128 ? 256 : pick_nt(M);
+    return (int64_t)sm_count * 2 * nt_max * TILE_F * 4;    // two partial pieces per CTA at most
 }
 
 int64_t gemm_tc_counter_bytes(int M, int N, int n_groups) {
-    const int nt = pick_nt(M);
-    return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ((M + nt - 1) / nt) * 4;
+    // token tiles: rows beyond 128 use tiles of at least 160 columns, so ceil(M / 128) bounds every smaller row count too
+    const int ttiles = M > 128 ? (M + 127) / 128 : 1;
+    return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ttiles * 4;
 }
 
 static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KParams& p) {
@@ -1404,6 +1418,8 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
         case 32: return slabs == 2 ? DFLASH_GEMM_CASE(32, 2) : DFLASH_GEMM_CASE(32, 1);
         case 64: return DFLASH_GEMM_CASE(64, 1);
         case 128: return DFLASH_GEMM_CASE(128, 1);
+        case 160: return DFLASH_GEMM_CASE(160, 1);
+        case 192: return DFLASH_GEMM_CASE(192, 1);
         default: return DFLASH_GEMM_CASE(256, 1);
     }
 #undef DFLASH_GEMM_CASE

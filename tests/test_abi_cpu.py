@@ -176,6 +176,19 @@ def test_attention_split_never_outgrows_its_partials_buffer(lib):
     lib.dflash_destroy(h)
 
 
+def test_workspace_grows_with_the_row_count(lib):
+    # a workspace sized for R rows must serve every call with fewer rows (a draft of 512 rows inside a workspace
+    # sized for the 544 rows of the projection that rides along): sizes never shrink as rows grow
+    h = C.c_void_p()
+    assert lib.dflash_create(C.byref(_qwen_cfg()), C.byref(h)) == 0
+    prev = 0
+    for rows in list(range(1, 300)) + list(range(300, 1200, 7)) + [2048, 4096]:
+        n = lib.dflash_workspace_bytes(h, 32, rows)
+        assert n >= prev, (rows, n, prev)
+        prev = n
+    lib.dflash_destroy(h)
+
+
 def test_attention_and_fused_projection_arguments_validated_on_the_host(lib):
     h = C.c_void_p()
     assert lib.dflash_create(C.byref(_cfg()), C.byref(h)) == 0
