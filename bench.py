@@ -710,6 +710,8 @@ def main():
     ap.add_argument("--separate-ctx", action="store_true",
                     help="run the context projection as its own call before the draft call instead of inside it")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--ctx-len", type=int, default=0,
+                    help="> 0: every sequence of the workload gets this context length (a small case of the same launches for profiler captures)")
     ap.add_argument("--repeats", type=int, default=7, help="timed regions of --steps steps each; ms_per_step is their median")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the extra key with the other benchmark configurations (cfg2, cfg3, cfg4) measured in the same run")
@@ -738,6 +740,10 @@ def main():
     from paper_2602_06036_b200 import build
     build.build()
     wl = synth.workload(args.workload)
+    if args.ctx_len > 0:
+        import dataclasses
+        wl = dataclasses.replace(wl, ctx_lens=tuple(args.ctx_len for _ in wl.ctx_lens))
+        args.no_other_workloads = True
     cfg = wl.cfg
     peaks = load_peaks()
     hbm = peaks["hbm_gbs"]

@@ -215,6 +215,9 @@ int32_t dflash_create(const dflash_config* cfg, dflash_handle** out) {
     dflash_handle* h = new (std::nothrow) dflash_handle();
     if (!h) return DFLASH_ERR_INVALID_ARG;
     h->cfg = c;
+    h->wmaps = new (std::nothrow) dflash_wmap_entry[DFLASH_WMAP_CACHE];
+    h->n_wmaps = 0;
+    if (!h->wmaps) { delete h; return DFLASH_ERR_INVALID_ARG; }
     h->has_weights = false;
     // SMs of the current device (grids of one CTA per SM, split heuristics and the partial-tile workspace follow
     // it); without a device - sizing queries on a host with no GPU - the B200's count
@@ -245,6 +248,7 @@ void dflash_destroy(dflash_handle* h) {
     }
     delete[] h->prof;
     delete[] h->trace_fam;
+    delete[] h->wmaps;
     delete h;
 }
 
@@ -302,6 +306,7 @@ int32_t dflash_set_weights(dflash_handle* h, const dflash_weights* w) {
     }
     h->w = *w;
     h->w.layers = h->layers;
+    h->n_wmaps = 0;      // maps of the previous weights are stale
     h->has_weights = true;
     return DFLASH_OK;
 }

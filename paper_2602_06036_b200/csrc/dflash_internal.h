@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of the library (not part of the ABI).
 #pragma once
 
+#include <cuda.h>  // CUtensorMap only
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -20,8 +21,20 @@ struct dflash_profile_rec {
     int family;
 };
 
+// Encoded tensor maps of weight matrices, kept per handle: the weights of a handle do not move between
+// dflash_set_weights calls, so a launch looks its maps up instead of encoding 6-8 of them (about 13 us of host
+// time per step for callers that launch eagerly).
+struct dflash_wmap_entry {
+    const void* base;
+    int rows, K, slabs;
+    CUtensorMap map;
+};
+constexpr int DFLASH_WMAP_CACHE = 8 * 64 + 8;      // per layer: QKV, K/V rows of QKV, O, gate/up, down (x slab variants) + fusion, LM head
+
 struct dflash_handle {
     dflash_config cfg;
+    dflash_wmap_entry* wmaps;      // [DFLASH_WMAP_CACHE], allocated at create
+    int n_wmaps;
     dflash_layer_weights layers[DFLASH_MAX_LAYERS];
     dflash_weights w;
     bool has_weights;

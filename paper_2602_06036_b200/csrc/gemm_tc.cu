@@ -1223,6 +1223,17 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows, i
 // Token-tile width: up to 128 rows the smallest width that holds them; beyond that the width (a multiple of 32 up
 // to 256) that pads the fewest token columns over all token tiles, the widest among equals (fewer token tiles =
 // fewer passes over the weights through L2): 136 rows -> 160, 544 -> 3 x 192, 512 -> 2 x 256.
+// The map of a weight matrix, from the handle's cache (encoded on first use; a full cache encodes without storing)
+bool weight_map(dflash_handle* h, CUtensorMap* m, const void* base, int rows, int K, int slabs) {
+    for (int i = 0; i < h->n_wmaps; ++i) {
+        const dflash_wmap_entry& e = h->wmaps[i];
+        if (e.base == base && e.rows == rows && e.K == K && e.slabs == slabs) { *m = e.map; return true; }
+    }
+    if (!make_map(m, base, rows, K, TILE_F, slabs)) return false;
+    if (h->n_wmaps < DFLASH_WMAP_CACHE) h->wmaps[h->n_wmaps++] = dflash_wmap_entry{base, rows, K, slabs, *m};
+    return true;
+}
+
 int pick_nt(int M) {
     for (int nt : {16, 32, 64, 128}) if (M <= nt) return nt;
     int best = 256;
@@ -1396,7 +1407,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
         if (n_maps + p.n_groups > GEMM_MAX_GROUPS) return DFLASH_ERR_UNSUPPORTED;
         p.w_map0 = n_maps;
         for (int g = 0; g < p.n_groups; ++g)
-            if (!make_map(&tw.m[n_maps++], a.W[g], a.N, a.K, TILE_F, slabs)) return DFLASH_ERR_CUDA;
+            if (!weight_map(L.h, &tw.m[n_maps++], a.W[g], a.N, a.K, slabs)) return DFLASH_ERR_CUDA;
         p.x_map = i;
         if (!make_map(&tx.m[i], a.X, a.M, a.K, nt, slabs)) return DFLASH_ERR_CUDA;
         const long long pairs = (long long)p.n_tiles * p.chunks_total;
