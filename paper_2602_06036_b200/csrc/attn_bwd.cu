@@ -11,8 +11,9 @@
 //                        order and accumulates the tile's dK, dV in TMEM, so the context gradients of all blocks add
 //                        up in a fixed order (bit-reproducible) without atomics.
 // Operands are staged by TMA in the 128-byte-swizzled layouts of the forward kernel. The 64 query rows of a kv
-// head (block rows x q heads of the group) are loaded twice to fill the 128-row operand; the probability rows of
-// the second copy are written as zeros, so contractions over the row index count every row once. Transposed
+// head (block rows x q heads of the group) are loaded twice to fill the 128-row operand, so that all four TMEM lane
+// quadrants share the row arithmetic (the second copy takes keys 32..63 of every tile); P and dS are written for rows
+// 0..63 only and rows 64..127 of their tiles stay zero, so contractions over the row index count every row once. Transposed
 // products (P^T dO, dS^T Q) cost nothing: the tensor core reads the same shared-memory tiles through MN-major
 // descriptors and produces dV^T, dK^T with head_dim on the TMEM lanes. One thread issues copies and tensor-core
 // instructions, 128 threads (one per TMEM lane) do the row arithmetic; every mbarrier wait is bounded.
@@ -34,9 +35,12 @@ constexpr int PG = 64;
 constexpr int QD_BYTES = 128 * HD * 2;           // one 128-row operand tile (Q or dO): two 64-column halves of 16 KiB
 constexpr int KV_TILE_BYTES = PG * HD * 2;       // K or V tile: two 64-column halves of 8 KiB
 constexpr int PS_BYTES = 128 * PG * 2;           // P or dS tile: 128 rows x 64 keys
-constexpr int N_THREADS = 160;                   // 4 row warps (TMEM lane quadrants 0..3) + the issuing warp
+constexpr int N_THREADS = 224;                   // 4 row warps (TMEM lane quadrants 0..3) + three single-thread roles: copies, scores, products
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S = 0, COL_DP = 64, COL_DQ = 128, COL_DVT = 256, COL_DKT = 320;
+// S and dP are double-buffered (the contractions of the next key tile run under the row arithmetic of the current one)
+constexpr uint32_t COL_S = 0, COL_DP = 64, COL_DQ = 128, COL_DVT = 256, COL_DKT = 320, COL_SDP2 = 384;
+__device__ __forceinline__ uint32_t sdp_col(int buf) { return buf ? COL_SDP2 : 0u; }
+constexpr int KV_STAGES = 3;
 constexpr float LOG2E = 1.4426950408889634f;
 
 struct BParams {
@@ -105,6 +109,7 @@ __device__ __forceinline__ void load_q_do(uint8_t* sQ, uint8_t* sDO, const CUten
 
 // S = Q K^T and dP = dO V^T of one 64-key tile (16 instructions)
 __device__ __forceinline__ void issue_s_dp(uint32_t tmem_base, uint32_t q_addr, uint32_t do_addr, uint32_t k_addr, uint32_t v_addr) {
+    // tmem_base already includes the S / dP buffer's first column
     constexpr uint32_t idesc = idesc_kk(128, PG);
 #pragma unroll
     for (int kk = 0; kk < HD / 16; ++kk)
@@ -129,39 +134,49 @@ __device__ __forceinline__ void issue_dkv_t(uint32_t tmem_base, uint32_t q_addr,
                  (accumulate || kk > 0) ? 1u : 0u);
 }
 
-// Row arithmetic of one tile, thread = operand row: reads its S and dP rows from TMEM, writes P and dS (bf16) into
-// the swizzled tiles. vis = keys of this tile the row sees (0 for rows that hold no query).
-__device__ __forceinline__ void row_math(uint32_t tmem_row, uint8_t* sP, uint8_t* sDS, int row, int vis, float lse2, float Dr,
+// Row arithmetic of one tile. The 64 query rows sit twice in the operand (TMEM lanes 0..63 and 64..127 hold the same
+// S and dP rows): the thread of lane l works on query row l & 63 and on keys [32 (l >> 6), +32) of the tile, so all
+// four lane quadrants (one warp each) share the work. It reads its half rows of S and dP from TMEM and writes P
+// and dS (bf16) into rows 0..63 of the swizzled tiles; rows 64..127 of those tiles stay zero (zeroed once at the
+// start), which is what makes contractions over the 128 operand rows count every query row once.
+// vis = keys of this tile the query row sees (0 for rows that hold no query).
+__device__ __forceinline__ void row_math(uint32_t tmem_row, uint8_t* sP, uint8_t* sDS, int lane_row, int vis, float lse2, float Dr,
                                          float scale, float scale_log2) {
-    uint8_t* prow = sP + row * 128;
-    uint8_t* drow = sDS + row * 128;
+    const int qrow = lane_row & 63, h = lane_row >> 6;
+    uint8_t* prow = sP + qrow * 128;
+    uint8_t* drow = sDS + qrow * 128;
+    float s[32], dp[32];
+    tmem_ld32(tmem_row + COL_S + h * 32, s);          // tmem_row includes the S / dP buffer's first column
+    tmem_ld32(tmem_row + COL_DP + h * 32, dp);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        float s[32], dp[32];
-        tmem_ld32(tmem_row + COL_S + h * 32, s);
-        tmem_ld32(tmem_row + COL_DP + h * 32, dp);
+    for (int c = 0; c < 32; ++c) {
+        const bool on = h * 32 + c < vis;
+        const float p = on ? fast_exp2(fmaf(s[c], scale_log2, -lse2)) : 0.f;
+        s[c] = p;
+        dp[c] = on ? p * (dp[c] - Dr) * scale : 0.f;
+    }
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const bool on = h * 32 + c < vis;
-            const float p = on ? fast_exp2(fmaf(s[c], scale_log2, -lse2)) : 0.f;
-            s[c] = p;
-            dp[c] = on ? p * (dp[c] - Dr) * scale : 0.f;
-        }
-#pragma unroll
-        for (int ck = 0; ck < 4; ++ck) {
-            uint4 w4, d4;
-            w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
-            w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
-            w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
-            w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
-            d4.x = pack_bf16(dp[ck * 8 + 0], dp[ck * 8 + 1]);
-            d4.y = pack_bf16(dp[ck * 8 + 2], dp[ck * 8 + 3]);
-            d4.z = pack_bf16(dp[ck * 8 + 4], dp[ck * 8 + 5]);
-            d4.w = pack_bf16(dp[ck * 8 + 6], dp[ck * 8 + 7]);
-            const int off = ((h * 4 + ck) ^ (row & 7)) << 4;
-            *reinterpret_cast<uint4*>(prow + off) = w4;
-            *reinterpret_cast<uint4*>(drow + off) = d4;
-        }
+    for (int ck = 0; ck < 4; ++ck) {
+        uint4 w4, d4;
+        w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
+        w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
+        w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
+        w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
+        d4.x = pack_bf16(dp[ck * 8 + 0], dp[ck * 8 + 1]);
+        d4.y = pack_bf16(dp[ck * 8 + 2], dp[ck * 8 + 3]);
+        d4.z = pack_bf16(dp[ck * 8 + 4], dp[ck * 8 + 5]);
+        d4.w = pack_bf16(dp[ck * 8 + 6], dp[ck * 8 + 7]);
+        const int off = ((h * 4 + ck) ^ (qrow & 7)) << 4;
+        *reinterpret_cast<uint4*>(prow + off) = w4;
+        *reinterpret_cast<uint4*>(drow + off) = d4;
+    }
+}
+// rows 64..127 of both P / dS buffer pairs := 0 (128 threads; visible to the tensor core after the first
+// fence.proxy.async + barrier arrival that follows)
+__device__ __forceinline__ void zero_upper_rows(uint8_t* sPS, int tid) {
+    for (int t = 0; t < 4; ++t) {
+        uint4* dst = reinterpret_cast<uint4*>(sPS + (size_t)t * PS_BYTES + 64 * 128);
+        for (int e = tid; e < 64 * 128 / 16; e += 128) dst[e] = make_uint4(0, 0, 0, 0);
     }
 }
 
@@ -178,26 +193,23 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;
     uint8_t* sDO = sQ + QD_BYTES;
-    uint8_t* sKV = sDO + QD_BYTES;                       // 2 stages x (K, V)
-    uint8_t* sP = sKV + 2 * 2 * KV_TILE_BYTES;
-    uint8_t* sDS = sP + PS_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sDS + PS_BYTES);
+    uint8_t* sKV = sDO + QD_BYTES;                       // KV_STAGES x (K, V)
+    uint8_t* sPS = sKV + KV_STAGES * 2 * KV_TILE_BYTES;  // 2 x (P, dS)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sPS + 2 * 2 * PS_BYTES);
     uint64_t* q_full = bars;
-    uint64_t* kv_full = bars + 1;      // [2]
-    uint64_t* kv_empty = bars + 3;     // [2]
-    uint64_t* s_full = bars + 5;
-    uint64_t* ds_full = bars + 6;
-    uint64_t* acc_done = bars + 7;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint64_t* kv_full = bars + 1;                  // [KV_STAGES]
+    uint64_t* kv_empty = kv_full + KV_STAGES;      // [KV_STAGES]
+    uint64_t* s_full = kv_empty + KV_STAGES;       // [2] S / dP buffer written by the tensor core
+    uint64_t* ds_full = s_full + 2;                // [2] P / dS buffer written by the row threads (and S / dP buffer read)
+    uint64_t* acc_done = ds_full + 2;              // [2] the products that read P / dS buffer are complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 2);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        mbar_init(s_full, 1);
-        mbar_init(ds_full, 4);
-        mbar_init(acc_done, 1);
+        for (int s = 0; s < KV_STAGES; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&ds_full[s], 4); mbar_init(&acc_done[s], 1); }
         flags[0] = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -215,12 +227,18 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int n_ctx_tiles = (L + PG - 1) / PG;
     const int n_tiles = n_ctx_tiles + 1;
 
+    // Three single-thread roles, each with its own chain of waits, so that a copy in flight never holds up a
+    // contraction whose operands are ready: copies (warp 4), S / dP of the next tile (warp 5), the accumulating
+    // products of the current tile (warp 6).
     if (warp == 4) {
         if (lane == 0) {
             const uint64_t pol_kv = policy_evict_last(), pol_q = policy_evict_first();
             bool ok = true;
-            auto load_tile = [&](int i) {
-                const int st = i & 1;
+            load_q_do(sQ, sDO, &tmQ, &tmDO, g, b * p.R, q_full, pol_q);
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                const int st = i % KV_STAGES;
+                // the stage held tile i - KV_STAGES: wait for that tile's products
+                if (i >= KV_STAGES && !mbar_wait(&kv_empty[st], ((i / KV_STAGES) - 1) & 1, &flags[0])) { ok = false; break; }
                 uint8_t* dK = sKV + (size_t)st * 2 * KV_TILE_BYTES;
                 uint8_t* dV = dK + KV_TILE_BYTES;
                 mbar_expect_tx(&kv_full[st], 2 * KV_TILE_BYTES);
@@ -242,33 +260,50 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     tma_load_2d(dV, &tmVb, g * HD, b * p.R, &kv_full[st], pol_q);
                     tma_load_2d(dV + KV_TILE_BYTES / 2, &tmVb, g * HD + 64, b * p.R, &kv_full[st], pol_q);
                 }
-            };
-            load_q_do(sQ, sDO, &tmQ, &tmDO, g, b * p.R, q_full, pol_q);
-            load_tile(0);
-            if (n_tiles > 1) load_tile(1);
-            ok = mbar_wait(q_full, 0, &flags[0]);
-            const uint32_t q_addr = smem_u32(sQ), do_addr = smem_u32(sDO), p_addr = smem_u32(sP), ds_addr = smem_u32(sDS);
+            }
+            if (!ok) {
+                flags[0] = 1;
+                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        if (lane == 0) {
+            const uint32_t q_addr = smem_u32(sQ), do_addr = smem_u32(sDO);
+            bool ok = mbar_wait(q_full, 0, &flags[0]);
             for (int i = 0; i < n_tiles && ok; ++i) {
-                const int st = i & 1;
-                if (!mbar_wait(&kv_full[st], (i >> 1) & 1, &flags[0])) { ok = false; break; }
+                const int st = i % KV_STAGES, buf = i & 1;
+                if (!mbar_wait(&kv_full[st], (i / KV_STAGES) & 1, &flags[0])) { ok = false; break; }
+                // S / dP buffer `buf` was last read by the row threads of tile i - 2
+                if (i >= 2 && !mbar_wait(&ds_full[buf], ((i - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t k_addr = smem_u32(sKV + (size_t)st * 2 * KV_TILE_BYTES), v_addr = k_addr + KV_TILE_BYTES;
-                issue_s_dp(tmem_base, q_addr, do_addr, k_addr, v_addr);
-                mma_commit(s_full);
-                // the tile after next takes the stage the previous tile used, once that tile's products are done
-                if (i >= 1 && i + 1 < n_tiles) {
-                    if (!mbar_wait(&kv_empty[st ^ 1], ((i - 1) >> 1) & 1, &flags[0])) { ok = false; break; }
-                    load_tile(i + 1);
-                }
-                if (!mbar_wait(ds_full, i & 1, &flags[0])) { ok = false; break; }
+                const uint32_t k_addr = smem_u32(sKV + (size_t)st * 2 * KV_TILE_BYTES);
+                issue_s_dp(tmem_base + sdp_col(buf), q_addr, do_addr, k_addr, k_addr + KV_TILE_BYTES);
+                mma_commit(&s_full[buf]);
+            }
+            if (!ok) {
+                flags[0] = 1;
+                if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 6) {
+        if (lane == 0) {
+            const uint32_t q_addr = smem_u32(sQ), do_addr = smem_u32(sDO);
+            bool ok = true;
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                const int st = i % KV_STAGES, buf = i & 1;
+                if (!mbar_wait(&ds_full[buf], (i >> 1) & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t k_addr = smem_u32(sKV + (size_t)st * 2 * KV_TILE_BYTES);
+                const uint32_t p_addr = smem_u32(sPS + (size_t)buf * 2 * PS_BYTES), ds_addr = p_addr + PS_BYTES;
                 constexpr uint32_t idesc_dq = idesc_k_mn(128, HD);
 #pragma unroll
                 for (int kk = 0; kk < PG / 16; ++kk)
                     mma_bf16(tmem_base + COL_DQ, smem_desc_sw128(ds_addr + kk * 32), smem_desc_mn(k_addr + kk * 2048, KV_TILE_BYTES / 2),
                              idesc_dq, (i > 0 || kk > 0) ? 1u : 0u);
                 if (i == n_tiles - 1) issue_dkv_t(tmem_base, q_addr, do_addr, p_addr, ds_addr, 0u);      // the block's own keys
-                mma_commit(acc_done);
+                mma_commit(&acc_done[buf]);
                 mma_commit(&kv_empty[st]);
             }
             if (!ok) {
@@ -278,11 +313,13 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         __syncwarp();
     } else {
-        const int row = warp * 32 + lane;                       // TMEM lane = operand row
+        const int row = warp * 32 + lane;                       // TMEM lane
         const uint32_t tmem_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const bool real = row < p.rows_valid;                   // rows from 64 on repeat rows 0..63 and count for nothing
-        const int r = real ? row / p.group : 0, j = real ? row % p.group : 0;
+        const int lrow = row & 63;                              // query row (lanes 64..127 repeat rows 0..63)
+        const bool real = lrow < p.rows_valid;
+        const int r = real ? lrow / p.group : 0, j = real ? lrow % p.group : 0;
         const size_t qrow = ((size_t)b * p.R + r) * p.Hq + g * p.group + j;
+        zero_upper_rows(sPS, row);
         // D = rowsum(dO * O) and the row's log-sum-exp in the log2 domain
         float Dr = 0.f, lse2 = 0.f;
         if (real) {
@@ -300,11 +337,12 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     Dr = fmaf(x.y, y.y, Dr);
                 }
             }
-            p.D[qrow] = Dr;
+            if (row < 64) p.D[qrow] = Dr;
             lse2 = __ldg(p.lse + qrow) * LOG2E;
         }
         bool ok = true;
         for (int i = 0; i < n_tiles; ++i) {
+            const int buf = i & 1;
             int n_valid, vis;
             if (i < n_ctx_tiles) {
                 n_valid = min(PG, L - i * PG);
@@ -314,14 +352,15 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 vis = p.causal ? min(r + 1, p.R) : p.R;
             }
             if (!real) vis = 0;
-            if (!mbar_wait(s_full, i & 1, &flags[0])) { ok = false; break; }
+            if (!mbar_wait(&s_full[buf], (i >> 1) & 1, &flags[0])) { ok = false; break; }
             tc_fence_after();
-            // P and dS of the previous tile are still being read by its products until acc_done
-            if (i > 0 && !mbar_wait(acc_done, (i - 1) & 1, &flags[0])) { ok = false; break; }
-            row_math(tmem_row, sP, sDS, row, vis, lse2, Dr, p.scale, p.scale_log2);
+            // P / dS buffer `buf` is still being read by the products of tile i - 2 until their acc_done
+            if (i >= 2 && !mbar_wait(&acc_done[buf], ((i - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
+            uint8_t* sP = sPS + (size_t)buf * 2 * PS_BYTES;
+            row_math(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
             // keys that do not exist must not poison dS K with whatever the page holds there
             if (n_valid < PG) {
-                uint8_t* dK = sKV + (size_t)(i & 1) * 2 * KV_TILE_BYTES;
+                uint8_t* dK = sKV + (size_t)(i % KV_STAGES) * 2 * KV_TILE_BYTES;
                 const int n_bad = PG - n_valid;
                 for (int e = row; e < n_bad * 16; e += 128) {
                     const int kr = n_valid + e / 16, part = e % 16;
@@ -331,9 +370,10 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tc_fence_before();
             fence_proxy_async();
             __syncwarp();
-            if (lane == 0) mbar_arrive(ds_full);
+            if (lane == 0) mbar_arrive(&ds_full[buf]);
         }
-        if (ok && !mbar_wait(acc_done, (n_tiles - 1) & 1, &flags[0])) ok = false;
+        // the tensor pipe completes in order: the last tile's products close the accumulators
+        if (ok && !mbar_wait(&acc_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, &flags[0])) ok = false;
         if (!ok) {
             flags[0] = 1;
             if (lane == 0 && p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
@@ -347,7 +387,7 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int c4 = 0; c4 < HD / 32; ++c4) {
                 float o[32];
                 tmem_ld32(tmem_row + COL_DQ + c4 * 32, o);
-                if (real) {
+                if (real && row < 64) {
 #pragma unroll
                     for (int d = 0; d < 32; d += 8) {
                         uint4 w4;
@@ -393,25 +433,24 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sKV = smem;                                  // K tile, V tile
     uint8_t* sQD = sKV + 2 * KV_TILE_BYTES;               // 2 stages x (Q, dO)
-    uint8_t* sP = sQD + 2 * 2 * QD_BYTES;
-    uint8_t* sDS = sP + PS_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sDS + PS_BYTES);
+    uint8_t* sPS = sQD + 2 * 2 * QD_BYTES;                // 2 x (P, dS)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sPS + 2 * 2 * PS_BYTES);
     uint64_t* kv_full = bars;
     uint64_t* qd_full = bars + 1;      // [2]
     uint64_t* qd_empty = bars + 3;     // [2]
-    uint64_t* s_full = bars + 5;
-    uint64_t* ds_full = bars + 6;
-    uint64_t* acc_done = bars + 7;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint64_t* s_full = bars + 5;       // [2]
+    uint64_t* ds_full = bars + 7;      // [2]
+    uint64_t* acc_done = bars + 9;     // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&qd_full[s], 1); mbar_init(&qd_empty[s], 1); }
-        mbar_init(s_full, 1);
-        mbar_init(ds_full, 4);
-        mbar_init(acc_done, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&qd_full[s], 1); mbar_init(&qd_empty[s], 1);
+            mbar_init(&s_full[s], 1); mbar_init(&ds_full[s], 4); mbar_init(&acc_done[s], 1);
+        }
         flags[0] = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -428,8 +467,9 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     int page = t < p.max_pages ? __ldg(p.page_table + (size_t)(p.shared_row ? 0 : owner) * p.max_pages + t) : -1;
     // a block sees this tile if its context is longer than the tile's first key
     auto sees = [&](int b) { return min(max(__ldg(p.ctx_len + b), 0), p.max_ctx_len) > key0; };
-    bool any = false;
-    for (int b = b_lo; b < b_hi && !any; ++b) any = sees(b);
+    int n_contrib = 0;       // blocks that see this tile
+    for (int b = b_lo; b < b_hi; ++b) n_contrib += sees(b) ? 1 : 0;
+    bool any = n_contrib > 0;
     const bool page_ok = page >= 0 && page < p.n_pages;
     if (any && !page_ok) {
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, DFLASH_DEV_BAD_PAGE);
@@ -440,7 +480,7 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     bool ok = true;
     if (any) {
         if (warp == 4) {
-            if (lane == 0) {
+            if (lane == 0) {      // copies: the key tile once, then Q / dO of every block that sees it
                 const uint64_t pol_kv = policy_evict_last(), pol_q = policy_evict_first();
                 const int rowK = ((((p.layer * p.n_pages + page) * 2 + 0) * p.Hkv + g) * PG);
                 const int rowV = rowK + p.Hkv * PG;
@@ -449,36 +489,50 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tma_load_2d(sKV + KV_TILE_BYTES / 2, &tmPool, 64, rowK, kv_full, pol_kv);
                 tma_load_2d(sKV + KV_TILE_BYTES, &tmPool, 0, rowV, kv_full, pol_kv);
                 tma_load_2d(sKV + KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmPool, 64, rowV, kv_full, pol_kv);
-                const uint32_t k_addr = smem_u32(sKV), v_addr = k_addr + KV_TILE_BYTES, p_addr = smem_u32(sP), ds_addr = smem_u32(sDS);
-                // next contributing block at or after b
-                auto next_from = [&](int b) { while (b < b_hi && !sees(b)) ++b; return b; };
-                int b_load = next_from(b_lo), n_loaded = 0;
-                auto load_next = [&]() {
-                    const int st = n_loaded & 1;
-                    load_q_do(sQD + (size_t)st * 2 * QD_BYTES, sQD + (size_t)st * 2 * QD_BYTES + QD_BYTES, &tmQ, &tmDO, g, b_load * p.R,
+                int k = 0;
+                for (int b = b_lo; b < b_hi && ok; ++b) {
+                    if (!sees(b)) continue;
+                    const int st = k & 1;
+                    if (k >= 2 && !mbar_wait(&qd_empty[st], ((k >> 1) - 1) & 1, &flags[0])) { ok = false; break; }
+                    load_q_do(sQD + (size_t)st * 2 * QD_BYTES, sQD + (size_t)st * 2 * QD_BYTES + QD_BYTES, &tmQ, &tmDO, g, b * p.R,
                               &qd_full[st], pol_q);
-                    ++n_loaded;
-                    b_load = next_from(b_load + 1);
-                };
-                load_next();
-                if (b_load < b_hi) load_next();
+                    ++k;
+                }
+                if (!ok) {
+                    flags[0] = 1;
+                    if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+                }
+            }
+            __syncwarp();
+        } else if (warp == 5) {
+            if (lane == 0) {      // scores of the k-th contributing block into buffer k & 1
+                const uint32_t k_addr = smem_u32(sKV), v_addr = k_addr + KV_TILE_BYTES;
                 ok = mbar_wait(kv_full, 0, &flags[0]);
-                for (int i = 0; ok; ++i) {
-                    if (i >= n_loaded) break;
-                    const int st = i & 1;
-                    if (!mbar_wait(&qd_full[st], (i >> 1) & 1, &flags[0])) { ok = false; break; }
+                for (int k = 0; k < n_contrib && ok; ++k) {
+                    const int st = k & 1;
+                    if (!mbar_wait(&qd_full[st], (k >> 1) & 1, &flags[0])) { ok = false; break; }
+                    if (k >= 2 && !mbar_wait(&ds_full[st], ((k - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t q_addr = smem_u32(sQD + (size_t)st * 2 * QD_BYTES);
+                    issue_s_dp(tmem_base + sdp_col(st), q_addr, q_addr + QD_BYTES, k_addr, v_addr);
+                    mma_commit(&s_full[st]);
+                }
+                if (!ok) {
+                    flags[0] = 1;
+                    if (p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
+                }
+            }
+            __syncwarp();
+        } else if (warp == 6) {
+            if (lane == 0) {      // accumulating products of the k-th contributing block
+                for (int k = 0; k < n_contrib && ok; ++k) {
+                    const int st = k & 1;
+                    if (!mbar_wait(&ds_full[st], (k >> 1) & 1, &flags[0])) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t q_addr = smem_u32(sQD + (size_t)st * 2 * QD_BYTES), do_addr = q_addr + QD_BYTES;
-                    issue_s_dp(tmem_base, q_addr, do_addr, k_addr, v_addr);
-                    mma_commit(s_full);
-                    if (i >= 1 && b_load < b_hi) {      // the block after next goes where the previous one was
-                        if (!mbar_wait(&qd_empty[st ^ 1], ((i - 1) >> 1) & 1, &flags[0])) { ok = false; break; }
-                        load_next();
-                    }
-                    if (!mbar_wait(ds_full, i & 1, &flags[0])) { ok = false; break; }
-                    tc_fence_after();
-                    issue_dkv_t(tmem_base, q_addr, do_addr, p_addr, ds_addr, i > 0 ? 1u : 0u);
-                    mma_commit(acc_done);
+                    const uint32_t p_addr = smem_u32(sPS + (size_t)st * 2 * PS_BYTES), ds_addr = p_addr + PS_BYTES;
+                    issue_dkv_t(tmem_base, q_addr, do_addr, p_addr, ds_addr, k > 0 ? 1u : 0u);
+                    mma_commit(&acc_done[st]);
                     mma_commit(&qd_empty[st]);
                 }
                 if (!ok) {
@@ -490,8 +544,10 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         } else {
             const int row = warp * 32 + lane;
             const uint32_t tmem_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-            const bool real = row < p.rows_valid;
-            const int r = real ? row / p.group : 0, j = real ? row % p.group : 0;
+            const int lrow = row & 63;
+            const bool real = lrow < p.rows_valid;
+            const int r = real ? lrow / p.group : 0, j = real ? lrow % p.group : 0;
+            zero_upper_rows(sPS, row);
             for (int b = b_lo; b < b_hi; ++b) {
                 const int Lb = min(max(__ldg(p.ctx_len + b), 0), p.max_ctx_len);
                 if (Lb <= key0) continue;
@@ -500,16 +556,18 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const float Dr = real ? __ldcg(p.D + qrow) : 0.f;
                 const float lse2 = real ? __ldg(p.lse + qrow) * LOG2E : 0.f;
                 const int vis = real ? min(PG, Lb - key0) : 0;
-                if (!mbar_wait(s_full, i & 1, &flags[0])) { ok = false; break; }
+                const int buf = i & 1;
+                if (!mbar_wait(&s_full[buf], (i >> 1) & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
-                if (i > 0 && !mbar_wait(acc_done, (i - 1) & 1, &flags[0])) { ok = false; break; }
-                row_math(tmem_row, sP, sDS, row, vis, lse2, Dr, p.scale, p.scale_log2);
+                if (i >= 2 && !mbar_wait(&acc_done[buf], ((i - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
+                uint8_t* sP = sPS + (size_t)buf * 2 * PS_BYTES;
+                row_math(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
                 tc_fence_before();
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(ds_full);
+                if (lane == 0) mbar_arrive(&ds_full[buf]);
             }
-            if (ok && n_done > 0 && !mbar_wait(acc_done, (n_done - 1) & 1, &flags[0])) ok = false;
+            if (ok && n_done > 0 && !mbar_wait(&acc_done[(n_done - 1) & 1], ((n_done - 1) >> 1) & 1, &flags[0])) ok = false;
             if (!ok) {
                 flags[0] = 1;
                 if (lane == 0 && p.status) atomicOr(p.status, DFLASH_DEV_TIMEOUT);
@@ -550,8 +608,8 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
 }
 
-constexpr int SMEM_Q = 1024 + 2 * QD_BYTES + 2 * 2 * KV_TILE_BYTES + 2 * PS_BYTES + 256;
-constexpr int SMEM_KV = 1024 + 2 * KV_TILE_BYTES + 2 * 2 * QD_BYTES + 2 * PS_BYTES + 256;
+constexpr int SMEM_Q = 1024 + 2 * QD_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 2 * 2 * PS_BYTES + 256;
+constexpr int SMEM_KV = 1024 + 2 * KV_TILE_BYTES + 2 * 2 * QD_BYTES + 2 * 2 * PS_BYTES + 256;
 static_assert(SMEM_Q <= 227 * 1024 && SMEM_KV <= 227 * 1024, "shared memory of one CTA");
 
 }  // namespace
