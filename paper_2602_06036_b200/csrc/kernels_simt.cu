@@ -499,16 +499,11 @@ __device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
 // V2: also track the runner-up value (for the margin). Without it (the accept step only needs the winner) the scan
 // is one compare and two selects per entry, which keeps the kernel memory-bound: the compare-and-shift chain of the
 // top-2 update was measured at 82 % instruction-issue utilisation and 31 % of DRAM bandwidth.
+// Scans entries [lo, hi) of a row with 16-byte loads (scalar at a misaligned head / tail), all 256 threads of the
+// CTA; the CTA's result is returned by thread 0 (sh: 8 entries of shared memory).
 template <typename T, bool V2>
-__global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict__ logits, int64_t row_stride,
-                                                             int vocab, int seg_len, float4* __restrict__ out) {
-    __shared__ Top2 sh[8];
+__device__ __forceinline__ Top2 scan_segment(const T* __restrict__ src, int lo, int hi, Top2* sh) {
     constexpr int VEC = 16 / (int)sizeof(T);
-    ptx::pdl_trigger();
-    ptx::pdl_wait();      // the scratch written below may alias what the previous kernel still uses
-    const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
-    const T* src = logits + (size_t)row * row_stride;
-    const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
     Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
     if (lo < hi) {
         // first index at or after lo whose address is 16-byte aligned
@@ -564,11 +559,22 @@ __global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     if (lane == 0) sh[w] = t;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        Top2 r = sh[0];
+    Top2 r = sh[0];
+    if (threadIdx.x == 0)
         for (int i = 1; i < (int)(blockDim.x >> 5); ++i) r = top2_merge(r, sh[i]);
-        out[(size_t)row * nseg + seg] = make_float4(r.v1, __int_as_float(r.i1), r.v2, 0.f);
-    }
+    return r;
+}
+
+template <typename T, bool V2>
+__global__ void __launch_bounds__(256) row_argmax_seg_kernel(const T* __restrict__ logits, int64_t row_stride,
+                                                             int vocab, int seg_len, float4* __restrict__ out) {
+    __shared__ Top2 sh[8];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();      // the scratch written below may alias what the previous kernel still uses
+    const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
+    const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
+    const Top2 r = scan_segment<T, V2>(logits + (size_t)row * row_stride, lo, hi, sh);
+    if (threadIdx.x == 0) out[(size_t)row * nseg + seg] = make_float4(r.v1, __int_as_float(r.i1), r.v2, 0.f);
 }
 
 // Stage 2: one warp per row merges the segments.
@@ -666,23 +672,17 @@ int launch_accept(const Launch& L, const dflash_verify_args& a, const int32_t* t
     return DFLASH_OK;
 }
 
-// Greedy verification from logits in two launches: the segment pass above, then one CTA per sequence
-// that merges the segments of its gamma + 1 rows (a warp per row) and applies the accept rule.
-__global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __restrict__ seg, int nseg,
-                                                            const int32_t* __restrict__ draft_ids, int draft_stride, int gamma,
-                                                            const int32_t* ctx_len, int32_t* __restrict__ accept_len,
-                                                            int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
-                                                            int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out) {
-    // new_ctx_len may alias ctx_len: neither is restrict, and the length is read before anything is written
-    __shared__ int32_t s_p[65];
-    ptx::pdl_trigger();
-    ptx::pdl_wait();
-    const int b = blockIdx.x, lane = threadIdx.x & 31;
+// Merges the segments of the gamma + 1 rows of sequence b (a warp per row) and applies the accept rule (one thread).
+__device__ __forceinline__ void merge_and_accept(const float4* seg, int nseg, int b, const int32_t* __restrict__ draft_ids, int draft_stride,
+                                                 int gamma, const int32_t* ctx_len, int32_t* __restrict__ accept_len,
+                                                 int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus, int32_t* new_ctx_len,
+                                                 int32_t* __restrict__ target_ids_out, int32_t* s_p) {
+    const int lane = threadIdx.x & 31;
     for (int j = threadIdx.x >> 5; j <= gamma; j += blockDim.x >> 5) {
         const size_t row = (size_t)b * (gamma + 1) + j;
         Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
         for (int i = lane; i < nseg; i += 32) {
-            const float4 e = seg[row * nseg + i];
+            const float4 e = __ldcg(seg + row * nseg + i);
             t = top2_merge(t, Top2{e.x, __float_as_int(e.y), e.z});
         }
 #pragma unroll
@@ -702,7 +702,7 @@ __global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __rest
     __syncthreads();
     if (threadIdx.x == 0) {
         const int32_t* d = draft_ids + (size_t)b * draft_stride;
-        const int32_t len = ctx_len[b];
+        const int32_t len = ctx_len[b];      // new_ctx_len may alias ctx_len: read before anything is written
         int a = 0;
         while (a < gamma && d[a] == s_p[a]) ++a;
         int32_t* o = out_tokens + (size_t)b * (gamma + 1);
@@ -713,6 +713,54 @@ __global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __rest
     }
 }
 
+// Second launch of the two-launch form (more sequences than tickets): one CTA per sequence.
+__global__ void __launch_bounds__(256) argmax_accept_kernel(const float4* __restrict__ seg, int nseg,
+                                                            const int32_t* __restrict__ draft_ids, int draft_stride, int gamma,
+                                                            const int32_t* ctx_len, int32_t* __restrict__ accept_len,
+                                                            int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
+                                                            int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out) {
+    __shared__ int32_t s_p[65];
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
+    merge_and_accept(seg, nseg, blockIdx.x, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus, new_ctx_len,
+                     target_ids_out, s_p);
+}
+
+// Greedy verification from logits in ONE launch: every CTA scans one segment of one row; the CTA that takes the last
+// ticket of its sequence merges the sequence's segments and applies the accept rule. The tickets live in the library
+// image (zero at load); atomicInc wraps the last ticket back to zero, so a call leaves them as it found them. Calls
+// that overlap on one GPU would mix their tickets: like every call of the library, verify calls run one after the other.
+constexpr int VERIFY_TICKETS = 4096;      // sequences per call on this path (more take the two-launch path)
+__device__ unsigned int g_verify_tickets[VERIFY_TICKETS];
+
+template <typename T>
+__global__ void __launch_bounds__(256) verify_fused_kernel(const T* __restrict__ logits, int64_t row_stride, int vocab, int seg_len,
+                                                           float4* seg_out, const int32_t* __restrict__ draft_ids, int draft_stride,
+                                                           int gamma, const int32_t* ctx_len, int32_t* __restrict__ accept_len,
+                                                           int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
+                                                           int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out) {
+    __shared__ Top2 sh[8];
+    __shared__ int32_t s_p[65];
+    __shared__ int s_last;
+    ptx::pdl_trigger();
+    ptx::pdl_wait();
+    const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
+    const int b = row / (gamma + 1);
+    const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
+    const Top2 r = scan_segment<T, false>(logits + (size_t)row * row_stride, lo, hi, sh);
+    if (threadIdx.x == 0) {
+        seg_out[(size_t)row * nseg + seg] = make_float4(r.v1, __int_as_float(r.i1), r.v2, 0.f);
+        __threadfence();
+        const unsigned int n = (unsigned int)nseg * (unsigned int)(gamma + 1);
+        s_last = atomicInc(&g_verify_tickets[b], n - 1) == n - 1 ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();      // the other CTAs' segment results are visible
+    merge_and_accept(seg_out, nseg, b, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus, new_ctx_len,
+                     target_ids_out, s_p);
+}
+
 int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t row_stride, float4* seg_scratch) {
     if (a.batch == 0) return DFLASH_OK;
     if (a.gamma > 64) return DFLASH_ERR_INVALID_ARG;
@@ -721,6 +769,18 @@ int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t r
     const int seg_len = ((a.vocab + nseg - 1) / nseg + 7) / 8 * 8;
     dim3 grid(nseg, rows);
     cudaError_t e;
+    if (a.batch <= VERIFY_TICKETS) {
+        if (a.logits_dtype == DFLASH_F32)
+            e = launch_pdl(verify_fused_kernel<float>, grid, dim3(256), 0, L.st, (const float*)a.logits, row_stride, a.vocab, seg_len,
+                           seg_scratch, a.draft_ids, a.draft_stride, a.gamma, a.ctx_len, a.accept_len, a.out_tokens, a.bonus,
+                           a.new_ctx_len, a.target_ids_out);
+        else
+            e = launch_pdl(verify_fused_kernel<__nv_bfloat16>, grid, dim3(256), 0, L.st, (const __nv_bfloat16*)a.logits, row_stride,
+                           a.vocab, seg_len, seg_scratch, a.draft_ids, a.draft_stride, a.gamma, a.ctx_len, a.accept_len, a.out_tokens,
+                           a.bonus, a.new_ctx_len, a.target_ids_out);
+        ++g_launches;
+        return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+    }
     if (a.logits_dtype == DFLASH_F32)
         e = launch_pdl(row_argmax_seg_kernel<float, false>, grid, dim3(256), 0, L.st, (const float*)a.logits, row_stride, a.vocab, seg_len,
                        seg_scratch);
