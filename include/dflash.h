@@ -216,6 +216,9 @@ typedef struct {
 int32_t dflash_target_verify(dflash_handle* h, const dflash_target_args* a /*[host]*/, void* stream);
 
 /* ---- greedy verify / accept (Sec. 3.1: tau in [1, gamma+1] incl. the bonus token) ----
+ * One launch in either mode. Mode LOGITS counts, per sequence, the CTAs that have finished scanning in a small
+ * ticket array inside the library image (16 KB per GPU, self-resetting; up to 4096 sequences per call, more take two
+ * launches): like all calls of this library, verify calls on one GPU must not overlap in time.
  * p_j = argmax_v logits[b, j, :] (mode LOGITS) or target_ids[b, j] (mode IDS), j = 0..gamma.
  * a = length of the longest prefix with draft[b, i] == p_i, i < a;  tau = a + 1;
  * out_tokens[b] = draft[b, 0..a-1], p_a, then -1; bonus[b] = p_a; new_ctx_len[b] = ctx_len[b]+tau. */
