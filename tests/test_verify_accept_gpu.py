@@ -100,3 +100,22 @@ def test_new_len_may_alias_ctx_len():
     lib.dflash_verify_accept(drafts, gamma, gamma, ctx, tau, toks, bonus, ctx, target_ids=tids)
     torch.cuda.synchronize()
     assert tau.tolist() == [4, 3, 2, 1] and ctx.tolist() == [14, 23, 32, 41]
+
+
+def test_more_sequences_than_tickets_take_two_launches_with_the_same_result():
+    # the one-launch form keeps one ticket per sequence for up to 4096 sequences; a larger batch runs the segment
+    # scan and the per-sequence merge as two launches. Both forms against numpy's first-occurrence argmax + the
+    # oracle's accept rule, and the one-launch form twice in a row (its tickets must be back at zero).
+    lib = _lib()
+    gamma, V = 2, 4099
+    for S in (4096, 4100):
+        logits, drafts, a = synth.make_verify_case(S, gamma, V, 0.5, 11, torch.bfloat16)
+        ctx = torch.arange(S, dtype=torch.int32) + 7
+        ref_ids = np.argmax(synth.to_numpy_f32(logits), axis=-1)
+        for _ in range(2):
+            got = _run(lib, drafts, gamma, ctx, logits=logits)
+            assert np.array_equal(got["tids"], ref_ids)
+            assert np.array_equal(got["tau"], a.numpy() + 1)
+            for b in (0, 1, S // 2, S - 1):
+                tau, out, bonus, new_len = orc.verify_accept(drafts[b].numpy(), ref_ids[b], int(ctx[b]))
+                assert got["toks"][b].tolist() == out.tolist() and got["bonus"][b] == bonus and got["new_len"][b] == new_len
