@@ -36,6 +36,7 @@ using namespace ptx;
 
 constexpr int HD = 128;          // head_dim
 constexpr int PG = 64;           // tokens per page = keys per tile
+constexpr int LPT_MAX = 256;      // batches up to this size are taken longest sequence first
 constexpr int NS = 5;            // K/V ring depth (the kernel is bound by the bytes it keeps in flight: 3 stages ran 1.37x slower than 4)
 constexpr int Q_BYTES = 128 * HD * 2;            // 32 KiB: two 64-wide halves of 128 rows
 constexpr int KV_STAGE_BYTES = 2 * PG * HD * 2;  // K (16 KiB) + V (16 KiB)
@@ -135,7 +136,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     pdl_trigger();
     const int chunk = blockIdx.x % p.n_chunks;
     const int g = (blockIdx.x / p.n_chunks) % p.Hkv;
-    const int b = blockIdx.x / (p.n_chunks * p.Hkv);
+    // CTAs are handed to the SMs in index order, so the sequences are taken longest first (a long sequence that
+    // starts in the last wave would hold the tail alone): the CTA group with number s works on the sequence whose
+    // length has rank s, ties by index. Every CTA finds that sequence itself from the call's lengths.
+    int b = blockIdx.x / (p.n_chunks * p.Hkv);
+    if (p.S > 1 && p.S <= LPT_MAX) {
+        __shared__ int s_len[LPT_MAX];
+        __shared__ int s_seq;
+        const int want = b;
+        for (int t = threadIdx.x; t < p.S; t += N_THREADS) s_len[t] = p.ctx_len[t];
+        __syncthreads();
+        if ((int)threadIdx.x < p.S) {
+            const int t = threadIdx.x, mine = s_len[t];
+            int rank = 0;
+            for (int j = 0; j < p.S; ++j) {
+                const int l = s_len[j];
+                rank += (l > mine || (l == mine && j < t)) ? 1 : 0;
+            }
+            if (rank == want) s_seq = t;
+        }
+        __syncthreads();
+        b = s_seq;
+    }
     const int L_given = p.ctx_len[b];
     const int L = min(max(L_given, 0), p.max_ctx_len);   // the ranges (and the partials buffer) cover max_ctx_len keys
     if (L_given > p.max_ctx_len && threadIdx.x == 0 && chunk == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);

@@ -348,10 +348,15 @@ def test_decode_step_appends_at_ctx_len():
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("mode", ["full", "causal"])
-def test_block_attention_building_block(dtype, mode):
+@pytest.mark.parametrize("n_seq", [8, 260])
+def test_block_attention_building_block(dtype, mode, n_seq):
+    # 8 sequences: lengths around the tile edges, with ties (the kernel takes the sequences longest first, equal
+    # lengths by index); 260 sequences: more than the kernel ranks by length, taken in index order
     from paper_2602_06036_b200 import binding
     cfg = synth.TINY if dtype == "fp32" else synth.MID
-    lens = (0, 1, 63, 64, 65, 300)
+    lens = (0, 1, 63, 64, 65, 300, 64, 300)
+    if n_seq > len(lens):
+        lens = tuple((37 * i) % 131 for i in range(n_seq))
     case = Case(cfg, lens, seed=7)
     case.fill_pool_synthetic()
     R = 9 if mode == "causal" else cfg.block_size
