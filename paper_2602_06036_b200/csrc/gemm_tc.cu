@@ -75,6 +75,9 @@ struct WMaps {
 
 struct KParams {
     int M, N, K, epi, chunks_total, n_groups, n_ftiles, n_ttiles, n_tiles, w_map0, x_map;
+    // A launch of CTA pairs walks PAIRS of neighbouring weight tiles: n_ftiles and n_tiles then count those pairs and
+    // n_ftiles_real the weight tiles themselves (an odd count leaves the last pair's odd CTA a tile beyond the matrix).
+    int n_ftiles_real;
     int cluster_k;     // the phase splits every tile's K range over the CTAs of a cluster (partial sums through their shared memory)
     float* part;
     int32_t* counters;
@@ -124,7 +127,18 @@ struct Unit {
     int slot;      // 0 = first piece of this CTA's range, 1 = a later one (partial pieces only: first or last)
     int full;      // covers every chunk of the tile
     int cl;        // this CTA's K share of a tile that its cluster finishes together
+    int ctr;       // index of the tile's ticket counter
+    int phantom;   // CTA pairs: this CTA's weight tile lies beyond the matrix (it only keeps the pair's protocol going)
 };
+// CTA pairs: the walk hands out pairs of weight tiles; CTA `prank` of the pair takes tile 2 * pair + prank.
+template <bool PAIR>
+__device__ __forceinline__ void own_tile(const KParams& p, Unit& u, int prank) {
+    if constexpr (PAIR) {
+        u.ft = u.ft * 2 + prank;
+        u.phantom = u.ft >= p.n_ftiles_real ? 1 : 0;
+        u.ctr = (u.g * p.n_ftiles_real + u.ft) * p.n_ttiles + u.tt;
+    }
+}
 
 // Work of CTA `cta` out of `n_ctas` in one phase. With at least one tile per CTA the tiles are split
 // into a SHARED part (the first n_tiles % n_ctas tiles) and whole tiles, the same number per CTA:
@@ -196,6 +210,8 @@ struct PieceWalk {
         t /= p.n_ttiles;
         u.ft = t % p.n_ftiles;
         u.g = t / p.n_ftiles;
+        u.ctr = u.tile;
+        u.phantom = 0;
         return u;
     }
 };
@@ -456,13 +472,20 @@ __device__ __forceinline__ void apply_epilogue(const KParams& p, float* sAcc, To
             if (p.logits_out && f < p.N)
                 for (int c = 0; c < n_tok; ++c) p.logits_out[(size_t)(tok0 + c) * p.N + f] = sAcc[row * ACC_LD + c];
             const int c = row % CH, g = row / CH;
-            T2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-#pragma unroll 16
+            // largest value, its first row and the second largest value of CH rows of one token column, without
+            // branches (rows come in increasing order, so a strict comparison keeps the smallest index among equals;
+            // data-dependent branches made this scan the slowest part of a wide token tile's epilogue)
+            float v1 = -CUDART_INF_F, v2 = -CUDART_INF_F;
+            int i1 = 0x7fffffff;
+            const int f_base = un.ft * TILE_F + g * CH;
+#pragma unroll
             for (int r = 0; r < CH; ++r) {
-                const int rr = g * CH + r, ff = un.ft * TILE_F + rr;
-                if (ff < p.N) t2_push(t, sAcc[rr * ACC_LD + c], ff);
+                const float x = (f_base + r < p.N) ? sAcc[(g * CH + r) * ACC_LD + c] : -CUDART_INF_F;
+                i1 = (x > v1) ? f_base + r : i1;
+                v2 = fmaxf(v2, fminf(v1, x));
+                v1 = fmaxf(v1, x);
             }
-            sRed[g * CH + c] = Top2Entry{t.v1, t.i1, t.v2, 0};
+            sRed[g * CH + c] = Top2Entry{v1, i1, v2, 0};
             epi_bar();
             if (row < n_tok) {
                 T2 m{sRed[row].v1, sRed[row].i1, sRed[row].v2};
@@ -630,15 +653,22 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 // Register cap: with small token tiles the kernel is kept at 232 registers, so that a warp of a small dependent
 // kernel (merge, finish) still fits into the register file partition that holds two of this CTA's six warps and
 // can become resident before this grid has drained.
-template <int NT, int SL, bool QKN>
+// PAIR: the launch runs as clusters of two CTAs that share every MMA (cta_group::2, M = 256): each CTA streams its own
+// 128-row weight tile but only HALF of the token tile, so a ring stage is a third smaller and the ring deeper - with
+// 160 to 256 token columns the single-CTA form is limited by the operand bytes an SM keeps in flight, not by the tensor
+// pipe. The even CTA's MMA thread issues for both; its commits arrive on both CTAs' barriers. Each CTA holds its own
+// 128 rows x NT columns of the accumulator in its own TMEM, so the epilogues are those of the single-CTA form.
+template <int NT, int SL, bool QKN, bool PAIR>
 __global__ void __maxnreg__(NT <= 32 ? 232 : 255)
 gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps tmX, const __grid_constant__ MParams mp) {
     if (threadIdx.x == 0) trace_min(mp.ph[0].trace, 0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int W_STAGE = W_STAGE_BYTES * SL;
-    constexpr int X_SLAB = NT * BK * 2;
+    constexpr int XR = PAIR ? NT / 2 : NT;           // token rows of the activation tile this CTA loads
+    constexpr int X_SLAB = XR * BK * 2;
     constexpr int X_STAGE = X_SLAB * SL;
+    static_assert(!PAIR || (SL == 1 && NT % 32 == 0 && NT >= 64), "CTA pairs: one slab per stage, halves of whole 16-row groups");
     constexpr int CH = pass_cols(NT);
     constexpr int ACC_LD = CH + 1;
     // partial pieces fetched together when finishing. More would shorten the tail further, but the register
@@ -669,7 +699,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); mbar_init(&xch_bar[b], 1); }
+        // a pair's leader frees an accumulator buffer when the epilogue warps of BOTH CTAs have read it
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], PAIR ? 8 : 4); mbar_init(&xch_bar[b], 1); }
         flags[0] = 0; flags[2] = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -686,8 +717,23 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     if (mp.cs > 1) cluster_arrive();
 
     const int G = gridDim.x;
+    // CTA pairs: the pair is the unit that walks the work; both CTAs take the same pieces
+    const int prank = PAIR ? (int)cluster_ctarank() : 0;
+    const int wid = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int WG = PAIR ? G >> 1 : G;
+    bool run = true;
+    if constexpr (PAIR) {
+        // Both CTAs' barriers exist before anyone arrives on a peer's; the MMA addresses both accumulators by ONE
+        // TMEM address, so the two allocations must have come out at the same columns (each CTA allocates once from
+        // an empty TMEM, so they do; checked, not assumed).
+        cluster_sync_all();
+        run = ld_shared_cluster_u32(mapa_shared(smem_u32(tmem_slot), (uint32_t)(prank ^ 1))) == tmem_base;
+        if (!run && threadIdx.x == 0 && mp.status) atomicOr(mp.status, DFLASH_DEV_TIMEOUT);
+    }
 
-    if (warp == 0) {
+    if (!run) {
+        // nothing: the other pairs' waits run out and the call reports the status word
+    } else if (warp == 0) {
         // ---------------- TMA producer ----------------
         // WEIGHT tiles are issued as soon as a ring slot is free. The ACTIVATION tile of a slot needs
         // the phase's inputs (phase 0: the grid dependency; later phases: every CTA has finished the
@@ -697,9 +743,12 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
             // chunk c of rows y.. : SL slabs of 64 K-elements
-            auto load = [&](void* dst, const CUtensorMap* m, int c, int y, uint64_t* bar, uint64_t pol) {
-                if constexpr (SL == 1) tma_load_2d(dst, m, c * BK, y, bar, pol);
-                else tma_load_3d(dst, m, 0, y, c * SL, bar, pol);
+            // CTA pairs: both CTAs' copies count their bytes on the LEADER's barrier of the stage
+            const uint32_t full_leader = PAIR ? mapa_shared(smem_u32(full), 0u) : 0u;
+            auto load = [&](void* dst, const CUtensorMap* m, int c, int y, int slot, uint64_t pol) {
+                if constexpr (PAIR) tma_load_2d_pair(dst, m, c * BK, y, full_leader + (uint32_t)slot * 8u, pol);
+                else if constexpr (SL == 1) tma_load_2d(dst, m, c * BK, y, &full[slot], pol);
+                else tma_load_3d(dst, m, 0, y, c * SL, &full[slot], pol);
             };
             int* q_ph = sPend;                      // queued slots: phase, chunk, token tile (ring order)
             int* q_c = sPend + MAX_STAGES;
@@ -725,7 +774,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         }
                         ready_ph = ph;
                     }
-                    load(sX + (size_t)q_head * X_STAGE, &tmX.m[mp.ph[ph].x_map], q_c[q_head], q_tt[q_head] * NT, &full[q_head], pol_x);
+                    load(sX + (size_t)q_head * X_STAGE, &tmX.m[mp.ph[ph].x_map], q_c[q_head], q_tt[q_head] * NT + prank * XR, q_head, pol_x);
                     q_head = (q_head + 1 == stages) ? 0 : q_head + 1;
                     --q_count;
                 }
@@ -733,10 +782,11 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
                 const CUtensorMap* xm = &tmX.m[p.x_map];
-                for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p) && ok;) {
-                    const Unit un = w.next(p);
+                for (PieceWalk w(p, wid, WG, mp.cs); !w.done(p) && ok;) {
+                    Unit un = w.next(p);
+                    own_tile<PAIR>(p, un, prank);
                     const CUtensorMap* wm = &tmW.m[p.w_map0 + un.g];
-                    const int y_w = un.ft * TILE_F, y_x = un.tt * NT;
+                    const int y_w = un.ft * TILE_F, y_x = un.tt * NT + prank * XR;      // rows beyond the matrix arrive as zeros
                     for (int c = un.c0; c < un.c1; ++c) {
                         if (!mbar_try_wait(&empty[st], par ^ 1)) {
                             const long long t0 = clock64();
@@ -746,10 +796,10 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                             }
                             if (!ok) break;
                         }
-                        mbar_expect_tx(&full[st], W_STAGE + X_STAGE);
-                        load(sW + (size_t)st * W_STAGE, wm, c, y_w, &full[st], pol_w);
+                        if (!PAIR || prank == 0) mbar_expect_tx(&full[st], (PAIR ? 2 : 1) * (W_STAGE + X_STAGE));
+                        load(sW + (size_t)st * W_STAGE, wm, c, y_w, st, pol_w);
                         if (q_count == 0 && ph <= ready_ph) {
-                            load(sX + (size_t)st * X_STAGE, xm, c, y_x, &full[st], pol_x);
+                            load(sX + (size_t)st * X_STAGE, xm, c, y_x, st, pol_x);
                         } else {
                             if (q_count == 0) q_head = st;
                             q_ph[st] = ph; q_c[st] = c; q_tt[st] = un.tt;
@@ -780,13 +830,14 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         if (mp.cs > 1) cluster_wait();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(TILE_F, NT);
+        // (the odd CTA of a pair issues nothing: the leader's MMAs read both CTAs' operands and write both accumulators)
+        if (lane == 0 && !(PAIR && prank == 1)) {
+            constexpr uint32_t idesc = instr_desc_bf16(PAIR ? 2 * TILE_F : TILE_F, NT);
             uint32_t it = 0, ui = 0;
             bool ok = true;
             for (int ph = 0; ph < mp.n_phases && ok; ++ph) {
                 const KParams& p = mp.ph[ph];
-                for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p) && ok; ++ui) {
+                for (PieceWalk w(p, wid, WG, mp.cs); !w.done(p) && ok; ++ui) {
                     const Unit un = w.next(p);
                     const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
                     if (!mbar_wait(&acc_empty[buf], aph ^ 1, &flags[0])) { ok = false; break; }
@@ -800,13 +851,20 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         const uint32_t a_addr = smem_u32(sW + (size_t)st * W_STAGE);
                         const uint32_t b_addr = smem_u32(sX + (size_t)st * X_STAGE);
 #pragma unroll
-                        for (int kk = 0; kk < SL * (BK / 16); ++kk)
-                            mma_bf16(d_tmem, smem_desc_sw128(a_addr + (kk >> 2) * W_STAGE_BYTES + (kk & 3) * 32),
-                                     smem_desc_sw128(b_addr + (kk >> 2) * X_SLAB + (kk & 3) * 32), idesc,
-                                     (c > un.c0 || kk > 0) ? 1u : 0u);
-                        mma_commit(&empty[st]);
+                        for (int kk = 0; kk < SL * (BK / 16); ++kk) {
+                            const uint64_t da = smem_desc_sw128(a_addr + (kk >> 2) * W_STAGE_BYTES + (kk & 3) * 32);
+                            const uint64_t db = smem_desc_sw128(b_addr + (kk >> 2) * X_SLAB + (kk & 3) * 32);
+                            const uint32_t acc = (c > un.c0 || kk > 0) ? 1u : 0u;
+                            if constexpr (PAIR) mma_bf16_pair(d_tmem, da, db, idesc, acc);
+                            else mma_bf16(d_tmem, da, db, idesc, acc);
+                        }
+                        if constexpr (PAIR) mma_commit_pair(&empty[st], 3);
+                        else mma_commit(&empty[st]);
                     }
-                    if (ok) mma_commit(&acc_full[buf]);
+                    if (ok) {
+                        if constexpr (PAIR) mma_commit_pair(&acc_full[buf], 3);
+                        else mma_commit(&acc_full[buf]);
+                    }
                 }
                 trace_max(p.trace, 2);
             }
@@ -836,7 +894,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
         if (mp.cs > 1) cluster_wait();      // every peer has set up its barriers (they arrived after doing so)
         for (int ph = 0; ph < mp.n_phases && alive; ++ph) {
             const KParams& p = mp.ph[ph];
-            const long long T = (long long)shared_tiles(p, G) * p.chunks_total;      // pairs of the shared part
+            const long long T = (long long)shared_tiles(p, WG) * p.chunks_total;     // (tile, chunk) pairs of the shared part
             const bool all_tok = p.M <= TOK_CACHE;   // per-token data cached for the whole phase (else per token tile)
             const bool need_info = p.epi == EPI_QKV_ROPE || p.epi == EPI_CTX_KV;
             int rstd_tt = -1, info_tt = -1;
@@ -872,8 +930,8 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     const int tok_base = un.tt * NT;
                     const int tok_off = all_tok ? tok_base : 0;
                     const long long x0 = (long long)un.tile * p.chunks_total;
-                    const int j0 = cta_of_pair(x0, T, G), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, G);
-                    const int n_contrib = j1 - j0 + 1, my_q = (int)blockIdx.x - j0;
+                    const int j0 = cta_of_pair(x0, T, WG), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, WG);
+                    const int n_contrib = j1 - j0 + 1, my_q = wid - j0;
                     const int n_ch = (min(NT, p.M - tok_base) + CH - 1) / CH;
                     if (my_q >= n_ch) continue;                      // more contributors than passes: nothing for this one
                     // residual rows of the first pass travel while the tickets are polled
@@ -881,7 +939,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                     if constexpr (CH <= 32) residual_load<CH>(p, un, tok_base + my_q * CH, row, xres, gain);
                     if (row == 0) {
                         const long long t0 = clock64();
-                        while (ld_acquire(p.counters + un.tile) < n_contrib) {
+                        while (ld_acquire(p.counters + un.ctr) < n_contrib) {
                             if (flags[0] || clock64() - t0 > SPIN_LIMIT) { flags[2] = 1; break; }
                         }
                     }
@@ -906,8 +964,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                             for (int u = 0; u < PF; ++u) {
                                 const int j = jb + u;
                                 if (j <= j1) {
-                                    const int sa = ((long long)j * T / G >= x0) ? 0 : 1;
-                                    const float* pa = p.part + (((size_t)j * 2 + sa) * NT + ch * CH) * TILE_F + row;
+                                    const int sa = ((long long)j * T / WG >= x0) ? 0 : 1;
+                                    const size_t jc = PAIR ? (size_t)j * 2 + prank : (size_t)j;      // the contributing CTA
+                                    const float* pa = p.part + ((jc * 2 + sa) * NT + ch * CH) * TILE_F + row;
 #pragma unroll
                                     for (int c = 0; c < CH; ++c) va[u][c] = __ldcg(pa + (size_t)c * TILE_F);
                                 } else {
@@ -930,8 +989,9 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 }
                 n_pend = 0;
             };
-            for (PieceWalk w(p, blockIdx.x, G, mp.cs); !w.done(p); ++ui) {
-                const Unit un = w.next(p);
+            for (PieceWalk w(p, wid, WG, mp.cs); !w.done(p); ++ui) {
+                Unit un = w.next(p);
+                own_tile<PAIR>(p, un, prank);
                 const int tok_base = un.tt * NT;
                 const uint32_t buf = ui & 1, aph = (ui >> 1) & 1;
                 const int tok_off = all_tok ? tok_base : 0;          // index of this tile's first token in the caches
@@ -944,6 +1004,16 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                 epi_bar();
                 if (flags[2]) { alive = false; break; }   // uniform over the four warps
                 tc_fence_after();
+                // the leader of a pair counts both CTAs' epilogue warps before it overwrites an accumulator buffer
+                auto release_acc = [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR && prank == 1) mbar_arrive_cluster(mapa_shared(smem_u32(&acc_empty[buf]), 0u));
+                        else mbar_arrive(&acc_empty[buf]);
+                    }
+                };
+                if (un.phantom) { release_acc(); continue; }
                 // The accumulator exists, so the previous phase is complete and its sums of squares are final.
                 if (p.ssq_in && !all_tok && rstd_tt != un.tt) {
                     token_rstd(p, tok_base, NT, row, sRstd);
@@ -1037,13 +1107,11 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
                         apply_epilogue<CH, QKN>(p, sAcc, sRed, un, tok_base + ch * CH, row, sPos + tok_off + ch * CH, sPage + tok_off + ch * CH, xres, gain, v);
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                release_acc();
                 if (!un.full) {
                     // the tile is shared: publish the piece, take a ticket, finish the tile at the end of the phase
                     epi_bar();
-                    if (row == 0) red_release_add(p.counters + un.tile, 1);
+                    if (row == 0) red_release_add(p.counters + un.ctr, 1);
                     pend[n_pend++] = un;
                     if (w.shared_done() && !w.done(p)) {      // whole tiles follow: reduce now, under their main loop
                         finish_shared();
@@ -1075,7 +1143,7 @@ gemm_tc_kernel(const __grid_constant__ WMaps tmW, const __grid_constant__ XMaps 
     }
     // no CTA of a cluster may go away while a peer can still write into its shared memory; every wait above is
     // bounded, so every CTA gets here
-    if (mp.cs > 1) cluster_sync_all();
+    if (mp.cs > 1 || PAIR) cluster_sync_all();
 }
 
 // Merge of the per-tile winners (index-aware, so order-independent). The entries are laid out
@@ -1253,6 +1321,7 @@ int pick_nt(int M) {
 constexpr int MAX_CLUSTERS = 32, MIN_CLUSTERS = 16;
 template <int NT, int SL, bool QKN>
 int cluster_capacity(int stages) {
+    constexpr bool PAIR = false;
     static int memo[MAX_DEVICES];
     static bool known[MAX_DEVICES] = {};
     const int dev = current_device_slot();
@@ -1269,7 +1338,7 @@ int cluster_capacity(int stages) {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<NT, SL, QKN>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<NT, SL, QKN, PAIR>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
     }
@@ -1279,12 +1348,48 @@ int cluster_capacity(int stages) {
     return n;
 }
 
-template <int NT, int SL, bool QKN>
+constexpr int pair_smem(int nt, int stages) { return 1024 + stages * (W_STAGE_BYTES + (nt / 2) * BK * 2) + smem_fixed(nt); }
+constexpr int pair_stages(int nt) { return std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (W_STAGE_BYTES + (nt / 2) * BK * 2)); }
+
+template <int NT, int SL, bool QKN, bool PAIR>
+int set_attr();
+
+// CTA pairs the device keeps resident at once for the pair form of a kernel (its CTAs wait for each other), asked of
+// the runtime once per device and kernel.
+template <int NT, bool QKN>
+int pair_capacity() {
+    static int memo[MAX_DEVICES];
+    static bool known[MAX_DEVICES] = {};
+    const int dev = current_device_slot();
+    if (dev >= 0 && known[dev]) return memo[dev];
+    int n = 0;
+    if (set_attr<NT, 1, QKN, true>() == DFLASH_OK) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 1024);
+        cfg.blockDim = dim3(N_THREADS);
+        cfg.dynamicSmemBytes = (size_t)pair_smem(NT, pair_stages(NT));
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<NT, 1, QKN, true>, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+    }
+    if (dev >= 0) { memo[dev] = n; known[dev] = true; }
+    return n;
+}
+
+template <int NT, int SL, bool QKN, bool PAIR>
 int set_attr() {
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = current_device_slot();
     if (dev < 0 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL, QKN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<NT, SL, QKN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         if (dev >= 0) attr_set[dev] = true;
     }
@@ -1296,7 +1401,8 @@ int set_attr() {
 // tiles than CTAs then split each tile's K range inside a cluster instead of through global memory.
 template <int NT, int SL, bool QKN>
 int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, MParams& mp, int grid_free) {
-    if (set_attr<NT, SL, QKN>() != DFLASH_OK) return DFLASH_ERR_CUDA;
+    constexpr bool PAIR = false;
+    if (set_attr<NT, SL, QKN, PAIR>() != DFLASH_OK) return DFLASH_ERR_CUDA;
     const int smem = 1024 + mp.stages * SL * (W_STAGE_BYTES + NT * BK * 2) + smem_fixed(NT);
     int grid = grid_free;
     mp.cs = 1;
@@ -1314,8 +1420,21 @@ int launch_nt(const Launch& L, const WMaps& tw, const XMaps& tx, MParams& mp, in
         mp.ph[i].cluster_k = (mp.cs > 1 && p.n_tiles < grid && p.chunks_total >= CS) ? 1 : 0;
     }
     const cudaError_t e =
-        mp.cs > 1 ? launch_pdl_cluster(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, CS, tw, tx, mp)
-                  : launch_pdl(gemm_tc_kernel<NT, SL, QKN>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
+        mp.cs > 1 ? launch_pdl_cluster(gemm_tc_kernel<NT, SL, QKN, PAIR>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, CS, tw, tx, mp)
+                  : launch_pdl(gemm_tc_kernel<NT, SL, QKN, PAIR>, dim3(grid), dim3(N_THREADS), (size_t)smem, L.st, tw, tx, mp);
+    ++g_launches;
+    return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
+}
+
+// The pair form: `pairs` clusters of two CTAs (the phases were filled for pairs of weight tiles, the activation maps
+// for half token tiles).
+template <int NT, bool QKN>
+int launch_pair(const Launch& L, const WMaps& tw, const XMaps& tx, MParams& mp, int pairs) {
+    if (set_attr<NT, 1, QKN, true>() != DFLASH_OK) return DFLASH_ERR_CUDA;
+    mp.cs = 1;
+    for (int i = 0; i < mp.n_phases; ++i) mp.ph[i].cluster_k = 0;
+    const cudaError_t e = launch_pdl_cluster(gemm_tc_kernel<NT, 1, QKN, true>, dim3(2 * pairs), dim3(N_THREADS),
+                                             (size_t)pair_smem(NT, mp.stages), L.st, 2, tw, tx, mp);
     ++g_launches;
     return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
 }
@@ -1337,14 +1456,15 @@ int64_t gemm_tc_counter_bytes(int M, int N, int n_groups) {
     return (int64_t)std::max(n_groups, 1) * ((N + TILE_F - 1) / TILE_F) * ttiles * 4;
 }
 
-static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, KParams& p) {
+static int fill_phase(const Launch& L, const GemmArgs& a, int nt, int slabs, bool pair, KParams& p) {
     if (a.K % 8 != 0) return DFLASH_ERR_UNSUPPORTED;
     const dflash_config& c = L.h->cfg;
     const int groups = std::max(a.n_groups, 1);
     p = KParams{};
     p.M = a.M; p.N = a.N; p.K = a.K; p.epi = a.epilogue;
     p.n_groups = groups;
-    p.n_ftiles = (a.N + TILE_F - 1) / TILE_F;
+    p.n_ftiles_real = (a.N + TILE_F - 1) / TILE_F;
+    p.n_ftiles = pair ? (p.n_ftiles_real + 1) / 2 : p.n_ftiles_real;
     p.n_ttiles = (a.M + nt - 1) / nt;
     p.chunks_total = (a.K + BK * slabs - 1) / (BK * slabs);
     p.n_tiles = groups * p.n_ftiles * p.n_ttiles;
@@ -1390,8 +1510,26 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     bool k64 = true;
     for (int i = 0; i < n_phases; ++i) k64 = k64 && phases[i].K % BK == 0;
     const int slabs = slabs_for(nt, k64);
+    bool qkn = false;
+    for (int i = 0; i < n_phases; ++i) {
+        qkn = qkn || phases[i].g_q != nullptr || phases[i].g_k != nullptr;
+        if (phases[i].epilogue == EPI_CTX_KV)
+            for (int g = 0; g < std::max(phases[i].n_groups, 1); ++g) qkn = qkn || phases[i].g_k_group[g] != nullptr;
+    }
+    // Token tiles of 160 columns and more run as CTA pairs where the device keeps pairs resident
+    int pair_cap = 0;
+    if (nt >= 160 && L.h->sm_count >= 2) {
+        switch (nt) {
+            case 160: pair_cap = qkn ? pair_capacity<160, true>() : pair_capacity<160, false>(); break;
+            case 192: pair_cap = qkn ? pair_capacity<192, true>() : pair_capacity<192, false>(); break;
+            default: pair_cap = qkn ? pair_capacity<256, true>() : pair_capacity<256, false>(); break;
+        }
+        pair_cap = std::min(pair_cap, L.h->sm_count / 2);
+    }
+    const bool pair = pair_cap >= 1;
     mp.n_phases = n_phases;
-    mp.stages = std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (slabs * (W_STAGE_BYTES + nt * BK * 2)));
+    mp.stages = pair ? pair_stages(nt)
+                     : std::min(MAX_STAGES, (SMEM_LIMIT - 1024 - smem_fixed(nt)) / (slabs * (W_STAGE_BYTES + nt * BK * 2)));
     mp.phase_done = phase_done;
     mp.status = L.status;
 
@@ -1400,7 +1538,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     for (int i = 0; i < n_phases; ++i) {
         const GemmArgs& a = phases[i];
         if (a.M <= 0 || a.N <= 0) return DFLASH_ERR_INVALID_ARG;
-        const int rc = fill_phase(L, a, nt, slabs, mp.ph[i]);
+        const int rc = fill_phase(L, a, nt, slabs, pair, mp.ph[i]);
         if (rc != DFLASH_OK) return rc;
         KParams& p = mp.ph[i];
         p.trace = traces ? traces[i] : nullptr;
@@ -1409,7 +1547,7 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
         for (int g = 0; g < p.n_groups; ++g)
             if (!weight_map(L.h, &tw.m[n_maps++], a.W[g], a.N, a.K, slabs)) return DFLASH_ERR_CUDA;
         p.x_map = i;
-        if (!make_map(&tx.m[i], a.X, a.M, a.K, nt, slabs)) return DFLASH_ERR_CUDA;
+        if (!make_map(&tx.m[i], a.X, a.M, a.K, pair ? nt / 2 : nt, slabs)) return DFLASH_ERR_CUDA;
         const long long pairs = (long long)p.n_tiles * p.chunks_total;
         min_pairs = min_pairs < 0 ? pairs : std::min(min_pairs, pairs);
     }
@@ -1417,10 +1555,14 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
     for (int i = n_phases; i < MAX_PHASES; ++i) tx.m[i] = tx.m[0];
     // one CTA per SM unless the smallest phase would leave ranges under 256 K-elements
     const int grid = (int)std::max<long long>(1, std::min<long long>(L.h->sm_count, min_pairs * slabs / 4));
-    bool qkn = false;
-    for (int i = 0; i < n_phases; ++i) {
-        qkn = qkn || mp.ph[i].gq != nullptr;
-        for (int g = 0; g < mp.ph[i].n_groups; ++g) qkn = qkn || mp.ph[i].gk[g] != nullptr;
+    if (pair) {
+        // one pair per two SMs unless the smallest phase would leave ranges under 256 K-elements
+        const int pairs = (int)std::max<long long>(1, std::min<long long>(pair_cap, min_pairs / 4));
+        switch (nt) {
+            case 160: return qkn ? launch_pair<160, true>(L, tw, tx, mp, pairs) : launch_pair<160, false>(L, tw, tx, mp, pairs);
+            case 192: return qkn ? launch_pair<192, true>(L, tw, tx, mp, pairs) : launch_pair<192, false>(L, tw, tx, mp, pairs);
+            default: return qkn ? launch_pair<256, true>(L, tw, tx, mp, pairs) : launch_pair<256, false>(L, tw, tx, mp, pairs);
+        }
     }
 #define DFLASH_GEMM_CASE(NT_, SL_) \
     (qkn ? launch_nt<NT_, SL_, true>(L, tw, tx, mp, grid) : launch_nt<NT_, SL_, false>(L, tw, tx, mp, grid))

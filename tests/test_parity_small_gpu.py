@@ -405,11 +405,14 @@ def test_many_anchor_blocks_over_one_cached_sequence():
         assert_close(out[b].float().cpu().numpy(), ref, cfg.dtype, f"block anchored at {a}")
 
 
-@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-def test_lmhead_argmax_building_block(dtype):
+@pytest.mark.parametrize("dtype,M", [("fp32", 70), ("bf16", 70), ("bf16", 136), ("bf16", 330), ("bf16", 512)])
+def test_lmhead_argmax_building_block(dtype, M):
+    # 70 rows: more than one logits staging chunk. 136 / 330 / 512 rows: token tiles of 160 / 192 / 256 columns, which
+    # run as CTA pairs (two CTAs per MMA); the vocabulary's odd number of 128-row tiles leaves the last pair half empty
     cfg = synth.TINY if dtype == "fp32" else synth.MID
+    if M == 330:
+        cfg = dataclasses.replace(cfg, vocab=4900)       # 39 tiles
     case = Case(cfg, (0,), seed=9)
-    M = 70                                   # more rows than one logits staging chunk
     hid = synth.normal((M, cfg.d_model), 1.0, 9, "lm.hidden", cfg.torch_dtype)
     dev = case.device
     ids = torch.zeros(M, dtype=torch.int32, device=dev)
