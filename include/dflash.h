@@ -469,6 +469,17 @@ int32_t dflash_trace_read(dflash_handle* h, int32_t* families /*[host] capacity 
  * clamped to it by the kernels and sets DFLASH_DEV_CTX_OVERFLOW. */
 int32_t dflash_attention_plan(const dflash_handle* h, int32_t batch, int32_t max_ctx_len, int64_t* out /*[host] [4]*/);
 
+/* How the chained contraction kernel splits one [M, K] x [N, K]^T product (n_groups weight matrices of N rows) over
+ * its CTAs, walked on the host with the kernel's own arithmetic (no CUDA work, no handle): sm_count CTAs at most,
+ * pair_cap = CTA pairs the device keeps resident (token tiles of 160+ columns run as pairs when >= 1; 74 on a B200),
+ * cluster_cap = 4-CTA clusters it keeps resident (token tiles of up to 32 columns; 33 on a B200). Returns 0 when
+ * every (tile, K chunk) is taken exactly once, no CTA holds more than two partial pieces (in different slots) and
+ * the contributors of every shared tile are the ones the finishing code looks for; a positive code names the first
+ * check that failed, -1 bad arguments. info (may be NULL): token tile width, pair form (0/1), grid size, CTAs per
+ * K-split cluster, tiles split across CTAs, K-split-cluster phase (0/1). The paper has no counterpart: a test aid. */
+int32_t dflash_gemm_plan_check(int32_t M, int32_t N, int32_t K, int32_t n_groups, int32_t sm_count, int32_t pair_cap,
+                               int32_t cluster_cap, int32_t* info /*[host] [6] or NULL*/);
+
 /* Static description of a return code. */
 const char* dflash_status_string(int32_t code);
 

@@ -29,7 +29,7 @@ EXPORTS = (
     "dflash_profile_read", "dflash_family_name", "dflash_trace_enable", "dflash_trace_read",
     "dflash_verify_accept_static", "dflash_sample_rows", "dflash_verify_accept_sample",
     "dflash_sample_workspace_bytes", "dflash_target_verify", "dflash_block_loss", "dflash_attention_plan",
-    "dflash_block_attention_bwd",
+    "dflash_block_attention_bwd", "dflash_gemm_plan_check",
 )
 N_FAMILIES = 15
 
@@ -164,6 +164,8 @@ def load():
     lib.dflash_sample_workspace_bytes.restype = C.c_int64
     lib.dflash_attention_plan.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
     lib.dflash_attention_plan.restype = C.c_int32
+    lib.dflash_gemm_plan_check.argtypes = [C.c_int32] * 7 + [C.POINTER(C.c_int32)]
+    lib.dflash_gemm_plan_check.restype = C.c_int32
     lib.dflash_status_string.argtypes = [C.c_int32]
     lib.dflash_status_string.restype = C.c_char_p
     lib.dflash_launch_count.argtypes = []

@@ -700,6 +700,11 @@ int32_t dflash_block_attention_bwd(dflash_handle* h, const dflash_attn_bwd_args*
     return DFLASH_OK;
 }
 
+int32_t dflash_gemm_plan_check(int32_t M, int32_t N, int32_t K, int32_t n_groups, int32_t sm_count, int32_t pair_cap,
+                               int32_t cluster_cap, int32_t* info) {
+    return dflash::gemm_plan_check(M, N, K, n_groups, sm_count, pair_cap, cluster_cap, info);
+}
+
 int32_t dflash_attention_plan(const dflash_handle* h, int32_t batch, int32_t max_ctx_len, int64_t* out) {
     if (!h || !out || batch < 1 || max_ctx_len < 0) return DFLASH_ERR_INVALID_ARG;
     const AttnPlan pl = attn_tc_plan(h->cfg, batch, max_ctx_len, h->sm_count);

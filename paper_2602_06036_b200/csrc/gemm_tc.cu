@@ -38,6 +38,8 @@
 #include <math_constants.h>
 
 #include <algorithm>
+#include <utility>
+#include <vector>
 
 namespace dflash {
 namespace {
@@ -132,7 +134,7 @@ struct Unit {
 };
 // CTA pairs: the walk hands out pairs of weight tiles; CTA `prank` of the pair takes tile 2 * pair + prank.
 template <bool PAIR>
-__device__ __forceinline__ void own_tile(const KParams& p, Unit& u, int prank) {
+__host__ __device__ __forceinline__ void own_tile(const KParams& p, Unit& u, int prank) {
     if constexpr (PAIR) {
         u.ft = u.ft * 2 + prank;
         u.phantom = u.ft >= p.n_ftiles_real ? 1 : 0;
@@ -150,7 +152,7 @@ __device__ __forceinline__ void own_tile(const KParams& p, Unit& u, int prank) {
 // Tiles are ordered token-tile fastest, so neighbouring CTAs share weight tiles through L2.
 // The shared part never leaves a CTA an empty range (every CTA between the first and the last
 // contributor of a tile publishes a piece): a remainder that small takes one more round of tiles with it.
-__device__ __forceinline__ int shared_tiles(const KParams& p, int n_ctas) {
+__host__ __device__ __forceinline__ int shared_tiles(const KParams& p, int n_ctas) {
     if (p.cluster_k) return 0;      // every tile is finished inside a cluster
     if (p.n_tiles < n_ctas) return p.n_tiles;
     const int r = p.n_tiles % n_ctas;
@@ -164,7 +166,7 @@ struct PieceWalk {
     int cl_c0, cl_c1;      // cluster mode: this CTA's chunk range of every tile its cluster takes (cl_c1 = 0: not cluster mode)
     // cs: CTAs per cluster. A cluster-mode phase gives its tiles to the clusters in turn; rank r of a cluster
     // streams chunks [r * C / cs, (r + 1) * C / cs) of each of its tiles.
-    __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas, int cs) {
+    __host__ __device__ __forceinline__ PieceWalk(const KParams& p, int cta, int n_ctas, int cs) {
         first = 1;
         n_shared = shared_tiles(p, n_ctas);
         const long long T = (long long)n_shared * p.chunks_total;
@@ -182,16 +184,16 @@ struct PieceWalk {
             dp_stride = n_ctas;
         }
     }
-    __device__ __forceinline__ bool shared_done() const { return cur >= hi; }
-    __device__ __forceinline__ bool done(const KParams& p) const { return cur >= hi && dp_next >= p.n_tiles; }
-    __device__ __forceinline__ Unit next(const KParams& p) {
+    __host__ __device__ __forceinline__ bool shared_done() const { return cur >= hi; }
+    __host__ __device__ __forceinline__ bool done(const KParams& p) const { return cur >= hi && dp_next >= p.n_tiles; }
+    __host__ __device__ __forceinline__ Unit next(const KParams& p) {
         Unit u;
         u.cl = 0;
         if (cur < hi) {
             u.tile = (int)(cur / p.chunks_total);
             u.c0 = (int)(cur % p.chunks_total);
             const long long left = hi - cur;
-            u.c1 = (int)min((long long)p.chunks_total, u.c0 + left);
+            u.c1 = (u.c0 + left < (long long)p.chunks_total) ? (int)(u.c0 + left) : p.chunks_total;
             u.full = (u.c0 == 0 && u.c1 == p.chunks_total) ? 1 : 0;
             u.slot = first ? 0 : 1;
             cur += u.c1 - u.c0;
@@ -216,7 +218,7 @@ struct PieceWalk {
     }
 };
 // CTA that owns pair number x of the shared part (T pairs):  largest j with floor(j*T/G) <= x
-__device__ __forceinline__ int cta_of_pair(long long x, long long T, int G) { return (int)(((x + 1) * G + T - 1) / T - 1); }
+__host__ __device__ __forceinline__ int cta_of_pair(long long x, long long T, int G) { return (int)(((x + 1) * G + T - 1) / T - 1); }
 
 // ---------------------------------------------------------------------------------------------
 // epilogues: 128 threads, thread `row` owns feature f0 + row; sAcc[row][c] holds 16 token columns
@@ -1576,6 +1578,92 @@ int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int
         default: return DFLASH_GEMM_CASE(256, 1);
     }
 #undef DFLASH_GEMM_CASE
+}
+
+// The work split of one phase, walked on the host exactly as the kernel's roles walk it (the same PieceWalk code):
+// every (tile, chunk) of the matrix covered once, at most two partial pieces per walker in different slots, the
+// contributors of a shared tile and their slots as the finishing code derives them. 0 = consistent.
+int gemm_plan_check(int M, int N, int K, int n_groups, int sm_count, int pair_cap, int cluster_cap, int32_t* info) {
+    if (M <= 0 || N <= 0 || K <= 0 || sm_count <= 0) return -1;
+    const int groups = std::max(n_groups, 1);
+    const int nt = pick_nt(M);
+    const int slabs = slabs_for(nt, K % BK == 0);
+    pair_cap = std::min(pair_cap, sm_count / 2);
+    const bool pair = nt >= 160 && sm_count >= 2 && pair_cap >= 1;
+    KParams p{};
+    p.M = M; p.N = N; p.K = K; p.n_groups = groups;
+    p.n_ftiles_real = (N + TILE_F - 1) / TILE_F;
+    p.n_ftiles = pair ? (p.n_ftiles_real + 1) / 2 : p.n_ftiles_real;
+    p.n_ttiles = (M + nt - 1) / nt;
+    p.chunks_total = (K + BK * slabs - 1) / (BK * slabs);
+    p.n_tiles = groups * p.n_ftiles * p.n_ttiles;
+    const long long pairs_tc = (long long)p.n_tiles * p.chunks_total;
+    int grid, cs = 1, walkers;
+    if (pair) {
+        walkers = (int)std::max<long long>(1, std::min<long long>(pair_cap, pairs_tc / 4));
+        grid = 2 * walkers;
+    } else {
+        grid = (int)std::max<long long>(1, std::min<long long>(sm_count, pairs_tc * slabs / 4));
+        if (nt <= 32 && grid >= CS) {
+            int cap = std::min(cluster_cap, MAX_CLUSTERS);      // as cluster_capacity() reports it
+            if (cap < MIN_CLUSTERS) cap = 0;
+            const int n_cl = std::min(cap, grid / CS);
+            if (n_cl >= 1) { cs = CS; grid = n_cl * CS; }
+        }
+        p.cluster_k = (cs > 1 && p.n_tiles < grid && p.chunks_total >= CS) ? 1 : 0;
+        walkers = grid;
+    }
+    if (info) { info[0] = nt; info[1] = pair ? 1 : 0; info[2] = grid; info[3] = cs; info[4] = shared_tiles(p, walkers); info[5] = p.cluster_k; }
+    const int real_tiles = groups * p.n_ftiles_real * p.n_ttiles;
+    std::vector<uint8_t> cover((size_t)real_tiles * p.chunks_total, 0);
+    const int n_shared = shared_tiles(p, walkers);
+    const long long T = (long long)n_shared * p.chunks_total;
+    std::vector<std::vector<std::pair<int, int>>> contrib((size_t)std::max(n_shared, 0));
+    for (int w = 0; w < walkers; ++w) {
+        for (int prank = 0; prank < (pair ? 2 : 1); ++prank) {
+            int n_partial = 0, slot_mask = 0;
+            for (PieceWalk pw(p, w, walkers, cs); !pw.done(p);) {
+                Unit u = pw.next(p);
+                if (pair) own_tile<true>(p, u, prank);
+                if (u.c0 < 0 || u.c1 > p.chunks_total || u.c0 >= u.c1) return 1;
+                if (u.full && u.tile < n_shared && prank == 0) contrib[(size_t)u.tile].push_back({w, -1});   // whole tile, one walker
+                if (!u.full && !u.cl) {
+                    if (u.tile >= n_shared) return 2;
+                    ++n_partial;
+                    if (slot_mask & (1 << u.slot)) return 3;            // two pieces of one CTA in the same partial slot
+                    slot_mask |= 1 << u.slot;
+                    if (prank == 0) contrib[(size_t)u.tile].push_back({w, u.slot});
+                }
+                if (u.phantom) continue;
+                if (u.ft >= p.n_ftiles_real || u.tt >= p.n_ttiles || u.g >= groups) return 4;
+                if (u.ctr != (u.g * p.n_ftiles_real + u.ft) * p.n_ttiles + u.tt) return 5;
+                for (int c = u.c0; c < u.c1; ++c) {
+                    uint8_t& k = cover[(size_t)u.ctr * p.chunks_total + c];
+                    if (k) return 6;                                    // a chunk of a tile handed out twice
+                    k = 1;
+                }
+            }
+            if (n_partial > 2) return 7;
+        }
+    }
+    for (uint8_t k : cover)
+        if (!k) return 8;                                               // a chunk nobody takes
+    for (int t = 0; t < n_shared; ++t) {
+        const long long x0 = (long long)t * p.chunks_total;
+        const int j0 = cta_of_pair(x0, T, walkers), j1 = cta_of_pair(x0 + p.chunks_total - 1, T, walkers);
+        const auto& cv = contrib[(size_t)t];
+        if ((int)cv.size() != j1 - j0 + 1) return 9;                    // the finishing code expects other contributors
+        if (cv.size() == 1 && cv[0].second == -1) {                     // a whole tile inside one walker's range: no exchange
+            if (cv[0].first != j0) return 12;
+            continue;
+        }
+        for (int j = j0; j <= j1; ++j) {
+            if (cv[(size_t)(j - j0)].first != j) return 10;
+            const int sa = ((long long)j * T / walkers >= x0) ? 0 : 1;
+            if (cv[(size_t)(j - j0)].second != sa) return 11;           // ... or looks for a piece in the other slot
+        }
+    }
+    return 0;
 }
 
 int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done) {

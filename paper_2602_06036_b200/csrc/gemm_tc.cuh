@@ -74,6 +74,8 @@ int64_t gemm_tc_counter_bytes(int M, int N, int n_groups);
 // them non-zero: one launch per zeroing).
 constexpr int GEMM_MAX_PHASES = 4;
 int launch_gemm_tc(const Launch& L, const GemmArgs& a, int32_t* phase_done);
+// Host-only consistency check of the work split of one contraction (see dflash_gemm_plan_check in dflash.h).
+int gemm_plan_check(int M, int N, int K, int n_groups, int sm_count, int pair_cap, int cluster_cap, int32_t* info);
 // A chain of contractions in ONE launch: phase i+1 may read what phase i's epilogues wrote. The
 // phases share the token-tile size (chosen for the largest row count) but not the row count. traces[i] (may be nullptr) = timeline record of phase i.
 int launch_gemm_chain(const Launch& L, const GemmArgs* phases, int n_phases, int32_t* phase_done,

@@ -176,6 +176,31 @@ def test_attention_split_never_outgrows_its_partials_buffer(lib):
     lib.dflash_destroy(h)
 
 
+def test_contraction_work_split_covers_every_chunk_once(lib):
+    # host arithmetic only, the kernel's own walk: every (weight tile, K chunk) is taken by exactly one CTA, no CTA
+    # holds more than two partial pieces, and the finishing code's idea of who contributed to a shared tile (and in
+    # which partial slot) is what the walk produced - for the three forms of the launch (K-split clusters with up to
+    # 32 token columns, plain CTAs, CTA pairs from 160 columns on) and for tile counts that are odd, ragged or tiny
+    shapes = [(4096, 4096, 1), (6144, 4096, 1), (24576, 4096, 1), (4096, 12288, 1), (151936, 4096, 1), (4096, 20480, 1),
+              (2048, 4096, 5), (1536, 512, 1), (5003, 512, 1), (4900, 512, 1), (512, 1536, 1), (128, 64, 1), (100, 200, 1),
+              (129, 72, 2), (768, 256, 1)]
+    rows = [1, 8, 16, 17, 32, 33, 64, 100, 128, 129, 136, 160, 161, 200, 256, 330, 512, 544, 1000]
+    info = (C.c_int32 * 6)()
+    forms = set()
+    for N, K, groups in shapes:
+        for M in rows:
+            for sms, pair_cap, cluster_cap in ((148, 74, 33), (148, 0, 0), (132, 66, 20), (64, 3, 16), (7, 1, 1), (1, 0, 0)):
+                rc = lib.dflash_gemm_plan_check(M, N, K, groups, sms, pair_cap, cluster_cap, info)
+                assert rc == 0, (rc, M, N, K, groups, sms, pair_cap, cluster_cap, list(info))
+                nt, pair, grid, cs = info[0], info[1], info[2], info[3]
+                assert nt >= min(M, 256) or M > 256
+                assert grid <= sms and (not pair or (grid % 2 == 0 and nt >= 160)) and (cs == 1 or (nt <= 32 and grid % cs == 0))
+                forms.add((bool(pair), cs > 1, info[5] == 1))
+    assert (True, False, False) in forms and (False, True, True) in forms and (False, True, False) in forms \
+        and (False, False, False) in forms
+    assert lib.dflash_gemm_plan_check(0, 128, 64, 1, 148, 74, 33, info) == -1
+
+
 def test_workspace_grows_with_the_row_count(lib):
     # a workspace sized for R rows must serve every call with fewer rows (a draft of 512 rows inside a workspace
     # sized for the 544 rows of the projection that rides along): sizes never shrink as rows grow
