@@ -96,13 +96,15 @@ def test_block_size_chosen_per_call(name):
 
 
 @pytest.mark.parametrize("base,over", [("tiny", {}), ("mid", {}), ("mid", dict(head_dim=64, n_q_heads=8, n_kv_heads=2)),
-                                       ("mid", dict(block_size=10, n_layers=3))])
+                                       ("mid", dict(block_size=10, n_layers=3)), ("mid12", {})])
 def test_per_head_qk_norm(base, over):
     # the optional attention variant: q and k heads RMS-normalised (own gains) before the rotation, for
     # block rows and for the injected context keys; CUDA-core path (tiny), tensor-core path with one head
-    # per 128-row weight tile (hd = 128) and with two (hd = 64)
+    # per 128-row weight tile (hd = 128) and with two (hd = 64); 12 sequences: 192 block rows, the contraction
+    # kernel's CTA-pair form with the head norms in its epilogues
     cfg = dataclasses.replace(synth.TINY if base == "tiny" else synth.MID, qk_norm=1, **over)
-    case = Case(cfg, (0, 70, 131) if base == "mid" else (65,), seed=23)
+    lens = {"tiny": (65,), "mid": (0, 70, 131), "mid12": (0, 70, 131, 5, 64, 65, 200, 17, 33, 128, 90, 1)}[base]
+    case = Case(cfg, lens, seed=23)
     case.project_prefill()
     _check_pool(case)
     got = case.run_draft()
