@@ -613,6 +613,8 @@ def measure(step, args, peaks, dist_on, rank, sampler=None, repeats=7, e2e_repea
     alg = algorithmic_bytes(cfg, wl.ctx_lens, step.rows_new)
     hbm = peaks["hbm_gbs"]
     es = 4 if cfg.dtype == "fp32" else 2
+    if not step.full_verify:      # greedy verify from the target's logits: one launch, every logit read once
+        alg["row_argmax"] = step.d_logits.numel() * step.d_logits.element_size()
     # device-side timeline of one extra eager step; the verify side of the serving-mix step runs on a second
     # handle (the target-shaped layer) and on the LM head of this one: traced separately and prefixed
     if step.full_verify:

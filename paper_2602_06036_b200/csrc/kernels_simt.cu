@@ -738,12 +738,15 @@ __global__ void __launch_bounds__(256) verify_fused_kernel(const T* __restrict__
                                                            float4* seg_out, const int32_t* __restrict__ draft_ids, int draft_stride,
                                                            int gamma, const int32_t* ctx_len, int32_t* __restrict__ accept_len,
                                                            int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus,
-                                                           int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out) {
+                                                           int32_t* new_ctx_len, int32_t* __restrict__ target_ids_out,
+                                                           unsigned long long* trace) {
     __shared__ Top2 sh[8];
     __shared__ int32_t s_p[65];
     __shared__ int s_last;
+    if (threadIdx.x == 0) ptx::trace_min(trace, 0);
     ptx::pdl_trigger();
     ptx::pdl_wait();
+    if (threadIdx.x == 0) ptx::trace_min(trace, 1);
     const int seg = blockIdx.x, nseg = gridDim.x, row = blockIdx.y;
     const int b = row / (gamma + 1);
     const int lo = seg * seg_len, hi = min(vocab, lo + seg_len);
@@ -755,10 +758,15 @@ __global__ void __launch_bounds__(256) verify_fused_kernel(const T* __restrict__
         s_last = atomicInc(&g_verify_tickets[b], n - 1) == n - 1 ? 1 : 0;
     }
     __syncthreads();
-    if (!s_last) return;
+    if (!s_last) {
+        if (threadIdx.x == 0) ptx::trace_max(trace, 3);
+        return;
+    }
     __threadfence();      // the other CTAs' segment results are visible
     merge_and_accept(seg_out, nseg, b, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus, new_ctx_len,
                      target_ids_out, s_p);
+    __syncthreads();
+    if (threadIdx.x == 0) ptx::trace_max(trace, 3);
 }
 
 int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t row_stride, float4* seg_scratch) {
@@ -773,11 +781,11 @@ int launch_verify_logits(const Launch& L, const dflash_verify_args& a, int64_t r
         if (a.logits_dtype == DFLASH_F32)
             e = launch_pdl(verify_fused_kernel<float>, grid, dim3(256), 0, L.st, (const float*)a.logits, row_stride, a.vocab, seg_len,
                            seg_scratch, a.draft_ids, a.draft_stride, a.gamma, a.ctx_len, a.accept_len, a.out_tokens, a.bonus,
-                           a.new_ctx_len, a.target_ids_out);
+                           a.new_ctx_len, a.target_ids_out, L.trace);
         else
             e = launch_pdl(verify_fused_kernel<__nv_bfloat16>, grid, dim3(256), 0, L.st, (const __nv_bfloat16*)a.logits, row_stride,
                            a.vocab, seg_len, seg_scratch, a.draft_ids, a.draft_stride, a.gamma, a.ctx_len, a.accept_len, a.out_tokens,
-                           a.bonus, a.new_ctx_len, a.target_ids_out);
+                           a.bonus, a.new_ctx_len, a.target_ids_out, L.trace);
         ++g_launches;
         return e == cudaSuccess ? DFLASH_OK : DFLASH_ERR_CUDA;
     }
