@@ -678,10 +678,28 @@ __device__ __forceinline__ void merge_and_accept(const float4* seg, int nseg, in
                                                  int32_t* __restrict__ out_tokens, int32_t* __restrict__ bonus, int32_t* new_ctx_len,
                                                  int32_t* __restrict__ target_ids_out, int32_t* s_p) {
     const int lane = threadIdx.x & 31;
-    for (int j = threadIdx.x >> 5; j <= gamma; j += blockDim.x >> 5) {
+    const int n_warps = blockDim.x >> 5;
+    // A warp takes rows w, w + n_warps, ...: the entries of up to RB of its rows are requested together (one round
+    // trip through L2 instead of one per row; up to 64 segments per row = two entries per lane).
+    constexpr int RB = 3;
+    for (int j0 = threadIdx.x >> 5; j0 <= gamma; j0 += RB * n_warps) {
+        float4 e0[RB], e1[RB];
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+            const int j = j0 + u * n_warps;
+            const size_t row = (size_t)b * (gamma + 1) + j;
+            const float4 none = make_float4(-CUDART_INF_F, __int_as_float(0x7fffffff), -CUDART_INF_F, 0.f);
+            e0[u] = (j <= gamma && lane < nseg) ? __ldcg(seg + row * nseg + lane) : none;
+            e1[u] = (j <= gamma && lane + 32 < nseg) ? __ldcg(seg + row * nseg + lane + 32) : none;
+        }
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+        const int j = j0 + u * n_warps;
+        if (j > gamma) break;
         const size_t row = (size_t)b * (gamma + 1) + j;
-        Top2 t{-CUDART_INF_F, 0x7fffffff, -CUDART_INF_F};
-        for (int i = lane; i < nseg; i += 32) {
+        Top2 t{e0[u].x, __float_as_int(e0[u].y), e0[u].z};
+        t = top2_merge(t, Top2{e1[u].x, __float_as_int(e1[u].y), e1[u].z});
+        for (int i = lane + 64; i < nseg; i += 32) {      // (never with the segment counts the launches choose)
             const float4 e = __ldcg(seg + row * nseg + i);
             t = top2_merge(t, Top2{e.x, __float_as_int(e.y), e.z});
         }
@@ -697,6 +715,7 @@ __device__ __forceinline__ void merge_and_accept(const float4* seg, int nseg, in
             const int32_t id = (t.i1 == 0x7fffffff) ? 0 : t.i1;      // nothing compared greater than -inf
             s_p[j] = id;
             if (target_ids_out) target_ids_out[row] = id;
+        }
         }
     }
     __syncthreads();
@@ -753,16 +772,18 @@ __global__ void __launch_bounds__(256) verify_fused_kernel(const T* __restrict__
     const Top2 r = scan_segment<T, false>(logits + (size_t)row * row_stride, lo, hi, sh);
     if (threadIdx.x == 0) {
         seg_out[(size_t)row * nseg + seg] = make_float4(r.v1, __int_as_float(r.i1), r.v2, 0.f);
-        __threadfence();
+        // one ticket with release (this CTA's result) and acquire (the results of the CTAs before it) semantics; the
+        // barrier below hands what thread 0 acquired to the rest of the CTA
         const unsigned int n = (unsigned int)nseg * (unsigned int)(gamma + 1);
-        s_last = atomicInc(&g_verify_tickets[b], n - 1) == n - 1 ? 1 : 0;
+        unsigned int old;
+        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(&g_verify_tickets[b]), "r"(n - 1) : "memory");
+        s_last = old == n - 1 ? 1 : 0;
     }
     __syncthreads();
     if (!s_last) {
         if (threadIdx.x == 0) ptx::trace_max(trace, 3);
         return;
     }
-    __threadfence();      // the other CTAs' segment results are visible
     merge_and_accept(seg_out, nseg, b, draft_ids, draft_stride, gamma, ctx_len, accept_len, out_tokens, bonus, new_ctx_len,
                      target_ids_out, s_p);
     __syncthreads();
