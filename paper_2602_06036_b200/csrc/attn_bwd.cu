@@ -107,6 +107,18 @@ __device__ __forceinline__ void load_q_do(uint8_t* sQ, uint8_t* sDO, const CUten
         }
 }
 
+// Q and dO of TWO blocks: rows 0..63 of the operand tiles hold block A's 64 rows, rows 64..127 block B's
+__device__ __forceinline__ void load_q_do_pair(uint8_t* sQ, uint8_t* sDO, const CUtensorMap* tmQ, const CUtensorMap* tmDO, int g, int rowA,
+                                               int rowB, uint64_t* bar, uint64_t pol) {
+    mbar_expect_tx(bar, 2 * QD_BYTES);
+    for (int hf = 0; hf < 2; ++hf)
+        for (int cp = 0; cp < 2; ++cp) {
+            const int row0 = cp ? rowB : rowA;
+            tma_load_4d(sQ + hf * (QD_BYTES / 2) + cp * (QD_BYTES / 4), tmQ, hf * 64, 0, g, row0, bar, pol);
+            tma_load_4d(sDO + hf * (QD_BYTES / 2) + cp * (QD_BYTES / 4), tmDO, hf * 64, 0, g, row0, bar, pol);
+        }
+}
+
 // S = Q K^T and dP = dO V^T of one 64-key tile (16 instructions)
 __device__ __forceinline__ void issue_s_dp(uint32_t tmem_base, uint32_t q_addr, uint32_t do_addr, uint32_t k_addr, uint32_t v_addr) {
     // tmem_base already includes the S / dP buffer's first column
@@ -169,6 +181,41 @@ __device__ __forceinline__ void row_math(uint32_t tmem_row, uint8_t* sP, uint8_t
         const int off = ((h * 4 + ck) ^ (qrow & 7)) << 4;
         *reinterpret_cast<uint4*>(prow + off) = w4;
         *reinterpret_cast<uint4*>(drow + off) = d4;
+    }
+}
+// Row arithmetic of one tile when the 128 operand rows are 64 query rows of each of TWO blocks (the context-gradient
+// kernel): the thread of lane l owns operand row l - all 64 keys of the tile - and writes row l of P and dS.
+__device__ __forceinline__ void row_math_full(uint32_t tmem_row, uint8_t* sP, uint8_t* sDS, int row, int vis, float lse2, float Dr,
+                                              float scale, float scale_log2) {
+    uint8_t* prow = sP + row * 128;
+    uint8_t* drow = sDS + row * 128;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        float s[32], dp[32];
+        tmem_ld32(tmem_row + COL_S + h * 32, s);
+        tmem_ld32(tmem_row + COL_DP + h * 32, dp);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const bool on = h * 32 + c < vis;
+            const float p = on ? fast_exp2(fmaf(s[c], scale_log2, -lse2)) : 0.f;
+            s[c] = p;
+            dp[c] = on ? p * (dp[c] - Dr) * scale : 0.f;
+        }
+#pragma unroll
+        for (int ck = 0; ck < 4; ++ck) {
+            uint4 w4, d4;
+            w4.x = pack_bf16(s[ck * 8 + 0], s[ck * 8 + 1]);
+            w4.y = pack_bf16(s[ck * 8 + 2], s[ck * 8 + 3]);
+            w4.z = pack_bf16(s[ck * 8 + 4], s[ck * 8 + 5]);
+            w4.w = pack_bf16(s[ck * 8 + 6], s[ck * 8 + 7]);
+            d4.x = pack_bf16(dp[ck * 8 + 0], dp[ck * 8 + 1]);
+            d4.y = pack_bf16(dp[ck * 8 + 2], dp[ck * 8 + 3]);
+            d4.z = pack_bf16(dp[ck * 8 + 4], dp[ck * 8 + 5]);
+            d4.w = pack_bf16(dp[ck * 8 + 6], dp[ck * 8 + 7]);
+            const int off = ((h * 4 + ck) ^ (row & 7)) << 4;
+            *reinterpret_cast<uint4*>(prow + off) = w4;
+            *reinterpret_cast<uint4*>(drow + off) = d4;
+        }
     }
 }
 // rows 64..127 of both P / dS buffer pairs := 0 (128 threads; visible to the tensor core after the first
@@ -422,7 +469,10 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// dK_ctx, dV_ctx: one CTA per (context tile, kv head, page-table row); the blocks that see the tile in batch order
+// dK_ctx, dV_ctx: one CTA per (context tile, kv head, page-table row); the blocks that see the tile in batch order,
+// TWO per step: the 128 operand rows are the 64 query rows of two consecutive contributing blocks, so a step's
+// contractions over the operand rows add both blocks' terms (half the steps, no duplicated rows; the order of the
+// sums is still fixed by the batch order). An odd block out rides with rows that see no key.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(N_THREADS, 1)
 attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
@@ -476,7 +526,8 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         any = false;
     }
 
-    int n_done = 0;      // contributing blocks processed (uniform over the CTA)
+    const int n_steps = (n_contrib + 1) / 2;      // two contributing blocks per step
+    int n_done = 0;      // steps processed (uniform over the CTA)
     bool ok = true;
     if (any) {
         if (warp == 4) {
@@ -489,14 +540,16 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tma_load_2d(sKV + KV_TILE_BYTES / 2, &tmPool, 64, rowK, kv_full, pol_kv);
                 tma_load_2d(sKV + KV_TILE_BYTES, &tmPool, 0, rowV, kv_full, pol_kv);
                 tma_load_2d(sKV + KV_TILE_BYTES + KV_TILE_BYTES / 2, &tmPool, 64, rowV, kv_full, pol_kv);
-                int k = 0;
-                for (int b = b_lo; b < b_hi && ok; ++b) {
-                    if (!sees(b)) continue;
+                int b = b_lo;
+                for (int k = 0; k < n_steps && ok; ++k) {
+                    while (!sees(b)) ++b;
+                    const int bA = b++;
+                    while (b < b_hi && !sees(b)) ++b;
+                    const int bB = b < b_hi ? b++ : bA;      // odd block out: its partner's rows see no key
                     const int st = k & 1;
                     if (k >= 2 && !mbar_wait(&qd_empty[st], ((k >> 1) - 1) & 1, &flags[0])) { ok = false; break; }
-                    load_q_do(sQD + (size_t)st * 2 * QD_BYTES, sQD + (size_t)st * 2 * QD_BYTES + QD_BYTES, &tmQ, &tmDO, g, b * p.R,
-                              &qd_full[st], pol_q);
-                    ++k;
+                    load_q_do_pair(sQD + (size_t)st * 2 * QD_BYTES, sQD + (size_t)st * 2 * QD_BYTES + QD_BYTES, &tmQ, &tmDO, g, bA * p.R,
+                                   bB * p.R, &qd_full[st], pol_q);
                 }
                 if (!ok) {
                     flags[0] = 1;
@@ -505,10 +558,10 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             __syncwarp();
         } else if (warp == 5) {
-            if (lane == 0) {      // scores of the k-th contributing block into buffer k & 1
+            if (lane == 0) {      // scores of the k-th pair of contributing blocks into buffer k & 1
                 const uint32_t k_addr = smem_u32(sKV), v_addr = k_addr + KV_TILE_BYTES;
                 ok = mbar_wait(kv_full, 0, &flags[0]);
-                for (int k = 0; k < n_contrib && ok; ++k) {
+                for (int k = 0; k < n_steps && ok; ++k) {
                     const int st = k & 1;
                     if (!mbar_wait(&qd_full[st], (k >> 1) & 1, &flags[0])) { ok = false; break; }
                     if (k >= 2 && !mbar_wait(&ds_full[st], ((k - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
@@ -524,8 +577,8 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             __syncwarp();
         } else if (warp == 6) {
-            if (lane == 0) {      // accumulating products of the k-th contributing block
-                for (int k = 0; k < n_contrib && ok; ++k) {
+            if (lane == 0) {      // accumulating products of the k-th pair of contributing blocks
+                for (int k = 0; k < n_steps && ok; ++k) {
                     const int st = k & 1;
                     if (!mbar_wait(&ds_full[st], (k >> 1) & 1, &flags[0])) { ok = false; break; }
                     tc_fence_after();
@@ -547,21 +600,27 @@ attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const int lrow = row & 63;
             const bool real = lrow < p.rows_valid;
             const int r = real ? lrow / p.group : 0, j = real ? lrow % p.group : 0;
-            zero_upper_rows(sPS, row);
-            for (int b = b_lo; b < b_hi; ++b) {
-                const int Lb = min(max(__ldg(p.ctx_len + b), 0), p.max_ctx_len);
-                if (Lb <= key0) continue;
-                const int i = n_done++;
-                const size_t qrow = ((size_t)b * p.R + r) * p.Hq + g * p.group + j;
-                const float Dr = real ? __ldcg(p.D + qrow) : 0.f;
-                const float lse2 = real ? __ldg(p.lse + qrow) * LOG2E : 0.f;
-                const int vis = real ? min(PG, Lb - key0) : 0;
+            int bn = b_lo;
+            for (int i = 0; i < n_steps; ++i) {
+                while (!sees(bn)) ++bn;
+                const int bA = bn++;
+                while (bn < b_hi && !sees(bn)) ++bn;
+                const int bB = bn < b_hi ? bn++ : -1;
+                n_done = i + 1;
+                // operand rows 0..63: block A, rows 64..127: block B (none: rows that see nothing)
+                const int b = row < 64 ? bA : bB;
+                const bool on = real && b >= 0;
+                const int Lb = on ? min(max(__ldg(p.ctx_len + b), 0), p.max_ctx_len) : 0;
+                const size_t qrow = on ? ((size_t)b * p.R + r) * p.Hq + g * p.group + j : 0;
+                const float Dr = on ? __ldcg(p.D + qrow) : 0.f;
+                const float lse2 = on ? __ldg(p.lse + qrow) * LOG2E : 0.f;
+                const int vis = on ? min(PG, Lb - key0) : 0;
                 const int buf = i & 1;
                 if (!mbar_wait(&s_full[buf], (i >> 1) & 1, &flags[0])) { ok = false; break; }
                 tc_fence_after();
                 if (i >= 2 && !mbar_wait(&acc_done[buf], ((i - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
                 uint8_t* sP = sPS + (size_t)buf * 2 * PS_BYTES;
-                row_math(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
+                row_math_full(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
                 tc_fence_before();
                 fence_proxy_async();
                 __syncwarp();
