@@ -478,7 +478,9 @@ __global__ void __launch_bounds__(N_THREADS, 1)
 attn_bwd_kv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                    const __grid_constant__ CUtensorMap tmPool, const BParams p) {
     pdl_trigger();
-    const int t = blockIdx.x, g = blockIdx.y, owner = blockIdx.z;
+    // kv head fastest, key tile next: CTAs reach the SMs in index order, and a tile is seen by at least as many blocks
+    // as every later one, so the longest CTAs (the first tiles, seen by every block) all start first
+    const int g = blockIdx.x, t = blockIdx.y, owner = blockIdx.z;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sKV = smem;                                  // K tile, V tile
@@ -732,7 +734,7 @@ int launch_attention_bwd(const Launch& L, const dflash_attn_bwd_args& a, float* 
     ++g_launches;
     const int n_ctx_tiles = (a.max_ctx_len + PG - 1) / PG;
     if (n_ctx_tiles > 0 && a.dkv_ctx) {
-        const dim3 grid(n_ctx_tiles, p.Hkv, p.shared_row ? 1 : a.batch);
+        const dim3 grid(p.Hkv, n_ctx_tiles, p.shared_row ? 1 : a.batch);
         if (launch_pdl(attn_bwd_kv_kernel, grid, dim3(N_THREADS), (size_t)SMEM_KV, L.st, tq, tdo, tpool, p) != cudaSuccess)
             return DFLASH_ERR_CUDA;
         ++g_launches;
