@@ -52,6 +52,7 @@ struct BParams {
     const __nv_bfloat16* dout;
     const float* lse;              // forward log-sum-exp (natural log)
     float* D;                      // [S, R, Hq] rowsum(dO * O): written by the first kernel, read by the second
+    const int32_t* order;          // [S] blocks by falling context length (ties by index): written by order_kernel
     __nv_bfloat16 *dq, *dk_blk, *dv_blk;
     float* dkv_ctx;                // [page][K|V][kv head][slot][hd] fp32 of the layer
     int32_t* status;
@@ -227,6 +228,30 @@ __device__ __forceinline__ void zero_upper_rows(uint8_t* sPS, int tid) {
     }
 }
 
+// Blocks by falling context length, ties by index (every thread ranks some blocks against all others; one CTA).
+// The first kernel takes its blocks in this order: the longest first, and - two blocks per CTA - neighbours of
+// similar length together.
+// More than ORDER_MAX blocks (the ranking is quadratic): index order.
+constexpr int ORDER_MAX = 4096;
+__global__ void __launch_bounds__(1024) order_kernel(const int32_t* __restrict__ ctx_len, int S, int32_t* __restrict__ order) {
+    extern __shared__ int32_t s_len[];
+    if (S > ORDER_MAX) {
+        for (int i = threadIdx.x; i < S; i += blockDim.x) order[i] = i;
+        return;
+    }
+    for (int i = threadIdx.x; i < S; i += blockDim.x) s_len[i] = ctx_len[i];
+    __syncthreads();
+    for (int t = threadIdx.x; t < S; t += blockDim.x) {
+        const int mine = s_len[t];
+        int rank = 0;
+        for (int j = 0; j < S; ++j) {
+            const int l = s_len[j];
+            rank += (l > mine || (l == mine && j < t)) ? 1 : 0;
+        }
+        order[rank] = t;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------------------
 // dQ, dK_blk, dV_blk: one CTA per (kv head, block)
 // ------------------------------------------------------------------------------------------------------------
@@ -235,7 +260,15 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                   const __grid_constant__ CUtensorMap tmPool, const __grid_constant__ CUtensorMap tmKb,
                   const __grid_constant__ CUtensorMap tmVb, const BParams p) {
     pdl_trigger();
-    const int g = blockIdx.x, b = blockIdx.y;
+    // Blocks are taken by falling context length (p.order). Blocks that share one page-table row (the training layout)
+    // go TWO per CTA: operand rows 0..63 are block A's query rows, rows 64..127 block B's; both walk the same key
+    // tiles (a row past its own context sees no key) and each block's own keys take a tile of their own. Otherwise
+    // one block per CTA, its rows loaded twice.
+    const int g = blockIdx.x;
+    const bool two = p.shared_row != 0;
+    const int ia0 = two ? 2 * (int)blockIdx.y : (int)blockIdx.y;
+    const int b = p.order[ia0];                                              // block A
+    const int bB = (two && ia0 + 1 < p.S) ? p.order[ia0 + 1] : -1;           // block B (or none)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;
@@ -249,12 +282,14 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint64_t* s_full = kv_empty + KV_STAGES;       // [2] S / dP buffer written by the tensor core
     uint64_t* ds_full = s_full + 2;                // [2] P / dS buffer written by the row threads (and S / dP buffer read)
     uint64_t* acc_done = ds_full + 2;              // [2] the products that read P / dS buffer are complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 2);
+    uint64_t* blk_read = acc_done + 2;             // [1] block A's own-key gradients have been read out of TMEM
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(blk_read + 1);
     volatile int* flags = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
+        mbar_init(blk_read, 4);
         for (int s = 0; s < KV_STAGES; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&ds_full[s], 4); mbar_init(&acc_done[s], 1); }
         flags[0] = 0;
@@ -268,11 +303,13 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();
 
-    const int L_given = p.ctx_len[b];
-    const int L = min(max(L_given, 0), p.max_ctx_len);
-    if (L_given > p.max_ctx_len && threadIdx.x == 0 && g == 0 && p.status) atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
+    const int LA_given = p.ctx_len[b], LB_given = bB >= 0 ? p.ctx_len[bB] : 0;
+    const int LA = min(max(LA_given, 0), p.max_ctx_len), LB = min(max(LB_given, 0), p.max_ctx_len);
+    if ((LA_given > p.max_ctx_len || LB_given > p.max_ctx_len) && threadIdx.x == 0 && g == 0 && p.status)
+        atomicOr(p.status, DFLASH_DEV_CTX_OVERFLOW);
+    const int L = max(LA, LB);                           // keys the CTA walks
     const int n_ctx_tiles = (L + PG - 1) / PG;
-    const int n_tiles = n_ctx_tiles + 1;
+    const int n_tiles = n_ctx_tiles + 1 + (bB >= 0 ? 1 : 0);      // + block A's own keys (+ block B's)
 
     // Three single-thread roles, each with its own chain of waits, so that a copy in flight never holds up a
     // contraction whose operands are ready: copies (warp 4), S / dP of the next tile (warp 5), the accumulating
@@ -281,7 +318,8 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (lane == 0) {
             const uint64_t pol_kv = policy_evict_last(), pol_q = policy_evict_first();
             bool ok = true;
-            load_q_do(sQ, sDO, &tmQ, &tmDO, g, b * p.R, q_full, pol_q);
+            if (two) load_q_do_pair(sQ, sDO, &tmQ, &tmDO, g, b * p.R, (bB >= 0 ? bB : b) * p.R, q_full, pol_q);
+            else load_q_do(sQ, sDO, &tmQ, &tmDO, g, b * p.R, q_full, pol_q);
             for (int i = 0; i < n_tiles && ok; ++i) {
                 const int st = i % KV_STAGES;
                 // the stage held tile i - KV_STAGES: wait for that tile's products
@@ -302,10 +340,11 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     tma_load_2d(dV, &tmPool, 0, rowV, &kv_full[st], pol_kv);
                     tma_load_2d(dV + KV_TILE_BYTES / 2, &tmPool, 64, rowV, &kv_full[st], pol_kv);
                 } else {
-                    tma_load_2d(dK, &tmKb, g * HD, b * p.R, &kv_full[st], pol_q);
-                    tma_load_2d(dK + KV_TILE_BYTES / 2, &tmKb, g * HD + 64, b * p.R, &kv_full[st], pol_q);
-                    tma_load_2d(dV, &tmVb, g * HD, b * p.R, &kv_full[st], pol_q);
-                    tma_load_2d(dV + KV_TILE_BYTES / 2, &tmVb, g * HD + 64, b * p.R, &kv_full[st], pol_q);
+                    const int bo = (i == n_ctx_tiles ? b : bB) * p.R;      // the own keys of block A, then of block B
+                    tma_load_2d(dK, &tmKb, g * HD, bo, &kv_full[st], pol_q);
+                    tma_load_2d(dK + KV_TILE_BYTES / 2, &tmKb, g * HD + 64, bo, &kv_full[st], pol_q);
+                    tma_load_2d(dV, &tmVb, g * HD, bo, &kv_full[st], pol_q);
+                    tma_load_2d(dV + KV_TILE_BYTES / 2, &tmVb, g * HD + 64, bo, &kv_full[st], pol_q);
                 }
             }
             if (!ok) {
@@ -349,7 +388,12 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int kk = 0; kk < PG / 16; ++kk)
                     mma_bf16(tmem_base + COL_DQ, smem_desc_sw128(ds_addr + kk * 32), smem_desc_mn(k_addr + kk * 2048, KV_TILE_BYTES / 2),
                              idesc_dq, (i > 0 || kk > 0) ? 1u : 0u);
-                if (i == n_tiles - 1) issue_dkv_t(tmem_base, q_addr, do_addr, p_addr, ds_addr, 0u);      // the block's own keys
+                if (i >= n_ctx_tiles) {      // a block's own keys (the other block's rows hold zeros in P / dS)
+                    // block B's gradients take the columns of block A's: those must have been read out
+                    if (i > n_ctx_tiles && !mbar_wait(blk_read, 0, &flags[0])) { ok = false; break; }
+                    tc_fence_after();
+                    issue_dkv_t(tmem_base, q_addr, do_addr, p_addr, ds_addr, 0u);
+                }
                 mma_commit(&acc_done[buf]);
                 mma_commit(&kv_empty[st]);
             }
@@ -362,11 +406,13 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     } else {
         const int row = warp * 32 + lane;                       // TMEM lane
         const uint32_t tmem_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const int lrow = row & 63;                              // query row (lanes 64..127 repeat rows 0..63)
-        const bool real = lrow < p.rows_valid;
+        const int lrow = row & 63;                              // query row (one block: lanes 64..127 repeat rows 0..63)
+        const int mine = (two && row >= 64) ? bB : b;           // the block this thread's operand row belongs to
+        const bool real = lrow < p.rows_valid && mine >= 0;
         const int r = real ? lrow / p.group : 0, j = real ? lrow % p.group : 0;
-        const size_t qrow = ((size_t)b * p.R + r) * p.Hq + g * p.group + j;
-        zero_upper_rows(sPS, row);
+        const size_t qrow = ((size_t)max(mine, 0) * p.R + r) * p.Hq + g * p.group + j;
+        const int L_mine = (two && row >= 64) ? LB : LA;
+        if (!two) zero_upper_rows(sPS, row);
         // D = rowsum(dO * O) and the row's log-sum-exp in the log2 domain
         float Dr = 0.f, lse2 = 0.f;
         if (real) {
@@ -384,19 +430,34 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     Dr = fmaf(x.y, y.y, Dr);
                 }
             }
-            if (row < 64) p.D[qrow] = Dr;
+            if (two || row < 64) p.D[qrow] = Dr;
             lse2 = __ldg(p.lse + qrow) * LOG2E;
         }
+        // a block's own-key gradients leave TMEM as soon as their tile's products are complete
+        auto write_own = [&](int blk) {
+            float tv[32], tk[32];      // dV_blk^T, dK_blk^T: lane = head_dim index, column = block row
+            tmem_ld32(tmem_row + COL_DVT, tv);
+            tmem_ld32(tmem_row + COL_DKT, tk);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                if (c < p.R) {
+                    const size_t at = (((size_t)blk * p.R + c) * p.Hkv + g) * HD + row;
+                    p.dv_blk[at] = __float2bfloat16_rn(tv[c]);
+                    p.dk_blk[at] = __float2bfloat16_rn(tk[c]);
+                }
+            }
+        };
         bool ok = true;
         for (int i = 0; i < n_tiles; ++i) {
             const int buf = i & 1;
             int n_valid, vis;
             if (i < n_ctx_tiles) {
                 n_valid = min(PG, L - i * PG);
-                vis = n_valid;
+                vis = min(max(L_mine - i * PG, 0), PG);
             } else {
                 n_valid = p.R;
-                vis = p.causal ? min(r + 1, p.R) : p.R;
+                const int owner = i == n_ctx_tiles ? b : bB;      // whose own keys these are
+                vis = mine == owner ? (p.causal ? min(r + 1, p.R) : p.R) : 0;
             }
             if (!real) vis = 0;
             if (!mbar_wait(&s_full[buf], (i >> 1) & 1, &flags[0])) { ok = false; break; }
@@ -404,7 +465,8 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // P / dS buffer `buf` is still being read by the products of tile i - 2 until their acc_done
             if (i >= 2 && !mbar_wait(&acc_done[buf], ((i - 2) >> 1) & 1, &flags[0])) { ok = false; break; }
             uint8_t* sP = sPS + (size_t)buf * 2 * PS_BYTES;
-            row_math(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
+            if (two) row_math_full(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
+            else row_math(tmem_row + sdp_col(buf), sP, sP + PS_BYTES, row, vis, lse2, Dr, p.scale, p.scale_log2);
             // keys that do not exist must not poison dS K with whatever the page holds there
             if (n_valid < PG) {
                 uint8_t* dK = sKV + (size_t)(i % KV_STAGES) * 2 * KV_TILE_BYTES;
@@ -418,6 +480,17 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(&ds_full[buf]);
+            if (bB >= 0 && i == n_tiles - 1) {
+                // block A's own-key tile was the one before: its products are complete once its acc_done fires;
+                // read its gradients out, then block B's products (waiting on blk_read) may take the columns
+                const int ia = n_ctx_tiles;
+                if (!mbar_wait(&acc_done[ia & 1], (ia >> 1) & 1, &flags[0])) { ok = false; break; }
+                tc_fence_after();
+                write_own(b);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(blk_read);
+            }
         }
         // the tensor pipe completes in order: the last tile's products close the accumulators
         if (ok && !mbar_wait(&acc_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, &flags[0])) ok = false;
@@ -434,7 +507,7 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int c4 = 0; c4 < HD / 32; ++c4) {
                 float o[32];
                 tmem_ld32(tmem_row + COL_DQ + c4 * 32, o);
-                if (real && row < 64) {
+                if (real && (two || row < 64)) {
 #pragma unroll
                     for (int d = 0; d < 32; d += 8) {
                         uint4 w4;
@@ -446,18 +519,7 @@ attn_bwd_q_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                 }
             }
-            // dV_blk^T, dK_blk^T: lane = head_dim index, column = block row
-            float tv[32], tk[32];
-            tmem_ld32(tmem_row + COL_DVT, tv);
-            tmem_ld32(tmem_row + COL_DKT, tk);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                if (c < p.R) {
-                    const size_t at = (((size_t)b * p.R + c) * p.Hkv + g) * HD + row;
-                    p.dv_blk[at] = __float2bfloat16_rn(tv[c]);
-                    p.dk_blk[at] = __float2bfloat16_rn(tk[c]);
-                }
-            }
+            write_own(bB >= 0 ? bB : b);      // the own-key gradients of the last own tile
         }
     }
     tc_fence_before();
@@ -728,7 +790,15 @@ int launch_attention_bwd(const Launch& L, const dflash_attn_bwd_args& a, float* 
             return DFLASH_ERR_CUDA;
         if (dev >= 0) attr_set[dev] = true;
     }
-    if (launch_ordered(attn_bwd_q_kernel, dim3(p.Hkv, a.batch), dim3(N_THREADS), (size_t)SMEM_Q, L.st, tq, tdo, tpool, tkb, tvb, p) !=
+    // the blocks by falling context length, behind D in the scratch (a.batch ints)
+    int32_t* order = reinterpret_cast<int32_t*>(D + (((size_t)a.batch * a.rows * c.n_q_heads + 63) / 64) * 64);
+    p.order = order;
+    if (launch_ordered(order_kernel, dim3(1), dim3(1024), (size_t)std::min(a.batch, ORDER_MAX) * 4, L.st, a.ctx_len, a.batch, order) !=
+        cudaSuccess)
+        return DFLASH_ERR_CUDA;
+    ++g_launches;
+    const int q_ctas = p.shared_row ? (a.batch + 1) / 2 : a.batch;      // blocks sharing one page-table row: two per CTA
+    if (launch_ordered(attn_bwd_q_kernel, dim3(p.Hkv, q_ctas), dim3(N_THREADS), (size_t)SMEM_Q, L.st, tq, tdo, tpool, tkb, tvb, p) !=
         cudaSuccess)
         return DFLASH_ERR_CUDA;
     ++g_launches;

@@ -92,11 +92,13 @@ def test_backward_of_separate_sequences(mode, R):
             assert np.all(dkv[last, :, :, n:, :] == 0)
 
 
-def test_backward_of_anchor_blocks_over_one_sequence_adds_context_gradients_in_order():
+@pytest.mark.parametrize("anchors", [(0, 16, 64, 65, 200, 313, 17, 130), (5, 300, 300, 64, 1, 129, 77), (250,)])
+def test_backward_of_anchor_blocks_over_one_sequence_adds_context_gradients_in_order(anchors):
+    # the kernels take these blocks two at a time (by falling context length, ties by index): an even count, an odd
+    # count with a tie, a single block
     cfg = synth.MID
     one = Case(cfg, (330,), seed=29)
     one.fill_pool_synthetic()
-    anchors = (0, 16, 64, 65, 200, 313, 17, 130)
     S, R, layer = len(anchors), cfg.block_size, 0
     table = one.page_table.repeat(S, 1).contiguous()
     ctx = torch.tensor(anchors, dtype=torch.int32, device=one.device)
