@@ -359,8 +359,8 @@ int32_t dflash_block_attention(dflash_handle* h, const dflash_attn_args* a /*[ho
  *     dkv_ctx[page][K=0|V=1][kv_head][slot][head_dim]
  * for every page that holds positions below max_ctx_len of a page-table row in use (whole pages are written,
  * zeros where no block sees a key); other pages are not touched. shared_page_row = 1 (the training layout): every
- * block reads page-table row 0 and the gradients of a position add up over all blocks that see it, in batch order
- * (bit-reproducible, no atomics). shared_page_row = 0: block b uses row b and owns its pages.
+ * block reads page-table row 0 and the gradients of a position add up over all blocks that see it in an order fixed
+ * by the batch order (two blocks at a time; bit-reproducible, no atomics). shared_page_row = 0: block b uses row b and owns its pages.
  * bf16 handles with head_dim 128, 64-token pages and rows * (Hq/Hkv) <= 64 only (DFLASH_ERR_UNSUPPORTED else).
  * Workspace as for dflash_block_attention. Errors as there; a ctx_len above max_ctx_len is clamped and flagged. */
 typedef struct {
